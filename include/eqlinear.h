@@ -1,0 +1,183 @@
+/*
+ * eqlinear.h -- C ABI of the Flash EQ-Linear hot path for NVIDIA B200 (sm_100a).
+ *
+ * The operator (Eq. 1 of the paper; circular-convolution reading of Eq. 3-5 and Eq. 19-21):
+ *
+ *     y[n, o, t] = bias[o] + sum_{i < C_in} sum_{s < T}  w[o, i, (t - s) mod T] * x[n, i, s]
+ *
+ * i.e. an ordinary linear layer whose dense weight is block-circulant over a cyclic group of
+ * order T.  The library never forms that dense weight: it evaluates Algorithm 1 -- a real DFT
+ * along the group axis, one complex channel-mixing product per retained frequency
+ * k = 0..floor(T/2), and the inverse real DFT plus bias -- for the forward pass and for both
+ * gradients.
+ *
+ * Conventions common to every entry point
+ *   - Features are dense row-major [N, C*T] with the group index fastest: element (n, c, t) is at
+ *     n*C*T + c*T + t.  The weight is [C_out, C_in, T] with the group offset r fastest; the bias
+ *     is [C_out].
+ *   - x, y, dy, dx, w and bias have the plan's dtype (EQL_FP32: float; EQL_FP16: IEEE half with
+ *     float accumulation).  dw and db are always float.
+ *   - Every tensor pointer is DEVICE memory owned by the caller, 16-byte aligned; outputs must not
+ *     alias inputs.  The *_host entry points are the only ones that take host pointers.
+ *   - The library allocates no device memory.  The plan keeps its derived weights in a
+ *     caller-owned device workspace; eqlinear_bwd_weight uses a caller-owned device scratch buffer.
+ *     Both must stay valid (and untouched by the caller) while in use.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Calls are
+ *     asynchronous on that stream and never synchronise the device, except where stated.
+ *   - Errors are return codes.  Argument errors are detected on the host before any launch.
+ *     N == 0 is a successful no-op.  Nothing traps or aborts on the device.
+ *   - A plan may be used from one stream at a time.
+ */
+#ifndef EQLINEAR_H_
+#define EQLINEAR_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct eqlinear_plan_s* eqlinear_plan_t;   /* opaque host object */
+
+typedef enum {
+    EQL_OK = 0,
+    EQL_ERR_INVALID_ARG = 1,      /* NULL pointer, negative size, bad enum                    */
+    EQL_ERR_UNSUPPORTED = 2,      /* group order or channel count outside the supported set   */
+    EQL_ERR_ALIGNMENT = 3,        /* pointer not 16-byte aligned, or row bytes not multiple of 16 */
+    EQL_ERR_WORKSPACE = 4,        /* workspace / scratch / staging buffer too small           */
+    EQL_ERR_ARCH = 5,             /* current device is not compute capability 10.x            */
+    EQL_ERR_CUDA = 6,             /* a CUDA runtime or driver call failed                      */
+    EQL_ERR_DEVICE_TIMEOUT = 7    /* a bounded wait inside a kernel ran out                    */
+} eql_status_t;
+
+typedef enum { EQL_FP32 = 0, EQL_FP16 = 1 } eql_dtype_t;
+
+/* Plan flags. */
+enum {
+    /* Use the index (s - t) mod T printed in Eq. 1-2 (circular correlation) instead of the
+     * (t - s) mod T of Eq. 3-5 / Eq. 19-21.  Costs nothing at run time (the weight spectrum is
+     * conjugated when the plan is built). */
+    EQL_FLAG_CORRELATION = 1u,
+    /* Force the CUDA-core (FFMA) kernels even where a tensor-core kernel exists. */
+    EQL_FLAG_FORCE_SIMT = 2u
+};
+
+typedef struct {
+    int32_t T, C_in, C_out, dtype;
+    uint32_t flags;
+    int32_t fwd_kernel;           /* 0 = CUDA-core FFMA kernel, 1 = tcgen05 tensor-core kernel */
+    int32_t bwd_data_kernel;
+    int32_t bwd_weight_kernel;
+    int64_t macs_per_token;       /* Step-2 multiply-accumulates of Algorithm 1 per token, exact count */
+    int64_t dense_macs_per_token; /* the naive dense layer's: (C_out*T)*(C_in*T)               */
+    int64_t bytes_per_token_fwd;  /* algorithmic HBM bytes per token of fwd: (C_in + C_out)*T*elem */
+    int64_t bytes_per_token_bwd_data;
+    int64_t bytes_per_token_bwd_weight;
+    size_t  workspace_bytes;
+} eql_info_t;
+
+/* ---- host-only helpers (no GPU needed) ------------------------------------------------------ */
+
+/* Text for a status code; never NULL. */
+const char* eqlinear_status_string(eql_status_t status);
+
+/* Multiply-accumulate counts for N tokens.  Step 2 of Algorithm 1 costs one real product per real
+ * frequency plane (k = 0 and, for even T, k = T/2) and four per complex one, so for even T
+ *   spectral = (2T - 2) * N * C_in * C_out   (6/16 of dense at T = 4, Theorem 1),
+ * for odd T (2T - 1) * N * C_in * C_out; dense = N * (C_out*T) * (C_in*T) (Eq. 1).
+ * Either output pointer may be NULL. */
+eql_status_t eqlinear_count_macs(int T, int C_in, int C_out, int64_t N,
+                                 int64_t* spectral_macs, int64_t* dense_macs);
+
+/* Size in bytes of the device workspace a plan of this shape needs. */
+eql_status_t eqlinear_workspace_bytes(int T, int C_in, int C_out, eql_dtype_t dtype, size_t* bytes);
+
+/* ---- plan (Algorithm 1, step 1 for the weight: the spectral weight, computed once) ---------- */
+
+/* Build a plan on the current device: validates the shape, takes the group DFT of w (Eq. 4),
+ * and stores the frequency planes of w -- in the operand layouts of the forward and of the
+ * conjugate-transposed data-gradient product, with the 1/T of the inverse DFT folded in -- and a
+ * copy of the bias in `workspace`.
+ *   T            group order, one of 2, 4, 8, 16, 32
+ *   C_in, C_out  channels per group element, >= 1; C_in*T*elem and C_out*T*elem must be
+ *                multiples of 16 bytes
+ *   w            device, [C_out, C_in, T], plan dtype
+ *   bias         device, [C_out], plan dtype, or NULL for no bias
+ *   workspace    device, 256-byte aligned, at least eqlinear_workspace_bytes() bytes; owned by the
+ *                caller, used by the plan until eqlinear_plan_destroy
+ * The weight transform is enqueued on `stream`; later calls on the same stream see it.
+ * On error *plan is set to NULL. */
+eql_status_t eqlinear_plan(eqlinear_plan_t* plan, int T, int C_in, int C_out, eql_dtype_t dtype,
+                           const void* w, const void* bias,
+                           void* workspace, size_t workspace_bytes,
+                           unsigned flags, void* stream);
+
+/* Recompute the spectral weight from new parameter values (after an optimiser step).
+ * bias == NULL keeps "no bias" only if the plan was built without one (else INVALID_ARG). */
+eql_status_t eqlinear_plan_set_weight(eqlinear_plan_t plan, const void* w, const void* bias, void* stream);
+
+eql_status_t eqlinear_plan_info(eqlinear_plan_t plan, eql_info_t* info);
+
+/* Reads the plan's device status word (synchronises `stream`): EQL_OK, or
+ * EQL_ERR_DEVICE_TIMEOUT if a bounded wait inside one of the plan's kernels gave up. */
+eql_status_t eqlinear_plan_device_status(eqlinear_plan_t plan, void* stream);
+
+/* Frees the host object only (the workspace is the caller's). NULL is accepted. */
+eql_status_t eqlinear_plan_destroy(eqlinear_plan_t plan);
+
+/* ---- the hot path ---------------------------------------------------------------------------- */
+
+/* Forward (Algorithm 1, steps 1-4; Eq. 4-7): y = circular-convolution layer of x, plus bias.
+ *   x  device [N, C_in*T]   y  device [N, C_out*T]   both plan dtype, N >= 0 tokens. */
+eql_status_t eqlinear_fwd(eqlinear_plan_t plan, const void* x, void* y, int64_t N, void* stream);
+
+/* Gradient with respect to the input: the same Fourier-domain decomposition with the conjugate
+ * transposed spectral weight, dx^_k = dy^_k . conj(w^_k) (appendix, "Forward and backward passes").
+ *   dy device [N, C_out*T]   dx device [N, C_in*T]. */
+eql_status_t eqlinear_bwd_data(eqlinear_plan_t plan, const void* dy, void* dx, int64_t N, void* stream);
+
+/* Bytes of device scratch eqlinear_bwd_weight needs for N tokens with this plan. */
+eql_status_t eqlinear_bwd_weight_scratch_bytes(eqlinear_plan_t plan, int64_t N, size_t* bytes);
+
+/* Gradients with respect to the original parameters (appendix, "Forward and backward passes"):
+ *   dw^_k[o, i] = sum_n dy^_k[n, o] * conj(x^_k[n, i]),  dw = inverse group DFT of dw^ (with 1/T),
+ *   db[o] = sum_n sum_t dy[n, o, t].
+ *   x device [N, C_in*T], dy device [N, C_out*T] (plan dtype);
+ *   dw device [C_out, C_in, T] float;  db device [C_out] float or NULL;
+ *   scratch device, 256-byte aligned, >= eqlinear_bwd_weight_scratch_bytes(); holds the per-split
+ *   partial spectra between the two kernels of this call; contents are undefined afterwards.
+ * dw and db are overwritten (not accumulated into); with N == 0 they are set to zero.
+ * The reduction order is fixed, so results are bit-reproducible run to run. */
+eql_status_t eqlinear_bwd_weight(eqlinear_plan_t plan, const void* x, const void* dy,
+                                 void* dw, void* db, int64_t N,
+                                 void* scratch, size_t scratch_bytes, void* stream);
+
+/* ---- host-buffer variants (end-to-end measurement, small-batch convenience) ------------------ */
+/* Same operations with HOST input/output buffers (pinned memory recommended).  Each call copies
+ * its inputs into the caller's device staging buffers on `stream`, runs the kernels above and
+ * copies the results back, all asynchronously on `stream`; the host buffers may be read once the
+ * stream has been synchronised.  Staging buffers are device memory with the sizes of the
+ * corresponding device-variant tensors. */
+eql_status_t eqlinear_fwd_host(eqlinear_plan_t plan, const void* x_host, void* y_host, int64_t N,
+                               void* x_staging, void* y_staging, void* stream);
+eql_status_t eqlinear_bwd_data_host(eqlinear_plan_t plan, const void* dy_host, void* dx_host, int64_t N,
+                                    void* dy_staging, void* dx_staging, void* stream);
+eql_status_t eqlinear_bwd_weight_host(eqlinear_plan_t plan, const void* x_host, const void* dy_host,
+                                      void* dw_host, void* db_host, int64_t N,
+                                      void* x_staging, void* dy_staging, void* dw_staging, void* db_staging,
+                                      void* scratch, size_t scratch_bytes, void* stream);
+
+/* One whole training step of the layer from host buffers: copies x and dy to the device once, runs
+ * eqlinear_fwd, eqlinear_bwd_data and eqlinear_bwd_weight, and copies y, dx, dw and db back, all
+ * asynchronously on `stream` (N > 0).  db_host / db_staging may both be NULL. */
+eql_status_t eqlinear_step_host(eqlinear_plan_t plan, const void* x_host, const void* dy_host,
+                                void* y_host, void* dx_host, void* dw_host, void* db_host, int64_t N,
+                                void* x_staging, void* dy_staging, void* y_staging, void* dx_staging,
+                                void* dw_staging, void* db_staging,
+                                void* scratch, size_t scratch_bytes, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* EQLINEAR_H_ */

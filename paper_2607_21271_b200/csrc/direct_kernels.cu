@@ -1,0 +1,435 @@
+// CUDA-core (FFMA) kernels of the EQ-Linear path: the FP32 production path, and the bring-up /
+// fallback path for FP16 I/O (half in, float math, half out).
+//
+// All three fuse Algorithm 1 into one GEMM-like dataflow: the group DFT (Eq. 4) is applied to each
+// group tuple as it is loaded, the per-frequency complex products (Eq. 5) accumulate in registers,
+// and the inverse DFT (Eq. 7) plus bias runs in the epilogue; no frequency-domain tensor touches
+// global memory except the weight-gradient's split partials.
+#include <cuda_fp16.h>
+
+#include "eql_internal.h"
+#include "rdft.cuh"
+
+namespace eql {
+namespace {
+
+// ---- group-tuple loads and stores (T contiguous elements, T*sizeof(IO) in {4, 8, 16, 32, ...} bytes)
+template <int BYTES>
+struct VecBytes { using type = uint4; static constexpr int n = BYTES / 16; };
+template <> struct VecBytes<8> { using type = uint2; static constexpr int n = 1; };
+template <> struct VecBytes<4> { using type = uint32_t; static constexpr int n = 1; };
+
+template <int T, typename IO>
+__device__ __forceinline__ void load_group(const IO* __restrict__ p, float* v) {
+    using V = VecBytes<T * sizeof(IO)>;
+    union { typename V::type vec[V::n]; IO e[T]; } u;
+#pragma unroll
+    for (int i = 0; i < V::n; ++i) u.vec[i] = __ldg(reinterpret_cast<const typename V::type*>(p) + i);
+#pragma unroll
+    for (int i = 0; i < T; ++i) {
+        if constexpr (sizeof(IO) == 4) v[i] = u.e[i]; else v[i] = __half2float(u.e[i]);
+    }
+}
+
+template <int T, typename IO>
+__device__ __forceinline__ void store_group(IO* __restrict__ p, const float* v) {
+    using V = VecBytes<T * sizeof(IO)>;
+    union { typename V::type vec[V::n]; IO e[T]; } u;
+#pragma unroll
+    for (int i = 0; i < T; ++i) {
+        if constexpr (sizeof(IO) == 4) u.e[i] = v[i]; else u.e[i] = __float2half_rn(v[i]);
+    }
+#pragma unroll
+    for (int i = 0; i < V::n; ++i) reinterpret_cast<typename V::type*>(p)[i] = u.vec[i];
+}
+
+// ---- tile shapes: 256 threads as 16 x 16, each owning TM x TN (row, column) pairs for all T planes
+template <int T> struct DirectCfg;
+template <> struct DirectCfg<2>  { static constexpr int TM = 8, TN = 4, BK = 8; };
+template <> struct DirectCfg<4>  { static constexpr int TM = 8, TN = 4, BK = 8; };
+template <> struct DirectCfg<8>  { static constexpr int TM = 4, TN = 4, BK = 8; };
+template <> struct DirectCfg<16> { static constexpr int TM = 4, TN = 2, BK = 4; };
+template <> struct DirectCfg<32> { static constexpr int TM = 2, TN = 2, BK = 4; };
+
+constexpr int kThreads = 256;
+constexpr int kPad = 4;
+
+// acc[p][i][j] += a[p][i] (x) b[p][j] over the real-packed planes: one product for the real
+// frequencies, the four-product complex multiply for the others (Eq. 5 written in real arithmetic,
+// as in Eq. 20).  CONJ_B multiplies by the conjugate of b instead.
+template <int T, int TM, int TN, bool CONJ_B>
+__device__ __forceinline__ void plane_mac(float (&acc)[T][TM][TN], const float (&a)[T][TM], const float (&b)[T][TN]) {
+#pragma unroll
+    for (int i = 0; i < TM; ++i)
+#pragma unroll
+        for (int j = 0; j < TN; ++j) {
+            acc[0][i][j] = fmaf(a[0][i], b[0][j], acc[0][i][j]);
+            acc[T - 1][i][j] = fmaf(a[T - 1][i], b[T - 1][j], acc[T - 1][i][j]);
+        }
+#pragma unroll
+    for (int k = 1; k < T / 2; ++k) {
+        const int pr = 2 * k - 1, pi = 2 * k;
+#pragma unroll
+        for (int i = 0; i < TM; ++i)
+#pragma unroll
+            for (int j = 0; j < TN; ++j) {
+                if constexpr (!CONJ_B) {
+                    acc[pr][i][j] = fmaf(a[pr][i], b[pr][j], acc[pr][i][j]);
+                    acc[pr][i][j] = fmaf(-a[pi][i], b[pi][j], acc[pr][i][j]);
+                    acc[pi][i][j] = fmaf(a[pr][i], b[pi][j], acc[pi][i][j]);
+                    acc[pi][i][j] = fmaf(a[pi][i], b[pr][j], acc[pi][i][j]);
+                } else {
+                    acc[pr][i][j] = fmaf(a[pr][i], b[pr][j], acc[pr][i][j]);
+                    acc[pr][i][j] = fmaf(a[pi][i], b[pi][j], acc[pr][i][j]);
+                    acc[pi][i][j] = fmaf(a[pi][i], b[pr][j], acc[pi][i][j]);
+                    acc[pi][i][j] = fmaf(-a[pr][i], b[pi][j], acc[pi][i][j]);
+                }
+            }
+    }
+}
+
+template <int N>
+__device__ __forceinline__ void lds_vec(const float* p, float* out) {
+    if constexpr (N % 4 == 0) {
+#pragma unroll
+        for (int i = 0; i < N / 4; ++i) {
+            float4 t = reinterpret_cast<const float4*>(p)[i];
+            out[4 * i] = t.x; out[4 * i + 1] = t.y; out[4 * i + 2] = t.z; out[4 * i + 3] = t.w;
+        }
+    } else {
+        static_assert(N % 2 == 0, "micro tile");
+#pragma unroll
+        for (int i = 0; i < N / 2; ++i) {
+            float2 t = reinterpret_cast<const float2*>(p)[i];
+            out[2 * i] = t.x; out[2 * i + 1] = t.y;
+        }
+    }
+}
+
+// ================================================================================================
+// Spectral weight (Algorithm 1, step 1 for the parameters): one thread per (o, i).
+// planes_fwd[p][i][o] = scale_p * W^_p[o][i];  planes_bwd[p][o][i] = scale_p * conj(W^)_p[o][i].
+// With the correlation flag the spectrum is conjugated (weight reversed along the group axis).
+template <int T, typename IO>
+__global__ void plan_weights_kernel(const IO* __restrict__ w, const IO* __restrict__ bias, int Ci, int Co,
+                                    bool correlation, float* __restrict__ pf, float* __restrict__ pb,
+                                    float* __restrict__ bias_f32) {
+    const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx < Co && bias_f32 != nullptr) {
+        if constexpr (sizeof(IO) == 4) bias_f32[idx] = bias[idx]; else bias_f32[idx] = __half2float(bias[idx]);
+    }
+    if (idx >= Ci * Co) return;
+    const int o = idx / Ci, i = idx - o * Ci;
+    float v[T];
+#pragma unroll
+    for (int r = 0; r < T; ++r) {
+        if constexpr (sizeof(IO) == 4) v[r] = w[(size_t)idx * T + r]; else v[r] = __half2float(w[(size_t)idx * T + r]);
+    }
+    rdft_forward<T>(v);
+#pragma unroll
+    for (int p = 0; p < T; ++p) {
+        const bool imag = (p != 0) && (p != T - 1) && ((p & 1) == 0);
+        float f = v[p] * plane_inverse_scale<T>(p);
+        if (imag && correlation) f = -f;
+        pf[((size_t)p * Ci + i) * Co + o] = f;
+        pb[((size_t)p * Co + o) * Ci + i] = imag ? -f : f;
+    }
+}
+
+// ================================================================================================
+// Fused forward / data-gradient kernel: out = IDFT( DFT(in) (x) planes ) + bias.
+// Block tile: BM rows (tokens) x BN output channels, all T planes; input channels streamed in chunks.
+template <int T, typename IO>
+__global__ void __launch_bounds__(kThreads)
+direct_linear_kernel(const IO* __restrict__ in, IO* __restrict__ out, int64_t N, int Cin, int Cout,
+                     const float* __restrict__ planes, const float* __restrict__ bias) {
+    using C = DirectCfg<T>;
+    constexpr int TM = C::TM, TN = C::TN, BK = C::BK, BM = 16 * TM, BN = 16 * TN;
+    __shared__ __align__(16) float xs[T][BK][BM + kPad];
+    __shared__ __align__(16) float ws[T][BK][BN + kPad];
+
+    const int tid = threadIdx.x, tm = tid & 15, tn = tid >> 4;
+    const int64_t m0 = (int64_t)blockIdx.x * BM;
+    const int n0 = blockIdx.y * BN;
+
+    float acc[T][TM][TN];
+#pragma unroll
+    for (int p = 0; p < T; ++p)
+#pragma unroll
+        for (int i = 0; i < TM; ++i)
+#pragma unroll
+            for (int j = 0; j < TN; ++j) acc[p][i][j] = 0.f;
+
+    for (int k0 = 0; k0 < Cin; k0 += BK) {
+        // group tuples of the input chunk -> DFT -> planes in shared memory
+        for (int item = tid; item < BM * BK; item += kThreads) {
+            const int kk = item % BK, m = item / BK;
+            float v[T];
+            const int64_t row = m0 + m;
+            if (row < N && k0 + kk < Cin) {
+                load_group<T, IO>(in + row * (int64_t)Cin * T + (int64_t)(k0 + kk) * T, v);
+                rdft_forward<T>(v);
+            } else {
+#pragma unroll
+                for (int p = 0; p < T; ++p) v[p] = 0.f;
+            }
+#pragma unroll
+            for (int p = 0; p < T; ++p) xs[p][kk][m] = v[p];
+        }
+        for (int idx = tid; idx < T * BK * BN; idx += kThreads) {
+            const int n = idx % BN, kk = (idx / BN) % BK, p = idx / (BN * BK);
+            float f = 0.f;
+            if (k0 + kk < Cin && n0 + n < Cout) f = __ldg(planes + ((size_t)p * Cin + k0 + kk) * Cout + n0 + n);
+            ws[p][kk][n] = f;
+        }
+        __syncthreads();
+#pragma unroll 2
+        for (int kk = 0; kk < BK; ++kk) {
+            float a[T][TM], b[T][TN];
+#pragma unroll
+            for (int p = 0; p < T; ++p) {
+                lds_vec<TM>(&xs[p][kk][tm * TM], a[p]);
+                lds_vec<TN>(&ws[p][kk][tn * TN], b[p]);
+            }
+            plane_mac<T, TM, TN, false>(acc, a, b);
+        }
+        __syncthreads();
+    }
+
+    // epilogue: inverse DFT over the planes, bias, one contiguous group tuple per (row, channel)
+#pragma unroll
+    for (int i = 0; i < TM; ++i) {
+        const int64_t row = m0 + tm * TM + i;
+        if (row >= N) continue;
+#pragma unroll
+        for (int j = 0; j < TN; ++j) {
+            const int n = n0 + tn * TN + j;
+            if (n >= Cout) continue;
+            float v[T];
+#pragma unroll
+            for (int p = 0; p < T; ++p) v[p] = acc[p][i][j];
+            if (bias != nullptr) v[0] += __ldg(bias + n);     // a constant over t lives in plane k = 0
+            rdft_inverse<T>(v);
+            store_group<T, IO>(out + row * (int64_t)Cout * T + (int64_t)n * T, v);
+        }
+    }
+}
+
+// ================================================================================================
+// Weight gradient, phase 1: per token range, dW^_p[o][i] += dY^_p[n][o] * conj(X^_p[n][i]).
+// Block tile: BO output channels x BI input channels, all planes; tokens streamed in chunks of BK.
+template <int T, typename IO>
+__global__ void __launch_bounds__(kThreads)
+direct_bwd_weight_kernel(const IO* __restrict__ x, const IO* __restrict__ dy, int64_t N, int Ci, int Co,
+                         int64_t tokens_per_split, float* __restrict__ part, float* __restrict__ db_part) {
+    using C = DirectCfg<T>;
+    constexpr int TO = C::TM, TI = C::TN, BK = C::BK, BO = 16 * TO, BI = 16 * TI;
+    __shared__ __align__(16) float gs[T][BK][BO + kPad];
+    __shared__ __align__(16) float xs[T][BK][BI + kPad];
+
+    const int tid = threadIdx.x, to = tid & 15, ti = tid >> 4;
+    const int o0 = blockIdx.x * BO, i0 = blockIdx.y * BI, split = blockIdx.z;
+    const int64_t nbeg = (int64_t)split * tokens_per_split;
+    const int64_t nend = (nbeg + tokens_per_split < N) ? nbeg + tokens_per_split : N;
+
+    float acc[T][TO][TI];
+    float dbacc[TO];
+#pragma unroll
+    for (int p = 0; p < T; ++p)
+#pragma unroll
+        for (int a = 0; a < TO; ++a)
+#pragma unroll
+            for (int b = 0; b < TI; ++b) acc[p][a][b] = 0.f;
+#pragma unroll
+    for (int a = 0; a < TO; ++a) dbacc[a] = 0.f;
+
+    for (int64_t n0 = nbeg; n0 < nend; n0 += BK) {
+        for (int item = tid; item < BO * BK; item += kThreads) {
+            const int o = item % BO, kk = item / BO;
+            float v[T];
+            if (n0 + kk < nend && o0 + o < Co) {
+                load_group<T, IO>(dy + (n0 + kk) * (int64_t)Co * T + (int64_t)(o0 + o) * T, v);
+                rdft_forward<T>(v);
+            } else {
+#pragma unroll
+                for (int p = 0; p < T; ++p) v[p] = 0.f;
+            }
+#pragma unroll
+            for (int p = 0; p < T; ++p) gs[p][kk][o] = v[p];
+        }
+        for (int item = tid; item < BI * BK; item += kThreads) {
+            const int i = item % BI, kk = item / BI;
+            float v[T];
+            if (n0 + kk < nend && i0 + i < Ci) {
+                load_group<T, IO>(x + (n0 + kk) * (int64_t)Ci * T + (int64_t)(i0 + i) * T, v);
+                rdft_forward<T>(v);
+            } else {
+#pragma unroll
+                for (int p = 0; p < T; ++p) v[p] = 0.f;
+            }
+#pragma unroll
+            for (int p = 0; p < T; ++p) xs[p][kk][i] = v[p];
+        }
+        __syncthreads();
+#pragma unroll 2
+        for (int kk = 0; kk < BK; ++kk) {
+            float a[T][TO], b[T][TI];
+#pragma unroll
+            for (int p = 0; p < T; ++p) {
+                lds_vec<TO>(&gs[p][kk][to * TO], a[p]);
+                lds_vec<TI>(&xs[p][kk][ti * TI], b[p]);
+            }
+            plane_mac<T, TO, TI, true>(acc, a, b);
+#pragma unroll
+            for (int q = 0; q < TO; ++q) dbacc[q] += a[0][q];     // db = sum_n Re dY^_0
+        }
+        __syncthreads();
+    }
+
+    const size_t plane_stride = (size_t)Co * Ci;
+    float* dst = part + (size_t)split * T * plane_stride;
+#pragma unroll
+    for (int a = 0; a < TO; ++a) {
+        const int o = o0 + to * TO + a;
+        if (o >= Co) continue;
+#pragma unroll
+        for (int b = 0; b < TI; ++b) {
+            const int i = i0 + ti * TI + b;
+            if (i >= Ci) continue;
+#pragma unroll
+            for (int p = 0; p < T; ++p) dst[p * plane_stride + (size_t)o * Ci + i] = acc[p][a][b];
+        }
+        if (blockIdx.y == 0 && ti == 0) db_part[(size_t)split * Co + o] = dbacc[a];
+    }
+}
+
+// Weight gradient, phase 2: fixed-order sum over the splits, inverse DFT with its 1/T, dw[o][i][:].
+template <int T>
+__global__ void bwd_weight_finalize_kernel(const float* __restrict__ part, const float* __restrict__ db_part,
+                                           int splits, int Ci, int Co, bool correlation,
+                                           float* __restrict__ dw, float* __restrict__ db) {
+    const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+    const size_t plane_stride = (size_t)Co * Ci;
+    if (idx < Co && db != nullptr) {
+        float s = 0.f;
+        for (int sp = 0; sp < splits; ++sp) s += db_part[(size_t)sp * Co + idx];
+        db[idx] = s;
+    }
+    if (idx >= Ci * Co) return;
+    float v[T];
+#pragma unroll
+    for (int p = 0; p < T; ++p) v[p] = 0.f;
+    for (int sp = 0; sp < splits; ++sp) {
+        const float* src = part + (size_t)sp * T * plane_stride + idx;
+#pragma unroll
+        for (int p = 0; p < T; ++p) v[p] += src[p * plane_stride];
+    }
+#pragma unroll
+    for (int p = 0; p < T; ++p) {
+        const bool imag = (p != 0) && (p != T - 1) && ((p & 1) == 0);
+        v[p] *= plane_inverse_scale<T>(p);
+        if (imag && correlation) v[p] = -v[p];
+    }
+    rdft_inverse<T>(v);
+#pragma unroll
+    for (int r = 0; r < T; ++r) dw[(size_t)idx * T + r] = v[r];
+}
+
+template <typename F>
+cudaError_t dispatch_T(int T, F&& f) {
+    switch (T) {
+        case 2: return f(std::integral_constant<int, 2>{});
+        case 4: return f(std::integral_constant<int, 4>{});
+        case 8: return f(std::integral_constant<int, 8>{});
+        case 16: return f(std::integral_constant<int, 16>{});
+        case 32: return f(std::integral_constant<int, 32>{});
+        default: return cudaErrorInvalidValue;
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_plan_weights(int T, eql_dtype_t dtype, bool correlation, const void* w, const void* bias,
+                                int Ci, int Co, float* planes_fwd, float* planes_bwd, float* bias_f32,
+                                cudaStream_t stream) {
+    const int total = Ci * Co > Co ? Ci * Co : Co;
+    const int threads = 128, blocks = (total + threads - 1) / threads;
+    return dispatch_T(T, [&](auto tc) {
+        constexpr int TT = decltype(tc)::value;
+        float* bdst = bias ? bias_f32 : nullptr;
+        if (dtype == EQL_FP32)
+            plan_weights_kernel<TT, float><<<blocks, threads, 0, stream>>>(
+                (const float*)w, (const float*)bias, Ci, Co, correlation, planes_fwd, planes_bwd, bdst);
+        else
+            plan_weights_kernel<TT, __half><<<blocks, threads, 0, stream>>>(
+                (const __half*)w, (const __half*)bias, Ci, Co, correlation, planes_fwd, planes_bwd, bdst);
+        return cudaGetLastError();
+    });
+}
+
+cudaError_t launch_direct_linear(int T, eql_dtype_t dtype, const void* in, void* out, int64_t N,
+                                 int Cin, int Cout, const float* planes, const float* bias_f32,
+                                 cudaStream_t stream) {
+    return dispatch_T(T, [&](auto tc) {
+        constexpr int TT = decltype(tc)::value;
+        using C = DirectCfg<TT>;
+        constexpr int BM = 16 * C::TM, BN = 16 * C::TN;
+        dim3 grid((unsigned)((N + BM - 1) / BM), (unsigned)((Cout + BN - 1) / BN));
+        if (dtype == EQL_FP32)
+            direct_linear_kernel<TT, float><<<grid, kThreads, 0, stream>>>(
+                (const float*)in, (float*)out, N, Cin, Cout, planes, bias_f32);
+        else
+            direct_linear_kernel<TT, __half><<<grid, kThreads, 0, stream>>>(
+                (const __half*)in, (__half*)out, N, Cin, Cout, planes, bias_f32);
+        return cudaGetLastError();
+    });
+}
+
+BwdWeightSplit direct_bwd_weight_split(int T, int Ci, int Co, int64_t N) {
+    int TO = 4, TI = 4, BK = 8;
+    switch (T) {
+        case 2: case 4: TO = 8; TI = 4; BK = 8; break;
+        case 8: TO = 4; TI = 4; BK = 8; break;
+        case 16: TO = 4; TI = 2; BK = 4; break;
+        default: TO = 2; TI = 2; BK = 4; break;
+    }
+    const int64_t tiles = (int64_t)((Co + 16 * TO - 1) / (16 * TO)) * ((Ci + 16 * TI - 1) / (16 * TI));
+    int64_t want = (2 * kNumSMs + tiles - 1) / tiles;            // about two blocks per SM in flight
+    const int64_t chunks = (N + BK - 1) / BK;
+    if (want > chunks) want = chunks;
+    if (want < 1) want = 1;
+    if (want > 65535) want = 65535;
+    BwdWeightSplit s;
+    s.tokens_per_split = ((chunks + want - 1) / want) * BK;
+    s.splits = (int)((N + s.tokens_per_split - 1) / s.tokens_per_split);
+    if (s.splits < 1) s.splits = 1;
+    s.scratch_bytes = align_up((size_t)s.splits * ((size_t)T * Co * Ci + Co) * sizeof(float), kWsAlign);
+    return s;
+}
+
+cudaError_t launch_direct_bwd_weight(int T, eql_dtype_t dtype, bool correlation, const void* x, const void* dy,
+                                     float* dw, float* db, int64_t N, int Ci, int Co,
+                                     const BwdWeightSplit& split, float* scratch, cudaStream_t stream) {
+    float* part = scratch;
+    float* db_part = scratch + (size_t)split.splits * T * Co * Ci;
+    return dispatch_T(T, [&](auto tc) {
+        constexpr int TT = decltype(tc)::value;
+        using C = DirectCfg<TT>;
+        constexpr int BO = 16 * C::TM, BI = 16 * C::TN;
+        dim3 grid((Co + BO - 1) / BO, (Ci + BI - 1) / BI, split.splits);
+        if (dtype == EQL_FP32)
+            direct_bwd_weight_kernel<TT, float><<<grid, kThreads, 0, stream>>>(
+                (const float*)x, (const float*)dy, N, Ci, Co, split.tokens_per_split, part, db_part);
+        else
+            direct_bwd_weight_kernel<TT, __half><<<grid, kThreads, 0, stream>>>(
+                (const __half*)x, (const __half*)dy, N, Ci, Co, split.tokens_per_split, part, db_part);
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+        const int total = Ci * Co > Co ? Ci * Co : Co;
+        bwd_weight_finalize_kernel<TT><<<(total + 127) / 128, 128, 0, stream>>>(
+            part, db_part, split.splits, Ci, Co, correlation, dw, db);
+        return cudaGetLastError();
+    });
+}
+
+}  // namespace eql

@@ -1,0 +1,56 @@
+// Internal declarations shared by the translation units of libeqlinear (not part of the C ABI).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "../../include/eqlinear.h"
+
+namespace eql {
+
+constexpr int kNumSMs = 148;            // B200
+constexpr size_t kWsAlign = 256;
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// Device workspace layout of a plan (offsets in bytes from the workspace base).
+struct WorkspaceLayout {
+    size_t status;        // int32 status word (+ padding)
+    size_t bias;          // float [Co]
+    size_t planes_fwd;    // float [T][Ci][Co]   pre-scaled spectral weight, forward operand order
+    size_t planes_bwd;    // float [T][Co][Ci]   conjugated, data-gradient operand order
+    size_t umma_fwd;      // half  tensor-core operand image for fwd       (FP16 plans only)
+    size_t umma_bwd;      // half  tensor-core operand image for bwd_data  (FP16 plans only)
+    size_t umma_fwd_bytes, umma_bwd_bytes;
+    size_t total;
+};
+WorkspaceLayout workspace_layout(int T, int Ci, int Co, eql_dtype_t dtype);
+
+inline bool supported_T(int T) { return T == 2 || T == 4 || T == 8 || T == 16 || T == 32; }
+
+// ---- CUDA-core (FFMA) kernels, direct_kernels.cu -------------------------------------------------
+// Spectral weight: w[Co][Ci][T] -> planes_fwd[T][Ci][Co], planes_bwd[T][Co][Ci] (float), bias -> float.
+cudaError_t launch_plan_weights(int T, eql_dtype_t dtype, bool correlation, const void* w, const void* bias,
+                                int Ci, int Co, float* planes_fwd, float* planes_bwd, float* bias_f32,
+                                cudaStream_t stream);
+
+// out[N, Cout*T] = inverse_dft( dft(in[N, Cin*T]) (x) planes[T][Cin][Cout] ) + bias   (bias may be NULL)
+cudaError_t launch_direct_linear(int T, eql_dtype_t dtype, const void* in, void* out, int64_t N,
+                                 int Cin, int Cout, const float* planes, const float* bias_f32,
+                                 cudaStream_t stream);
+
+// Split-K layout of the weight-gradient reduction.
+struct BwdWeightSplit {
+    int splits;               // number of token ranges
+    int64_t tokens_per_split; // multiple of the kernel's token chunk
+    size_t scratch_bytes;     // splits * (T*Co*Ci + Co) floats, rounded up
+};
+BwdWeightSplit direct_bwd_weight_split(int T, int Ci, int Co, int64_t N);
+
+// Partial spectra part[split][T][Co][Ci], db partials [split][Co] -> dw[Co][Ci][T], db[Co].
+cudaError_t launch_direct_bwd_weight(int T, eql_dtype_t dtype, bool correlation, const void* x, const void* dy,
+                                     float* dw, float* db, int64_t N, int Ci, int Co,
+                                     const BwdWeightSplit& split, float* scratch, cudaStream_t stream);
+
+}  // namespace eql

@@ -1,0 +1,319 @@
+// C ABI of libeqlinear: argument validation, the plan object, kernel selection, host-buffer variants.
+// Every step of the path itself runs in the kernels of the other translation units.
+#include <cuda_fp16.h>
+
+#include <new>
+
+#include "eql_internal.h"
+
+struct eqlinear_plan_s {
+    int T, Ci, Co;
+    eql_dtype_t dtype;
+    unsigned flags;
+    bool has_bias;
+    int device;
+    char* ws;
+    eql::WorkspaceLayout lay;
+    int fwd_kernel, bwd_data_kernel, bwd_weight_kernel;
+};
+
+namespace eql {
+
+WorkspaceLayout workspace_layout(int T, int Ci, int Co, eql_dtype_t dtype) {
+    WorkspaceLayout l{};
+    size_t off = 0;
+    l.status = off;      off += kWsAlign;
+    l.bias = off;        off += align_up((size_t)Co * sizeof(float), kWsAlign);
+    l.planes_fwd = off;  off += align_up((size_t)T * Ci * Co * sizeof(float), kWsAlign);
+    l.planes_bwd = off;  off += align_up((size_t)T * Ci * Co * sizeof(float), kWsAlign);
+    l.umma_fwd = off;    l.umma_fwd_bytes = 0;
+    l.umma_bwd = off;    l.umma_bwd_bytes = 0;
+    (void)dtype;
+    l.total = off;
+    return l;
+}
+
+}  // namespace eql
+
+namespace {
+
+using namespace eql;
+
+inline size_t elem_size(eql_dtype_t d) { return d == EQL_FP32 ? 4 : 2; }
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+eql_status_t check_shape(int T, int Ci, int Co, int dtype) {
+    if (dtype != EQL_FP32 && dtype != EQL_FP16) return EQL_ERR_INVALID_ARG;
+    if (T < 1 || Ci < 1 || Co < 1) return EQL_ERR_INVALID_ARG;
+    if (!supported_T(T)) return EQL_ERR_UNSUPPORTED;
+    if ((int64_t)Ci * T > (1 << 20) || (int64_t)Co * T > (1 << 20)) return EQL_ERR_UNSUPPORTED;
+    const size_t e = elem_size((eql_dtype_t)dtype);
+    if (((size_t)Ci * T * e) % 16 != 0 || ((size_t)Co * T * e) % 16 != 0) return EQL_ERR_ALIGNMENT;
+    return EQL_OK;
+}
+
+eql_status_t check_tokens(int64_t N) {
+    if (N < 0) return EQL_ERR_INVALID_ARG;
+    if (N > ((int64_t)1 << 31) - 1024) return EQL_ERR_UNSUPPORTED;
+    return EQL_OK;
+}
+
+eql_status_t build_weights(eqlinear_plan_t p, const void* w, const void* bias, cudaStream_t s) {
+    cudaError_t e = launch_plan_weights(p->T, p->dtype, (p->flags & EQL_FLAG_CORRELATION) != 0, w, bias, p->Ci, p->Co,
+                                        (float*)(p->ws + p->lay.planes_fwd), (float*)(p->ws + p->lay.planes_bwd),
+                                        (float*)(p->ws + p->lay.bias), s);
+    return e == cudaSuccess ? EQL_OK : EQL_ERR_CUDA;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* eqlinear_status_string(eql_status_t status) {
+    switch (status) {
+        case EQL_OK: return "ok";
+        case EQL_ERR_INVALID_ARG: return "invalid argument";
+        case EQL_ERR_UNSUPPORTED: return "unsupported shape (group order must be 2, 4, 8, 16 or 32)";
+        case EQL_ERR_ALIGNMENT: return "pointer or row size not 16-byte aligned";
+        case EQL_ERR_WORKSPACE: return "workspace, scratch or staging buffer too small";
+        case EQL_ERR_ARCH: return "device is not compute capability 10.x (B200)";
+        case EQL_ERR_CUDA: return "CUDA call failed";
+        case EQL_ERR_DEVICE_TIMEOUT: return "a bounded wait inside a kernel ran out";
+    }
+    return "unknown status";
+}
+
+eql_status_t eqlinear_count_macs(int T, int C_in, int C_out, int64_t N, int64_t* spectral_macs, int64_t* dense_macs) {
+    if (T < 1 || C_in < 1 || C_out < 1 || N < 0) return EQL_ERR_INVALID_ARG;
+    const int64_t n_real = (T % 2 == 0) ? 2 : 1;            // k = 0 and, for even T, k = T/2
+    const int64_t n_cplx = (T - n_real) / 2;                // 0 < k < T/2
+    if (spectral_macs) *spectral_macs = (n_real + 4 * n_cplx) * N * C_in * C_out;
+    if (dense_macs) *dense_macs = N * ((int64_t)C_out * T) * ((int64_t)C_in * T);
+    return EQL_OK;
+}
+
+eql_status_t eqlinear_workspace_bytes(int T, int C_in, int C_out, eql_dtype_t dtype, size_t* bytes) {
+    if (!bytes) return EQL_ERR_INVALID_ARG;
+    eql_status_t st = check_shape(T, C_in, C_out, dtype);
+    if (st != EQL_OK) return st;
+    *bytes = workspace_layout(T, C_in, C_out, dtype).total;
+    return EQL_OK;
+}
+
+eql_status_t eqlinear_plan(eqlinear_plan_t* plan, int T, int C_in, int C_out, eql_dtype_t dtype, const void* w,
+                           const void* bias, void* workspace, size_t workspace_bytes, unsigned flags, void* stream) {
+    if (!plan) return EQL_ERR_INVALID_ARG;
+    *plan = nullptr;
+    eql_status_t st = check_shape(T, C_in, C_out, dtype);
+    if (st != EQL_OK) return st;
+    if (!w || !workspace) return EQL_ERR_INVALID_ARG;
+    if (flags & ~(unsigned)(EQL_FLAG_CORRELATION | EQL_FLAG_FORCE_SIMT)) return EQL_ERR_INVALID_ARG;
+    if (!aligned16(w) || (bias && !aligned16(bias))) return EQL_ERR_ALIGNMENT;
+    if (reinterpret_cast<uintptr_t>(workspace) % kWsAlign != 0) return EQL_ERR_ALIGNMENT;
+    WorkspaceLayout lay = workspace_layout(T, C_in, C_out, dtype);
+    if (workspace_bytes < lay.total) return EQL_ERR_WORKSPACE;
+
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return EQL_ERR_CUDA;
+    int major = 0;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return EQL_ERR_CUDA;
+    if (major != 10) return EQL_ERR_ARCH;
+
+    eqlinear_plan_s* p = new (std::nothrow) eqlinear_plan_s();
+    if (!p) return EQL_ERR_INVALID_ARG;
+    p->T = T; p->Ci = C_in; p->Co = C_out; p->dtype = dtype; p->flags = flags;
+    p->has_bias = bias != nullptr; p->device = dev; p->ws = (char*)workspace; p->lay = lay;
+    p->fwd_kernel = p->bwd_data_kernel = p->bwd_weight_kernel = 0;
+
+    cudaStream_t s = (cudaStream_t)stream;
+    if (cudaMemsetAsync(p->ws + lay.status, 0, kWsAlign, s) != cudaSuccess) { delete p; return EQL_ERR_CUDA; }
+    st = build_weights(p, w, bias, s);
+    if (st != EQL_OK) { delete p; return st; }
+    *plan = p;
+    return EQL_OK;
+}
+
+eql_status_t eqlinear_plan_set_weight(eqlinear_plan_t plan, const void* w, const void* bias, void* stream) {
+    if (!plan || !w) return EQL_ERR_INVALID_ARG;
+    if ((bias != nullptr) != plan->has_bias) return EQL_ERR_INVALID_ARG;
+    if (!aligned16(w) || (bias && !aligned16(bias))) return EQL_ERR_ALIGNMENT;
+    return build_weights(plan, w, bias, (cudaStream_t)stream);
+}
+
+eql_status_t eqlinear_plan_info(eqlinear_plan_t plan, eql_info_t* info) {
+    if (!plan || !info) return EQL_ERR_INVALID_ARG;
+    const int64_t e = (int64_t)elem_size(plan->dtype);
+    info->T = plan->T; info->C_in = plan->Ci; info->C_out = plan->Co; info->dtype = plan->dtype;
+    info->flags = plan->flags;
+    info->fwd_kernel = plan->fwd_kernel;
+    info->bwd_data_kernel = plan->bwd_data_kernel;
+    info->bwd_weight_kernel = plan->bwd_weight_kernel;
+    eqlinear_count_macs(plan->T, plan->Ci, plan->Co, 1, &info->macs_per_token, &info->dense_macs_per_token);
+    info->bytes_per_token_fwd = (int64_t)(plan->Ci + plan->Co) * plan->T * e;
+    info->bytes_per_token_bwd_data = info->bytes_per_token_fwd;
+    info->bytes_per_token_bwd_weight = info->bytes_per_token_fwd;
+    info->workspace_bytes = plan->lay.total;
+    return EQL_OK;
+}
+
+eql_status_t eqlinear_plan_device_status(eqlinear_plan_t plan, void* stream) {
+    if (!plan) return EQL_ERR_INVALID_ARG;
+    int word = 0;
+    cudaStream_t s = (cudaStream_t)stream;
+    if (cudaMemcpyAsync(&word, plan->ws + plan->lay.status, sizeof(int), cudaMemcpyDeviceToHost, s) != cudaSuccess)
+        return EQL_ERR_CUDA;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return EQL_ERR_CUDA;
+    return word == 0 ? EQL_OK : EQL_ERR_DEVICE_TIMEOUT;
+}
+
+eql_status_t eqlinear_plan_destroy(eqlinear_plan_t plan) {
+    delete plan;
+    return EQL_OK;
+}
+
+eql_status_t eqlinear_fwd(eqlinear_plan_t plan, const void* x, void* y, int64_t N, void* stream) {
+    if (!plan) return EQL_ERR_INVALID_ARG;
+    eql_status_t st = check_tokens(N);
+    if (st != EQL_OK) return st;
+    if (N == 0) return EQL_OK;
+    if (!x || !y || x == y) return EQL_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(y)) return EQL_ERR_ALIGNMENT;
+    const float* bias = plan->has_bias ? (const float*)(plan->ws + plan->lay.bias) : nullptr;
+    cudaError_t e = launch_direct_linear(plan->T, plan->dtype, x, y, N, plan->Ci, plan->Co,
+                                         (const float*)(plan->ws + plan->lay.planes_fwd), bias, (cudaStream_t)stream);
+    return e == cudaSuccess ? EQL_OK : EQL_ERR_CUDA;
+}
+
+eql_status_t eqlinear_bwd_data(eqlinear_plan_t plan, const void* dy, void* dx, int64_t N, void* stream) {
+    if (!plan) return EQL_ERR_INVALID_ARG;
+    eql_status_t st = check_tokens(N);
+    if (st != EQL_OK) return st;
+    if (N == 0) return EQL_OK;
+    if (!dy || !dx || dy == dx) return EQL_ERR_INVALID_ARG;
+    if (!aligned16(dy) || !aligned16(dx)) return EQL_ERR_ALIGNMENT;
+    cudaError_t e = launch_direct_linear(plan->T, plan->dtype, dy, dx, N, plan->Co, plan->Ci,
+                                         (const float*)(plan->ws + plan->lay.planes_bwd), nullptr, (cudaStream_t)stream);
+    return e == cudaSuccess ? EQL_OK : EQL_ERR_CUDA;
+}
+
+eql_status_t eqlinear_bwd_weight_scratch_bytes(eqlinear_plan_t plan, int64_t N, size_t* bytes) {
+    if (!plan || !bytes) return EQL_ERR_INVALID_ARG;
+    eql_status_t st = check_tokens(N);
+    if (st != EQL_OK) return st;
+    *bytes = direct_bwd_weight_split(plan->T, plan->Ci, plan->Co, N > 0 ? N : 1).scratch_bytes;
+    return EQL_OK;
+}
+
+eql_status_t eqlinear_bwd_weight(eqlinear_plan_t plan, const void* x, const void* dy, void* dw, void* db, int64_t N,
+                                 void* scratch, size_t scratch_bytes, void* stream) {
+    if (!plan) return EQL_ERR_INVALID_ARG;
+    eql_status_t st = check_tokens(N);
+    if (st != EQL_OK) return st;
+    if (!dw) return EQL_ERR_INVALID_ARG;
+    if (!aligned16(dw) || (db && !aligned16(db))) return EQL_ERR_ALIGNMENT;
+    cudaStream_t s = (cudaStream_t)stream;
+    if (N == 0) {
+        if (cudaMemsetAsync(dw, 0, (size_t)plan->Co * plan->Ci * plan->T * sizeof(float), s) != cudaSuccess) return EQL_ERR_CUDA;
+        if (db && cudaMemsetAsync(db, 0, (size_t)plan->Co * sizeof(float), s) != cudaSuccess) return EQL_ERR_CUDA;
+        return EQL_OK;
+    }
+    if (!x || !dy || !scratch) return EQL_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(dy)) return EQL_ERR_ALIGNMENT;
+    if (reinterpret_cast<uintptr_t>(scratch) % kWsAlign != 0) return EQL_ERR_ALIGNMENT;
+    BwdWeightSplit split = direct_bwd_weight_split(plan->T, plan->Ci, plan->Co, N);
+    if (scratch_bytes < split.scratch_bytes) return EQL_ERR_WORKSPACE;
+    cudaError_t e = launch_direct_bwd_weight(plan->T, plan->dtype, (plan->flags & EQL_FLAG_CORRELATION) != 0, x, dy,
+                                             (float*)dw, (float*)db, N, plan->Ci, plan->Co, split, (float*)scratch, s);
+    return e == cudaSuccess ? EQL_OK : EQL_ERR_CUDA;
+}
+
+// ---- host-buffer variants ---------------------------------------------------------------------
+eql_status_t eqlinear_fwd_host(eqlinear_plan_t plan, const void* x_host, void* y_host, int64_t N, void* x_staging,
+                               void* y_staging, void* stream) {
+    if (!plan) return EQL_ERR_INVALID_ARG;
+    eql_status_t st = check_tokens(N);
+    if (st != EQL_OK) return st;
+    if (N == 0) return EQL_OK;
+    if (!x_host || !y_host || !x_staging || !y_staging) return EQL_ERR_INVALID_ARG;
+    cudaStream_t s = (cudaStream_t)stream;
+    const size_t e = elem_size(plan->dtype);
+    const size_t xb = (size_t)N * plan->Ci * plan->T * e, yb = (size_t)N * plan->Co * plan->T * e;
+    if (cudaMemcpyAsync(x_staging, x_host, xb, cudaMemcpyHostToDevice, s) != cudaSuccess) return EQL_ERR_CUDA;
+    st = eqlinear_fwd(plan, x_staging, y_staging, N, stream);
+    if (st != EQL_OK) return st;
+    if (cudaMemcpyAsync(y_host, y_staging, yb, cudaMemcpyDeviceToHost, s) != cudaSuccess) return EQL_ERR_CUDA;
+    return EQL_OK;
+}
+
+eql_status_t eqlinear_bwd_data_host(eqlinear_plan_t plan, const void* dy_host, void* dx_host, int64_t N,
+                                    void* dy_staging, void* dx_staging, void* stream) {
+    if (!plan) return EQL_ERR_INVALID_ARG;
+    eql_status_t st = check_tokens(N);
+    if (st != EQL_OK) return st;
+    if (N == 0) return EQL_OK;
+    if (!dy_host || !dx_host || !dy_staging || !dx_staging) return EQL_ERR_INVALID_ARG;
+    cudaStream_t s = (cudaStream_t)stream;
+    const size_t e = elem_size(plan->dtype);
+    const size_t xb = (size_t)N * plan->Ci * plan->T * e, yb = (size_t)N * plan->Co * plan->T * e;
+    if (cudaMemcpyAsync(dy_staging, dy_host, yb, cudaMemcpyHostToDevice, s) != cudaSuccess) return EQL_ERR_CUDA;
+    st = eqlinear_bwd_data(plan, dy_staging, dx_staging, N, stream);
+    if (st != EQL_OK) return st;
+    if (cudaMemcpyAsync(dx_host, dx_staging, xb, cudaMemcpyDeviceToHost, s) != cudaSuccess) return EQL_ERR_CUDA;
+    return EQL_OK;
+}
+
+eql_status_t eqlinear_bwd_weight_host(eqlinear_plan_t plan, const void* x_host, const void* dy_host, void* dw_host,
+                                      void* db_host, int64_t N, void* x_staging, void* dy_staging, void* dw_staging,
+                                      void* db_staging, void* scratch, size_t scratch_bytes, void* stream) {
+    if (!plan) return EQL_ERR_INVALID_ARG;
+    eql_status_t st = check_tokens(N);
+    if (st != EQL_OK) return st;
+    if (!dw_host || !dw_staging || (db_host && !db_staging)) return EQL_ERR_INVALID_ARG;
+    if (N > 0 && (!x_host || !dy_host || !x_staging || !dy_staging)) return EQL_ERR_INVALID_ARG;
+    cudaStream_t s = (cudaStream_t)stream;
+    const size_t e = elem_size(plan->dtype);
+    const size_t xb = (size_t)N * plan->Ci * plan->T * e, yb = (size_t)N * plan->Co * plan->T * e;
+    if (N > 0) {
+        if (cudaMemcpyAsync(x_staging, x_host, xb, cudaMemcpyHostToDevice, s) != cudaSuccess) return EQL_ERR_CUDA;
+        if (cudaMemcpyAsync(dy_staging, dy_host, yb, cudaMemcpyHostToDevice, s) != cudaSuccess) return EQL_ERR_CUDA;
+    }
+    st = eqlinear_bwd_weight(plan, x_staging, dy_staging, dw_staging, db_host ? db_staging : nullptr, N, scratch,
+                             scratch_bytes, stream);
+    if (st != EQL_OK) return st;
+    if (cudaMemcpyAsync(dw_host, dw_staging, (size_t)plan->Co * plan->Ci * plan->T * sizeof(float),
+                        cudaMemcpyDeviceToHost, s) != cudaSuccess) return EQL_ERR_CUDA;
+    if (db_host && cudaMemcpyAsync(db_host, db_staging, (size_t)plan->Co * sizeof(float), cudaMemcpyDeviceToHost, s) !=
+                       cudaSuccess) return EQL_ERR_CUDA;
+    return EQL_OK;
+}
+
+eql_status_t eqlinear_step_host(eqlinear_plan_t plan, const void* x_host, const void* dy_host, void* y_host,
+                                void* dx_host, void* dw_host, void* db_host, int64_t N, void* x_staging,
+                                void* dy_staging, void* y_staging, void* dx_staging, void* dw_staging,
+                                void* db_staging, void* scratch, size_t scratch_bytes, void* stream) {
+    if (!plan) return EQL_ERR_INVALID_ARG;
+    eql_status_t st = check_tokens(N);
+    if (st != EQL_OK) return st;
+    if (N == 0) return EQL_ERR_INVALID_ARG;
+    if (!x_host || !dy_host || !y_host || !dx_host || !dw_host) return EQL_ERR_INVALID_ARG;
+    if (!x_staging || !dy_staging || !y_staging || !dx_staging || !dw_staging) return EQL_ERR_INVALID_ARG;
+    if ((db_host != nullptr) != (db_staging != nullptr)) return EQL_ERR_INVALID_ARG;
+    cudaStream_t s = (cudaStream_t)stream;
+    const size_t e = elem_size(plan->dtype);
+    const size_t xb = (size_t)N * plan->Ci * plan->T * e, yb = (size_t)N * plan->Co * plan->T * e;
+    if (cudaMemcpyAsync(x_staging, x_host, xb, cudaMemcpyHostToDevice, s) != cudaSuccess) return EQL_ERR_CUDA;
+    if (cudaMemcpyAsync(dy_staging, dy_host, yb, cudaMemcpyHostToDevice, s) != cudaSuccess) return EQL_ERR_CUDA;
+    if ((st = eqlinear_fwd(plan, x_staging, y_staging, N, stream)) != EQL_OK) return st;
+    if (cudaMemcpyAsync(y_host, y_staging, yb, cudaMemcpyDeviceToHost, s) != cudaSuccess) return EQL_ERR_CUDA;
+    if ((st = eqlinear_bwd_data(plan, dy_staging, dx_staging, N, stream)) != EQL_OK) return st;
+    if (cudaMemcpyAsync(dx_host, dx_staging, xb, cudaMemcpyDeviceToHost, s) != cudaSuccess) return EQL_ERR_CUDA;
+    if ((st = eqlinear_bwd_weight(plan, x_staging, dy_staging, dw_staging, db_staging, N, scratch, scratch_bytes,
+                                  stream)) != EQL_OK) return st;
+    if (cudaMemcpyAsync(dw_host, dw_staging, (size_t)plan->Co * plan->Ci * plan->T * sizeof(float),
+                        cudaMemcpyDeviceToHost, s) != cudaSuccess) return EQL_ERR_CUDA;
+    if (db_host && cudaMemcpyAsync(db_host, db_staging, (size_t)plan->Co * sizeof(float), cudaMemcpyDeviceToHost, s) !=
+                       cudaSuccess) return EQL_ERR_CUDA;
+    return EQL_OK;
+}
+
+}  // extern "C"

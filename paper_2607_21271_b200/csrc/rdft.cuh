@@ -1,0 +1,172 @@
+// Real DFT / inverse real DFT of length T in {1, 2, 4, 8, 16, 32} along the group axis, held entirely
+// in registers (Algorithm 1, steps 1 and 4; Eq. 4 and Eq. 7; the T = 4 case reduces to Eq. 19 and Eq. 21).
+//
+// Real-packed plane order used everywhere in the library (T values in, T values out):
+//   plane 0        : k = 0                    (real)
+//   plane 2k-1, 2k : Re, Im of frequency k    for 0 < k < T/2
+//   plane T-1      : k = T/2                  (real; T >= 2)
+//
+// Forward:  X_k = sum_s x_s e^{-2 pi i k s / T}                 (unnormalised, Eq. 4)
+// Inverse:  y_t = P_0 + (-1)^t P_{T-1} + sum_{0<k<T/2} ( P_{2k-1} cos(2 pi k t/T) - P_{2k} sin(2 pi k t/T) )
+//           i.e. the inverse DFT of Eq. 7 / Eq. 15 for planes that were pre-scaled by 1/T (real
+//           frequencies) and 2/T (complex frequencies).  The library folds those scales into the
+//           spectral weight, so the inverse here is adds, subtracts and twiddle products only.
+#pragma once
+
+#include <utility>
+
+#if defined(__CUDACC__)
+#define EQL_HD __host__ __device__ __forceinline__
+#else
+#define EQL_HD inline
+#endif
+
+namespace eql {
+
+// cos(2*pi*j/32), j = 0..8; sin(2*pi*j/32) = cos(2*pi*(8-j)/32).
+template <int J32>
+struct Tw32 {
+    static_assert(J32 >= 0 && J32 <= 8, "twiddle index");
+    static constexpr float value() {
+        constexpr float t[9] = {1.0f,
+                                0.98078528040323044913f,
+                                0.92387953251128675613f,
+                                0.83146961230254523708f,
+                                0.70710678118654752440f,
+                                0.55557023301960222474f,
+                                0.38268343236508977173f,
+                                0.19509032201612826785f,
+                                0.0f};
+        return t[J32];
+    }
+};
+
+template <int N, class F, int... Is>
+EQL_HD void static_for_impl(F&& f, std::integer_sequence<int, Is...>) {
+    (f(std::integral_constant<int, Is>{}), ...);
+}
+// Calls f(integral_constant<int, 0>) ... f(integral_constant<int, N-1>) (compile-time indices).
+template <int N, class F>
+EQL_HD void static_for(F&& f) {
+    static_for_impl<N>(static_cast<F&&>(f), std::make_integer_sequence<int, N>{});
+}
+
+// Half spectrum of a real sequence x[0], x[S], ..., x[(T-1)S]: re[k], im[k] for k = 0..T/2.
+// Radix-2 decimation in time on half spectra: with E, O the half spectra of the even / odd samples,
+//   X_k = E_k + w^k O_k,   X_{T/2-k} = conj(E_k - w^k O_k),   w = e^{-2 pi i / T},  k = 0..T/4.
+template <int T, int S>
+EQL_HD void rfft_half(const float* x, float* re, float* im) {
+    if constexpr (T == 1) {
+        re[0] = x[0]; im[0] = 0.f;
+    } else if constexpr (T == 2) {
+        re[0] = x[0] + x[S]; re[1] = x[0] - x[S];
+        im[0] = 0.f; im[1] = 0.f;
+    } else {
+        constexpr int H = T / 2, Q = T / 4;
+        float er[Q + 1], ei[Q + 1], orr[Q + 1], oi[Q + 1];
+        rfft_half<H, 2 * S>(x, er, ei);
+        rfft_half<H, 2 * S>(x + S, orr, oi);
+        re[0] = er[0] + orr[0]; im[0] = 0.f;
+        re[H] = er[0] - orr[0]; im[H] = 0.f;
+        re[Q] = er[Q]; im[Q] = -orr[Q];                 // w^{T/4} = -i, and E_Q, O_Q are real
+        static_for<(Q > 1 ? Q - 1 : 0)>([&](auto kk) {
+            constexpr int k = decltype(kk)::value + 1;   // 0 < k < T/4
+            constexpr int j = k * (32 / T);
+            float tr, ti;
+            if constexpr (2 * j == 8) {                  // k = T/8: cos = sin
+                constexpr float c = Tw32<4>::value();
+                tr = c * (orr[k] + oi[k]);
+                ti = c * (oi[k] - orr[k]);
+            } else {
+                constexpr float c = Tw32<j>::value();
+                constexpr float s = Tw32<8 - j>::value();
+                tr = c * orr[k] + s * oi[k];             // (c - i s)(Or + i Oi)
+                ti = c * oi[k] - s * orr[k];
+            }
+            re[k] = er[k] + tr;     im[k] = ei[k] + ti;
+            re[H - k] = er[k] - tr; im[H - k] = ti - ei[k];
+        });
+    }
+}
+
+// Forward real DFT, in place: v[0..T) group samples -> v[0..T) real-packed planes.
+template <int T>
+EQL_HD void rdft_forward(float* v) {
+    if constexpr (T == 1) {
+    } else {
+        float re[T / 2 + 1], im[T / 2 + 1];
+        rfft_half<T, 1>(v, re, im);
+        v[0] = re[0];
+        v[T - 1] = re[T / 2];
+        static_for<T / 2 - 1>([&](auto kk) {
+            constexpr int k = decltype(kk)::value + 1;
+            v[2 * k - 1] = re[k];
+            v[2 * k] = im[k];
+        });
+    }
+}
+
+// Inverse on the scaled half spectrum (real frequencies x1, complex frequencies x2, see the header):
+// y[0], y[S], ... y[(T-1)S] from re[k], im[k], k = 0..T/2.  Decimation in time run backwards:
+//   A_k = X_k + conj(X_{T/2-k}) -> even samples,  B_k = (X_k - conj(X_{T/2-k})) w^{-k} -> odd samples.
+template <int T, int S>
+EQL_HD void irfft_half(const float* re, const float* im, float* y) {
+    if constexpr (T == 1) {
+        y[0] = re[0];
+    } else if constexpr (T == 2) {
+        y[0] = re[0] + re[1];
+        y[S] = re[0] - re[1];
+    } else {
+        constexpr int H = T / 2, Q = T / 4;
+        float ar[Q + 1], ai[Q + 1], br[Q + 1], bi[Q + 1];
+        ar[0] = re[0] + re[H]; ai[0] = 0.f;
+        br[0] = re[0] - re[H]; bi[0] = 0.f;
+        ar[Q] = re[Q];  ai[Q] = 0.f;                     // the sub-transforms' k = T/4 planes are real
+        br[Q] = -im[Q]; bi[Q] = 0.f;
+        static_for<(Q > 1 ? Q - 1 : 0)>([&](auto kk) {
+            constexpr int k = decltype(kk)::value + 1;
+            constexpr int j = k * (32 / T);
+            ar[k] = re[k] + re[H - k];
+            ai[k] = im[k] - im[H - k];
+            const float dr = re[k] - re[H - k];
+            const float di = im[k] + im[H - k];
+            if constexpr (2 * j == 8) {
+                constexpr float c = Tw32<4>::value();
+                br[k] = c * (dr - di);
+                bi[k] = c * (di + dr);
+            } else {
+                constexpr float c = Tw32<j>::value();
+                constexpr float s = Tw32<8 - j>::value();
+                br[k] = c * dr - s * di;                 // (dr + i di)(c + i s)
+                bi[k] = c * di + s * dr;
+            }
+        });
+        irfft_half<H, 2 * S>(ar, ai, y);
+        irfft_half<H, 2 * S>(br, bi, y + S);
+    }
+}
+
+// Inverse real DFT, in place: v[0..T) real-packed pre-scaled planes -> v[0..T) group samples.
+template <int T>
+EQL_HD void rdft_inverse(float* v) {
+    if constexpr (T == 1) {
+    } else {
+        float re[T / 2 + 1], im[T / 2 + 1];
+        re[0] = v[0]; im[0] = 0.f;
+        re[T / 2] = v[T - 1]; im[T / 2] = 0.f;
+        static_for<T / 2 - 1>([&](auto kk) {
+            constexpr int k = decltype(kk)::value + 1;
+            re[k] = v[2 * k - 1];
+            im[k] = v[2 * k];
+        });
+        irfft_half<T, 1>(re, im, v);
+    }
+}
+
+// Scale that turns a true (unnormalised) spectrum plane into the pre-scaled plane rdft_inverse expects.
+template <int T>
+EQL_HD float plane_inverse_scale(int plane) {
+    return (plane == 0 || plane == T - 1) ? (1.0f / T) : (2.0f / T);
+}
+
+}  // namespace eql

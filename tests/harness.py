@@ -1,0 +1,121 @@
+"""Shared helpers for the GPU parity tests: run the C-ABI library on a workload and compare with the oracle."""
+
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+import paper_2607_21271_b200 as eq
+from oracle import eqlinear_oracle as orc
+
+TOL = {"fp32": 1e-5, "fp16": 3e-3}          # max|err| / max|ref|, the stated parity bars
+CANARY = 64                                  # guard elements after every output buffer
+
+
+def torch_dtype(dtype: str):
+    return torch.float32 if dtype == "fp32" else torch.float16
+
+
+def eql_dtype(dtype: str) -> int:
+    return eq.EQL_FP32 if dtype == "fp32" else eq.EQL_FP16
+
+
+def rel_max_err(got: np.ndarray, ref: np.ndarray) -> float:
+    scale = float(np.abs(ref).max())
+    err = float(np.abs(got.astype(np.float64) - ref).max())
+    return err / scale if scale > 0 else err
+
+
+class GpuLayer:
+    """One plan plus its buffers, all through the C ABI."""
+
+    def __init__(self, T, Ci, Co, dtype, w, bias, flags=0, device="cuda:0"):
+        self.T, self.Ci, self.Co, self.dtype = T, Ci, Co, dtype
+        self.dev = torch.device(device)
+        self.td = torch_dtype(dtype)
+        self.w = torch.from_numpy(np.ascontiguousarray(w)).to(self.dev)
+        self.bias = None if bias is None else torch.from_numpy(np.ascontiguousarray(bias)).to(self.dev)
+        self.ws_bytes = eq.eqlinear_workspace_bytes(T, Ci, Co, eql_dtype(dtype))
+        self.ws = torch.empty(self.ws_bytes + 256, dtype=torch.uint8, device=self.dev)
+        assert self.ws.data_ptr() % 256 == 0
+        self.stream = torch.cuda.current_stream(self.dev).cuda_stream
+        self.plan = eq.eqlinear_plan(T, Ci, Co, eql_dtype(dtype), self.w, self.bias, self.ws, self.ws_bytes,
+                                     flags, self.stream)
+
+    def close(self):
+        if self.plan:
+            torch.cuda.synchronize(self.dev)
+            eq.eqlinear_plan_destroy(self.plan)
+            self.plan = None
+
+    def _out(self, rows, cols, dtype=None):
+        """Output buffer with a canary tail; returns (flat buffer, view)."""
+        dtype = dtype or self.td
+        n = rows * cols
+        buf = torch.full((n + CANARY,), -77.0, dtype=dtype, device=self.dev)
+        return buf, buf[:n].view(rows, cols) if rows > 0 else buf[:0].view(0, cols)
+
+    @staticmethod
+    def _canary_ok(buf, n):
+        return bool((buf[n:] == -77.0).all().item())
+
+    def fwd(self, x_np):
+        N = x_np.shape[0]
+        x = torch.from_numpy(np.ascontiguousarray(x_np)).to(self.dev)
+        buf, y = self._out(N, self.Co * self.T)
+        eq.eqlinear_fwd(self.plan, x if N else None, buf if N else None, N, self.stream)
+        torch.cuda.synchronize(self.dev)
+        assert self._canary_ok(buf, N * self.Co * self.T), "fwd wrote past its output"
+        return y.cpu().numpy()
+
+    def bwd_data(self, dy_np):
+        N = dy_np.shape[0]
+        dy = torch.from_numpy(np.ascontiguousarray(dy_np)).to(self.dev)
+        buf, dx = self._out(N, self.Ci * self.T)
+        eq.eqlinear_bwd_data(self.plan, dy if N else None, buf if N else None, N, self.stream)
+        torch.cuda.synchronize(self.dev)
+        assert self._canary_ok(buf, N * self.Ci * self.T), "bwd_data wrote past its output"
+        return dx.cpu().numpy()
+
+    def bwd_weight(self, x_np, dy_np, want_db=True):
+        N = x_np.shape[0]
+        x = torch.from_numpy(np.ascontiguousarray(x_np)).to(self.dev)
+        dy = torch.from_numpy(np.ascontiguousarray(dy_np)).to(self.dev)
+        nw = self.Co * self.Ci * self.T
+        wbuf, _ = self._out(1, nw, torch.float32)
+        bbuf, _ = self._out(1, self.Co, torch.float32)
+        sb = eq.eqlinear_bwd_weight_scratch_bytes(self.plan, N)
+        scratch = torch.empty(sb + 256, dtype=torch.uint8, device=self.dev)
+        eq.eqlinear_bwd_weight(self.plan, x if N else None, dy if N else None, wbuf, bbuf if want_db else None, N,
+                               scratch, sb, self.stream)
+        torch.cuda.synchronize(self.dev)
+        assert self._canary_ok(wbuf, nw), "bwd_weight wrote past dw"
+        assert self._canary_ok(bbuf, self.Co), "bwd_weight wrote past db"
+        dw = wbuf[:nw].view(self.Co, self.Ci, self.T).cpu().numpy()
+        db = bbuf[:self.Co].cpu().numpy() if want_db else None
+        return dw, db
+
+
+def check_workload(wl, passes=None, flags=0, data=None):
+    """Runs the named passes on the GPU and returns {tensor: max|err|/max|ref|} against the oracle."""
+    data = data or eq.workloads.generate(wl)
+    passes = passes or wl.passes
+    corr = bool(flags & eq.EQL_FLAG_CORRELATION)
+    layer = GpuLayer(wl.T, wl.Ci, wl.Co, wl.dtype, data["w"], data["bias"], flags)
+    errs = {}
+    try:
+        if "fwd" in passes:
+            y = layer.fwd(data["x"])
+            errs["y"] = rel_max_err(y, orc.fwd(data["x"], data["w"], data["bias"], corr))
+        if "bwd_data" in passes:
+            dx = layer.bwd_data(data["dy"])
+            errs["dx"] = rel_max_err(dx, orc.bwd_data(data["dy"], data["w"], corr))
+        if "bwd_weight" in passes:
+            dw, db = layer.bwd_weight(data["x"], data["dy"])
+            rdw, rdb = orc.bwd_weight(data["x"], data["dy"], wl.T, corr)
+            errs["dw"] = rel_max_err(dw, rdw)
+            errs["db"] = rel_max_err(db, rdb)
+        assert eq.eqlinear_plan_device_status(layer.plan, layer.stream) == eq.binding.EQL_OK
+    finally:
+        layer.close()
+    return errs

@@ -1,0 +1,194 @@
+"""GPU parity: the CUDA library (through its C ABI) against the float64 oracle, element by element.
+
+Bars (max|gpu - ref| / max|ref| over the whole tensor): 1e-5 for FP32, 3e-3 for FP16 I/O with
+float accumulation.
+"""
+
+import numpy as np
+import pytest
+import torch
+
+import paper_2607_21271_b200 as eq
+from oracle import eqlinear_oracle as orc
+from paper_2607_21271_b200.workloads import CONFIGS, Workload, generate
+from tests.harness import TOL, GpuLayer, check_workload, rel_max_err
+
+pytestmark = pytest.mark.gpu
+
+
+# ------------------------------------------------------------------ the five configurations, full size
+@pytest.mark.parametrize("name", list(CONFIGS))
+def test_config_matches_oracle(name):
+    wl = CONFIGS[name]
+    errs = check_workload(wl)
+    print(name, {k: f"{v:.2e}" for k, v in errs.items()})
+    assert set(errs) >= {"y"}
+    for k, v in errs.items():
+        assert v <= TOL[wl.dtype], f"{name}: {k} error {v:.3e} above {TOL[wl.dtype]:.0e}"
+
+
+# ------------------------------------------------------------------ ragged token counts, several tiles
+@pytest.mark.parametrize("dtype", ["fp32", "fp16"])
+@pytest.mark.parametrize("N", [1, 2, 127, 128, 129, 197, 1000])
+def test_ragged_token_counts(dtype, N):
+    wl = Workload(f"ragged{N}", dtype, 8, 24, 40, N, "normal", ("fwd", "bwd_data", "bwd_weight"), 11)
+    for k, v in check_workload(wl).items():
+        assert v <= TOL[dtype], f"N={N} {dtype}: {k} error {v:.3e}"
+
+
+@pytest.mark.parametrize("dtype", ["fp32", "fp16"])
+@pytest.mark.parametrize("T,Ci,Co", [(2, 8, 16), (4, 64, 64), (4, 6, 10), (8, 96, 384), (8, 384, 96),
+                                       (16, 17, 33), (32, 32, 32), (32, 5, 3)])
+def test_shapes(dtype, T, Ci, Co):
+    wl = Workload("shape", dtype, T, Ci, Co, 333, "normal", ("fwd", "bwd_data", "bwd_weight"), 12)
+    for k, v in check_workload(wl).items():
+        assert v <= TOL[dtype], f"T={T} Ci={Ci} Co={Co} {dtype}: {k} error {v:.3e}"
+
+
+@pytest.mark.parametrize("dtype", ["fp32", "fp16"])
+def test_paper_parity_shape(dtype):
+    """The shape of the paper's numerical-equivalence table (Table 4): (B, N, c, T) = (32, 1024, 64, 4)."""
+    wl = Workload("table4", dtype, 4, 64, 64, 32 * 1024, "normal", ("fwd", "bwd_data", "bwd_weight"), 13)
+    for k, v in check_workload(wl).items():
+        assert v <= TOL[dtype], f"{k} error {v:.3e}"
+
+
+@pytest.mark.parametrize("dtype", ["fp32", "fp16"])
+def test_correlation_flag_and_no_bias(dtype):
+    wl = Workload("corr", dtype, 8, 16, 24, 300, "none", ("fwd", "bwd_data", "bwd_weight"), 14)
+    for k, v in check_workload(wl, flags=eq.EQL_FLAG_CORRELATION).items():
+        assert v <= TOL[dtype], f"{k} error {v:.3e}"
+
+
+# ------------------------------------------------------------------ plan life cycle
+def test_empty_batch_and_repeated_calls_and_set_weight():
+    wl = Workload("life", "fp32", 4, 8, 12, 200, "normal", ("fwd",), 15)
+    d = generate(wl)
+    layer = GpuLayer(wl.T, wl.Ci, wl.Co, wl.dtype, d["w"], d["bias"])
+    try:
+        # N = 0 is a no-op / zero gradients
+        assert layer.fwd(d["x"][:0]).shape == (0, wl.Co * wl.T)
+        dw0, db0 = layer.bwd_weight(d["x"][:0], d["dy"][:0])
+        assert not dw0.any() and not db0.any()
+        ref = orc.fwd(d["x"], d["w"], d["bias"])
+        y1, y2 = layer.fwd(d["x"]), layer.fwd(d["x"])
+        assert np.array_equal(y1, y2)
+        assert rel_max_err(y1, ref) <= TOL["fp32"]
+        # new parameter values through set_weight
+        w2 = (d["w"] * 0.5 + 0.25).astype(np.float32)
+        b2 = (d["bias"] - 1.0).astype(np.float32)
+        w2_t, b2_t = torch.from_numpy(w2).cuda(), torch.from_numpy(b2).cuda()
+        eq.eqlinear_plan_set_weight(layer.plan, w2_t, b2_t, layer.stream)
+        assert rel_max_err(layer.fwd(d["x"]), orc.fwd(d["x"], w2, b2)) <= TOL["fp32"]
+        assert rel_max_err(layer.bwd_data(d["dy"]), orc.bwd_data(d["dy"], w2)) <= TOL["fp32"]
+        # weight gradient is bit-reproducible (fixed reduction order)
+        a, _ = layer.bwd_weight(d["x"], d["dy"])
+        b, _ = layer.bwd_weight(d["x"], d["dy"])
+        assert np.array_equal(a, b)
+        # db may be omitted
+        dw, db = layer.bwd_weight(d["x"], d["dy"], want_db=False)
+        assert db is None and np.array_equal(dw, a)
+    finally:
+        layer.close()
+
+
+def test_two_plans_interleaved_on_one_stream():
+    wa = Workload("a", "fp16", 4, 24, 96, 500, "normal", ("fwd",), 16)
+    wb = Workload("b", "fp32", 8, 48, 48, 300, "normal", ("fwd",), 17)
+    da, db_ = generate(wa), generate(wb)
+    la = GpuLayer(wa.T, wa.Ci, wa.Co, wa.dtype, da["w"], da["bias"])
+    lb = GpuLayer(wb.T, wb.Ci, wb.Co, wb.dtype, db_["w"], db_["bias"])
+    try:
+        ya1 = la.fwd(da["x"]); yb1 = lb.fwd(db_["x"]); ya2 = la.fwd(da["x"])
+        assert np.array_equal(ya1, ya2)
+        assert rel_max_err(ya1, orc.fwd(da["x"], da["w"], da["bias"])) <= TOL["fp16"]
+        assert rel_max_err(yb1, orc.fwd(db_["x"], db_["w"], db_["bias"])) <= TOL["fp32"]
+    finally:
+        la.close(); lb.close()
+
+
+def test_runtime_argument_errors():
+    wl = Workload("err", "fp32", 4, 8, 8, 16, "none", ("fwd",), 18)
+    d = generate(wl)
+    layer = GpuLayer(wl.T, wl.Ci, wl.Co, wl.dtype, d["w"], None)
+    lib = eq.load_library()
+    B = eq.binding
+    try:
+        x = torch.zeros(16 * 32 + 4, dtype=torch.float32, device="cuda")
+        y = torch.zeros(16 * 32 + 4, dtype=torch.float32, device="cuda")
+        p = layer.plan
+        assert lib.eqlinear_fwd(p, x.data_ptr(), y.data_ptr(), -1, None) == B.EQL_ERR_INVALID_ARG
+        assert lib.eqlinear_fwd(p, None, y.data_ptr(), 4, None) == B.EQL_ERR_INVALID_ARG
+        assert lib.eqlinear_fwd(p, x.data_ptr(), x.data_ptr(), 4, None) == B.EQL_ERR_INVALID_ARG
+        assert lib.eqlinear_fwd(p, x.data_ptr() + 4, y.data_ptr(), 4, None) == B.EQL_ERR_ALIGNMENT
+        assert lib.eqlinear_bwd_data(p, x.data_ptr(), y.data_ptr() + 8, 4, None) == B.EQL_ERR_ALIGNMENT
+        dw = torch.zeros(8 * 8 * 4, dtype=torch.float32, device="cuda")
+        sc = torch.zeros(1 << 16, dtype=torch.uint8, device="cuda")
+        assert lib.eqlinear_bwd_weight(p, x.data_ptr(), y.data_ptr(), dw.data_ptr(), None, 16, sc.data_ptr(), 8,
+                                       None) == B.EQL_ERR_WORKSPACE
+        assert lib.eqlinear_plan_set_weight(p, layer.w.data_ptr(), layer.w.data_ptr(), None) == B.EQL_ERR_INVALID_ARG
+        info = eq.eqlinear_plan_info(p)
+        assert (info.T, info.C_in, info.C_out) == (4, 8, 8)
+        assert info.macs_per_token == 6 * 8 * 8 and info.dense_macs_per_token == 32 * 32
+        assert info.bytes_per_token_fwd == (8 + 8) * 4 * 4
+    finally:
+        layer.close()
+
+
+# ------------------------------------------------------------------ invariants on the GPU output alone
+@pytest.mark.parametrize("dtype,T", [("fp32", 4), ("fp32", 8), ("fp16", 16)])
+def test_gpu_equivariance_and_adjoint(dtype, T):
+    wl = Workload("inv", dtype, T, 16, 24, 512, "normal", ("fwd", "bwd_data", "bwd_weight"), 19)
+    d = generate(wl)
+    layer = GpuLayer(wl.T, wl.Ci, wl.Co, wl.dtype, d["w"], d["bias"])
+    try:
+        y = layer.fwd(d["x"]).astype(np.float64).reshape(wl.N, wl.Co, T)
+        for r in (1, T - 1):
+            xr = np.roll(d["x"].reshape(wl.N, wl.Ci, T), r, axis=-1).reshape(wl.N, wl.Ci * T)
+            yr = layer.fwd(np.ascontiguousarray(xr)).astype(np.float64).reshape(wl.N, wl.Co, T)
+            nmse = ((yr - np.roll(y, r, axis=-1)) ** 2).sum() / (y ** 2).sum()
+            assert nmse <= (1e-12 if dtype == "fp32" else 1e-5), nmse   # paper's Table 5: 4e-8 in FP32
+    finally:
+        layer.close()
+    # adjoint identity <dy, fwd0(x)> = <dx, x> = <dw, w> with the bias-free layer
+    layer = GpuLayer(wl.T, wl.Ci, wl.Co, wl.dtype, d["w"], None)
+    try:
+        f64 = lambda a: a.astype(np.float64)
+        lhs = np.vdot(f64(d["dy"]), f64(layer.fwd(d["x"])))
+        dx = layer.bwd_data(d["dy"])
+        dw, _ = layer.bwd_weight(d["x"], d["dy"])
+        tol = 1e-5 if dtype == "fp32" else 3e-3
+        assert abs(lhs - np.vdot(f64(dx), f64(d["x"]))) <= tol * abs(lhs)
+        assert abs(lhs - np.vdot(f64(dw), f64(d["w"]))) <= tol * abs(lhs)
+    finally:
+        layer.close()
+
+
+# ------------------------------------------------------------------ host-buffer variants
+def test_host_buffer_variants():
+    wl = Workload("host", "fp16", 8, 24, 40, 700, "normal", ("fwd", "bwd_data", "bwd_weight"), 20)
+    d = generate(wl)
+    layer = GpuLayer(wl.T, wl.Ci, wl.Co, wl.dtype, d["w"], d["bias"])
+    try:
+        N = wl.N
+        xh = torch.from_numpy(d["x"]).pin_memory(); dyh = torch.from_numpy(d["dy"]).pin_memory()
+        yh = torch.empty(N, wl.Dout, dtype=torch.float16).pin_memory()
+        dxh = torch.empty(N, wl.Din, dtype=torch.float16).pin_memory()
+        dwh = torch.empty(wl.Co, wl.Ci, wl.T, dtype=torch.float32).pin_memory()
+        dbh = torch.empty(wl.Co, dtype=torch.float32).pin_memory()
+        xs = torch.empty(N, wl.Din, dtype=torch.float16, device="cuda"); dys = torch.empty(N, wl.Dout, dtype=torch.float16, device="cuda")
+        ys = torch.empty_like(dys); dxs = torch.empty_like(xs)
+        dws = torch.empty(wl.Co, wl.Ci, wl.T, dtype=torch.float32, device="cuda"); dbs = torch.empty(wl.Co, dtype=torch.float32, device="cuda")
+        sb = eq.eqlinear_bwd_weight_scratch_bytes(layer.plan, N)
+        sc = torch.empty(sb, dtype=torch.uint8, device="cuda")
+        eq.eqlinear_fwd_host(layer.plan, xh, yh, N, xs, ys, layer.stream)
+        eq.eqlinear_bwd_data_host(layer.plan, dyh, dxh, N, dys, dxs, layer.stream)
+        eq.eqlinear_bwd_weight_host(layer.plan, xh, dyh, dwh, dbh, N, xs, dys, dws, dbs, sc, sb, layer.stream)
+        torch.cuda.synchronize()
+        assert rel_max_err(yh.numpy(), orc.fwd(d["x"], d["w"], d["bias"])) <= TOL["fp16"]
+        assert rel_max_err(dxh.numpy(), orc.bwd_data(d["dy"], d["w"])) <= TOL["fp16"]
+        rdw, rdb = orc.bwd_weight(d["x"], d["dy"], wl.T)
+        assert rel_max_err(dwh.numpy(), rdw) <= TOL["fp16"]
+        assert rel_max_err(dbh.numpy(), rdb) <= TOL["fp16"]
+    finally:
+        layer.close()
