@@ -54,3 +54,15 @@ cudaError_t launch_direct_bwd_weight(int T, eql_dtype_t dtype, bool correlation,
                                      const BwdWeightSplit& split, float* scratch, cudaStream_t stream);
 
 }  // namespace eql
+
+// The host object behind eqlinear_plan_t.
+struct eqlinear_plan_s {
+    int T, Ci, Co;
+    eql_dtype_t dtype;
+    unsigned flags;
+    bool has_bias;
+    int device;
+    char* ws;                       // caller-owned device workspace
+    eql::WorkspaceLayout lay;
+    int fwd_kernel, bwd_data_kernel, bwd_weight_kernel;
+};

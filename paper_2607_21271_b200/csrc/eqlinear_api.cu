@@ -6,17 +6,6 @@
 
 #include "eql_internal.h"
 
-struct eqlinear_plan_s {
-    int T, Ci, Co;
-    eql_dtype_t dtype;
-    unsigned flags;
-    bool has_bias;
-    int device;
-    char* ws;
-    eql::WorkspaceLayout lay;
-    int fwd_kernel, bwd_data_kernel, bwd_weight_kernel;
-};
-
 namespace eql {
 
 WorkspaceLayout workspace_layout(int T, int Ci, int Co, eql_dtype_t dtype) {
