@@ -153,6 +153,34 @@ eql_status_t eqlinear_bwd_weight(eqlinear_plan_t plan, const void* x, const void
                                  void* dw, void* db, int64_t N,
                                  void* scratch, size_t scratch_bytes, void* stream);
 
+/* Size of the scratch array that is built into the library for eqlinear_bwd_weight_static. */
+#define EQL_STATIC_SCRATCH_BYTES (32u << 20)
+
+/* eqlinear_bwd_weight without a scratch argument.  (The paper has no counterpart: this entry point
+ * exists for the library's users, not for the method.)
+ *
+ * Who it is for: code that must compute the weight gradient at a point where it cannot obtain
+ * device memory -- a plug-in running inside a host application that owns the allocator and gives
+ * the plug-in none, a service whose memory pool has already claimed the whole GPU so that a fresh
+ * cudaMalloc would fail, or a latency-critical loop that may not risk the device-wide stall an
+ * allocation can cause.  Such callers still pass their inputs and outputs (x, dy, dw, db, as for
+ * eqlinear_bwd_weight); only the scratch for the per-split partial spectra comes from the library,
+ * from a fixed device array of EQL_STATIC_SCRATCH_BYTES (32 MiB) that every GPU which loads the
+ * library holds until the process exits.  This call allocates nothing and frees nothing.
+ *
+ *   - Returns EQL_ERR_WORKSPACE, and launches nothing, when eqlinear_bwd_weight_scratch_bytes(plan, N)
+ *     is larger than EQL_STATIC_SCRATCH_BYTES; use eqlinear_bwd_weight with your own buffer then.
+ *   - The first call on each device looks up the array's device address (the plan's device must be
+ *     the current device; EQL_ERR_INVALID_ARG otherwise).  Make that first call before any stream
+ *     capture begins.
+ *   - All calls, from every plan and stream, share the one array, and it keeps whatever the last
+ *     call left in it.  Nothing in it has to start at zero: each call overwrites every partial it
+ *     later reads.  Two calls that overlap in time on the GPU race on it; order them on one stream
+ *     (or with events).
+ *   - Results are identical to eqlinear_bwd_weight's for the same plan and N. */
+eql_status_t eqlinear_bwd_weight_static(eqlinear_plan_t plan, const void* x, const void* dy,
+                                        void* dw, void* db, int64_t N, void* stream);
+
 /* ---- host-buffer variants (end-to-end measurement, small-batch convenience) ------------------ */
 /* Same operations with HOST input/output buffers (pinned memory recommended).  Each call copies
  * its inputs into the caller's device staging buffers on `stream`, runs the kernels above and

@@ -29,12 +29,14 @@ EQL_FP16 = 1
 EQL_FLAG_CORRELATION = 1
 EQL_FLAG_FORCE_SIMT = 2
 
+EQL_STATIC_SCRATCH_BYTES = 32 << 20
+
 # Every symbol include/eqlinear.h declares.
 EXPORTED_SYMBOLS = (
     "eqlinear_status_string", "eqlinear_count_macs", "eqlinear_workspace_bytes", "eqlinear_plan",
     "eqlinear_plan_set_weight", "eqlinear_plan_info", "eqlinear_plan_device_status", "eqlinear_plan_destroy",
     "eqlinear_fwd", "eqlinear_bwd_data", "eqlinear_bwd_weight_scratch_bytes", "eqlinear_bwd_weight",
-    "eqlinear_fwd_host", "eqlinear_bwd_data_host", "eqlinear_bwd_weight_host", "eqlinear_step_host",
+    "eqlinear_fwd_host", "eqlinear_bwd_data_host", "eqlinear_bwd_weight_host", "eqlinear_step_host", "eqlinear_bwd_weight_static",
 )
 
 
@@ -88,6 +90,7 @@ def load_library(path: str | None = None) -> ctypes.CDLL:
         "eqlinear_fwd_host": [V, V, V, I64, V, V, V],
         "eqlinear_bwd_data_host": [V, V, V, I64, V, V, V],
         "eqlinear_bwd_weight_host": [V, V, V, V, V, I64, V, V, V, V, V, SZ, V],
+        "eqlinear_bwd_weight_static": [V, V, V, V, V, I64, V],
         "eqlinear_step_host": [V, V, V, V, V, V, V, I64, V, V, V, V, V, V, V, SZ, V],
     }
     for name, argtypes in sigs.items():
@@ -202,3 +205,10 @@ def eqlinear_step_host(plan, x_host, dy_host, y_host, dx_host, dw_host, db_host,
                                              _ptr(dw_host), _ptr(db_host), N, _ptr(x_staging), _ptr(dy_staging),
                                              _ptr(y_staging), _ptr(dx_staging), _ptr(dw_staging), _ptr(db_staging),
                                              _ptr(scratch), scratch_bytes, stream or None), "eqlinear_step_host")
+
+
+def eqlinear_bwd_weight_static(plan, x, dy, dw, db, N, stream=0) -> None:
+    """eqlinear_bwd_weight for callers that cannot allocate device scratch: the library's built-in
+    32 MiB device array is used instead (shared by all calls; do not overlap two of them)."""
+    _check(load_library().eqlinear_bwd_weight_static(plan, _ptr(x), _ptr(dy), _ptr(dw), _ptr(db), N, stream or None),
+           "eqlinear_bwd_weight_static")
