@@ -53,6 +53,23 @@ cudaError_t launch_direct_bwd_weight(int T, eql_dtype_t dtype, bool correlation,
                                      float* dw, float* db, int64_t N, int Ci, int Co,
                                      const BwdWeightSplit& split, float* scratch, cudaStream_t stream);
 
+// ---- tcgen05 tensor-core kernels (FP16 I/O), umma_linear.cu ----------------------------------------
+struct UmmaLinearShape {
+    int T, Cin, Cout;
+    int CoT;            // output channels per tile: multiple of 16, T*CoT <= 512 TMEM columns
+    int nTiles;         // output-channel tiles
+    int nK;             // 16-channel chunks of the reduction dimension
+    int rowsB;          // (2T-2)*CoT rows of the weight image per (tile, chunk)
+    size_t image_bytes;
+};
+bool umma_linear_supported(int T, eql_dtype_t dtype);
+UmmaLinearShape umma_linear_shape(int T, int Cin, int Cout);
+// planes[T][Cin][Cout] (float) -> operand image for umma_linear_kernel.
+cudaError_t launch_build_umma_image(const UmmaLinearShape& s, const float* planes, void* image, cudaStream_t stream);
+// out[N, Cout*T] = IDFT( DFT(in[N, Cin*T]) (x) image ) + bias, fp16 I/O, tcgen05 MMA with FP32 accumulation in TMEM.
+cudaError_t launch_umma_linear(const UmmaLinearShape& s, const void* in, void* out, int64_t N, const void* image,
+                               const float* bias_f32, int* status, int num_sms, cudaStream_t stream);
+
 }  // namespace eql
 
 // The host object behind eqlinear_plan_t.
@@ -65,4 +82,6 @@ struct eqlinear_plan_s {
     char* ws;                       // caller-owned device workspace
     eql::WorkspaceLayout lay;
     int fwd_kernel, bwd_data_kernel, bwd_weight_kernel;
+    int num_sms;
+    eql::UmmaLinearShape umma_fwd, umma_bwd;
 };

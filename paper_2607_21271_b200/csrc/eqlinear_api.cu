@@ -17,7 +17,12 @@ WorkspaceLayout workspace_layout(int T, int Ci, int Co, eql_dtype_t dtype) {
     l.planes_bwd = off;  off += align_up((size_t)T * Ci * Co * sizeof(float), kWsAlign);
     l.umma_fwd = off;    l.umma_fwd_bytes = 0;
     l.umma_bwd = off;    l.umma_bwd_bytes = 0;
-    (void)dtype;
+    if (umma_linear_supported(T, dtype)) {
+        l.umma_fwd_bytes = umma_linear_shape(T, Ci, Co).image_bytes;
+        l.umma_bwd_bytes = umma_linear_shape(T, Co, Ci).image_bytes;
+        l.umma_fwd = off;  off += l.umma_fwd_bytes;
+        l.umma_bwd = off;  off += l.umma_bwd_bytes;
+    }
     l.total = off;
     return l;
 }
@@ -51,7 +56,16 @@ eql_status_t build_weights(eqlinear_plan_t p, const void* w, const void* bias, c
     cudaError_t e = launch_plan_weights(p->T, p->dtype, (p->flags & EQL_FLAG_CORRELATION) != 0, w, bias, p->Ci, p->Co,
                                         (float*)(p->ws + p->lay.planes_fwd), (float*)(p->ws + p->lay.planes_bwd),
                                         (float*)(p->ws + p->lay.bias), s);
-    return e == cudaSuccess ? EQL_OK : EQL_ERR_CUDA;
+    if (e != cudaSuccess) return EQL_ERR_CUDA;
+    if (p->fwd_kernel == 1) {
+        e = launch_build_umma_image(p->umma_fwd, (const float*)(p->ws + p->lay.planes_fwd), p->ws + p->lay.umma_fwd, s);
+        if (e != cudaSuccess) return EQL_ERR_CUDA;
+    }
+    if (p->bwd_data_kernel == 1) {
+        e = launch_build_umma_image(p->umma_bwd, (const float*)(p->ws + p->lay.planes_bwd), p->ws + p->lay.umma_bwd, s);
+        if (e != cudaSuccess) return EQL_ERR_CUDA;
+    }
+    return EQL_OK;
 }
 
 }  // namespace
@@ -113,6 +127,13 @@ eql_status_t eqlinear_plan(eqlinear_plan_t* plan, int T, int C_in, int C_out, eq
     p->T = T; p->Ci = C_in; p->Co = C_out; p->dtype = dtype; p->flags = flags;
     p->has_bias = bias != nullptr; p->device = dev; p->ws = (char*)workspace; p->lay = lay;
     p->fwd_kernel = p->bwd_data_kernel = p->bwd_weight_kernel = 0;
+    p->num_sms = kNumSMs;
+    if (cudaDeviceGetAttribute(&p->num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) { delete p; return EQL_ERR_CUDA; }
+    if (umma_linear_supported(T, dtype) && !(flags & EQL_FLAG_FORCE_SIMT)) {
+        p->fwd_kernel = p->bwd_data_kernel = 1;
+        p->umma_fwd = umma_linear_shape(T, C_in, C_out);
+        p->umma_bwd = umma_linear_shape(T, C_out, C_in);
+    }
 
     cudaStream_t s = (cudaStream_t)stream;
     if (cudaMemsetAsync(p->ws + lay.status, 0, kWsAlign, s) != cudaSuccess) { delete p; return EQL_ERR_CUDA; }
@@ -168,6 +189,11 @@ eql_status_t eqlinear_fwd(eqlinear_plan_t plan, const void* x, void* y, int64_t 
     if (!x || !y || x == y) return EQL_ERR_INVALID_ARG;
     if (!aligned16(x) || !aligned16(y)) return EQL_ERR_ALIGNMENT;
     const float* bias = plan->has_bias ? (const float*)(plan->ws + plan->lay.bias) : nullptr;
+    if (plan->fwd_kernel == 1) {
+        cudaError_t e = launch_umma_linear(plan->umma_fwd, x, y, N, plan->ws + plan->lay.umma_fwd, bias,
+                                           (int*)(plan->ws + plan->lay.status), plan->num_sms, (cudaStream_t)stream);
+        return e == cudaSuccess ? EQL_OK : EQL_ERR_CUDA;
+    }
     cudaError_t e = launch_direct_linear(plan->T, plan->dtype, x, y, N, plan->Ci, plan->Co,
                                          (const float*)(plan->ws + plan->lay.planes_fwd), bias, (cudaStream_t)stream);
     return e == cudaSuccess ? EQL_OK : EQL_ERR_CUDA;
@@ -180,6 +206,11 @@ eql_status_t eqlinear_bwd_data(eqlinear_plan_t plan, const void* dy, void* dx, i
     if (N == 0) return EQL_OK;
     if (!dy || !dx || dy == dx) return EQL_ERR_INVALID_ARG;
     if (!aligned16(dy) || !aligned16(dx)) return EQL_ERR_ALIGNMENT;
+    if (plan->bwd_data_kernel == 1) {
+        cudaError_t e = launch_umma_linear(plan->umma_bwd, dy, dx, N, plan->ws + plan->lay.umma_bwd, nullptr,
+                                           (int*)(plan->ws + plan->lay.status), plan->num_sms, (cudaStream_t)stream);
+        return e == cudaSuccess ? EQL_OK : EQL_ERR_CUDA;
+    }
     cudaError_t e = launch_direct_linear(plan->T, plan->dtype, dy, dx, N, plan->Co, plan->Ci,
                                          (const float*)(plan->ws + plan->lay.planes_bwd), nullptr, (cudaStream_t)stream);
     return e == cudaSuccess ? EQL_OK : EQL_ERR_CUDA;

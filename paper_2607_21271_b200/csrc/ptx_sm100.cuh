@@ -40,13 +40,14 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 
 // Bounded wait.  Returns false if the barrier did not flip within the poll budget or if another
 // thread of the CTA has already given up (abort flag); on its own time-out it raises the flag and
-// records `code` in the global status word.  Nothing here traps or spins forever.
-constexpr uint32_t kWaitPolls = 1u << 22;
+// records `code` in the global status word.  With heed_abort = false (used while draining copies and
+// MMAs that are already in flight) only the poll budget ends the wait.  Nothing here traps or spins forever.
+constexpr uint32_t kWaitPolls = 1u << 20;
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status,
-                                          int code) {
+                                          int code, bool heed_abort = true) {
     for (uint32_t it = 0; it < kWaitPolls; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
-        if ((it & 63u) == 63u && *abort_flag != 0) return false;
+        if (heed_abort && (it & 63u) == 63u && *abort_flag != 0) return false;
     }
     *abort_flag = 1;
     atomicCAS(status, 0, code);

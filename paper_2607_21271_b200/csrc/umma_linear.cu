@@ -1,0 +1,504 @@
+// Fused EQ-Linear forward / data-gradient on the 5th-generation tensor cores (tcgen05 + TMEM), FP16 I/O,
+// FP32 accumulation.  One persistent CTA per SM; a work unit is (128-token tile, output-channel tile).
+//
+//   TMA (2-D, 128B swizzle)      raw rows of x            -> shared "slabs" [128 rows x 128 B]
+//   8 transform warps            group DFT (Eq. 4) in registers, planes rounded to fp16 once
+//                                -> shared A operands, one [128 x 16] K-major tile per real-packed plane
+//   TMA (1-D bulk)               spectral-weight image of this (tile, 16-channel chunk) -> shared B operands
+//   1 thread                     tcgen05.mma kind::f16: one product per real frequency, and the complex
+//                                product of Eq. 5 as the real 2x2 block [Xr|Xi] x [[Wr,Wi],[-Wi,Wr]] -> TMEM
+//   4 epilogue warps             tcgen05.ld, bias on plane k = 0, inverse DFT (Eq. 7) in registers,
+//                                fp16 rounding, group tuples stored contiguously to global memory
+//
+// Frequency-domain data never leaves the SM (registers, shared memory, TMEM).  The data gradient is the
+// same kernel run on dy with the conjugate-transposed weight image and no bias.
+//
+// Every wait on an mbarrier is bounded: on a time-out the CTA raises an abort flag, records a status
+// code for the host, drains its outstanding copies and MMAs, frees its TMEM and returns.
+#include <cuda_fp16.h>
+
+#include <cstring>
+#include <mutex>
+
+#include "eql_internal.h"
+#include "ptx_sm100.cuh"
+#include "rdft.cuh"
+
+namespace eql {
+namespace {
+
+constexpr int kTileM = 128;            // tokens per tile = UMMA M = TMEM lanes
+constexpr int kChunkK = 16;            // input channels per pipeline stage = one UMMA K step for f16
+constexpr int kSlabBytes = kTileM * 128;
+constexpr int kThreadsUmma = 512;
+constexpr int kTmemCols = 512;
+
+// warp roles
+constexpr int kWarpTmaX = 0, kWarpMma = 1, kWarpTmaB = 2, kWarpEpi0 = 4, kWarpDft0 = 8;
+
+template <int T> struct UmmaCfg;
+template <> struct UmmaCfg<4>  { static constexpr int SR = 4, SA = 4, SB = 3; };
+template <> struct UmmaCfg<8>  { static constexpr int SR = 4, SA = 3, SB = 2; };
+template <> struct UmmaCfg<16> { static constexpr int SR = 2, SA = 2, SB = 2; };
+template <> struct UmmaCfg<32> { static constexpr int SR = 4, SA = 1, SB = 1; };
+
+struct UmmaParams {
+    __half* out;                 // [N, Cout*T]
+    const __half* image;         // spectral-weight operand image, see build_image_kernel
+    const float* bias;           // [Cout] or nullptr
+    int* status;                 // device status word of the plan
+    int64_t N;
+    int Cin, Cout;
+    int CoT, nTiles, nK, rowsB;
+    int b_slot_bytes;            // bytes of one B ring slot (rowsB*32 rounded up to 128)
+    int64_t num_units;
+};
+
+__device__ __forceinline__ float2 unpack_h2(uint32_t u) {
+    __half2 h;
+    memcpy(&h, &u, 4);
+    return __half22float2(h);
+}
+__device__ __forceinline__ uint32_t pack_h2(float lo, float hi) {
+    __half2 h = __floats2half2_rn(lo, hi);
+    uint32_t u;
+    memcpy(&u, &h, 4);
+    return u;
+}
+
+struct SmemBarriers {
+    uint64_t full_raw[4], empty_raw[4];
+    uint64_t full_a[4], empty_a[4];
+    uint64_t full_b[4], empty_b[4];
+    uint64_t full_d, empty_d, mma_done;
+    uint32_t tmem_base;
+    int abort_flag;
+};
+
+// ------------------------------------------------------------------------------------------------
+// Operand image of the spectral weight for the tensor-core kernel.
+// planes[p][cin][cout] (float, already scaled by 1/T resp. 2/T, conjugated for the data gradient) ->
+// for every (output tile, 16-channel chunk) one blob of rowsB rows x 16 k in the no-swizzle K-major
+// core-matrix layout [k half][row][8 k]: element (row n, k) at ((k/8)*rowsB + n)*8 + k%8 halves.
+// Rows of a blob (CoT = output channels per tile):
+//   [0, CoT)                         plane 0 (k = 0)
+//   per complex frequency f (4*CoT): Wr | Wi   (multiplied by Re x^)   then   -Wi | Wr   (by Im x^)
+//   [rowsB - CoT, rowsB)             plane T-1 (k = T/2)
+template <int T>
+__global__ void build_image_kernel(const float* __restrict__ planes, int Cin, int Cout, int CoT, int nTiles, int nK,
+                                   int rowsB, __half* __restrict__ image) {
+    const int64_t total = (int64_t)nTiles * nK * rowsB * kChunkK;
+    for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
+         idx += (int64_t)gridDim.x * blockDim.x) {
+        const int within = (int)(idx % ((int64_t)rowsB * kChunkK));
+        const int64_t blob = idx / ((int64_t)rowsB * kChunkK);
+        const int kc = (int)(blob % nK), tile = (int)(blob / nK);
+        const int khalf = within / (rowsB * 8);
+        const int n = (within / 8) % rowsB;
+        const int kk = khalf * 8 + (within & 7);
+        int plane, local;
+        float sign = 1.f;
+        if (n < CoT) {
+            plane = 0; local = n;
+        } else if (n >= rowsB - CoT) {
+            plane = T - 1; local = n - (rowsB - CoT);
+        } else {
+            const int m = n - CoT, f = m / (4 * CoT) + 1, part = (m / CoT) & 3;
+            local = m % CoT;
+            if (part == 0) plane = 2 * f - 1;                     // Wr  -> Re y^
+            else if (part == 1) plane = 2 * f;                    // Wi  -> Im y^
+            else if (part == 2) { plane = 2 * f; sign = -1.f; }   // -Wi -> Re y^
+            else plane = 2 * f - 1;                               // Wr  -> Im y^
+        }
+        const int cin = kc * kChunkK + kk, cout = tile * CoT + local;
+        float v = 0.f;
+        if (cin < Cin && cout < Cout) v = sign * planes[((size_t)plane * Cin + cin) * Cout + cout];
+        image[idx] = __float2half_rn(v);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+template <int T>
+__global__ void __launch_bounds__(kThreadsUmma, 1)
+umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const UmmaParams prm) {
+    using Cfg = UmmaCfg<T>;
+    constexpr int SR = Cfg::SR, SA = Cfg::SA, SB = Cfg::SB;
+    constexpr int NCH = 64 / T;                 // channels per raw slab row (128 B)
+    constexpr int SPK = kChunkK / NCH;          // slabs per 16-channel chunk (= T/4)
+    constexpr int kAStage = T * 4096;           // T planes x [128 x 16] halves
+
+    extern __shared__ uint8_t smem_raw_base[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw_base) + 1023) & ~(uintptr_t)1023);
+    uint8_t* raw = smem;                                   // SR slabs
+    uint8_t* xhat = raw + SR * kSlabBytes;                 // SA stages
+    uint8_t* bsm = xhat + SA * kAStage;                    // SB slots
+    SmemBarriers* bar = reinterpret_cast<SmemBarriers*>(bsm + SB * prm.b_slot_bytes);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    volatile int* abort_flag = &bar->abort_flag;
+    int* status = prm.status;
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < SR; ++i) { ptx::mbar_init(&bar->full_raw[i], 1); ptx::mbar_init(&bar->empty_raw[i], 4); }
+        for (int i = 0; i < SA; ++i) { ptx::mbar_init(&bar->full_a[i], 4 * SPK); ptx::mbar_init(&bar->empty_a[i], 1); }
+        for (int i = 0; i < SB; ++i) { ptx::mbar_init(&bar->full_b[i], 1); ptx::mbar_init(&bar->empty_b[i], 1); }
+        ptx::mbar_init(&bar->full_d, 1);
+        ptx::mbar_init(&bar->empty_d, 4);
+        ptx::mbar_init(&bar->mma_done, 1);
+        bar->abort_flag = 0;
+        ptx::fence_mbar_init();
+        ptx::prefetch_tensormap(&tmap_in);
+    }
+    if (warp == kWarpMma) {
+        ptx::tmem_alloc(&bar->tmem_base, kTmemCols);
+        ptx::tmem_relinquish();
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::tc_fence_after_sync();
+    const uint32_t tmem_base = bar->tmem_base;
+
+    const int nK = prm.nK, nTiles = prm.nTiles, CoT = prm.CoT, rowsB = prm.rowsB;
+    const int64_t first = blockIdx.x, stride = gridDim.x;
+
+    if (warp == kWarpTmaX) {
+        // ---------------------------------------------------------------- raw activation rows via TMA
+        if (lane == 0) {
+            uint32_t cr = 0;
+            bool ok = true;
+            for (int64_t u = first; u < prm.num_units && ok; u += stride) {
+                const int row0 = (int)(u / nTiles) * kTileM;
+                for (int kc = 0; kc < nK && ok; ++kc) {
+                    for (int q = 0; q < SPK; ++q, ++cr) {
+                        const int slot = cr % SR;
+                        ok = ptx::mbar_wait(&bar->empty_raw[slot], ((cr / SR) & 1) ^ 1, abort_flag, status, 101);
+                        if (!ok) break;
+                        ptx::mbar_arrive_expect_tx(&bar->full_raw[slot], kSlabBytes);
+                        ptx::tma_load_2d(raw + slot * kSlabBytes, &tmap_in, (kc * kChunkK + q * NCH) * T, row0,
+                                         &bar->full_raw[slot]);
+                    }
+                }
+            }
+            if (!ok) {   // drain: every copy this thread issued must have landed before the CTA may exit
+                const uint32_t lo = cr > (uint32_t)SR ? cr - SR : 0;
+                for (uint32_t c = lo; c < cr; ++c)
+                    ptx::mbar_wait(&bar->full_raw[c % SR], (c / SR) & 1, abort_flag, status, 111, false);
+            }
+        }
+    } else if (warp == kWarpTmaB) {
+        // ---------------------------------------------------------------- spectral-weight blobs via bulk copy
+        if (lane == 0) {
+            uint32_t cb = 0;
+            bool ok = true;
+            const uint32_t blob_bytes = (uint32_t)rowsB * 32u;
+            for (int64_t u = first; u < prm.num_units && ok; u += stride) {
+                const int tile = (int)(u % nTiles);
+                for (int kc = 0; kc < nK; ++kc, ++cb) {
+                    const int slot = cb % SB;
+                    ok = ptx::mbar_wait(&bar->empty_b[slot], ((cb / SB) & 1) ^ 1, abort_flag, status, 102);
+                    if (!ok) break;
+                    ptx::mbar_arrive_expect_tx(&bar->full_b[slot], blob_bytes);
+                    ptx::bulk_load_1d(bsm + slot * prm.b_slot_bytes,
+                                      prm.image + ((size_t)tile * nK + kc) * (size_t)rowsB * kChunkK, blob_bytes,
+                                      &bar->full_b[slot]);
+                }
+            }
+            if (!ok) {
+                const uint32_t lo = cb > (uint32_t)SB ? cb - SB : 0;
+                for (uint32_t c = lo; c < cb; ++c)
+                    ptx::mbar_wait(&bar->full_b[c % SB], (c / SB) & 1, abort_flag, status, 112, false);
+            }
+        }
+    } else if (warp == kWarpMma) {
+        // ---------------------------------------------------------------- tensor-core issue (one thread)
+        if (lane == 0) {
+            uint32_t ca = 0, cb = 0, cu = 0;
+            bool ok = true;
+            const uint32_t idesc_real = ptx::umma_idesc_f16_f32(kTileM, CoT);
+            const uint32_t idesc_cplx = ptx::umma_idesc_f16_f32(kTileM, 2 * CoT);
+            const uint32_t b_lbo = (uint32_t)rowsB * 16u;
+            for (int64_t u = first; u < prm.num_units && ok; u += stride, ++cu) {
+                ok = ptx::mbar_wait(&bar->empty_d, (cu & 1) ^ 1, abort_flag, status, 103);
+                if (!ok) break;
+                ptx::tc_fence_after_sync();
+                for (int kc = 0; kc < nK; ++kc, ++ca, ++cb) {
+                    const int sa = ca % SA, sb = cb % SB;
+                    ok = ptx::mbar_wait(&bar->full_a[sa], (ca / SA) & 1, abort_flag, status, 104) &&
+                         ptx::mbar_wait(&bar->full_b[sb], (cb / SB) & 1, abort_flag, status, 105);
+                    if (!ok) break;
+                    ptx::tc_fence_after_sync();
+                    const uint32_t a0 = ptx::smem_u32(xhat + sa * kAStage);
+                    const uint32_t b0 = ptx::smem_u32(bsm + sb * prm.b_slot_bytes);
+                    const uint32_t acc = kc > 0 ? 1u : 0u;
+                    // k = 0
+                    ptx::umma_f16(tmem_base, ptx::umma_smem_desc(a0, 2048, 128), ptx::umma_smem_desc(b0, b_lbo, 128),
+                                  idesc_real, acc);
+                    // complex frequencies: [Re y^ | Im y^] (+)= Re x^ [Wr|Wi] + Im x^ [-Wi|Wr]
+#pragma unroll
+                    for (int f = 1; f < T / 2; ++f) {
+                        const uint32_t d = tmem_base + (uint32_t)((2 * f - 1) * CoT);
+                        const uint32_t rb = (uint32_t)(CoT + (f - 1) * 4 * CoT);
+                        ptx::umma_f16(d, ptx::umma_smem_desc(a0 + (2 * f - 1) * 4096, 2048, 128),
+                                      ptx::umma_smem_desc(b0 + rb * 16u, b_lbo, 128), idesc_cplx, acc);
+                        ptx::umma_f16(d, ptx::umma_smem_desc(a0 + (2 * f) * 4096, 2048, 128),
+                                      ptx::umma_smem_desc(b0 + (rb + 2 * CoT) * 16u, b_lbo, 128), idesc_cplx, 1u);
+                    }
+                    // k = T/2
+                    ptx::umma_f16(tmem_base + (uint32_t)((T - 1) * CoT),
+                                  ptx::umma_smem_desc(a0 + (T - 1) * 4096, 2048, 128),
+                                  ptx::umma_smem_desc(b0 + (uint32_t)(rowsB - CoT) * 16u, b_lbo, 128), idesc_real, acc);
+                    ptx::umma_commit(&bar->empty_a[sa]);
+                    ptx::umma_commit(&bar->empty_b[sb]);
+                }
+                if (ok) ptx::umma_commit(&bar->full_d);
+            }
+            // all MMAs issued by this thread must have retired before shared memory and TMEM go away
+            ptx::umma_commit(&bar->mma_done);
+            ptx::mbar_wait(&bar->mma_done, 0, abort_flag, status, 113, false);
+        }
+    } else if (warp >= kWarpDft0) {
+        // ---------------------------------------------------------------- group DFT: raw slab row -> A operands
+        const int w = warp - kWarpDft0, quarter = w & 3, par = w >> 2;
+        const int r = quarter * 32 + lane;
+        uint32_t cr = 0, ca = 0;
+        bool ok = true;
+        for (int64_t u = first; u < prm.num_units && ok; u += stride) {
+            for (int kc = 0; kc < nK && ok; ++kc, ++ca) {
+                const int sa = ca % SA;
+                for (int q = 0; q < SPK; ++q, ++cr) {
+                    if ((int)(cr & 1) != par) continue;
+                    const int slot = cr % SR;
+                    ok = ptx::mbar_wait(&bar->full_raw[slot], (cr / SR) & 1, abort_flag, status, 106) &&
+                         ptx::mbar_wait(&bar->empty_a[sa], ((ca / SA) & 1) ^ 1, abort_flag, status, 107);
+                    if (!ok) break;
+                    const uint8_t* src = raw + slot * kSlabBytes + r * 128;
+                    uint32_t wd[32];
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const uint4 c = *reinterpret_cast<const uint4*>(src + ((j ^ (r & 7)) << 4));
+                        wd[4 * j] = c.x; wd[4 * j + 1] = c.y; wd[4 * j + 2] = c.z; wd[4 * j + 3] = c.w;
+                    }
+                    uint32_t packed[T][NCH / 2];
+#pragma unroll
+                    for (int cp = 0; cp < NCH / 2; ++cp) {
+                        float v0[T], v1[T];
+#pragma unroll
+                        for (int t = 0; t < T; t += 2) {
+                            const float2 a = unpack_h2(wd[((2 * cp) * T + t) / 2]);
+                            const float2 b = unpack_h2(wd[((2 * cp + 1) * T + t) / 2]);
+                            v0[t] = a.x; v0[t + 1] = a.y;
+                            v1[t] = b.x; v1[t + 1] = b.y;
+                        }
+                        rdft_forward<T>(v0);
+                        rdft_forward<T>(v1);
+#pragma unroll
+                        for (int p = 0; p < T; ++p) packed[p][cp] = pack_h2(v0[p], v1[p]);
+                    }
+                    uint8_t* dst = xhat + sa * kAStage + r * 16;
+                    const int kfirst = q * NCH;                  // first k of this slab inside the 16-channel chunk
+#pragma unroll
+                    for (int p = 0; p < T; ++p) {
+                        uint8_t* d = dst + p * 4096 + (kfirst >> 3) * 2048 + (kfirst & 7) * 2;
+                        if constexpr (NCH == 16) {
+                            *reinterpret_cast<uint4*>(d) = make_uint4(packed[p][0], packed[p][1], packed[p][2], packed[p][3]);
+                            *reinterpret_cast<uint4*>(d + 2048) = make_uint4(packed[p][4], packed[p][5], packed[p][6], packed[p][7]);
+                        } else if constexpr (NCH == 8) {
+                            *reinterpret_cast<uint4*>(d) = make_uint4(packed[p][0], packed[p][1], packed[p][2], packed[p][3]);
+                        } else if constexpr (NCH == 4) {
+                            *reinterpret_cast<uint2*>(d) = make_uint2(packed[p][0], packed[p][1]);
+                        } else {
+                            *reinterpret_cast<uint32_t*>(d) = packed[p][0];
+                        }
+                    }
+                    ptx::fence_proxy_async_smem();               // generic-proxy writes -> visible to the MMA (async proxy)
+                    __syncwarp();
+                    if (lane == 0) {
+                        ptx::mbar_arrive(&bar->empty_raw[slot]);
+                        ptx::mbar_arrive(&bar->full_a[sa]);
+                    }
+                }
+            }
+        }
+    } else if (warp >= kWarpEpi0 && warp < kWarpEpi0 + 4) {
+        // ---------------------------------------------------------------- epilogue: TMEM -> inverse DFT -> global
+        constexpr int G = 64 / T;                                // channels per TMEM read group
+        const int quad = warp & 3;
+        const uint32_t lane_base = tmem_base + ((uint32_t)(quad * 32) << 16);
+        uint32_t cu = 0;
+        bool ok = true;
+        for (int64_t u = first; u < prm.num_units && ok; u += stride, ++cu) {
+            const int tile = (int)(u % nTiles);
+            const int64_t row = (u / nTiles) * kTileM + quad * 32 + lane;
+            ok = ptx::mbar_wait(&bar->full_d, cu & 1, abort_flag, status, 108);
+            if (!ok) break;
+            ptx::tc_fence_after_sync();
+            __half* orow = prm.out + row * (int64_t)prm.Cout * T;
+            for (int c0 = 0; c0 < CoT; c0 += G) {
+                uint32_t in[T][G];
+#pragma unroll
+                for (int p = 0; p < T; ++p) ptx::tmem_ld<G>(lane_base + (uint32_t)(p * CoT + c0), in[p]);
+                ptx::tmem_ld_wait();
+                if (c0 + G >= CoT) {                             // last read of this accumulator: hand TMEM back
+                    ptx::tc_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) ptx::mbar_arrive(&bar->empty_d);
+                }
+                if (row >= prm.N) continue;
+                if constexpr (T == 4) {
+#pragma unroll
+                    for (int g = 0; g < G; g += 2) {
+                        const int co = tile * CoT + c0 + g;
+                        float v0[4], v1[4];
+#pragma unroll
+                        for (int p = 0; p < 4; ++p) { v0[p] = __uint_as_float(in[p][g]); v1[p] = __uint_as_float(in[p][g + 1]); }
+                        if (prm.bias != nullptr) {
+                            if (co < prm.Cout) v0[0] += __ldg(prm.bias + co);
+                            if (co + 1 < prm.Cout) v1[0] += __ldg(prm.bias + co + 1);
+                        }
+                        rdft_inverse<4>(v0);
+                        rdft_inverse<4>(v1);
+                        if (co + 1 < prm.Cout) {
+                            ptx::st_global_v4(orow + (int64_t)co * 4, pack_h2(v0[0], v0[1]), pack_h2(v0[2], v0[3]),
+                                              pack_h2(v1[0], v1[1]), pack_h2(v1[2], v1[3]));
+                        } else if (co < prm.Cout) {
+                            *reinterpret_cast<uint2*>(orow + (int64_t)co * 4) =
+                                make_uint2(pack_h2(v0[0], v0[1]), pack_h2(v0[2], v0[3]));
+                        }
+                    }
+                } else {
+#pragma unroll
+                    for (int g = 0; g < G; ++g) {
+                        const int co = tile * CoT + c0 + g;
+                        if (co >= prm.Cout) continue;
+                        float v[T];
+#pragma unroll
+                        for (int p = 0; p < T; ++p) v[p] = __uint_as_float(in[p][g]);
+                        if (prm.bias != nullptr) v[0] += __ldg(prm.bias + co);
+                        rdft_inverse<T>(v);
+                        __half* dst = orow + (int64_t)co * T;
+#pragma unroll
+                        for (int t = 0; t < T; t += 8)
+                            ptx::st_global_v4(dst + t, pack_h2(v[t], v[t + 1]), pack_h2(v[t + 2], v[t + 3]),
+                                              pack_h2(v[t + 4], v[t + 5]), pack_h2(v[t + 6], v[t + 7]));
+                    }
+                }
+            }
+        }
+    }
+
+    // ---------------------------------------------------------------- teardown (reached by every thread)
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    if (warp == kWarpMma) {
+        ptx::tc_fence_after_sync();
+        ptx::tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------ host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    });
+    return fn;
+}
+
+template <int T>
+size_t umma_smem_bytes(int b_slot_bytes) {
+    using Cfg = UmmaCfg<T>;
+    return 1024 + (size_t)Cfg::SR * kSlabBytes + (size_t)Cfg::SA * T * 4096 + (size_t)Cfg::SB * b_slot_bytes +
+           sizeof(SmemBarriers) + 64;
+}
+
+template <typename F>
+cudaError_t dispatch_umma_T(int T, F&& f) {
+    switch (T) {
+        case 4: return f(std::integral_constant<int, 4>{});
+        case 8: return f(std::integral_constant<int, 8>{});
+        case 16: return f(std::integral_constant<int, 16>{});
+        case 32: return f(std::integral_constant<int, 32>{});
+        default: return cudaErrorInvalidValue;
+    }
+}
+
+}  // namespace
+
+bool umma_linear_supported(int T, eql_dtype_t dtype) {
+    return dtype == EQL_FP16 && (T == 4 || T == 8 || T == 16 || T == 32);
+}
+
+UmmaLinearShape umma_linear_shape(int T, int Cin, int Cout) {
+    UmmaLinearShape s{};
+    s.T = T; s.Cin = Cin; s.Cout = Cout;
+    const int max_cot = kTmemCols / T;                           // T planes x CoT fp32 columns <= 512
+    s.nTiles = (Cout + max_cot - 1) / max_cot;
+    const int per = (Cout + s.nTiles - 1) / s.nTiles;
+    s.CoT = (per + 15) / 16 * 16;
+    s.nK = (Cin + kChunkK - 1) / kChunkK;
+    s.rowsB = (2 * T - 2) * s.CoT;
+    s.image_bytes = align_up((size_t)s.nTiles * s.nK * s.rowsB * kChunkK * sizeof(__half), kWsAlign);
+    return s;
+}
+
+cudaError_t launch_build_umma_image(const UmmaLinearShape& s, const float* planes, void* image, cudaStream_t stream) {
+    return dispatch_umma_T(s.T, [&](auto tc) {
+        constexpr int TT = decltype(tc)::value;
+        const int64_t total = (int64_t)s.nTiles * s.nK * s.rowsB * kChunkK;
+        const int blocks = (int)((total + 255) / 256 < 4096 ? (total + 255) / 256 : 4096);
+        build_image_kernel<TT><<<blocks, 256, 0, stream>>>(planes, s.Cin, s.Cout, s.CoT, s.nTiles, s.nK, s.rowsB,
+                                                            (__half*)image);
+        return cudaGetLastError();
+    });
+}
+
+cudaError_t launch_umma_linear(const UmmaLinearShape& s, const void* in, void* out, int64_t N, const void* image,
+                               const float* bias_f32, int* status, int num_sms, cudaStream_t stream) {
+    EncodeTiledFn enc = encode_tiled_fn();
+    if (enc == nullptr) return cudaErrorNotSupported;
+    CUtensorMap tmap;
+    const cuuint64_t gdim[2] = {(cuuint64_t)s.Cin * s.T, (cuuint64_t)N};
+    const cuuint64_t gstr[1] = {(cuuint64_t)s.Cin * s.T * sizeof(__half)};
+    const cuuint32_t box[2] = {64, (cuuint32_t)kTileM};
+    const cuuint32_t estr[2] = {1, 1};
+    if (enc(&tmap, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(in), gdim, gstr, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return cudaErrorInvalidValue;
+
+    UmmaParams prm{};
+    prm.out = (__half*)out; prm.image = (const __half*)image; prm.bias = bias_f32; prm.status = status;
+    prm.N = N; prm.Cin = s.Cin; prm.Cout = s.Cout;
+    prm.CoT = s.CoT; prm.nTiles = s.nTiles; prm.nK = s.nK; prm.rowsB = s.rowsB;
+    prm.b_slot_bytes = (int)align_up((size_t)s.rowsB * 32, 128);
+    prm.num_units = ((N + kTileM - 1) / kTileM) * s.nTiles;
+    const int grid = (int)(prm.num_units < num_sms ? prm.num_units : num_sms);
+
+    return dispatch_umma_T(s.T, [&](auto tc) {
+        constexpr int TT = decltype(tc)::value;
+        const size_t smem = umma_smem_bytes<TT>(prm.b_slot_bytes);
+        static unsigned long long attr_done = 0;              // one bit per device (per instantiation)
+        int dev = 0;
+        cudaGetDevice(&dev);
+        if (!((attr_done >> (dev & 63)) & 1ull)) {
+            cudaError_t e = cudaFuncSetAttribute(umma_linear_kernel<TT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                 227 * 1024);
+            if (e != cudaSuccess) return e;
+            attr_done |= 1ull << (dev & 63);
+        }
+        if (smem > 227 * 1024) return cudaErrorInvalidConfiguration;
+        umma_linear_kernel<TT><<<grid, kThreadsUmma, smem, stream>>>(tmap, prm);
+        return cudaGetLastError();
+    });
+}
+
+}  // namespace eql
