@@ -407,6 +407,19 @@ BwdWeightSplit direct_bwd_weight_split(int T, int Ci, int Co, int64_t N) {
     return s;
 }
 
+cudaError_t launch_bwd_weight_finalize(int T, bool correlation, const float* scratch, int splits, int Ci, int Co,
+                                       float* dw, float* db, cudaStream_t stream) {
+    const float* part = scratch;
+    const float* db_part = scratch + (size_t)splits * T * Co * Ci;
+    return dispatch_T(T, [&](auto tc) {
+        constexpr int TT = decltype(tc)::value;
+        const int total = Ci * Co > Co ? Ci * Co : Co;
+        bwd_weight_finalize_kernel<TT><<<(total + 127) / 128, 128, 0, stream>>>(part, db_part, splits, Ci, Co,
+                                                                                 correlation, dw, db);
+        return cudaGetLastError();
+    });
+}
+
 cudaError_t launch_direct_bwd_weight(int T, eql_dtype_t dtype, bool correlation, const void* x, const void* dy,
                                      float* dw, float* db, int64_t N, int Ci, int Co,
                                      const BwdWeightSplit& split, float* scratch, cudaStream_t stream) {

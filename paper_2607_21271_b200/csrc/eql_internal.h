@@ -70,6 +70,25 @@ cudaError_t launch_build_umma_image(const UmmaLinearShape& s, const float* plane
 cudaError_t launch_umma_linear(const UmmaLinearShape& s, const void* in, void* out, int64_t N, const void* image,
                                const float* bias_f32, int* status, int num_sms, cudaStream_t stream);
 
+// ---- tcgen05 weight-gradient kernel (FP16 inputs), umma_bwd_weight.cu --------------------------------
+struct UmmaBwdWeightShape {
+    int T, Ci, Co;
+    int CiT, nCiTiles;          // input-channel tile (UMMA M side, <= 128 lanes, CiT*T <= 1024)
+    int CoT, nCoTiles;          // output-channel tile (UMMA N side, T*CoT <= 512 TMEM columns)
+    int nXs, nYs;               // 64-element raw slabs of x / dy per 16-token chunk
+    int splits;                 // token ranges
+    int64_t chunks_per_split;   // 16-token chunks per range
+    size_t scratch_bytes;       // splits * (T*Co*Ci + Co) floats
+};
+bool umma_bwd_weight_supported(int T, eql_dtype_t dtype);
+UmmaBwdWeightShape umma_bwd_weight_shape(int T, int Ci, int Co, int64_t N, int num_sms);
+// Phase 1 only: partial spectra + db partials into scratch (same layout as the CUDA-core kernel's).
+cudaError_t launch_umma_bwd_weight(const UmmaBwdWeightShape& s, const void* x, const void* dy, int64_t N,
+                                   float* scratch, int* status, cudaStream_t stream);
+// Phase 2 (direct_kernels.cu): fixed-order sum over splits, 1/T, inverse DFT -> dw, db.
+cudaError_t launch_bwd_weight_finalize(int T, bool correlation, const float* scratch, int splits, int Ci, int Co,
+                                       float* dw, float* db, cudaStream_t stream);
+
 }  // namespace eql
 
 // The host object behind eqlinear_plan_t.

@@ -133,6 +133,7 @@ eql_status_t eqlinear_plan(eqlinear_plan_t* plan, int T, int C_in, int C_out, eq
         p->fwd_kernel = p->bwd_data_kernel = 1;
         p->umma_fwd = umma_linear_shape(T, C_in, C_out);
         p->umma_bwd = umma_linear_shape(T, C_out, C_in);
+        if (umma_bwd_weight_supported(T, dtype)) p->bwd_weight_kernel = 1;
     }
 
     cudaStream_t s = (cudaStream_t)stream;
@@ -220,7 +221,10 @@ eql_status_t eqlinear_bwd_weight_scratch_bytes(eqlinear_plan_t plan, int64_t N, 
     if (!plan || !bytes) return EQL_ERR_INVALID_ARG;
     eql_status_t st = check_tokens(N);
     if (st != EQL_OK) return st;
-    *bytes = direct_bwd_weight_split(plan->T, plan->Ci, plan->Co, N > 0 ? N : 1).scratch_bytes;
+    if (plan->bwd_weight_kernel == 1)
+        *bytes = umma_bwd_weight_shape(plan->T, plan->Ci, plan->Co, N > 0 ? N : 1, plan->num_sms).scratch_bytes;
+    else
+        *bytes = direct_bwd_weight_split(plan->T, plan->Ci, plan->Co, N > 0 ? N : 1).scratch_bytes;
     return EQL_OK;
 }
 
@@ -240,6 +244,15 @@ eql_status_t eqlinear_bwd_weight(eqlinear_plan_t plan, const void* x, const void
     if (!x || !dy || !scratch) return EQL_ERR_INVALID_ARG;
     if (!aligned16(x) || !aligned16(dy)) return EQL_ERR_ALIGNMENT;
     if (reinterpret_cast<uintptr_t>(scratch) % kWsAlign != 0) return EQL_ERR_ALIGNMENT;
+    if (plan->bwd_weight_kernel == 1) {
+        UmmaBwdWeightShape bs = umma_bwd_weight_shape(plan->T, plan->Ci, plan->Co, N, plan->num_sms);
+        if (scratch_bytes < bs.scratch_bytes) return EQL_ERR_WORKSPACE;
+        cudaError_t e = launch_umma_bwd_weight(bs, x, dy, N, (float*)scratch, (int*)(plan->ws + plan->lay.status), s);
+        if (e != cudaSuccess) return EQL_ERR_CUDA;
+        e = launch_bwd_weight_finalize(plan->T, (plan->flags & EQL_FLAG_CORRELATION) != 0, (const float*)scratch, bs.splits,
+                                       plan->Ci, plan->Co, (float*)dw, (float*)db, s);
+        return e == cudaSuccess ? EQL_OK : EQL_ERR_CUDA;
+    }
     BwdWeightSplit split = direct_bwd_weight_split(plan->T, plan->Ci, plan->Co, N);
     if (scratch_bytes < split.scratch_bytes) return EQL_ERR_WORKSPACE;
     cudaError_t e = launch_direct_bwd_weight(plan->T, plan->dtype, (plan->flags & EQL_FLAG_CORRELATION) != 0, x, dy,

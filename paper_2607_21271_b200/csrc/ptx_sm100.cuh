@@ -118,6 +118,10 @@ __device__ __forceinline__ uint32_t umma_idesc_f16_f32(uint32_t M, uint32_t N) {
            | ((N >> 3) << 17)       // N / 8
            | ((M >> 4) << 24);      // M / 16
 }
+// Same, with both operands MN-major ("transposed": the M resp. N index is the contiguous one in shared memory).
+__device__ __forceinline__ uint32_t umma_idesc_f16_f32_mn_major(uint32_t M, uint32_t N) {
+    return umma_idesc_f16_f32(M, N) | (1u << 15) | (1u << 16);
+}
 // D[tmem] (+)= A[smem] * B[smem]^T; issued by ONE thread.
 __device__ __forceinline__ void umma_f16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
                                          uint32_t accumulate) {

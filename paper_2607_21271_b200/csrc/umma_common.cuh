@@ -1,0 +1,75 @@
+// Device helpers shared by the tcgen05 kernels: half2 packing and the "slab row" transform
+// (128 bytes = 64 consecutive fp16 elements of one token, read from a 128B-swizzled TMA slab,
+// group DFT of the 64/T channels they hold, planes rounded to fp16 once and packed channel-pairwise).
+#pragma once
+
+#include <cuda_fp16.h>
+
+#include <cstring>
+
+#include "rdft.cuh"
+
+namespace eql {
+
+__device__ __forceinline__ float2 unpack_h2(uint32_t u) {
+    __half2 h;
+    memcpy(&h, &u, 4);
+    return __half22float2(h);
+}
+__device__ __forceinline__ uint32_t pack_h2(float lo, float hi) {
+    __half2 h = __floats2half2_rn(lo, hi);
+    uint32_t u;
+    memcpy(&u, &h, 4);
+    return u;
+}
+
+// row_base: start of this token's 128-byte row inside a slab written by TMA with 128B swizzle
+// (slab base 1024-byte aligned, rows 128 bytes apart); r: row index inside the slab.
+// packed[p][cp] = (plane p of channel 2cp, plane p of channel 2cp+1) as half2.
+// plane0[c] (optional, float) = unrounded k = 0 plane of channel c (the sum over the group axis).
+template <int T, bool WANT_PLANE0>
+__device__ __forceinline__ void dft_slab_row(const uint8_t* row_base, int r, uint32_t (&packed)[T][(64 / T) / 2],
+                                             float* plane0) {
+    constexpr int NCH = 64 / T;
+    uint32_t wd[32];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const uint4 c = *reinterpret_cast<const uint4*>(row_base + ((j ^ (r & 7)) << 4));
+        wd[4 * j] = c.x; wd[4 * j + 1] = c.y; wd[4 * j + 2] = c.z; wd[4 * j + 3] = c.w;
+    }
+#pragma unroll
+    for (int cp = 0; cp < NCH / 2; ++cp) {
+        float v0[T], v1[T];
+#pragma unroll
+        for (int t = 0; t < T; t += 2) {
+            const float2 a = unpack_h2(wd[((2 * cp) * T + t) / 2]);
+            const float2 b = unpack_h2(wd[((2 * cp + 1) * T + t) / 2]);
+            v0[t] = a.x; v0[t + 1] = a.y;
+            v1[t] = b.x; v1[t + 1] = b.y;
+        }
+        rdft_forward<T>(v0);
+        rdft_forward<T>(v1);
+        if constexpr (WANT_PLANE0) { plane0[2 * cp] = v0[0]; plane0[2 * cp + 1] = v1[0]; }
+#pragma unroll
+        for (int p = 0; p < T; ++p) packed[p][cp] = pack_h2(v0[p], v1[p]);
+    }
+}
+
+// Stores the NCH = 64/T packed channel values of one plane as one contiguous run of NCH halves.
+// NCH = 16 -> two 16-byte stores `second_half_stride` bytes apart, 8 -> one 16-byte store, 4 -> 8 bytes, 2 -> 4 bytes.
+template <int NCH>
+__device__ __forceinline__ void store_plane_run(uint8_t* d, const uint32_t* pk, int second_half_stride, uint32_t xor_mask = 0u) {
+    if constexpr (NCH == 16) {
+        *reinterpret_cast<uint4*>(d) = make_uint4(pk[0] ^ xor_mask, pk[1] ^ xor_mask, pk[2] ^ xor_mask, pk[3] ^ xor_mask);
+        *reinterpret_cast<uint4*>(d + second_half_stride) =
+            make_uint4(pk[4] ^ xor_mask, pk[5] ^ xor_mask, pk[6] ^ xor_mask, pk[7] ^ xor_mask);
+    } else if constexpr (NCH == 8) {
+        *reinterpret_cast<uint4*>(d) = make_uint4(pk[0] ^ xor_mask, pk[1] ^ xor_mask, pk[2] ^ xor_mask, pk[3] ^ xor_mask);
+    } else if constexpr (NCH == 4) {
+        *reinterpret_cast<uint2*>(d) = make_uint2(pk[0] ^ xor_mask, pk[1] ^ xor_mask);
+    } else {
+        *reinterpret_cast<uint32_t*>(d) = pk[0] ^ xor_mask;
+    }
+}
+
+}  // namespace eql

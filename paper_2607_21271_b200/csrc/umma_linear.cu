@@ -23,6 +23,7 @@
 #include "eql_internal.h"
 #include "ptx_sm100.cuh"
 #include "rdft.cuh"
+#include "umma_common.cuh"
 
 namespace eql {
 namespace {
@@ -53,18 +54,6 @@ struct UmmaParams {
     int b_slot_bytes;            // bytes of one B ring slot (rowsB*32 rounded up to 128)
     int64_t num_units;
 };
-
-__device__ __forceinline__ float2 unpack_h2(uint32_t u) {
-    __half2 h;
-    memcpy(&h, &u, 4);
-    return __half22float2(h);
-}
-__device__ __forceinline__ uint32_t pack_h2(float lo, float hi) {
-    __half2 h = __floats2half2_rn(lo, hi);
-    uint32_t u;
-    memcpy(&u, &h, 4);
-    return u;
-}
 
 struct SmemBarriers {
     uint64_t full_raw[4], empty_raw[4];
@@ -271,45 +260,12 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const UmmaParams
                     ok = ptx::mbar_wait(&bar->full_raw[slot], (cr / SR) & 1, abort_flag, status, 106) &&
                          ptx::mbar_wait(&bar->empty_a[sa], ((ca / SA) & 1) ^ 1, abort_flag, status, 107);
                     if (!ok) break;
-                    const uint8_t* src = raw + slot * kSlabBytes + r * 128;
-                    uint32_t wd[32];
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        const uint4 c = *reinterpret_cast<const uint4*>(src + ((j ^ (r & 7)) << 4));
-                        wd[4 * j] = c.x; wd[4 * j + 1] = c.y; wd[4 * j + 2] = c.z; wd[4 * j + 3] = c.w;
-                    }
                     uint32_t packed[T][NCH / 2];
-#pragma unroll
-                    for (int cp = 0; cp < NCH / 2; ++cp) {
-                        float v0[T], v1[T];
-#pragma unroll
-                        for (int t = 0; t < T; t += 2) {
-                            const float2 a = unpack_h2(wd[((2 * cp) * T + t) / 2]);
-                            const float2 b = unpack_h2(wd[((2 * cp + 1) * T + t) / 2]);
-                            v0[t] = a.x; v0[t + 1] = a.y;
-                            v1[t] = b.x; v1[t + 1] = b.y;
-                        }
-                        rdft_forward<T>(v0);
-                        rdft_forward<T>(v1);
-#pragma unroll
-                        for (int p = 0; p < T; ++p) packed[p][cp] = pack_h2(v0[p], v1[p]);
-                    }
-                    uint8_t* dst = xhat + sa * kAStage + r * 16;
+                    dft_slab_row<T, false>(raw + slot * kSlabBytes + r * 128, r, packed, nullptr);
                     const int kfirst = q * NCH;                  // first k of this slab inside the 16-channel chunk
+                    uint8_t* dst = xhat + sa * kAStage + r * 16 + (kfirst >> 3) * 2048 + (kfirst & 7) * 2;
 #pragma unroll
-                    for (int p = 0; p < T; ++p) {
-                        uint8_t* d = dst + p * 4096 + (kfirst >> 3) * 2048 + (kfirst & 7) * 2;
-                        if constexpr (NCH == 16) {
-                            *reinterpret_cast<uint4*>(d) = make_uint4(packed[p][0], packed[p][1], packed[p][2], packed[p][3]);
-                            *reinterpret_cast<uint4*>(d + 2048) = make_uint4(packed[p][4], packed[p][5], packed[p][6], packed[p][7]);
-                        } else if constexpr (NCH == 8) {
-                            *reinterpret_cast<uint4*>(d) = make_uint4(packed[p][0], packed[p][1], packed[p][2], packed[p][3]);
-                        } else if constexpr (NCH == 4) {
-                            *reinterpret_cast<uint2*>(d) = make_uint2(packed[p][0], packed[p][1]);
-                        } else {
-                            *reinterpret_cast<uint32_t*>(d) = packed[p][0];
-                        }
-                    }
+                    for (int p = 0; p < T; ++p) store_plane_run<NCH>(dst + p * 4096, packed[p], 2048);
                     ptx::fence_proxy_async_smem();               // generic-proxy writes -> visible to the MMA (async proxy)
                     __syncwarp();
                     if (lane == 0) {

@@ -47,7 +47,7 @@ def test_static_scratch_matches_caller_scratch_twice(dtype, T, Ci, Co, N):
 
 
 def test_static_scratch_rejects_sizes_beyond_the_array():
-    T, Ci, Co, N = 32, 64, 64, 4096
+    T, Ci, Co, N = 8, 256, 256, 8192
     wl = Workload("big", "fp16", T, Ci, Co, N, "none", ("bwd_weight",), 23)
     d = generate(wl)
     layer = GpuLayer(T, Ci, Co, "fp16", d["w"], None)
