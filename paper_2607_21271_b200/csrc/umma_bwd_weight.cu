@@ -174,11 +174,15 @@ umma_bwd_weight_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
             ok = ptx::mbar_wait(&bar->full_raw[slot], (uint32_t)((c / kRawSlots) & 1), abort_flag, status, 203) &&
                  ptx::mbar_wait(&bar->empty_ab[st], (uint32_t)((c / kStages) & 1) ^ 1, abort_flag, status, 204);
             if (!ok) break;
+            uint32_t wd[32];
+            if (active)
+                load_slab_row(raw + slot * kRawSlot + ((is_y ? kMaxXSlabs : 0) + slab) * kSlab + row * 128, row, wd);
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(&bar->empty_raw[slot]);     // the slot can be refilled while we transform
             if (active) {
-                const uint8_t* src = raw + slot * kRawSlot + ((is_y ? kMaxXSlabs : 0) + slab) * kSlab + row * 128;
                 uint32_t packed[T][NCH / 2];
                 float p0[NCH];
-                dft_slab_row<T, true>(src, row, packed, p0);
+                dft_words<T, true>(wd, packed, p0);
                 const int mn0 = slab * NCH;                      // first channel of this slab inside the tile
                 // MN-major tile: (channel mn, token k) at (mn/8)*256 + (k/8)*128 + (k%8)*16 + (mn%8)*2
                 const int off = (mn0 >> 3) * 256 + (row >> 3) * 128 + (row & 7) * 16 + (mn0 & 7) * 2;
@@ -204,10 +208,7 @@ umma_bwd_weight_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
             }
             ptx::fence_proxy_async_smem();
             __syncwarp();
-            if (lane == 0) {
-                ptx::mbar_arrive(&bar->empty_raw[slot]);
-                ptx::mbar_arrive(&bar->full_ab[st]);
-            }
+            if (lane == 0) ptx::mbar_arrive(&bar->full_ab[st]);
         }
         // db partial of this token range: sum over the 16 token rows of each half warp
         if (is_y) {

@@ -25,18 +25,21 @@ __device__ __forceinline__ uint32_t pack_h2(float lo, float hi) {
 
 // row_base: start of this token's 128-byte row inside a slab written by TMA with 128B swizzle
 // (slab base 1024-byte aligned, rows 128 bytes apart); r: row index inside the slab.
-// packed[p][cp] = (plane p of channel 2cp, plane p of channel 2cp+1) as half2.
-// plane0[c] (optional, float) = unrounded k = 0 plane of channel c (the sum over the group axis).
-template <int T, bool WANT_PLANE0>
-__device__ __forceinline__ void dft_slab_row(const uint8_t* row_base, int r, uint32_t (&packed)[T][(64 / T) / 2],
-                                             float* plane0) {
-    constexpr int NCH = 64 / T;
-    uint32_t wd[32];
+// wd[0..32) = the row's 64 halves in logical order.
+__device__ __forceinline__ void load_slab_row(const uint8_t* row_base, int r, uint32_t (&wd)[32]) {
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
         const uint4 c = *reinterpret_cast<const uint4*>(row_base + ((j ^ (r & 7)) << 4));
         wd[4 * j] = c.x; wd[4 * j + 1] = c.y; wd[4 * j + 2] = c.z; wd[4 * j + 3] = c.w;
     }
+}
+
+// Group DFT of the 64/T channels held in wd.
+// packed[p][cp] = (plane p of channel 2cp, plane p of channel 2cp+1) as half2.
+// plane0[c] (optional, float) = unrounded k = 0 plane of channel c (the sum over the group axis).
+template <int T, bool WANT_PLANE0>
+__device__ __forceinline__ void dft_words(const uint32_t (&wd)[32], uint32_t (&packed)[T][(64 / T) / 2], float* plane0) {
+    constexpr int NCH = 64 / T;
 #pragma unroll
     for (int cp = 0; cp < NCH / 2; ++cp) {
         float v0[T], v1[T];

@@ -2,13 +2,13 @@
 // FP32 accumulation.  One persistent CTA per SM; a work unit is (128-token tile, output-channel tile).
 //
 //   TMA (2-D, 128B swizzle)      raw rows of x            -> shared "slabs" [128 rows x 128 B]
-//   8 transform warps            group DFT (Eq. 4) in registers, planes rounded to fp16 once
+//   12 compute warps, phase 1    group DFT (Eq. 4) in registers, planes rounded to fp16 once
 //                                -> shared A operands, one [128 x 16] K-major tile per real-packed plane
 //   TMA (1-D bulk)               spectral-weight image of this (tile, 16-channel chunk) -> shared B operands
 //   1 thread                     tcgen05.mma kind::f16: one product per real frequency, and the complex
 //                                product of Eq. 5 as the real 2x2 block [Xr|Xi] x [[Wr,Wi],[-Wi,Wr]] -> TMEM
-//   4 epilogue warps             tcgen05.ld, bias on plane k = 0, inverse DFT (Eq. 7) in registers,
-//                                fp16 rounding, group tuples stored contiguously to global memory
+//   12 compute warps, phase 2    tcgen05.ld, bias on plane k = 0, inverse DFT (Eq. 7) in registers,
+//                                fp16 rounding, 128 contiguous bytes per token stored with 32-byte stores
 //
 // Frequency-domain data never leaves the SM (registers, shared memory, TMEM).  The data gradient is the
 // same kernel run on dy with the conjugate-transposed weight image and no bias.
@@ -35,7 +35,8 @@ constexpr int kThreadsUmma = 512;
 constexpr int kTmemCols = 512;
 
 // warp roles
-constexpr int kWarpTmaX = 0, kWarpMma = 1, kWarpTmaB = 2, kWarpEpi0 = 4, kWarpDft0 = 8;
+constexpr int kWarpTmaX = 0, kWarpMma = 1, kWarpTmaB = 2, kWarpCompute0 = 4;
+constexpr int kNumComputeWarps = 12;
 
 template <int T> struct UmmaCfg;
 template <> struct UmmaCfg<4>  { static constexpr int SR = 4, SA = 4, SB = 3; };
@@ -128,11 +129,11 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const UmmaParams
     int* status = prm.status;
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < SR; ++i) { ptx::mbar_init(&bar->full_raw[i], 1); ptx::mbar_init(&bar->empty_raw[i], 4); }
+        for (int i = 0; i < SR; ++i) { ptx::mbar_init(&bar->full_raw[i], 1); ptx::mbar_init(&bar->empty_raw[i], kNumComputeWarps); }
         for (int i = 0; i < SA; ++i) { ptx::mbar_init(&bar->full_a[i], 4 * SPK); ptx::mbar_init(&bar->empty_a[i], 1); }
         for (int i = 0; i < SB; ++i) { ptx::mbar_init(&bar->full_b[i], 1); ptx::mbar_init(&bar->empty_b[i], 1); }
         ptx::mbar_init(&bar->full_d, 1);
-        ptx::mbar_init(&bar->empty_d, 4);
+        ptx::mbar_init(&bar->empty_d, kNumComputeWarps);
         ptx::mbar_init(&bar->mma_done, 1);
         bar->abort_flag = 0;
         ptx::fence_mbar_init();
@@ -245,99 +246,124 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const UmmaParams
             ptx::umma_commit(&bar->mma_done);
             ptx::mbar_wait(&bar->mma_done, 0, abort_flag, status, 113, false);
         }
-    } else if (warp >= kWarpDft0) {
-        // ---------------------------------------------------------------- group DFT: raw slab row -> A operands
-        const int w = warp - kWarpDft0, quarter = w & 3, par = w >> 2;
-        const int r = quarter * 32 + lane;
-        uint32_t cr = 0, ca = 0;
+    } else if (warp >= kWarpCompute0) {
+        // ---------------------------------------------------------------- compute warps: transform, then epilogue
+        // Per unit every compute warp first transforms its share of the raw slab rows (group DFT -> A operands)
+        // and then drains its share of the accumulator (inverse DFT -> global).  Work items of the transform
+        // are (slab, 32-row quarter); they are dealt round-robin over the 12 warps across chunks.
+        constexpr int G = 64 / T;                                // channels per TMEM read group
+        constexpr int kItemsPerChunk = 4 * SPK;
+        // A warp's consecutive items are kNumComputeWarps items apart; that must stay below SA chunks so that the
+        // owner-only wait on empty_a is never more than one phase ahead of the barrier.
+        static_assert(kNumComputeWarps < SA * kItemsPerChunk, "empty_a parity wait would be ambiguous");
+        const int cw = warp - kWarpCompute0;
+        const int quad = warp & 3;                               // TMEM lane quadrant this warp may read
+        const int third = cw >> 2;                               // which share of the column groups
+        const uint32_t lane_base = tmem_base + ((uint32_t)(quad * 32) << 16);
+        const bool vec32 = ((reinterpret_cast<uintptr_t>(prm.out) & 31u) == 0) && (((int64_t)prm.Cout * T * 2) % 32 == 0);
+        uint32_t ca = 0, cu = 0;
+        uint32_t item_mod = 0;                                   // (index of the next slab's first work item) mod 12
         bool ok = true;
-        for (int64_t u = first; u < prm.num_units && ok; u += stride) {
+        for (int64_t u = first; u < prm.num_units && ok; u += stride, ++cu) {
+            // ---- transform
             for (int kc = 0; kc < nK && ok; ++kc, ++ca) {
                 const int sa = ca % SA;
-                for (int q = 0; q < SPK; ++q, ++cr) {
-                    if ((int)(cr & 1) != par) continue;
+#pragma unroll 1
+                for (int q = 0; q < SPK; ++q) {
+                    const uint32_t cr = ca * SPK + q;            // running slab counter
                     const int slot = cr % SR;
-                    ok = ptx::mbar_wait(&bar->full_raw[slot], (cr / SR) & 1, abort_flag, status, 106) &&
-                         ptx::mbar_wait(&bar->empty_a[sa], ((ca / SA) & 1) ^ 1, abort_flag, status, 107);
+                    // A parity wait is only unambiguous while the waiter is at most one phase behind the barrier,
+                    // so every compute warp both observes and releases every phase of every slot barrier:
+                    // owners of one of the slab's four row quarters release after loading their rows, the
+                    // other warps right away.
+                    ok = ptx::mbar_wait(&bar->full_raw[slot], (cr / SR) & 1, abort_flag, status, 106);
                     if (!ok) break;
+                    int d = cw - (int)item_mod;                  // which quarter of this slab is ours, if any
+                    if (d < 0) d += kNumComputeWarps;
+                    item_mod = (item_mod + 4) % kNumComputeWarps;
+                    if (d >= 4) {
+                        if (lane == 0) ptx::mbar_arrive(&bar->empty_raw[slot]);
+                        continue;
+                    }
+                    const int r = d * 32 + lane;
+                    uint32_t wd[32];
+                    load_slab_row(raw + slot * kSlabBytes + r * 128, r, wd);
+                    __syncwarp();
+                    if (lane == 0) ptx::mbar_arrive(&bar->empty_raw[slot]);     // refill can start while we transform
                     uint32_t packed[T][NCH / 2];
-                    dft_slab_row<T, false>(raw + slot * kSlabBytes + r * 128, r, packed, nullptr);
+                    dft_words<T, false>(wd, packed, nullptr);
+                    ok = ptx::mbar_wait(&bar->empty_a[sa], ((ca / SA) & 1) ^ 1, abort_flag, status, 107);
+                    if (!ok) break;
                     const int kfirst = q * NCH;                  // first k of this slab inside the 16-channel chunk
                     uint8_t* dst = xhat + sa * kAStage + r * 16 + (kfirst >> 3) * 2048 + (kfirst & 7) * 2;
 #pragma unroll
                     for (int p = 0; p < T; ++p) store_plane_run<NCH>(dst + p * 4096, packed[p], 2048);
                     ptx::fence_proxy_async_smem();               // generic-proxy writes -> visible to the MMA (async proxy)
                     __syncwarp();
-                    if (lane == 0) {
-                        ptx::mbar_arrive(&bar->empty_raw[slot]);
-                        ptx::mbar_arrive(&bar->full_a[sa]);
-                    }
+                    if (lane == 0) ptx::mbar_arrive(&bar->full_a[sa]);
                 }
             }
-        }
-    } else if (warp >= kWarpEpi0 && warp < kWarpEpi0 + 4) {
-        // ---------------------------------------------------------------- epilogue: TMEM -> inverse DFT -> global
-        constexpr int G = 64 / T;                                // channels per TMEM read group
-        const int quad = warp & 3;
-        const uint32_t lane_base = tmem_base + ((uint32_t)(quad * 32) << 16);
-        uint32_t cu = 0;
-        bool ok = true;
-        for (int64_t u = first; u < prm.num_units && ok; u += stride, ++cu) {
+            if (!ok) break;
+            // ---- epilogue
             const int tile = (int)(u % nTiles);
             const int64_t row = (u / nTiles) * kTileM + quad * 32 + lane;
             ok = ptx::mbar_wait(&bar->full_d, cu & 1, abort_flag, status, 108);
             if (!ok) break;
             ptx::tc_fence_after_sync();
             __half* orow = prm.out + row * (int64_t)prm.Cout * T;
-            for (int c0 = 0; c0 < CoT; c0 += G) {
+            const int ngroups = CoT / G;
+            for (int gi = third; gi < ngroups; gi += 3) {
+                const int c0 = gi * G;
                 uint32_t in[T][G];
 #pragma unroll
                 for (int p = 0; p < T; ++p) ptx::tmem_ld<G>(lane_base + (uint32_t)(p * CoT + c0), in[p]);
                 ptx::tmem_ld_wait();
-                if (c0 + G >= CoT) {                             // last read of this accumulator: hand TMEM back
+                if (gi + 3 >= ngroups) {                         // this warp's last read of the accumulator
                     ptx::tc_fence_before_sync();
                     __syncwarp();
                     if (lane == 0) ptx::mbar_arrive(&bar->empty_d);
                 }
                 if (row >= prm.N) continue;
-                if constexpr (T == 4) {
+                const int co0 = tile * CoT + c0;
+                uint32_t o[32];                                  // G channels x T halves = 64 halves = 128 bytes
 #pragma unroll
-                    for (int g = 0; g < G; g += 2) {
-                        const int co = tile * CoT + c0 + g;
-                        float v0[4], v1[4];
+                for (int g = 0; g < G; ++g) {
+                    float v[T];
 #pragma unroll
-                        for (int p = 0; p < 4; ++p) { v0[p] = __uint_as_float(in[p][g]); v1[p] = __uint_as_float(in[p][g + 1]); }
-                        if (prm.bias != nullptr) {
-                            if (co < prm.Cout) v0[0] += __ldg(prm.bias + co);
-                            if (co + 1 < prm.Cout) v1[0] += __ldg(prm.bias + co + 1);
-                        }
-                        rdft_inverse<4>(v0);
-                        rdft_inverse<4>(v1);
-                        if (co + 1 < prm.Cout) {
-                            ptx::st_global_v4(orow + (int64_t)co * 4, pack_h2(v0[0], v0[1]), pack_h2(v0[2], v0[3]),
-                                              pack_h2(v1[0], v1[1]), pack_h2(v1[2], v1[3]));
-                        } else if (co < prm.Cout) {
-                            *reinterpret_cast<uint2*>(orow + (int64_t)co * 4) =
-                                make_uint2(pack_h2(v0[0], v0[1]), pack_h2(v0[2], v0[3]));
-                        }
+                    for (int p = 0; p < T; ++p) v[p] = __uint_as_float(in[p][g]);
+                    if (prm.bias != nullptr && co0 + g < prm.Cout) v[0] += __ldg(prm.bias + co0 + g);
+                    rdft_inverse<T>(v);
+#pragma unroll
+                    for (int t = 0; t < T; t += 2) o[(g * T + t) / 2] = pack_h2(v[t], v[t + 1]);
+                }
+                __half* dst = orow + (int64_t)co0 * T;
+                if (co0 + G <= prm.Cout) {
+                    if (vec32) {
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) ptx::st_global_v8(dst + i * 16, &o[i * 8]);
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) ptx::st_global_v4(dst + i * 8, o[4 * i], o[4 * i + 1], o[4 * i + 2], o[4 * i + 3]);
                     }
-                } else {
+                } else {                                         // ragged channel tail: one channel at a time
 #pragma unroll
                     for (int g = 0; g < G; ++g) {
-                        const int co = tile * CoT + c0 + g;
-                        if (co >= prm.Cout) continue;
-                        float v[T];
+                        if (co0 + g >= prm.Cout) continue;
+                        if constexpr (T == 4) {
+                            *reinterpret_cast<uint2*>(dst + g * 4) = make_uint2(o[2 * g], o[2 * g + 1]);
+                        } else {
 #pragma unroll
-                        for (int p = 0; p < T; ++p) v[p] = __uint_as_float(in[p][g]);
-                        if (prm.bias != nullptr) v[0] += __ldg(prm.bias + co);
-                        rdft_inverse<T>(v);
-                        __half* dst = orow + (int64_t)co * T;
-#pragma unroll
-                        for (int t = 0; t < T; t += 8)
-                            ptx::st_global_v4(dst + t, pack_h2(v[t], v[t + 1]), pack_h2(v[t + 2], v[t + 3]),
-                                              pack_h2(v[t + 4], v[t + 5]), pack_h2(v[t + 6], v[t + 7]));
+                            for (int t = 0; t < T; t += 8)
+                                ptx::st_global_v4(dst + g * T + t, o[(g * T + t) / 2], o[(g * T + t) / 2 + 1],
+                                                  o[(g * T + t) / 2 + 2], o[(g * T + t) / 2 + 3]);
+                        }
                     }
                 }
+            }
+            if (third >= ngroups) {                              // fewer column groups than shares: nothing to read
+                ptx::tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(&bar->empty_d);
             }
         }
     }

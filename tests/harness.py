@@ -42,6 +42,11 @@ class GpuLayer:
         self.plan = eq.eqlinear_plan(T, Ci, Co, eql_dtype(dtype), self.w, self.bias, self.ws, self.ws_bytes,
                                      flags, self.stream)
 
+    def raw_status(self) -> int:
+        """The plan's device status word (0 = ok, else the code of the wait that gave up)."""
+        torch.cuda.synchronize(self.dev)
+        return int(self.ws[:4].view(torch.int32).item())
+
     def close(self):
         if self.plan:
             torch.cuda.synchronize(self.dev)
