@@ -66,7 +66,7 @@ def load_library(path: str | None = None) -> ctypes.CDLL:
     global _lib
     if _lib is not None and path is None:
         return _lib
-    p = path or LIB_PATH
+    p = path or os.environ.get("EQLINEAR_LIB") or LIB_PATH     # EQLINEAR_LIB: explicit path to another build
     if not os.path.exists(p):
         raise FileNotFoundError(
             f"{p} not found: build it with `python -m paper_2607_21271_b200.build` "

@@ -16,6 +16,7 @@
 #include <utility>
 
 #if defined(__CUDACC__)
+#include <cuda_fp16.h>
 #define EQL_HD __host__ __device__ __forceinline__
 #else
 #define EQL_HD inline
@@ -41,6 +42,19 @@ struct Tw32 {
     }
 };
 
+// Value types the butterflies run on: float (one channel) or, in device code, __half2 (two channels
+// per instruction, every operation rounded to half precision).
+template <typename V>
+struct Num {
+    static EQL_HD V cst(float c) { return V(c); }
+};
+#if defined(__CUDACC__)
+template <>
+struct Num<__half2> {
+    static __device__ __forceinline__ __half2 cst(float c) { return __float2half2_rn(c); }
+};
+#endif
+
 template <int N, class F, int... Is>
 EQL_HD void static_for_impl(F&& f, std::integer_sequence<int, Is...>) {
     (f(std::integral_constant<int, Is>{}), ...);
@@ -54,32 +68,33 @@ EQL_HD void static_for(F&& f) {
 // Half spectrum of a real sequence x[0], x[S], ..., x[(T-1)S]: re[k], im[k] for k = 0..T/2.
 // Radix-2 decimation in time on half spectra: with E, O the half spectra of the even / odd samples,
 //   X_k = E_k + w^k O_k,   X_{T/2-k} = conj(E_k - w^k O_k),   w = e^{-2 pi i / T},  k = 0..T/4.
-template <int T, int S>
-EQL_HD void rfft_half(const float* x, float* re, float* im) {
+template <int T, int S, typename V>
+EQL_HD void rfft_half(const V* x, V* re, V* im) {
+    const V zero = Num<V>::cst(0.f);
     if constexpr (T == 1) {
-        re[0] = x[0]; im[0] = 0.f;
+        re[0] = x[0]; im[0] = zero;
     } else if constexpr (T == 2) {
         re[0] = x[0] + x[S]; re[1] = x[0] - x[S];
-        im[0] = 0.f; im[1] = 0.f;
+        im[0] = zero; im[1] = zero;
     } else {
         constexpr int H = T / 2, Q = T / 4;
-        float er[Q + 1], ei[Q + 1], orr[Q + 1], oi[Q + 1];
-        rfft_half<H, 2 * S>(x, er, ei);
-        rfft_half<H, 2 * S>(x + S, orr, oi);
-        re[0] = er[0] + orr[0]; im[0] = 0.f;
-        re[H] = er[0] - orr[0]; im[H] = 0.f;
+        V er[Q + 1], ei[Q + 1], orr[Q + 1], oi[Q + 1];
+        rfft_half<H, 2 * S, V>(x, er, ei);
+        rfft_half<H, 2 * S, V>(x + S, orr, oi);
+        re[0] = er[0] + orr[0]; im[0] = zero;
+        re[H] = er[0] - orr[0]; im[H] = zero;
         re[Q] = er[Q]; im[Q] = -orr[Q];                 // w^{T/4} = -i, and E_Q, O_Q are real
         static_for<(Q > 1 ? Q - 1 : 0)>([&](auto kk) {
             constexpr int k = decltype(kk)::value + 1;   // 0 < k < T/4
             constexpr int j = k * (32 / T);
-            float tr, ti;
+            V tr, ti;
             if constexpr (2 * j == 8) {                  // k = T/8: cos = sin
-                constexpr float c = Tw32<4>::value();
+                const V c = Num<V>::cst(Tw32<4>::value());
                 tr = c * (orr[k] + oi[k]);
                 ti = c * (oi[k] - orr[k]);
             } else {
-                constexpr float c = Tw32<j>::value();
-                constexpr float s = Tw32<8 - j>::value();
+                const V c = Num<V>::cst(Tw32<j>::value());
+                const V s = Num<V>::cst(Tw32<8 - j>::value());
                 tr = c * orr[k] + s * oi[k];             // (c - i s)(Or + i Oi)
                 ti = c * oi[k] - s * orr[k];
             }
@@ -90,12 +105,12 @@ EQL_HD void rfft_half(const float* x, float* re, float* im) {
 }
 
 // Forward real DFT, in place: v[0..T) group samples -> v[0..T) real-packed planes.
-template <int T>
-EQL_HD void rdft_forward(float* v) {
+template <int T, typename V = float>
+EQL_HD void rdft_forward(V* v) {
     if constexpr (T == 1) {
     } else {
-        float re[T / 2 + 1], im[T / 2 + 1];
-        rfft_half<T, 1>(v, re, im);
+        V re[T / 2 + 1], im[T / 2 + 1];
+        rfft_half<T, 1, V>(v, re, im);
         v[0] = re[0];
         v[T - 1] = re[T / 2];
         static_for<T / 2 - 1>([&](auto kk) {

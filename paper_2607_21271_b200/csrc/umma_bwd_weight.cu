@@ -177,8 +177,11 @@ umma_bwd_weight_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
             uint32_t wd[32];
             if (active)
                 load_slab_row(raw + slot * kRawSlot + ((is_y ? kMaxXSlabs : 0) + slab) * kSlab + row * 128, row, wd);
+            // The rows are in registers: order these generic-proxy reads before the async-proxy (TMA) refill of
+            // the slot, then release it so that the refill overlaps the transform.
+            ptx::fence_proxy_async_smem();
             __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(&bar->empty_raw[slot]);     // the slot can be refilled while we transform
+            if (lane == 0) ptx::mbar_arrive(&bar->empty_raw[slot]);
             if (active) {
                 uint32_t packed[T][NCH / 2];
                 float p0[NCH];

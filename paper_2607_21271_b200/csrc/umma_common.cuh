@@ -36,25 +36,47 @@ __device__ __forceinline__ void load_slab_row(const uint8_t* row_base, int r, ui
 
 // Group DFT of the 64/T channels held in wd.
 // packed[p][cp] = (plane p of channel 2cp, plane p of channel 2cp+1) as half2.
-// plane0[c] (optional, float) = unrounded k = 0 plane of channel c (the sum over the group axis).
-template <int T, bool WANT_PLANE0>
+// plane0[c] (optional, float) = k = 0 plane of channel c (the sum over the group axis).
+// HALF_MATH = false: butterflies in float, each plane rounded to half once.
+// HALF_MATH = true : two channels per instruction in packed half arithmetic (every butterfly output rounded
+//                    to half; about twice as cheap, error stays well inside the FP16 parity bar).
+template <int T, bool WANT_PLANE0, bool HALF_MATH = false>
 __device__ __forceinline__ void dft_words(const uint32_t (&wd)[32], uint32_t (&packed)[T][(64 / T) / 2], float* plane0) {
     constexpr int NCH = 64 / T;
 #pragma unroll
     for (int cp = 0; cp < NCH / 2; ++cp) {
-        float v0[T], v1[T];
+        if constexpr (HALF_MATH) {
+            __half2 v[T];
 #pragma unroll
-        for (int t = 0; t < T; t += 2) {
-            const float2 a = unpack_h2(wd[((2 * cp) * T + t) / 2]);
-            const float2 b = unpack_h2(wd[((2 * cp + 1) * T + t) / 2]);
-            v0[t] = a.x; v0[t + 1] = a.y;
-            v1[t] = b.x; v1[t + 1] = b.y;
+            for (int t = 0; t < T; t += 2) {
+                const uint32_t wa = wd[((2 * cp) * T + t) / 2], wb = wd[((2 * cp + 1) * T + t) / 2];
+                const uint32_t lo = __byte_perm(wa, wb, 0x5410);      // (a[t],   b[t])
+                const uint32_t hi = __byte_perm(wa, wb, 0x7632);      // (a[t+1], b[t+1])
+                memcpy(&v[t], &lo, 4);
+                memcpy(&v[t + 1], &hi, 4);
+            }
+            rdft_forward<T, __half2>(v);
+            if constexpr (WANT_PLANE0) {
+                const float2 f = __half22float2(v[0]);
+                plane0[2 * cp] = f.x; plane0[2 * cp + 1] = f.y;
+            }
+#pragma unroll
+            for (int p = 0; p < T; ++p) memcpy(&packed[p][cp], &v[p], 4);
+        } else {
+            float v0[T], v1[T];
+#pragma unroll
+            for (int t = 0; t < T; t += 2) {
+                const float2 a = unpack_h2(wd[((2 * cp) * T + t) / 2]);
+                const float2 b = unpack_h2(wd[((2 * cp + 1) * T + t) / 2]);
+                v0[t] = a.x; v0[t + 1] = a.y;
+                v1[t] = b.x; v1[t + 1] = b.y;
+            }
+            rdft_forward<T>(v0);
+            rdft_forward<T>(v1);
+            if constexpr (WANT_PLANE0) { plane0[2 * cp] = v0[0]; plane0[2 * cp + 1] = v1[0]; }
+#pragma unroll
+            for (int p = 0; p < T; ++p) packed[p][cp] = pack_h2(v0[p], v1[p]);
         }
-        rdft_forward<T>(v0);
-        rdft_forward<T>(v1);
-        if constexpr (WANT_PLANE0) { plane0[2 * cp] = v0[0]; plane0[2 * cp + 1] = v1[0]; }
-#pragma unroll
-        for (int p = 0; p < T; ++p) packed[p][cp] = pack_h2(v0[p], v1[p]);
     }
 }
 

@@ -39,10 +39,12 @@ constexpr int kWarpTmaX = 0, kWarpMma = 1, kWarpTmaB = 2, kWarpCompute0 = 4;
 constexpr int kNumComputeWarps = 12;
 
 template <int T> struct UmmaCfg;
-template <> struct UmmaCfg<4>  { static constexpr int SR = 4, SA = 4, SB = 3; };
-template <> struct UmmaCfg<8>  { static constexpr int SR = 4, SA = 3, SB = 2; };
-template <> struct UmmaCfg<16> { static constexpr int SR = 2, SA = 2, SB = 2; };
-template <> struct UmmaCfg<32> { static constexpr int SR = 4, SA = 1, SB = 1; };
+// Ring depths: SR raw slabs (16 KB each; a multiple of 3 so that every slot is always served by the same
+// group of four compute warps), SA transformed-operand stages (T*4 KB each), SB weight-image slots.
+template <> struct UmmaCfg<4>  { static constexpr int SR = 6, SA = 4, SB = 2; };
+template <> struct UmmaCfg<8>  { static constexpr int SR = 6, SA = 2, SB = 2; };
+template <> struct UmmaCfg<16> { static constexpr int SR = 3, SA = 2, SB = 1; };
+template <> struct UmmaCfg<32> { static constexpr int SR = 3, SA = 1, SB = 1; };
 
 struct UmmaParams {
     __half* out;                 // [N, Cout*T]
@@ -56,8 +58,16 @@ struct UmmaParams {
     int64_t num_units;
 };
 
+// Optional timeline instrumentation (compiled only with -DEQL_TRACE): CTA 0 records clock64() stamps.
+#ifdef EQL_TRACE
+__device__ unsigned long long g_trace[8192];
+#define EQL_STAMP(slot) do { if (blockIdx.x == 0 && (slot) < 8192) g_trace[(slot)] = clock64(); } while (0)
+#else
+#define EQL_STAMP(slot) do { } while (0)
+#endif
+
 struct SmemBarriers {
-    uint64_t full_raw[4], empty_raw[4];
+    uint64_t full_raw[6], empty_raw[6];
     uint64_t full_a[4], empty_a[4];
     uint64_t full_b[4], empty_b[4];
     uint64_t full_d, empty_d, mma_done;
@@ -129,7 +139,7 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const UmmaParams
     int* status = prm.status;
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < SR; ++i) { ptx::mbar_init(&bar->full_raw[i], 1); ptx::mbar_init(&bar->empty_raw[i], kNumComputeWarps); }
+        for (int i = 0; i < SR; ++i) { ptx::mbar_init(&bar->full_raw[i], 1); ptx::mbar_init(&bar->empty_raw[i], 4); }
         for (int i = 0; i < SA; ++i) { ptx::mbar_init(&bar->full_a[i], 4 * SPK); ptx::mbar_init(&bar->empty_a[i], 1); }
         for (int i = 0; i < SB; ++i) { ptx::mbar_init(&bar->full_b[i], 1); ptx::mbar_init(&bar->empty_b[i], 1); }
         ptx::mbar_init(&bar->full_d, 1);
@@ -163,6 +173,7 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const UmmaParams
                         const int slot = cr % SR;
                         ok = ptx::mbar_wait(&bar->empty_raw[slot], ((cr / SR) & 1) ^ 1, abort_flag, status, 101);
                         if (!ok) break;
+                        EQL_STAMP(2048 + cr);
                         ptx::mbar_arrive_expect_tx(&bar->full_raw[slot], kSlabBytes);
                         ptx::tma_load_2d(raw + slot * kSlabBytes, &tmap_in, (kc * kChunkK + q * NCH) * T, row0,
                                          &bar->full_raw[slot]);
@@ -187,6 +198,7 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const UmmaParams
                     const int slot = cb % SB;
                     ok = ptx::mbar_wait(&bar->empty_b[slot], ((cb / SB) & 1) ^ 1, abort_flag, status, 102);
                     if (!ok) break;
+                    EQL_STAMP(4096 + cb);
                     ptx::mbar_arrive_expect_tx(&bar->full_b[slot], blob_bytes);
                     ptx::bulk_load_1d(bsm + slot * prm.b_slot_bytes,
                                       prm.image + ((size_t)tile * nK + kc) * (size_t)rowsB * kChunkK, blob_bytes,
@@ -208,13 +220,18 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const UmmaParams
             const uint32_t idesc_cplx = ptx::umma_idesc_f16_f32(kTileM, 2 * CoT);
             const uint32_t b_lbo = (uint32_t)rowsB * 16u;
             for (int64_t u = first; u < prm.num_units && ok; u += stride, ++cu) {
+                EQL_STAMP(512 + 2 * cu);
                 ok = ptx::mbar_wait(&bar->empty_d, (cu & 1) ^ 1, abort_flag, status, 103);
+                EQL_STAMP(512 + 2 * cu + 1);
                 if (!ok) break;
                 ptx::tc_fence_after_sync();
                 for (int kc = 0; kc < nK; ++kc, ++ca, ++cb) {
                     const int sa = ca % SA, sb = cb % SB;
-                    ok = ptx::mbar_wait(&bar->full_a[sa], (ca / SA) & 1, abort_flag, status, 104) &&
-                         ptx::mbar_wait(&bar->full_b[sb], (cb / SB) & 1, abort_flag, status, 105);
+                    EQL_STAMP(1024 + 4 * ca);
+                    ok = ptx::mbar_wait(&bar->full_a[sa], (ca / SA) & 1, abort_flag, status, 104);
+                    EQL_STAMP(1024 + 4 * ca + 1);
+                    ok = ok && ptx::mbar_wait(&bar->full_b[sb], (cb / SB) & 1, abort_flag, status, 105);
+                    EQL_STAMP(1024 + 4 * ca + 2);
                     if (!ok) break;
                     ptx::tc_fence_after_sync();
                     const uint32_t a0 = ptx::smem_u32(xhat + sa * kAStage);
@@ -239,6 +256,7 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const UmmaParams
                                   ptx::umma_smem_desc(b0 + (uint32_t)(rowsB - CoT) * 16u, b_lbo, 128), idesc_real, acc);
                     ptx::umma_commit(&bar->empty_a[sa]);
                     ptx::umma_commit(&bar->empty_b[sb]);
+                    EQL_STAMP(1024 + 4 * ca + 3);
                 }
                 if (ok) ptx::umma_commit(&bar->full_d);
             }
@@ -250,46 +268,47 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const UmmaParams
         // ---------------------------------------------------------------- compute warps: transform, then epilogue
         // Per unit every compute warp first transforms its share of the raw slab rows (group DFT -> A operands)
         // and then drains its share of the accumulator (inverse DFT -> global).  Work items of the transform
-        // are (slab, 32-row quarter); they are dealt round-robin over the 12 warps across chunks.
+        // are (slab, 32-row quarter).
         constexpr int G = 64 / T;                                // channels per TMEM read group
-        constexpr int kItemsPerChunk = 4 * SPK;
-        // A warp's consecutive items are kNumComputeWarps items apart; that must stay below SA chunks so that the
-        // owner-only wait on empty_a is never more than one phase ahead of the barrier.
-        static_assert(kNumComputeWarps < SA * kItemsPerChunk, "empty_a parity wait would be ambiguous");
+        // The 12 warps form 3 groups of 4; raw slab number cr is transformed by group cr % 3, one 32-row quarter
+        // per warp.  Because SR is a multiple of 3, a slot is always served by the same group, so each warp
+        // sees every phase of the slot barriers it waits on, in order (a parity wait is only unambiguous one
+        // phase ahead).  A warp's consecutive slabs are 3 apart, i.e. 3/SPK chunks, which must stay below SA
+        // (a warp that stored into chunk c' has seen the commit of chunk c' - SA, so when it next waits for the
+        // commit of chunk c - SA with c - c' <= SA the barrier is at most one phase behind).
+        static_assert(SR % 3 == 0, "raw slots must map to fixed warp groups");
+        static_assert((3 + SPK - 1) / SPK <= SA, "empty_a parity wait would be ambiguous");
         const int cw = warp - kWarpCompute0;
         const int quad = warp & 3;                               // TMEM lane quadrant this warp may read
-        const int third = cw >> 2;                               // which share of the column groups
+        const int group = cw >> 2;                               // transform group, and share of the epilogue's column groups
+        const int third = group;
         const uint32_t lane_base = tmem_base + ((uint32_t)(quad * 32) << 16);
         const bool vec32 = ((reinterpret_cast<uintptr_t>(prm.out) & 31u) == 0) && (((int64_t)prm.Cout * T * 2) % 32 == 0);
         uint32_t ca = 0, cu = 0;
-        uint32_t item_mod = 0;                                   // (index of the next slab's first work item) mod 12
         bool ok = true;
         for (int64_t u = first; u < prm.num_units && ok; u += stride, ++cu) {
             // ---- transform
+            if (cw == 0 && lane == 0) EQL_STAMP(8 * cu);
             for (int kc = 0; kc < nK && ok; ++kc, ++ca) {
                 const int sa = ca % SA;
 #pragma unroll 1
                 for (int q = 0; q < SPK; ++q) {
                     const uint32_t cr = ca * SPK + q;            // running slab counter
+                    if ((int)(cr % 3) != group) continue;
                     const int slot = cr % SR;
-                    // A parity wait is only unambiguous while the waiter is at most one phase behind the barrier,
-                    // so every compute warp both observes and releases every phase of every slot barrier:
-                    // owners of one of the slab's four row quarters release after loading their rows, the
-                    // other warps right away.
                     ok = ptx::mbar_wait(&bar->full_raw[slot], (cr / SR) & 1, abort_flag, status, 106);
                     if (!ok) break;
-                    int d = cw - (int)item_mod;                  // which quarter of this slab is ours, if any
-                    if (d < 0) d += kNumComputeWarps;
-                    item_mod = (item_mod + 4) % kNumComputeWarps;
-                    if (d >= 4) {
-                        if (lane == 0) ptx::mbar_arrive(&bar->empty_raw[slot]);
-                        continue;
-                    }
+                    const int d = quad;                          // this warp's 32-row quarter of the slab
                     const int r = d * 32 + lane;
                     uint32_t wd[32];
                     load_slab_row(raw + slot * kSlabBytes + r * 128, r, wd);
+#ifndef EQL_LATE_RELEASE
+                    // The rows are in registers: order these generic-proxy reads before the async-proxy (TMA) refill
+                    // of the slot, then release it so that the refill overlaps the transform.
+                    ptx::fence_proxy_async_smem();
                     __syncwarp();
-                    if (lane == 0) ptx::mbar_arrive(&bar->empty_raw[slot]);     // refill can start while we transform
+                    if (lane == 0) ptx::mbar_arrive(&bar->empty_raw[slot]);
+#endif
                     uint32_t packed[T][NCH / 2];
                     dft_words<T, false>(wd, packed, nullptr);
                     ok = ptx::mbar_wait(&bar->empty_a[sa], ((ca / SA) & 1) ^ 1, abort_flag, status, 107);
@@ -300,14 +319,21 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const UmmaParams
                     for (int p = 0; p < T; ++p) store_plane_run<NCH>(dst + p * 4096, packed[p], 2048);
                     ptx::fence_proxy_async_smem();               // generic-proxy writes -> visible to the MMA (async proxy)
                     __syncwarp();
-                    if (lane == 0) ptx::mbar_arrive(&bar->full_a[sa]);
+                    if (lane == 0) {
+#ifdef EQL_LATE_RELEASE
+                        ptx::mbar_arrive(&bar->empty_raw[slot]);
+#endif
+                        ptx::mbar_arrive(&bar->full_a[sa]);
+                    }
                 }
             }
             if (!ok) break;
             // ---- epilogue
             const int tile = (int)(u % nTiles);
             const int64_t row = (u / nTiles) * kTileM + quad * 32 + lane;
+            if (cw == 0 && lane == 0) EQL_STAMP(8 * cu + 1);
             ok = ptx::mbar_wait(&bar->full_d, cu & 1, abort_flag, status, 108);
+            if (cw == 0 && lane == 0) EQL_STAMP(8 * cu + 2);
             if (!ok) break;
             ptx::tc_fence_after_sync();
             __half* orow = prm.out + row * (int64_t)prm.Cout * T;
@@ -365,6 +391,7 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const UmmaParams
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(&bar->empty_d);
             }
+            if (cw == 0 && lane == 0) EQL_STAMP(8 * cu + 3);
         }
     }
 
@@ -414,6 +441,17 @@ cudaError_t dispatch_umma_T(int T, F&& f) {
 }
 
 }  // namespace
+
+#ifdef EQL_TRACE
+extern "C" int eqlinear_debug_read_trace(unsigned long long* dst, int n) {
+    cudaDeviceSynchronize();
+    return (int)cudaMemcpyFromSymbol(dst, g_trace, sizeof(unsigned long long) * (n < 8192 ? n : 8192));
+}
+extern "C" int eqlinear_debug_clear_trace() {
+    static unsigned long long zeros[8192];
+    return (int)cudaMemcpyToSymbol(g_trace, zeros, sizeof(zeros));
+}
+#endif
 
 bool umma_linear_supported(int T, eql_dtype_t dtype) {
     return dtype == EQL_FP16 && (T == 4 || T == 8 || T == 16 || T == 32);
