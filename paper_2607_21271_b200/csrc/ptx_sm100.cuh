@@ -38,13 +38,30 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
     return ok != 0;
 }
 
+// Non-suspending poll of a phase (about 50 cycles); mbarrier.try_wait instead may put the thread to sleep, and
+// waking it after the phase completes costs a few hundred cycles.
+__device__ __forceinline__ bool mbar_test_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+
 // Bounded wait.  Returns false if the barrier did not flip within the poll budget or if another
 // thread of the CTA has already given up (abort flag); on its own time-out it raises the flag and
 // records `code` in the global status word.  With heed_abort = false (used while draining copies and
 // MMAs that are already in flight) only the poll budget ends the wait.  Nothing here traps or spins forever.
 constexpr uint32_t kWaitPolls = 1u << 20;
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status,
-                                          int code, bool heed_abort = true) {
+                                          int code, bool heed_abort = true, uint32_t spin_polls = 0) {
+    // latency-critical single-thread roles first spin without suspending
+    for (uint32_t it = 0; it < spin_polls; ++it)
+        if (mbar_test_wait(bar, parity)) return true;
     for (uint32_t it = 0; it < kWaitPolls; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
         if (heed_abort && (it & 63u) == 63u && *abort_flag != 0) return false;

@@ -39,12 +39,16 @@ constexpr int kWarpTmaX = 0, kWarpMma = 1, kWarpTmaB = 2, kWarpCompute0 = 4;
 constexpr int kNumComputeWarps = 12;
 
 template <int T> struct UmmaCfg;
-// Ring depths: SR raw slabs (16 KB each; a multiple of 3 so that every slot is always served by the same
-// group of four compute warps), SA transformed-operand stages (T*4 KB each), SB weight-image slots.
-template <> struct UmmaCfg<4>  { static constexpr int SR = 6, SA = 4, SB = 2; };
-template <> struct UmmaCfg<8>  { static constexpr int SR = 6, SA = 2, SB = 2; };
-template <> struct UmmaCfg<16> { static constexpr int SR = 3, SA = 2, SB = 1; };
-template <> struct UmmaCfg<32> { static constexpr int SR = 3, SA = 1, SB = 1; };
+// Ring depths.  The raw ring has 3 slots of SPS slabs (16 KB each) that complete on one barrier: a slot hand-off
+// costs several hundred cycles whatever its size, so slots are made fat where shared memory allows.  With 3 slots
+// every slot is always served by the same warp groups (slab number mod 3 selects the group).  SA transformed-operand
+// stages (T*4 KB each), SB weight-image slots.
+template <> struct UmmaCfg<4>  { static constexpr int SPS = 2, SA = 4, SB = 2; };
+template <> struct UmmaCfg<8>  { static constexpr int SPS = 2, SA = 2, SB = 2; };
+template <> struct UmmaCfg<16> { static constexpr int SPS = 1, SA = 2, SB = 1; };
+template <> struct UmmaCfg<32> { static constexpr int SPS = 1, SA = 1, SB = 1; };
+constexpr int kRawSlots = 3;
+constexpr uint32_t kSpin = 256;               // test_wait polls before a single-thread role falls back to try_wait
 
 struct UmmaParams {
     __half* out;                 // [N, Cout*T]
@@ -122,7 +126,8 @@ template <int T>
 __global__ void __launch_bounds__(kThreadsUmma, 1)
 umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const UmmaParams prm) {
     using Cfg = UmmaCfg<T>;
-    constexpr int SR = Cfg::SR, SA = Cfg::SA, SB = Cfg::SB;
+    constexpr int SPS = Cfg::SPS, SA = Cfg::SA, SB = Cfg::SB;
+    constexpr int SR = kRawSlots * SPS;         // slabs in the raw ring
     constexpr int NCH = 64 / T;                 // channels per raw slab row (128 B)
     constexpr int SPK = kChunkK / NCH;          // slabs per 16-channel chunk (= T/4)
     constexpr int kAStage = T * 4096;           // T planes x [128 x 16] halves
@@ -139,7 +144,7 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const UmmaParams
     int* status = prm.status;
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < SR; ++i) { ptx::mbar_init(&bar->full_raw[i], 1); ptx::mbar_init(&bar->empty_raw[i], 4); }
+        for (int i = 0; i < kRawSlots; ++i) { ptx::mbar_init(&bar->full_raw[i], 1); ptx::mbar_init(&bar->empty_raw[i], 4 * SPS); }
         for (int i = 0; i < SA; ++i) { ptx::mbar_init(&bar->full_a[i], 4 * SPK); ptx::mbar_init(&bar->empty_a[i], 1); }
         for (int i = 0; i < SB; ++i) { ptx::mbar_init(&bar->full_b[i], 1); ptx::mbar_init(&bar->empty_b[i], 1); }
         ptx::mbar_init(&bar->full_d, 1);
@@ -164,26 +169,39 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const UmmaParams
     if (warp == kWarpTmaX) {
         // ---------------------------------------------------------------- raw activation rows via TMA
         if (lane == 0) {
-            uint32_t cr = 0;
+            uint32_t cr = 0;                                     // running slab counter; slot phase = cr / SPS
             bool ok = true;
             for (int64_t u = first; u < prm.num_units && ok; u += stride) {
                 const int row0 = (int)(u / nTiles) * kTileM;
                 for (int kc = 0; kc < nK && ok; ++kc) {
                     for (int q = 0; q < SPK; ++q, ++cr) {
-                        const int slot = cr % SR;
-                        ok = ptx::mbar_wait(&bar->empty_raw[slot], ((cr / SR) & 1) ^ 1, abort_flag, status, 101);
-                        if (!ok) break;
-                        EQL_STAMP(2048 + cr);
-                        ptx::mbar_arrive_expect_tx(&bar->full_raw[slot], kSlabBytes);
-                        ptx::tma_load_2d(raw + slot * kSlabBytes, &tmap_in, (kc * kChunkK + q * NCH) * T, row0,
+                        const uint32_t ph = cr / SPS;            // slot phase counter
+                        const int slot = ph % kRawSlots;
+                        if (cr % SPS == 0) {
+                            ok = ptx::mbar_wait(&bar->empty_raw[slot], ((ph / kRawSlots) & 1) ^ 1, abort_flag, status, 101, true, kSpin);
+                            if (!ok) break;
+                            EQL_STAMP(2048 + cr);
+                            ptx::mbar_arrive_expect_tx(&bar->full_raw[slot], SPS * kSlabBytes);
+                        }
+                        ptx::tma_load_2d(raw + (slot * SPS + cr % SPS) * kSlabBytes, &tmap_in, (kc * kChunkK + q * NCH) * T, row0,
                                          &bar->full_raw[slot]);
                     }
                 }
             }
-            if (!ok) {   // drain: every copy this thread issued must have landed before the CTA may exit
-                const uint32_t lo = cr > (uint32_t)SR ? cr - SR : 0;
-                for (uint32_t c = lo; c < cr; ++c)
-                    ptx::mbar_wait(&bar->full_raw[c % SR], (c / SR) & 1, abort_flag, status, 111, false);
+            // A slot phase must receive all SPS loads it was armed for, also at the very end of the work.
+            if (ok) {
+                while (cr % SPS != 0) {
+                    const uint32_t ph = cr / SPS;
+                    ptx::tma_load_2d(raw + ((ph % kRawSlots) * SPS + cr % SPS) * kSlabBytes, &tmap_in, 0, 0, &bar->full_raw[ph % kRawSlots]);
+                    ++cr;
+                }
+            }
+            // drain: every copy this thread issued must have landed before the CTA may exit
+            {
+                const uint32_t nph = (cr + SPS - 1) / SPS;
+                const uint32_t lo = nph > (uint32_t)kRawSlots ? nph - kRawSlots : 0;
+                for (uint32_t c = lo; c < nph; ++c)
+                    ptx::mbar_wait(&bar->full_raw[c % kRawSlots], (c / kRawSlots) & 1, abort_flag, status, 111, false);
             }
         }
     } else if (warp == kWarpTmaB) {
@@ -196,7 +214,7 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const UmmaParams
                 const int tile = (int)(u % nTiles);
                 for (int kc = 0; kc < nK; ++kc, ++cb) {
                     const int slot = cb % SB;
-                    ok = ptx::mbar_wait(&bar->empty_b[slot], ((cb / SB) & 1) ^ 1, abort_flag, status, 102);
+                    ok = ptx::mbar_wait(&bar->empty_b[slot], ((cb / SB) & 1) ^ 1, abort_flag, status, 102, true, kSpin);
                     if (!ok) break;
                     EQL_STAMP(4096 + cb);
                     ptx::mbar_arrive_expect_tx(&bar->full_b[slot], blob_bytes);
@@ -221,16 +239,16 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const UmmaParams
             const uint32_t b_lbo = (uint32_t)rowsB * 16u;
             for (int64_t u = first; u < prm.num_units && ok; u += stride, ++cu) {
                 EQL_STAMP(512 + 2 * cu);
-                ok = ptx::mbar_wait(&bar->empty_d, (cu & 1) ^ 1, abort_flag, status, 103);
+                ok = ptx::mbar_wait(&bar->empty_d, (cu & 1) ^ 1, abort_flag, status, 103, true, kSpin);
                 EQL_STAMP(512 + 2 * cu + 1);
                 if (!ok) break;
                 ptx::tc_fence_after_sync();
                 for (int kc = 0; kc < nK; ++kc, ++ca, ++cb) {
                     const int sa = ca % SA, sb = cb % SB;
                     EQL_STAMP(1024 + 4 * ca);
-                    ok = ptx::mbar_wait(&bar->full_a[sa], (ca / SA) & 1, abort_flag, status, 104);
+                    ok = ptx::mbar_wait(&bar->full_a[sa], (ca / SA) & 1, abort_flag, status, 104, true, kSpin);
                     EQL_STAMP(1024 + 4 * ca + 1);
-                    ok = ok && ptx::mbar_wait(&bar->full_b[sb], (cb / SB) & 1, abort_flag, status, 105);
+                    ok = ok && ptx::mbar_wait(&bar->full_b[sb], (cb / SB) & 1, abort_flag, status, 105, true, kSpin);
                     EQL_STAMP(1024 + 4 * ca + 2);
                     if (!ok) break;
                     ptx::tc_fence_after_sync();
@@ -271,12 +289,12 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const UmmaParams
         // are (slab, 32-row quarter).
         constexpr int G = 64 / T;                                // channels per TMEM read group
         // The 12 warps form 3 groups of 4; raw slab number cr is transformed by group cr % 3, one 32-row quarter
-        // per warp.  Because SR is a multiple of 3, a slot is always served by the same group, so each warp
+        // per warp.  Because the ring has 3 slots, a slot is always served by the same groups, so each warp
         // sees every phase of the slot barriers it waits on, in order (a parity wait is only unambiguous one
         // phase ahead).  A warp's consecutive slabs are 3 apart, i.e. 3/SPK chunks, which must stay below SA
         // (a warp that stored into chunk c' has seen the commit of chunk c' - SA, so when it next waits for the
         // commit of chunk c - SA with c - c' <= SA the barrier is at most one phase behind).
-        static_assert(SR % 3 == 0, "raw slots must map to fixed warp groups");
+        static_assert(kRawSlots == 3 && SPS <= 3, "raw slots must map to fixed warp groups");
         static_assert((3 + SPK - 1) / SPK <= SA, "empty_a parity wait would be ambiguous");
         const int cw = warp - kWarpCompute0;
         const int quad = warp & 3;                               // TMEM lane quadrant this warp may read
@@ -295,13 +313,14 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const UmmaParams
                 for (int q = 0; q < SPK; ++q) {
                     const uint32_t cr = ca * SPK + q;            // running slab counter
                     if ((int)(cr % 3) != group) continue;
-                    const int slot = cr % SR;
-                    ok = ptx::mbar_wait(&bar->full_raw[slot], (cr / SR) & 1, abort_flag, status, 106);
+                    const uint32_t ph = cr / SPS;                // raw-ring slot phase this slab arrives in
+                    const int slot = ph % kRawSlots;
+                    ok = ptx::mbar_wait(&bar->full_raw[slot], (ph / kRawSlots) & 1, abort_flag, status, 106, true, 16);
                     if (!ok) break;
                     const int d = quad;                          // this warp's 32-row quarter of the slab
                     const int r = d * 32 + lane;
                     uint32_t wd[32];
-                    load_slab_row(raw + slot * kSlabBytes + r * 128, r, wd);
+                    load_slab_row(raw + (slot * SPS + cr % SPS) * kSlabBytes + r * 128, r, wd);
 #ifndef EQL_LATE_RELEASE
                     // The rows are in registers: order these generic-proxy reads before the async-proxy (TMA) refill
                     // of the slot, then release it so that the refill overlaps the transform.
@@ -311,7 +330,7 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const UmmaParams
 #endif
                     uint32_t packed[T][NCH / 2];
                     dft_words<T, false>(wd, packed, nullptr);
-                    ok = ptx::mbar_wait(&bar->empty_a[sa], ((ca / SA) & 1) ^ 1, abort_flag, status, 107);
+                    ok = ptx::mbar_wait(&bar->empty_a[sa], ((ca / SA) & 1) ^ 1, abort_flag, status, 107, true, 16);
                     if (!ok) break;
                     const int kfirst = q * NCH;                  // first k of this slab inside the 16-channel chunk
                     uint8_t* dst = xhat + sa * kAStage + r * 16 + (kfirst >> 3) * 2048 + (kfirst & 7) * 2;
@@ -332,7 +351,7 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const UmmaParams
             const int tile = (int)(u % nTiles);
             const int64_t row = (u / nTiles) * kTileM + quad * 32 + lane;
             if (cw == 0 && lane == 0) EQL_STAMP(8 * cu + 1);
-            ok = ptx::mbar_wait(&bar->full_d, cu & 1, abort_flag, status, 108);
+            ok = ptx::mbar_wait(&bar->full_d, cu & 1, abort_flag, status, 108, true, 16);
             if (cw == 0 && lane == 0) EQL_STAMP(8 * cu + 2);
             if (!ok) break;
             ptx::tc_fence_after_sync();
@@ -425,7 +444,7 @@ EncodeTiledFn encode_tiled_fn() {
 template <int T>
 size_t umma_smem_bytes(int b_slot_bytes) {
     using Cfg = UmmaCfg<T>;
-    return 1024 + (size_t)Cfg::SR * kSlabBytes + (size_t)Cfg::SA * T * 4096 + (size_t)Cfg::SB * b_slot_bytes +
+    return 1024 + (size_t)kRawSlots * Cfg::SPS * kSlabBytes + (size_t)Cfg::SA * T * 4096 + (size_t)Cfg::SB * b_slot_bytes +
            sizeof(SmemBarriers) + 64;
 }
 
