@@ -45,6 +45,7 @@ struct BwParams {
     int splits;
     int64_t chunks_per_split;    // 16-token chunks per token range
     int xhat_bytes, stage_bytes;
+    int x3d, y3d;                // tensor maps are 3-D (64 elements, rows, slab index): one load per chunk and tensor
 };
 
 struct BwBarriers {
@@ -113,11 +114,21 @@ umma_bwd_weight_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
                 ptx::mbar_arrive_expect_tx(&bar->full_raw[slot], bytes);
                 const int row = (int)((chunk0 + c) * kChunkTok);
                 uint8_t* dst = raw + slot * kRawSlot;
-                for (int s = 0; s < prm.nXs; ++s)
-                    ptx::tma_load_2d(dst + s * kSlab, &tmap_x, ci_tile * CiT * T + s * 64, row, &bar->full_raw[slot]);
-                for (int s = 0; s < prm.nYs; ++s)
-                    ptx::tma_load_2d(dst + (kMaxXSlabs + s) * kSlab, &tmap_dy, co_tile * CoT * T + s * 64, row,
-                                     &bar->full_raw[slot]);
+                // One 3-D box [slab][16 rows][64 elements] per tensor where the row length is a whole number of
+                // slabs; otherwise one 2-D box per slab (the same shared-memory layout either way).
+                if (prm.x3d) {
+                    ptx::tma_load_3d(dst, &tmap_x, 0, row, ci_tile * CiT * T / 64, &bar->full_raw[slot]);
+                } else {
+                    for (int s = 0; s < prm.nXs; ++s)
+                        ptx::tma_load_2d(dst + s * kSlab, &tmap_x, ci_tile * CiT * T + s * 64, row, &bar->full_raw[slot]);
+                }
+                if (prm.y3d) {
+                    ptx::tma_load_3d(dst + kMaxXSlabs * kSlab, &tmap_dy, 0, row, co_tile * CoT * T / 64, &bar->full_raw[slot]);
+                } else {
+                    for (int s = 0; s < prm.nYs; ++s)
+                        ptx::tma_load_2d(dst + (kMaxXSlabs + s) * kSlab, &tmap_dy, co_tile * CoT * T + s * 64, row,
+                                         &bar->full_raw[slot]);
+                }
             }
             if (!ok) {
                 const int64_t lo = c > kRawSlots ? c - kRawSlots : 0;
@@ -294,6 +305,19 @@ bool encode_rows16(EncodeTiledFn enc, CUtensorMap* map, const void* base, int64_
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// 3-D view of a [rows, cols] half tensor whose row length is a multiple of 64 elements:
+// dim0 = 64 contiguous elements, dim1 = rows (stride = row pitch), dim2 = slab index (stride = 128 bytes).
+// A box [64, 16, nslabs] lands in shared memory as nslabs consecutive [16 x 128 B] slabs.
+bool encode_slabs3d(EncodeTiledFn enc, CUtensorMap* map, const void* base, int64_t cols, int64_t rows, int nslabs) {
+    const cuuint64_t gdim[3] = {64, (cuuint64_t)rows, (cuuint64_t)(cols / 64)};
+    const cuuint64_t gstr[2] = {(cuuint64_t)cols * sizeof(__half), 128};
+    const cuuint32_t box[3] = {64, (cuuint32_t)kChunkTok, (cuuint32_t)nslabs};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, const_cast<void*>(base), gdim, gstr, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 int balanced_tile(int C, int max_tile, int round) {
     const int n = (C + max_tile - 1) / max_tile;
     const int per = (C + n - 1) / n;
@@ -333,9 +357,13 @@ cudaError_t launch_umma_bwd_weight(const UmmaBwdWeightShape& s, const void* x, c
     EncodeTiledFn enc = encode_fn();
     if (enc == nullptr) return cudaErrorNotSupported;
     CUtensorMap mx, my;
-    if (!encode_rows16(enc, &mx, x, (int64_t)s.Ci * s.T, N) || !encode_rows16(enc, &my, dy, (int64_t)s.Co * s.T, N))
-        return cudaErrorInvalidValue;
+    const int64_t xcols = (int64_t)s.Ci * s.T, ycols = (int64_t)s.Co * s.T;
+    const bool x3d = (xcols % 64 == 0) && encode_slabs3d(enc, &mx, x, xcols, N, s.nXs);
+    const bool y3d = (ycols % 64 == 0) && encode_slabs3d(enc, &my, dy, ycols, N, s.nYs);
+    if (!x3d && !encode_rows16(enc, &mx, x, xcols, N)) return cudaErrorInvalidValue;
+    if (!y3d && !encode_rows16(enc, &my, dy, ycols, N)) return cudaErrorInvalidValue;
     BwParams prm{};
+    prm.x3d = x3d; prm.y3d = y3d;
     prm.part = scratch;
     prm.db_part = scratch + (size_t)s.splits * s.T * s.Co * s.Ci;
     prm.status = status;

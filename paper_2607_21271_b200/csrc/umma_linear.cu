@@ -315,8 +315,16 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const UmmaParams
                     if ((int)(cr % 3) != group) continue;
                     const uint32_t ph = cr / SPS;                // raw-ring slot phase this slab arrives in
                     const int slot = ph % kRawSlots;
+#ifdef EQL_TRACE
+                    const bool tr = (cw == 0 && lane == 0);
+                    const int tb = 6000 + 8 * (int)(cr / 3);
+                    if (tr) EQL_STAMP(tb);
+#endif
                     ok = ptx::mbar_wait(&bar->full_raw[slot], (ph / kRawSlots) & 1, abort_flag, status, 106, true, 16);
                     if (!ok) break;
+#ifdef EQL_TRACE
+                    if (tr) EQL_STAMP(tb + 1);
+#endif
                     const int d = quad;                          // this warp's 32-row quarter of the slab
                     const int r = d * 32 + lane;
                     uint32_t wd[32];
@@ -328,10 +336,19 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const UmmaParams
                     __syncwarp();
                     if (lane == 0) ptx::mbar_arrive(&bar->empty_raw[slot]);
 #endif
+#ifdef EQL_TRACE
+                    if (tr) EQL_STAMP(tb + 2);
+#endif
                     uint32_t packed[T][NCH / 2];
                     dft_words<T, false>(wd, packed, nullptr);
+#ifdef EQL_TRACE
+                    if (tr) { if (packed[0][0] == 0x12345678u) EQL_STAMP(tb + 7); EQL_STAMP(tb + 3); }
+#endif
                     ok = ptx::mbar_wait(&bar->empty_a[sa], ((ca / SA) & 1) ^ 1, abort_flag, status, 107, true, 16);
                     if (!ok) break;
+#ifdef EQL_TRACE
+                    if (tr) EQL_STAMP(tb + 4);
+#endif
                     const int kfirst = q * NCH;                  // first k of this slab inside the 16-channel chunk
                     uint8_t* dst = xhat + sa * kAStage + r * 16 + (kfirst >> 3) * 2048 + (kfirst & 7) * 2;
 #pragma unroll
@@ -344,6 +361,9 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const UmmaParams
 #endif
                         ptx::mbar_arrive(&bar->full_a[sa]);
                     }
+#ifdef EQL_TRACE
+                    if (tr) EQL_STAMP(tb + 5);
+#endif
                 }
             }
             if (!ok) break;
@@ -359,10 +379,18 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const UmmaParams
             const int ngroups = CoT / G;
             for (int gi = third; gi < ngroups; gi += 3) {
                 const int c0 = gi * G;
+#ifdef EQL_TRACE
+                const bool tre = (cw == 0 && lane == 0 && cu < 4);
+                const int te = 7000 + 16 * (int)cu + 4 * (gi / 3);
+                if (tre) EQL_STAMP(te);
+#endif
                 uint32_t in[T][G];
 #pragma unroll
                 for (int p = 0; p < T; ++p) ptx::tmem_ld<G>(lane_base + (uint32_t)(p * CoT + c0), in[p]);
                 ptx::tmem_ld_wait();
+#ifdef EQL_TRACE
+                if (tre) { if (in[0][0] == 0x7fc12345u) EQL_STAMP(te + 3); EQL_STAMP(te + 1); }
+#endif
                 if (gi + 3 >= ngroups) {                         // this warp's last read of the accumulator
                     ptx::tc_fence_before_sync();
                     __syncwarp();
@@ -382,6 +410,9 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const UmmaParams
                     for (int t = 0; t < T; t += 2) o[(g * T + t) / 2] = pack_h2(v[t], v[t + 1]);
                 }
                 __half* dst = orow + (int64_t)co0 * T;
+#ifdef EQL_TRACE
+                if (tre) { if (o[0] == 0x7fc12345u) EQL_STAMP(te + 3); EQL_STAMP(te + 2); }
+#endif
                 if (co0 + G <= prm.Cout) {
                     if (vec32) {
 #pragma unroll
@@ -405,6 +436,9 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const UmmaParams
                     }
                 }
             }
+#ifdef EQL_TRACE
+            if (cw == 0 && lane == 0 && cu < 4) EQL_STAMP(7000 + 16 * (int)cu + 15);
+#endif
             if (third >= ngroups) {                              // fewer column groups than shares: nothing to read
                 ptx::tc_fence_before_sync();
                 __syncwarp();
