@@ -33,9 +33,13 @@ if ROOT not in sys.path:
 FALLBACK_HBM_GBS = 6650.0        # earlier measurement on this machine, used only without MEASURED_PEAKS.json
 FALLBACK_BF16_TFLOPS = 1590.0
 
-# DRAM bytes (read + write) per launch of the dominant kernel from the committed ncu captures
-# under profiles/ (None = not captured for that workload).
-NCU_TRAFFIC_BYTES = {}
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per launch from the committed ncu capture
+# profiles/umma_kernels_fp16_vit_b_fc1.md (None = not captured for that workload / kernel).
+NCU_TRAFFIC_BYTES = {
+    ("vit_b_fc1_fp16", "fwd"): 39.8e6 + 101.1e6,
+    ("vit_b_fc1_fp16", "bwd_data"): 156.3e6 + 17.9e6,
+    ("vit_b_fc1_fp16", "bwd_weight"): 193.7e6 + 3.8e6,
+}
 
 
 def load_peaks():
@@ -179,7 +183,7 @@ def metric_name(wl):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
@@ -321,7 +325,8 @@ def main():
                 "hbm_bound_us": hbm_time * 1e6, "tensor_bound_us": tc_time * 1e6,
                 "per_kernel": {n: {"ms": kern_ms[n], "GBps": alg_bytes[n] / (kern_ms[n] * 1e-3) / 1e9,
                                    "hbm_frac": alg_bytes[n] / (kern_ms[n] * 1e-3) / 1e9 / peaks["hbm_gbs"],
-                                   "tcgen05": bool(kernel_kind[n])} for n in names}}
+                                   "tcgen05": bool(kernel_kind[n]),
+                                   "traffic": NCU_TRAFFIC_BYTES.get((wl.name, n))} for n in names}}
 
     # end to end through the host-buffer C-ABI call: pinned host buffers, copies inside the timed region
     e2e = None
