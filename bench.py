@@ -205,6 +205,7 @@ def main():
     import torch.distributed as dist
 
     import paper_2607_21271_b200 as eq
+    from paper_2607_21271_b200 import parallel
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -265,8 +266,7 @@ def main():
             if events is not None:
                 events[3].record()
             if world > 1:
-                dist.all_reduce(dw)
-                dist.all_reduce(db)
+                parallel.allreduce_weight_grads(dw, db)
 
     def barrier():
         if world > 1:

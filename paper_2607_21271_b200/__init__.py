@@ -1,6 +1,6 @@
 """Flash EQ-Linear hot path for NVIDIA B200 (sm_100a): a C-ABI CUDA library plus this thin binding."""
 
-from . import binding, workloads  # noqa: F401
+from . import binding, parallel, workloads  # noqa: F401
 from .binding import (  # noqa: F401
     EQL_FLAG_CORRELATION, EQL_FLAG_FORCE_SIMT, EQL_FP16, EQL_FP32, EqlError,
     eqlinear_bwd_data, eqlinear_bwd_data_host, eqlinear_bwd_weight, eqlinear_bwd_weight_host,

@@ -1,0 +1,29 @@
+"""Data-parallel plumbing of the EQ-Linear path: token sharding and the one exchange step.
+
+The forward pass and the data gradient are independent per token, so tokens are split over ranks and the
+spectral weight is replicated.  The weight and bias gradients are sums over tokens, so their per-rank
+partial results are summed over ranks (one all-reduce of T*C_out*C_in + C_out floats).  torch.distributed is
+plumbing only; the arithmetic of the layer stays in the CUDA library.
+"""
+
+from __future__ import annotations
+
+
+def shard_tokens(N: int, rank: int, world: int) -> tuple[int, int]:
+    """Contiguous, balanced token range [begin, end) of `rank` out of `world` (sizes differ by at most 1)."""
+    if world < 1 or not 0 <= rank < world or N < 0:
+        raise ValueError("bad shard arguments")
+    base, extra = divmod(N, world)
+    begin = rank * base + min(rank, extra)
+    return begin, begin + base + (1 if rank < extra else 0)
+
+
+def allreduce_weight_grads(dw, db=None, group=None) -> None:
+    """Sum dw (and db) over the ranks of `group`, in place.  No-op without an initialised process group."""
+    import torch.distributed as dist
+
+    if not dist.is_available() or not dist.is_initialized() or dist.get_world_size(group) == 1:
+        return
+    dist.all_reduce(dw, op=dist.ReduceOp.SUM, group=group)
+    if db is not None:
+        dist.all_reduce(db, op=dist.ReduceOp.SUM, group=group)
