@@ -39,14 +39,16 @@ constexpr int kWarpTmaX = 0, kWarpMma = 1, kWarpTmaB = 2, kWarpCompute0 = 4;
 constexpr int kNumComputeWarps = 12;
 
 template <int T> struct UmmaCfg;
-// Ring depths.  The raw ring has 3 slots of SPS slabs (16 KB each) that complete on one barrier: a slot hand-off
-// costs several hundred cycles whatever its size, so slots are made fat where shared memory allows.  With 3 slots
-// every slot is always served by the same warp groups (slab number mod 3 selects the group).  SA transformed-operand
-// stages (T*4 KB each), SB weight-image slots.
-template <> struct UmmaCfg<4>  { static constexpr int SPS = 2, SA = 4, SB = 2; };
-template <> struct UmmaCfg<8>  { static constexpr int SPS = 2, SA = 2, SB = 2; };
-template <> struct UmmaCfg<16> { static constexpr int SPS = 1, SA = 2, SB = 1; };
-template <> struct UmmaCfg<32> { static constexpr int SPS = 1, SA = 1, SB = 1; };
+// Ring depths.  The raw ring has 3 slots of SPS slabs (16 KB each) that complete on one barrier; with 3 slots every
+// slot is always served by the same warp groups (slab number mod 3 selects the group).  SA transformed-operand
+// stages (T*4 KB each), SB weight-image slots.  Measured on the EQ-ViT-B shape: a raw slot is released only after its
+// rows have been transformed and stored, so a deep raw ring (6 slabs) matters more than a third weight-image slot.
+// EARLY: release a raw slot as soon as its rows are in registers (one more fence + arrive per item) instead of after
+// the transformed rows have been stored; pays off only where the raw ring cannot be deep (T >= 16).
+template <> struct UmmaCfg<4>  { static constexpr int SPS = 2, SA = 4, SB = 2; static constexpr bool EARLY = false; };
+template <> struct UmmaCfg<8>  { static constexpr int SPS = 2, SA = 2, SB = 2; static constexpr bool EARLY = false; };
+template <> struct UmmaCfg<16> { static constexpr int SPS = 1, SA = 2, SB = 1; static constexpr bool EARLY = true; };
+template <> struct UmmaCfg<32> { static constexpr int SPS = 1, SA = 1, SB = 1; static constexpr bool EARLY = true; };
 constexpr int kRawSlots = 3;
 constexpr uint32_t kSpin = 256;               // test_wait polls before a single-thread role falls back to try_wait
 
@@ -73,7 +75,7 @@ __device__ unsigned long long g_trace[8192];
 struct SmemBarriers {
     uint64_t full_raw[6], empty_raw[6];
     uint64_t full_a[4], empty_a[4];
-    uint64_t full_b[4], empty_b[4];
+    uint64_t full_b[4], empty_b[4];      // SB <= 4
     uint64_t full_d, empty_d, mma_done;
     uint32_t tmem_base;
     int abort_flag;
@@ -329,13 +331,13 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const UmmaParams
                     const int r = d * 32 + lane;
                     uint32_t wd[32];
                     load_slab_row(raw + (slot * SPS + cr % SPS) * kSlabBytes + r * 128, r, wd);
-#ifndef EQL_LATE_RELEASE
-                    // The rows are in registers: order these generic-proxy reads before the async-proxy (TMA) refill
-                    // of the slot, then release it so that the refill overlaps the transform.
-                    ptx::fence_proxy_async_smem();
-                    __syncwarp();
-                    if (lane == 0) ptx::mbar_arrive(&bar->empty_raw[slot]);
-#endif
+                    if constexpr (Cfg::EARLY) {
+                        // The rows are in registers: order these generic-proxy reads before the async-proxy (TMA)
+                        // refill of the slot, then release it so that the refill overlaps the transform.
+                        ptx::fence_proxy_async_smem();
+                        __syncwarp();
+                        if (lane == 0) ptx::mbar_arrive(&bar->empty_raw[slot]);
+                    }
 #ifdef EQL_TRACE
                     if (tr) EQL_STAMP(tb + 2);
 #endif
@@ -355,10 +357,10 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const UmmaParams
                     for (int p = 0; p < T; ++p) store_plane_run<NCH>(dst + p * 4096, packed[p], 2048);
                     ptx::fence_proxy_async_smem();               // generic-proxy writes -> visible to the MMA (async proxy)
                     __syncwarp();
+                    // The same fence also orders this thread's earlier generic-proxy reads of the raw slab before the
+                    // async-proxy (TMA) refill that the release below allows.
                     if (lane == 0) {
-#ifdef EQL_LATE_RELEASE
-                        ptx::mbar_arrive(&bar->empty_raw[slot]);
-#endif
+                        if constexpr (!Cfg::EARLY) ptx::mbar_arrive(&bar->empty_raw[slot]);
                         ptx::mbar_arrive(&bar->full_a[sa]);
                     }
 #ifdef EQL_TRACE
