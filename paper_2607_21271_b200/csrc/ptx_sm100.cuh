@@ -97,6 +97,15 @@ __device__ __forceinline__ void tma_load_3d(void* smem_dst, const CUtensorMap* m
         ::"r"(smem_u32(smem_dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(c2), "r"(smem_u32(bar))
         : "memory");
 }
+// 2-D tiled store shared -> global as part of the thread's current bulk async-group (rows / columns outside the
+// tensor are clipped by the hardware); commit the group, later wait until the source has been read.
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, int c0, int c1, const void* smem_src) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
+                 ::"l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(smem_u32(smem_src))
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_commit_group() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_group_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 // 1-D bulk copy global -> shared; both addresses 16-byte aligned, bytes a multiple of 16.
 __device__ __forceinline__ void bulk_load_1d(void* smem_dst, const void* gmem_src, uint32_t bytes, uint64_t* bar) {
     asm volatile(
@@ -134,6 +143,18 @@ __device__ __forceinline__ uint64_t umma_smem_desc(uint32_t smem_addr, uint32_t 
     d |= (uint64_t)1 << 46;                       // descriptor version for sm_100
     return d;                                     // base offset 0, layout type 0 (no swizzle)
 }
+// K-major operand whose rows are 32 bytes (16 halves = one UMMA K step), 32-byte swizzle: rows are stored 32 bytes
+// apart, 8-row groups (256 B) back to back, and the two 16-byte chunks of row r are exchanged when bit 2 of r is set
+// (address bit 4 ^= address bit 7).  Tile base must be 256-byte aligned.
+__device__ __forceinline__ uint64_t umma_smem_desc_k_sw32(uint32_t smem_addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)1 << 16;                       // leading byte offset: unused for swizzled K-major
+    d |= (uint64_t)(256 >> 4) << 32;              // stride between 8-row groups
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)6 << 61;                       // SWIZZLE_32B
+    return d;
+}
 // Instruction descriptor for kind::f16 with F16 A/B (both K-major), F32 accumulator, M x N tile.
 __device__ __forceinline__ uint32_t umma_idesc_f16_f32(uint32_t M, uint32_t N) {
     return (1u << 4)                // D format: F32
@@ -149,6 +170,9 @@ __device__ __forceinline__ uint32_t umma_idesc_f16_f32_mn_major(uint32_t M, uint
 // D[tmem] (+)= A[smem] * B[smem]^T; issued by ONE thread.
 __device__ __forceinline__ void umma_f16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
                                          uint32_t accumulate) {
+#ifdef EQL_ABLATE_MMA
+    return;
+#endif
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
         "setp.ne.b32 p, %4, 0;\n\t"

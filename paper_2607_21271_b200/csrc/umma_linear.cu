@@ -7,8 +7,9 @@
 //   TMA (1-D bulk)               spectral-weight image of this (tile, 16-channel chunk) -> shared B operands
 //   1 thread                     tcgen05.mma kind::f16: one product per real frequency, and the complex
 //                                product of Eq. 5 as the real 2x2 block [Xr|Xi] x [[Wr,Wi],[-Wi,Wr]] -> TMEM
-//   12 compute warps, phase 2    tcgen05.ld, bias on plane k = 0, inverse DFT (Eq. 7) in registers,
-//                                fp16 rounding, 128 contiguous bytes per token stored with 32-byte stores
+//   12 compute warps, phase 2    tcgen05.ld, bias on plane k = 0, inverse DFT (Eq. 7) in registers, fp16 rounding,
+//                                [32 tokens x 128 B] staged in shared memory (the idle A-operand stages) and written
+//                                with asynchronous, fully coalesced TMA tensor stores
 //
 // Frequency-domain data never leaves the SM (registers, shared memory, TMEM).  The data gradient is the
 // same kernel run on dy with the conjugate-transposed weight image and no bias.
@@ -76,7 +77,7 @@ struct SmemBarriers {
     uint64_t full_raw[6], empty_raw[6];
     uint64_t full_a[4], empty_a[4];
     uint64_t full_b[4], empty_b[4];      // SB <= 4
-    uint64_t full_d, empty_d, mma_done;
+    uint64_t full_d, empty_d, mma_done, staging_free;
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -84,8 +85,8 @@ struct SmemBarriers {
 // ------------------------------------------------------------------------------------------------
 // Operand image of the spectral weight for the tensor-core kernel.
 // planes[p][cin][cout] (float, already scaled by 1/T resp. 2/T, conjugated for the data gradient) ->
-// for every (output tile, 16-channel chunk) one blob of rowsB rows x 16 k in the no-swizzle K-major
-// core-matrix layout [k half][row][8 k]: element (row n, k) at ((k/8)*rowsB + n)*8 + k%8 halves.
+// for every (output tile, 16-channel chunk) one blob of rowsB rows x 16 k in the canonical K-major layout with
+// 32-byte swizzle: element (row n, k) at n*16 + ((k/8) ^ ((n>>2)&1))*8 + k%8 halves.
 // Rows of a blob (CoT = output channels per tile):
 //   [0, CoT)                         plane 0 (k = 0)
 //   per complex frequency f (4*CoT): Wr | Wi   (multiplied by Re x^)   then   -Wi | Wr   (by Im x^)
@@ -99,9 +100,11 @@ __global__ void build_image_kernel(const float* __restrict__ planes, int Cin, in
         const int within = (int)(idx % ((int64_t)rowsB * kChunkK));
         const int64_t blob = idx / ((int64_t)rowsB * kChunkK);
         const int kc = (int)(blob % nK), tile = (int)(blob / nK);
-        const int khalf = within / (rowsB * 8);
-        const int n = (within / 8) % rowsB;
-        const int kk = khalf * 8 + (within & 7);
+        // destination element `within` of the blob: row n = within / 16, 16-byte chunk c, element e; the chunk
+        // holds k-half (c ^ bit 2 of n) (32-byte swizzle)
+        const int n = within / kChunkK;
+        const int c = (within >> 3) & 1;
+        const int kk = ((c ^ ((n >> 2) & 1)) << 3) + (within & 7);
         int plane, local;
         float sign = 1.f;
         if (n < CoT) {
@@ -126,7 +129,8 @@ __global__ void build_image_kernel(const float* __restrict__ planes, int Cin, in
 // ------------------------------------------------------------------------------------------------
 template <int T>
 __global__ void __launch_bounds__(kThreadsUmma, 1)
-umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const UmmaParams prm) {
+umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_constant__ CUtensorMap tmap_out,
+                   const UmmaParams prm) {
     using Cfg = UmmaCfg<T>;
     constexpr int SPS = Cfg::SPS, SA = Cfg::SA, SB = Cfg::SB;
     constexpr int SR = kRawSlots * SPS;         // slabs in the raw ring
@@ -152,9 +156,11 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const UmmaParams
         ptx::mbar_init(&bar->full_d, 1);
         ptx::mbar_init(&bar->empty_d, kNumComputeWarps);
         ptx::mbar_init(&bar->mma_done, 1);
+        ptx::mbar_init(&bar->staging_free, kNumComputeWarps);
         bar->abort_flag = 0;
         ptx::fence_mbar_init();
         ptx::prefetch_tensormap(&tmap_in);
+        ptx::prefetch_tensormap(&tmap_out);
     }
     if (warp == kWarpMma) {
         ptx::tmem_alloc(&bar->tmem_base, kTmemCols);
@@ -238,7 +244,6 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const UmmaParams
             bool ok = true;
             const uint32_t idesc_real = ptx::umma_idesc_f16_f32(kTileM, CoT);
             const uint32_t idesc_cplx = ptx::umma_idesc_f16_f32(kTileM, 2 * CoT);
-            const uint32_t b_lbo = (uint32_t)rowsB * 16u;
             for (int64_t u = first; u < prm.num_units && ok; u += stride, ++cu) {
                 EQL_STAMP(512 + 2 * cu);
                 ok = ptx::mbar_wait(&bar->empty_d, (cu & 1) ^ 1, abort_flag, status, 103, true, kSpin);
@@ -258,22 +263,22 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const UmmaParams
                     const uint32_t b0 = ptx::smem_u32(bsm + sb * prm.b_slot_bytes);
                     const uint32_t acc = kc > 0 ? 1u : 0u;
                     // k = 0
-                    ptx::umma_f16(tmem_base, ptx::umma_smem_desc(a0, 2048, 128), ptx::umma_smem_desc(b0, b_lbo, 128),
+                    ptx::umma_f16(tmem_base, ptx::umma_smem_desc_k_sw32(a0), ptx::umma_smem_desc_k_sw32(b0),
                                   idesc_real, acc);
                     // complex frequencies: [Re y^ | Im y^] (+)= Re x^ [Wr|Wi] + Im x^ [-Wi|Wr]
 #pragma unroll
                     for (int f = 1; f < T / 2; ++f) {
                         const uint32_t d = tmem_base + (uint32_t)((2 * f - 1) * CoT);
                         const uint32_t rb = (uint32_t)(CoT + (f - 1) * 4 * CoT);
-                        ptx::umma_f16(d, ptx::umma_smem_desc(a0 + (2 * f - 1) * 4096, 2048, 128),
-                                      ptx::umma_smem_desc(b0 + rb * 16u, b_lbo, 128), idesc_cplx, acc);
-                        ptx::umma_f16(d, ptx::umma_smem_desc(a0 + (2 * f) * 4096, 2048, 128),
-                                      ptx::umma_smem_desc(b0 + (rb + 2 * CoT) * 16u, b_lbo, 128), idesc_cplx, 1u);
+                        ptx::umma_f16(d, ptx::umma_smem_desc_k_sw32(a0 + (2 * f - 1) * 4096),
+                                      ptx::umma_smem_desc_k_sw32(b0 + rb * 32u), idesc_cplx, acc);
+                        ptx::umma_f16(d, ptx::umma_smem_desc_k_sw32(a0 + (2 * f) * 4096),
+                                      ptx::umma_smem_desc_k_sw32(b0 + (rb + 2 * CoT) * 32u), idesc_cplx, 1u);
                     }
                     // k = T/2
                     ptx::umma_f16(tmem_base + (uint32_t)((T - 1) * CoT),
-                                  ptx::umma_smem_desc(a0 + (T - 1) * 4096, 2048, 128),
-                                  ptx::umma_smem_desc(b0 + (uint32_t)(rowsB - CoT) * 16u, b_lbo, 128), idesc_real, acc);
+                                  ptx::umma_smem_desc_k_sw32(a0 + (T - 1) * 4096),
+                                  ptx::umma_smem_desc_k_sw32(b0 + (uint32_t)(rowsB - CoT) * 32u), idesc_real, acc);
                     ptx::umma_commit(&bar->empty_a[sa]);
                     ptx::umma_commit(&bar->empty_b[sb]);
                     EQL_STAMP(1024 + 4 * ca + 3);
@@ -303,9 +308,10 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const UmmaParams
         const int group = cw >> 2;                               // transform group, and share of the epilogue's column groups
         const int third = group;
         const uint32_t lane_base = tmem_base + ((uint32_t)(quad * 32) << 16);
-        const bool vec32 = ((reinterpret_cast<uintptr_t>(prm.out) & 31u) == 0) && (((int64_t)prm.Cout * T * 2) % 32 == 0);
         uint32_t ca = 0, cu = 0;
         bool ok = true;
+        bool staging_pending = false;                            // previous unit's TMA stores may still be reading the stage
+        uint8_t* staging = xhat + cw * 4096;                     // this warp's [32 tokens x 128 B] output stage (128B swizzle)
         for (int64_t u = first; u < prm.num_units && ok; u += stride, ++cu) {
             // ---- transform
             if (cw == 0 && lane == 0) EQL_STAMP(8 * cu);
@@ -342,19 +348,34 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const UmmaParams
                     if (tr) EQL_STAMP(tb + 2);
 #endif
                     uint32_t packed[T][NCH / 2];
+#ifdef EQL_ABLATE_DFT
+#pragma unroll
+                    for (int p = 0; p < T; ++p)
+#pragma unroll
+                        for (int c2 = 0; c2 < NCH / 2; ++c2) packed[p][c2] = wd[(p * (NCH / 2) + c2) & 31];
+#else
                     dft_words<T, false>(wd, packed, nullptr);
+#endif
 #ifdef EQL_TRACE
                     if (tr) { if (packed[0][0] == 0x12345678u) EQL_STAMP(tb + 7); EQL_STAMP(tb + 3); }
 #endif
                     ok = ptx::mbar_wait(&bar->empty_a[sa], ((ca / SA) & 1) ^ 1, abort_flag, status, 107, true, 16);
                     if (!ok) break;
+                    if (staging_pending) {                       // the previous unit's output stage lives in the A-operand stages
+                        ok = ptx::mbar_wait(&bar->staging_free, (cu - 1) & 1, abort_flag, status, 109, true, 16);
+                        if (!ok) break;
+                        staging_pending = false;
+                    }
 #ifdef EQL_TRACE
                     if (tr) EQL_STAMP(tb + 4);
 #endif
                     const int kfirst = q * NCH;                  // first k of this slab inside the 16-channel chunk
-                    uint8_t* dst = xhat + sa * kAStage + r * 16 + (kfirst >> 3) * 2048 + (kfirst & 7) * 2;
+                    // A tile of a plane: row r at r*32, its two 16-byte chunks exchanged when bit 2 of r is set (32B swizzle)
+                    const int sw = (r >> 2) & 1;
+                    uint8_t* dst = xhat + sa * kAStage + r * 32 + (((kfirst >> 3) ^ sw) << 4) + (kfirst & 7) * 2;
+                    const int second = sw ? -16 : 16;            // where the other k-half of the same row lives (NCH = 16 only)
 #pragma unroll
-                    for (int p = 0; p < T; ++p) store_plane_run<NCH>(dst + p * 4096, packed[p], 2048);
+                    for (int p = 0; p < T; ++p) store_plane_run<NCH>(dst + p * 4096, packed[p], second);
                     ptx::fence_proxy_async_smem();               // generic-proxy writes -> visible to the MMA (async proxy)
                     __syncwarp();
                     // The same fence also orders this thread's earlier generic-proxy reads of the raw slab before the
@@ -371,13 +392,11 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const UmmaParams
             if (!ok) break;
             // ---- epilogue
             const int tile = (int)(u % nTiles);
-            const int64_t row = (u / nTiles) * kTileM + quad * 32 + lane;
             if (cw == 0 && lane == 0) EQL_STAMP(8 * cu + 1);
             ok = ptx::mbar_wait(&bar->full_d, cu & 1, abort_flag, status, 108, true, 16);
             if (cw == 0 && lane == 0) EQL_STAMP(8 * cu + 2);
             if (!ok) break;
             ptx::tc_fence_after_sync();
-            __half* orow = prm.out + row * (int64_t)prm.Cout * T;
             const int ngroups = CoT / G;
             for (int gi = third; gi < ngroups; gi += 3) {
                 const int c0 = gi * G;
@@ -398,7 +417,9 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const UmmaParams
                     __syncwarp();
                     if (lane == 0) ptx::mbar_arrive(&bar->empty_d);
                 }
-                if (row >= prm.N) continue;
+#ifdef EQL_ABLATE_EPI
+                if (in[0][0] != 0x7fc54321u) continue;
+#endif
                 const int co0 = tile * CoT + c0;
                 uint32_t o[32];                                  // G channels x T halves = 64 halves = 128 bytes
 #pragma unroll
@@ -411,33 +432,31 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const UmmaParams
 #pragma unroll
                     for (int t = 0; t < T; t += 2) o[(g * T + t) / 2] = pack_h2(v[t], v[t + 1]);
                 }
-                __half* dst = orow + (int64_t)co0 * T;
 #ifdef EQL_TRACE
                 if (tre) { if (o[0] == 0x7fc12345u) EQL_STAMP(te + 3); EQL_STAMP(te + 2); }
 #endif
-                if (co0 + G <= prm.Cout) {
-                    if (vec32) {
+                // stage the warp's 32 rows of 128 bytes (chunk j of row l at j ^ (l & 7): the tensor map's 128B swizzle) and
+                // hand them to one asynchronous TMA store; rows >= N and channels >= Cout are clipped by the hardware
+                if (lane == 0) ptx::bulk_wait_group_read0();     // previous group's stage has been read
+                __syncwarp();
 #pragma unroll
-                        for (int i = 0; i < 4; ++i) ptx::st_global_v8(dst + i * 16, &o[i * 8]);
-                    } else {
-#pragma unroll
-                        for (int i = 0; i < 8; ++i) ptx::st_global_v4(dst + i * 8, o[4 * i], o[4 * i + 1], o[4 * i + 2], o[4 * i + 3]);
-                    }
-                } else {                                         // ragged channel tail: one channel at a time
-#pragma unroll
-                    for (int g = 0; g < G; ++g) {
-                        if (co0 + g >= prm.Cout) continue;
-                        if constexpr (T == 4) {
-                            *reinterpret_cast<uint2*>(dst + g * 4) = make_uint2(o[2 * g], o[2 * g + 1]);
-                        } else {
-#pragma unroll
-                            for (int t = 0; t < T; t += 8)
-                                ptx::st_global_v4(dst + g * T + t, o[(g * T + t) / 2], o[(g * T + t) / 2 + 1],
-                                                  o[(g * T + t) / 2 + 2], o[(g * T + t) / 2 + 3]);
-                        }
-                    }
+                for (int jj = 0; jj < 8; ++jj)
+                    *reinterpret_cast<uint4*>(staging + lane * 128 + ((jj ^ (lane & 7)) << 4)) =
+                        make_uint4(o[4 * jj], o[4 * jj + 1], o[4 * jj + 2], o[4 * jj + 3]);
+                ptx::fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0 && co0 < prm.Cout) {
+                    ptx::tma_store_2d(&tmap_out, co0 * T, (int)((u / nTiles) * kTileM) + quad * 32, staging);
+                    ptx::bulk_commit_group();
                 }
             }
+            // the A-operand stages double as the output stage: the next unit's transform may overwrite them only after
+            // every warp's stores have read their source
+            if (lane == 0) {
+                ptx::bulk_wait_group_read0();
+                ptx::mbar_arrive(&bar->staging_free);
+            }
+            staging_pending = true;
 #ifdef EQL_TRACE
             if (cw == 0 && lane == 0 && cu < 4) EQL_STAMP(7000 + 16 * (int)cu + 15);
 #endif
@@ -550,6 +569,15 @@ cudaError_t launch_umma_linear(const UmmaLinearShape& s, const void* in, void* o
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return cudaErrorInvalidValue;
 
+    CUtensorMap tmap_out;
+    {
+        const cuuint64_t odim[2] = {(cuuint64_t)s.Cout * s.T, (cuuint64_t)N};
+        const cuuint64_t ostr[1] = {(cuuint64_t)s.Cout * s.T * sizeof(__half)};
+        const cuuint32_t obox[2] = {64, 32};
+        if (enc(&tmap_out, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, out, odim, ostr, obox, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return cudaErrorInvalidValue;
+    }
     UmmaParams prm{};
     prm.out = (__half*)out; prm.image = (const __half*)image; prm.bias = bias_f32; prm.status = status;
     prm.N = N; prm.Cin = s.Cin; prm.Cout = s.Cout;
@@ -571,7 +599,7 @@ cudaError_t launch_umma_linear(const UmmaLinearShape& s, const void* in, void* o
             attr_done |= 1ull << (dev & 63);
         }
         if (smem > 227 * 1024) return cudaErrorInvalidConfiguration;
-        umma_linear_kernel<TT><<<grid, kThreadsUmma, smem, stream>>>(tmap, prm);
+        umma_linear_kernel<TT><<<grid, kThreadsUmma, smem, stream>>>(tmap, tmap_out, prm);
         return cudaGetLastError();
     });
 }
