@@ -304,35 +304,49 @@ direct_bwd_weight_kernel(const IO* __restrict__ x, const IO* __restrict__ dy, in
 }
 
 // Weight gradient, phase 2: fixed-order sum over the splits, inverse DFT with its 1/T, dw[o][i][:].
+// Block = 32 (o, i) pairs x T planes: thread (pair, plane) sums its plane over the splits (coalesced over the
+// pairs), the planes meet in shared memory, and the first 32 threads run the inverse transform.
 template <int T>
-__global__ void bwd_weight_finalize_kernel(const float* __restrict__ part, const float* __restrict__ db_part,
-                                           int splits, int Ci, int Co, bool correlation,
-                                           float* __restrict__ dw, float* __restrict__ db) {
-    const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+__global__ void __launch_bounds__(32 * T)
+bwd_weight_finalize_kernel(const float* __restrict__ part, const float* __restrict__ db_part, int splits, int Ci,
+                           int Co, bool correlation, float* __restrict__ dw, float* __restrict__ db) {
+    __shared__ float planes[T][33];
+    const int pair = threadIdx.x & 31, p = threadIdx.x >> 5;
+    const int idx = blockIdx.x * 32 + pair;
     const size_t plane_stride = (size_t)Co * Ci;
-    if (idx < Co && db != nullptr) {
-        float s = 0.f;
-        for (int sp = 0; sp < splits; ++sp) s += db_part[(size_t)sp * Co + idx];
-        db[idx] = s;
+    // db: the first blocks also reduce the bias partials (one thread per output channel)
+    {
+        const int o = blockIdx.x * blockDim.x + threadIdx.x;
+        if (o < Co && db != nullptr) {
+            float s = 0.f;
+            for (int sp = 0; sp < splits; ++sp) s += db_part[(size_t)sp * Co + o];
+            db[o] = s;
+        }
     }
-    if (idx >= Ci * Co) return;
-    float v[T];
-#pragma unroll
-    for (int p = 0; p < T; ++p) v[p] = 0.f;
-    for (int sp = 0; sp < splits; ++sp) {
-        const float* src = part + (size_t)sp * T * plane_stride + idx;
-#pragma unroll
-        for (int p = 0; p < T; ++p) v[p] += src[p * plane_stride];
+    float acc = 0.f;
+    if (idx < Ci * Co) {
+        const float* src = part + (size_t)p * plane_stride + idx;
+        for (int sp = 0; sp < splits; ++sp) acc += src[(size_t)sp * T * plane_stride];
     }
+    const bool imag = (p != 0) && (p != T - 1) && ((p & 1) == 0);
+    acc *= plane_inverse_scale<T>(p);
+    if (imag && correlation) acc = -acc;
+    planes[p][pair] = acc;
+    __syncthreads();
+    if (p == 0 && idx < Ci * Co) {
+        float v[T];
 #pragma unroll
-    for (int p = 0; p < T; ++p) {
-        const bool imag = (p != 0) && (p != T - 1) && ((p & 1) == 0);
-        v[p] *= plane_inverse_scale<T>(p);
-        if (imag && correlation) v[p] = -v[p];
+        for (int q = 0; q < T; ++q) v[q] = planes[q][pair];
+        rdft_inverse<T>(v);
+#pragma unroll
+        for (int r = 0; r < T; ++r) dw[(size_t)idx * T + r] = v[r];
     }
-    rdft_inverse<T>(v);
-#pragma unroll
-    for (int r = 0; r < T; ++r) dw[(size_t)idx * T + r] = v[r];
+}
+
+// Enough blocks of 32*T threads to cover the (o, i) pairs (32 per block) and, with one thread each, the Co bias sums.
+inline int finalize_blocks(int T, int Ci, int Co) {
+    const int by_pairs = (Ci * Co + 31) / 32, by_bias = (Co + 32 * T - 1) / (32 * T);
+    return by_pairs > by_bias ? by_pairs : by_bias;
 }
 
 template <typename F>
@@ -413,9 +427,8 @@ cudaError_t launch_bwd_weight_finalize(int T, bool correlation, const float* scr
     const float* db_part = scratch + (size_t)splits * T * Co * Ci;
     return dispatch_T(T, [&](auto tc) {
         constexpr int TT = decltype(tc)::value;
-        const int total = Ci * Co > Co ? Ci * Co : Co;
-        bwd_weight_finalize_kernel<TT><<<(total + 127) / 128, 128, 0, stream>>>(part, db_part, splits, Ci, Co,
-                                                                                 correlation, dw, db);
+        bwd_weight_finalize_kernel<TT><<<finalize_blocks(TT, Ci, Co), 32 * TT, 0, stream>>>(part, db_part, splits, Ci, Co,
+                                                                                             correlation, dw, db);
         return cudaGetLastError();
     });
 }
@@ -438,8 +451,7 @@ cudaError_t launch_direct_bwd_weight(int T, eql_dtype_t dtype, bool correlation,
                 (const __half*)x, (const __half*)dy, N, Ci, Co, split.tokens_per_split, part, db_part);
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return e;
-        const int total = Ci * Co > Co ? Ci * Co : Co;
-        bwd_weight_finalize_kernel<TT><<<(total + 127) / 128, 128, 0, stream>>>(
+        bwd_weight_finalize_kernel<TT><<<finalize_blocks(TT, Ci, Co), 32 * TT, 0, stream>>>(
             part, db_part, split.splits, Ci, Co, correlation, dw, db);
         return cudaGetLastError();
     });

@@ -196,7 +196,16 @@ umma_bwd_weight_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
             if (active) {
                 uint32_t packed[T][NCH / 2];
                 float p0[NCH];
+#ifdef EQL_ABLATE_DFT
+#pragma unroll
+                for (int p = 0; p < T; ++p)
+#pragma unroll
+                    for (int c2 = 0; c2 < NCH / 2; ++c2) packed[p][c2] = wd[(p * (NCH / 2) + c2) & 31];
+#pragma unroll
+                for (int i = 0; i < NCH; ++i) p0[i] = 0.f;
+#else
                 dft_words<T, true>(wd, packed, p0);
+#endif
                 const int mn0 = slab * NCH;                      // first channel of this slab inside the tile
                 // MN-major tile: (channel mn, token k) at (mn/8)*256 + (k/8)*128 + (k%8)*16 + (mn%8)*2
                 const int off = (mn0 >> 3) * 256 + (row >> 3) * 128 + (row & 7) * 16 + (mn0 & 7) * 2;
