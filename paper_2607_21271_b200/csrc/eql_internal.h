@@ -56,14 +56,15 @@ cudaError_t launch_direct_bwd_weight(int T, eql_dtype_t dtype, bool correlation,
 // ---- tcgen05 tensor-core kernels (FP16 I/O), umma_linear.cu ----------------------------------------
 struct UmmaLinearShape {
     int T, Cin, Cout;
+    int elem_bytes;     // 2: half I/O (kind::f16), 4: float I/O (kind::tf32, 3xTF32 split)
     int CoT;            // output channels per tile: multiple of 16, T*CoT <= 512 TMEM columns
     int nTiles;         // output-channel tiles
-    int nK;             // 16-channel chunks of the reduction dimension
+    int nK;             // chunks of the reduction dimension (16 channels for half, 8 for float)
     int rowsB;          // (2T-2)*CoT rows of the weight image per (tile, chunk)
     size_t image_bytes;
 };
 bool umma_linear_supported(int T, eql_dtype_t dtype);
-UmmaLinearShape umma_linear_shape(int T, int Cin, int Cout);
+UmmaLinearShape umma_linear_shape(int T, int Cin, int Cout, eql_dtype_t dtype);
 // planes[T][Cin][Cout] (float) -> operand image for umma_linear_kernel.
 cudaError_t launch_build_umma_image(const UmmaLinearShape& s, const float* planes, void* image, cudaStream_t stream);
 // out[N, Cout*T] = IDFT( DFT(in[N, Cin*T]) (x) image ) + bias, fp16 I/O, tcgen05 MMA with FP32 accumulation in TMEM.

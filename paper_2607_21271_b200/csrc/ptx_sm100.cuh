@@ -166,6 +166,10 @@ __device__ __forceinline__ uint32_t umma_idesc_f16_f32(uint32_t M, uint32_t N) {
            | ((N >> 3) << 17)       // N / 8
            | ((M >> 4) << 24);      // M / 16
 }
+// kind::tf32 with TF32 A/B (32-bit containers, both K-major), F32 accumulator.
+__device__ __forceinline__ uint32_t umma_idesc_tf32_f32(uint32_t M, uint32_t N) {
+    return (1u << 4) | (2u << 7) | (2u << 10) | ((N >> 3) << 17) | ((M >> 4) << 24);
+}
 // Same, with both operands MN-major ("transposed": the M resp. N index is the contiguous one in shared memory).
 __device__ __forceinline__ uint32_t umma_idesc_f16_f32_mn_major(uint32_t M, uint32_t N) {
     return umma_idesc_f16_f32(M, N) | (1u << 15) | (1u << 16);
@@ -180,6 +184,18 @@ __device__ __forceinline__ void umma_f16(uint32_t d_tmem, uint64_t a_desc, uint6
         "{\n\t.reg .pred p;\n\t"
         "setp.ne.b32 p, %4, 0;\n\t"
         "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void umma_tf32(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                          uint32_t accumulate) {
+#ifdef EQL_ABLATE_MMA
+    return;
+#endif
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
 }

@@ -80,8 +80,37 @@ __device__ __forceinline__ void dft_words(const uint32_t (&wd)[32], uint32_t (&p
     }
 }
 
-// Stores the NCH = 64/T packed channel values of one plane as one contiguous run of NCH halves.
-// NCH = 16 -> two 16-byte stores `second_half_stride` bytes apart, 8 -> one 16-byte store, 4 -> 8 bytes, 2 -> 4 bytes.
+// Group DFT of the 32/T float channels held in wd (a 128-byte slab row of an FP32 tensor), in place:
+// afterwards wd[c*T + p] is plane p of channel c.
+template <int T>
+__device__ __forceinline__ void dft_words_f32(uint32_t (&wd)[32]) {
+    constexpr int NCH = 32 / T;
+#pragma unroll
+    for (int c = 0; c < NCH; ++c) {
+        float v[T];
+#pragma unroll
+        for (int t = 0; t < T; ++t) v[t] = __uint_as_float(wd[c * T + t]);
+        rdft_forward<T>(v);
+#pragma unroll
+        for (int t = 0; t < T; ++t) wd[c * T + t] = __float_as_uint(v[t]);
+    }
+}
+
+// 3xTF32 split of a float: hi = v rounded to TF32 (10 mantissa bits), lo = (v - hi) rounded to TF32;
+// hi*hi + hi*lo + lo*hi reproduces the float product to ~2^-22 (the tensor core itself would truncate, so both
+// parts are rounded here).
+__device__ __forceinline__ uint32_t round_tf32(float v) {
+    uint32_t r;
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(v));
+    return r;
+}
+__device__ __forceinline__ void split_tf32(float v, uint32_t& hi, uint32_t& lo) {
+    hi = round_tf32(v);
+    lo = round_tf32(v - __uint_as_float(hi));
+}
+
+// Stores W 32-bit words of one plane as one contiguous run.
+// W = 8 -> two 16-byte stores `second_half_stride` bytes apart, 4 -> one 16-byte store, 2 -> 8 bytes, 1 -> 4 bytes.
 template <int NCH>
 __device__ __forceinline__ void store_plane_run(uint8_t* d, const uint32_t* pk, int second_half_stride, uint32_t xor_mask = 0u) {
     if constexpr (NCH == 16) {

@@ -30,7 +30,7 @@ namespace eql {
 namespace {
 
 constexpr int kTileM = 128;            // tokens per tile = UMMA M = TMEM lanes
-constexpr int kChunkK = 16;            // input channels per pipeline stage = one UMMA K step for f16
+constexpr int kRowBytes = 32;           // operand row of one pipeline stage = one UMMA K step (16 halves / 8 floats)
 constexpr int kSlabBytes = kTileM * 128;
 constexpr int kThreadsUmma = 512;
 constexpr int kTmemCols = 512;
@@ -39,29 +39,33 @@ constexpr int kTmemCols = 512;
 constexpr int kWarpTmaX = 0, kWarpMma = 1, kWarpTmaB = 2, kWarpCompute0 = 4;
 constexpr int kNumComputeWarps = 12;
 
-template <int T> struct UmmaCfg;
+template <int T, int E> struct UmmaCfg;          // E = bytes per element of the I/O tensors (2: half, 4: float)
 // Ring depths.  The raw ring has 3 slots of SPS slabs (16 KB each) that complete on one barrier; with 3 slots every
 // slot is always served by the same warp groups (slab number mod 3 selects the group).  SA transformed-operand
-// stages (T*4 KB each), SB weight-image slots.  Measured on the EQ-ViT-B shape: a raw slot is released only after its
-// rows have been transformed and stored, so a deep raw ring (6 slabs) matters more than a third weight-image slot.
+// stages (T*4 KB each, twice that for the hi/lo halves of FP32), SB weight-image slots.  Measured on the EQ-ViT-B
+// shape: a raw slot is released only after its rows have been transformed and stored, so a deep raw ring (6 slabs)
+// matters more than a third weight-image slot.
 // EARLY: release a raw slot as soon as its rows are in registers (one more fence + arrive per item) instead of after
-// the transformed rows have been stored; pays off only where the raw ring cannot be deep (T >= 16).
-template <> struct UmmaCfg<4>  { static constexpr int SPS = 2, SA = 4, SB = 2; static constexpr bool EARLY = false; };
-template <> struct UmmaCfg<8>  { static constexpr int SPS = 2, SA = 2, SB = 2; static constexpr bool EARLY = false; };
-template <> struct UmmaCfg<16> { static constexpr int SPS = 1, SA = 2, SB = 1; static constexpr bool EARLY = true; };
-template <> struct UmmaCfg<32> { static constexpr int SPS = 1, SA = 1, SB = 1; static constexpr bool EARLY = true; };
+// the transformed rows have been stored; used where the raw ring cannot be deep.
+// MAXCOT: output channels per tile (T*CoT fp32 TMEM columns <= 512, and the weight-image slot must fit).
+template <> struct UmmaCfg<4, 2>  { static constexpr int SPS = 2, SA = 4, SB = 2, MAXCOT = 128; static constexpr bool EARLY = false; };
+template <> struct UmmaCfg<8, 2>  { static constexpr int SPS = 2, SA = 2, SB = 2, MAXCOT = 64;  static constexpr bool EARLY = false; };
+template <> struct UmmaCfg<16, 2> { static constexpr int SPS = 1, SA = 2, SB = 1, MAXCOT = 32;  static constexpr bool EARLY = true; };
+template <> struct UmmaCfg<32, 2> { static constexpr int SPS = 1, SA = 1, SB = 1, MAXCOT = 16;  static constexpr bool EARLY = true; };
+template <> struct UmmaCfg<4, 4>  { static constexpr int SPS = 1, SA = 3, SB = 1, MAXCOT = 128; static constexpr bool EARLY = true; };
+template <> struct UmmaCfg<8, 4>  { static constexpr int SPS = 1, SA = 2, SB = 1, MAXCOT = 48;  static constexpr bool EARLY = true; };
 constexpr int kRawSlots = 3;
 constexpr uint32_t kSpin = 256;               // test_wait polls before a single-thread role falls back to try_wait
 
 struct UmmaParams {
-    __half* out;                 // [N, Cout*T]
-    const __half* image;         // spectral-weight operand image, see build_image_kernel
+    void* out;                   // [N, Cout*T]
+    const uint8_t* image;        // spectral-weight operand image, see build_image_kernel
     const float* bias;           // [Cout] or nullptr
     int* status;                 // device status word of the plan
     int64_t N;
     int Cin, Cout;
     int CoT, nTiles, nK, rowsB;
-    int b_slot_bytes;            // bytes of one B ring slot (rowsB*32 rounded up to 128)
+    int b_slot_bytes;            // bytes of one B ring slot (rowsB*32, twice that for FP32, rounded up to 128)
     int64_t num_units;
 };
 
@@ -85,26 +89,30 @@ struct SmemBarriers {
 // ------------------------------------------------------------------------------------------------
 // Operand image of the spectral weight for the tensor-core kernel.
 // planes[p][cin][cout] (float, already scaled by 1/T resp. 2/T, conjugated for the data gradient) ->
-// for every (output tile, 16-channel chunk) one blob of rowsB rows x 16 k in the canonical K-major layout with
-// 32-byte swizzle: element (row n, k) at n*16 + ((k/8) ^ ((n>>2)&1))*8 + k%8 halves.
+// for every (output tile, channel chunk of one UMMA K step) one blob of rowsB rows x 32 bytes in the canonical K-major
+// layout with 32-byte swizzle: byte b of row n lives at n*32 + (((b>>4) ^ ((n>>2)&1))<<4) + (b&15).
+// FP32 plans store two such blobs back to back: the TF32 "hi" parts and the "lo" remainders (3xTF32).
 // Rows of a blob (CoT = output channels per tile):
 //   [0, CoT)                         plane 0 (k = 0)
 //   per complex frequency f (4*CoT): Wr | Wi   (multiplied by Re x^)   then   -Wi | Wr   (by Im x^)
 //   [rowsB - CoT, rowsB)             plane T-1 (k = T/2)
-template <int T>
+template <int T, typename IO>
 __global__ void build_image_kernel(const float* __restrict__ planes, int Cin, int Cout, int CoT, int nTiles, int nK,
-                                   int rowsB, __half* __restrict__ image) {
-    const int64_t total = (int64_t)nTiles * nK * rowsB * kChunkK;
+                                   int rowsB, IO* __restrict__ image) {
+    constexpr int E = sizeof(IO), KCH = kRowBytes / E, EPC = 16 / E, NSPLIT = E == 4 ? 2 : 1;
+    const int64_t per_blob = (int64_t)NSPLIT * rowsB * KCH;
+    const int64_t total = (int64_t)nTiles * nK * per_blob;
     for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
          idx += (int64_t)gridDim.x * blockDim.x) {
-        const int within = (int)(idx % ((int64_t)rowsB * kChunkK));
-        const int64_t blob = idx / ((int64_t)rowsB * kChunkK);
+        const int within_all = (int)(idx % per_blob);
+        const int64_t blob = idx / per_blob;
         const int kc = (int)(blob % nK), tile = (int)(blob / nK);
-        // destination element `within` of the blob: row n = within / 16, 16-byte chunk c, element e; the chunk
-        // holds k-half (c ^ bit 2 of n) (32-byte swizzle)
-        const int n = within / kChunkK;
-        const int c = (within >> 3) & 1;
-        const int kk = ((c ^ ((n >> 2) & 1)) << 3) + (within & 7);
+        const int part = within_all / (rowsB * KCH), within = within_all % (rowsB * KCH);
+        // destination element `within` of the blob: row n, 16-byte chunk c, element e of the chunk; the chunk holds
+        // k-half (c ^ bit 2 of n) (32-byte swizzle)
+        const int n = within / KCH;
+        const int c = (within % KCH) / EPC;
+        const int kk = (c ^ ((n >> 2) & 1)) * EPC + within % EPC;
         int plane, local;
         float sign = 1.f;
         if (n < CoT) {
@@ -112,31 +120,43 @@ __global__ void build_image_kernel(const float* __restrict__ planes, int Cin, in
         } else if (n >= rowsB - CoT) {
             plane = T - 1; local = n - (rowsB - CoT);
         } else {
-            const int m = n - CoT, f = m / (4 * CoT) + 1, part = (m / CoT) & 3;
+            const int m = n - CoT, f = m / (4 * CoT) + 1, quarter = (m / CoT) & 3;
             local = m % CoT;
-            if (part == 0) plane = 2 * f - 1;                     // Wr  -> Re y^
-            else if (part == 1) plane = 2 * f;                    // Wi  -> Im y^
-            else if (part == 2) { plane = 2 * f; sign = -1.f; }   // -Wi -> Re y^
-            else plane = 2 * f - 1;                               // Wr  -> Im y^
+            if (quarter == 0) plane = 2 * f - 1;                     // Wr  -> Re y^
+            else if (quarter == 1) plane = 2 * f;                    // Wi  -> Im y^
+            else if (quarter == 2) { plane = 2 * f; sign = -1.f; }   // -Wi -> Re y^
+            else plane = 2 * f - 1;                                  // Wr  -> Im y^
         }
-        const int cin = kc * kChunkK + kk, cout = tile * CoT + local;
+        const int cin = kc * KCH + kk, cout = tile * CoT + local;
         float v = 0.f;
         if (cin < Cin && cout < Cout) v = sign * planes[((size_t)plane * Cin + cin) * Cout + cout];
-        image[idx] = __float2half_rn(v);
+        if constexpr (E == 2) {
+            image[idx] = __float2half_rn(v);
+        } else {
+            uint32_t hi, lo;
+            split_tf32(v, hi, lo);
+            image[idx] = __uint_as_float(part == 0 ? hi : lo);
+        }
     }
 }
 
 // ------------------------------------------------------------------------------------------------
-template <int T>
+template <int T, typename IO>
 __global__ void __launch_bounds__(kThreadsUmma, 1)
 umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_constant__ CUtensorMap tmap_out,
                    const UmmaParams prm) {
-    using Cfg = UmmaCfg<T>;
+    constexpr int E = sizeof(IO);               // 2: half I/O, kind::f16;  4: float I/O, kind::tf32 with the 3xTF32 split
+    using Cfg = UmmaCfg<T, E>;
     constexpr int SPS = Cfg::SPS, SA = Cfg::SA, SB = Cfg::SB;
     constexpr int SR = kRawSlots * SPS;         // slabs in the raw ring
-    constexpr int NCH = 64 / T;                 // channels per raw slab row (128 B)
-    constexpr int SPK = kChunkK / NCH;          // slabs per 16-channel chunk (= T/4)
-    constexpr int kAStage = T * 4096;           // T planes x [128 x 16] halves
+    constexpr int EPR = 128 / E;                // elements per raw slab row (128 B)
+    constexpr int NCH = EPR / T;                // channels per raw slab row
+    constexpr int KCH = kRowBytes / E;          // channels per chunk = one UMMA K step (16 halves / 8 floats)
+    constexpr int SPK = KCH / NCH;              // slabs per chunk (= T/4)
+    constexpr int NSPLIT = E == 4 ? 2 : 1;      // operand copies: FP32 keeps TF32 hi parts and lo remainders
+    constexpr int kAPart = T * 4096;            // T planes x [128 rows x 32 B]
+    constexpr int kAStage = kAPart * NSPLIT;
+    constexpr int W = NCH * E / 4;              // 32-bit words one slab row contributes to one plane
 
     extern __shared__ uint8_t smem_raw_base[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw_base) + 1023) & ~(uintptr_t)1023);
@@ -191,7 +211,7 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
                             EQL_STAMP(2048 + cr);
                             ptx::mbar_arrive_expect_tx(&bar->full_raw[slot], SPS * kSlabBytes);
                         }
-                        ptx::tma_load_2d(raw + (slot * SPS + cr % SPS) * kSlabBytes, &tmap_in, (kc * kChunkK + q * NCH) * T, row0,
+                        ptx::tma_load_2d(raw + (slot * SPS + cr % SPS) * kSlabBytes, &tmap_in, (kc * KCH + q * NCH) * T, row0,
                                          &bar->full_raw[slot]);
                     }
                 }
@@ -217,7 +237,7 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
         if (lane == 0) {
             uint32_t cb = 0;
             bool ok = true;
-            const uint32_t blob_bytes = (uint32_t)rowsB * 32u;
+            const uint32_t blob_bytes = (uint32_t)rowsB * kRowBytes * NSPLIT;
             for (int64_t u = first; u < prm.num_units && ok; u += stride) {
                 const int tile = (int)(u % nTiles);
                 for (int kc = 0; kc < nK; ++kc, ++cb) {
@@ -227,7 +247,7 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
                     EQL_STAMP(4096 + cb);
                     ptx::mbar_arrive_expect_tx(&bar->full_b[slot], blob_bytes);
                     ptx::bulk_load_1d(bsm + slot * prm.b_slot_bytes,
-                                      prm.image + ((size_t)tile * nK + kc) * (size_t)rowsB * kChunkK, blob_bytes,
+                                      prm.image + ((size_t)tile * nK + kc) * (size_t)blob_bytes, blob_bytes,
                                       &bar->full_b[slot]);
                 }
             }
@@ -242,8 +262,15 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
         if (lane == 0) {
             uint32_t ca = 0, cb = 0, cu = 0;
             bool ok = true;
-            const uint32_t idesc_real = ptx::umma_idesc_f16_f32(kTileM, CoT);
-            const uint32_t idesc_cplx = ptx::umma_idesc_f16_f32(kTileM, 2 * CoT);
+            const uint32_t idesc_real = E == 2 ? ptx::umma_idesc_f16_f32(kTileM, CoT) : ptx::umma_idesc_tf32_f32(kTileM, CoT);
+            const uint32_t idesc_cplx = E == 2 ? ptx::umma_idesc_f16_f32(kTileM, 2 * CoT) : ptx::umma_idesc_tf32_f32(kTileM, 2 * CoT);
+            auto mma = [](uint32_t d, uint32_t a_addr, uint32_t b_addr, uint32_t idesc, uint32_t accumulate) {
+                if constexpr (E == 2)
+                    ptx::umma_f16(d, ptx::umma_smem_desc_k_sw32(a_addr), ptx::umma_smem_desc_k_sw32(b_addr), idesc, accumulate);
+                else
+                    ptx::umma_tf32(d, ptx::umma_smem_desc_k_sw32(a_addr), ptx::umma_smem_desc_k_sw32(b_addr), idesc, accumulate);
+            };
+            const uint32_t b_part = (uint32_t)rowsB * kRowBytes;
             for (int64_t u = first; u < prm.num_units && ok; u += stride, ++cu) {
                 EQL_STAMP(512 + 2 * cu);
                 ok = ptx::mbar_wait(&bar->empty_d, (cu & 1) ^ 1, abort_flag, status, 103, true, kSpin);
@@ -259,26 +286,26 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
                     EQL_STAMP(1024 + 4 * ca + 2);
                     if (!ok) break;
                     ptx::tc_fence_after_sync();
-                    const uint32_t a0 = ptx::smem_u32(xhat + sa * kAStage);
-                    const uint32_t b0 = ptx::smem_u32(bsm + sb * prm.b_slot_bytes);
-                    const uint32_t acc = kc > 0 ? 1u : 0u;
-                    // k = 0
-                    ptx::umma_f16(tmem_base, ptx::umma_smem_desc_k_sw32(a0), ptx::umma_smem_desc_k_sw32(b0),
-                                  idesc_real, acc);
-                    // complex frequencies: [Re y^ | Im y^] (+)= Re x^ [Wr|Wi] + Im x^ [-Wi|Wr]
+                    // FP16: one pass.  FP32 (3xTF32): hi*hi, hi*lo, lo*hi accumulate into the same columns.
 #pragma unroll
-                    for (int f = 1; f < T / 2; ++f) {
-                        const uint32_t d = tmem_base + (uint32_t)((2 * f - 1) * CoT);
-                        const uint32_t rb = (uint32_t)(CoT + (f - 1) * 4 * CoT);
-                        ptx::umma_f16(d, ptx::umma_smem_desc_k_sw32(a0 + (2 * f - 1) * 4096),
-                                      ptx::umma_smem_desc_k_sw32(b0 + rb * 32u), idesc_cplx, acc);
-                        ptx::umma_f16(d, ptx::umma_smem_desc_k_sw32(a0 + (2 * f) * 4096),
-                                      ptx::umma_smem_desc_k_sw32(b0 + (rb + 2 * CoT) * 32u), idesc_cplx, 1u);
+                    for (int pass = 0; pass < (E == 4 ? 3 : 1); ++pass) {
+                        const uint32_t a0 = ptx::smem_u32(xhat + sa * kAStage) + (pass == 2 ? kAPart : 0);
+                        const uint32_t b0 = ptx::smem_u32(bsm + sb * prm.b_slot_bytes) + (pass == 1 ? b_part : 0);
+                        const uint32_t acc = (kc > 0 || pass > 0) ? 1u : 0u;
+                        // k = 0
+                        mma(tmem_base, a0, b0, idesc_real, acc);
+                        // complex frequencies: [Re y^ | Im y^] (+)= Re x^ [Wr|Wi] + Im x^ [-Wi|Wr]
+#pragma unroll
+                        for (int f = 1; f < T / 2; ++f) {
+                            const uint32_t d = tmem_base + (uint32_t)((2 * f - 1) * CoT);
+                            const uint32_t rb = (uint32_t)(CoT + (f - 1) * 4 * CoT);
+                            mma(d, a0 + (2 * f - 1) * 4096, b0 + rb * kRowBytes, idesc_cplx, acc);
+                            mma(d, a0 + (2 * f) * 4096, b0 + (rb + 2 * CoT) * kRowBytes, idesc_cplx, 1u);
+                        }
+                        // k = T/2
+                        mma(tmem_base + (uint32_t)((T - 1) * CoT), a0 + (T - 1) * 4096,
+                            b0 + (uint32_t)(rowsB - CoT) * kRowBytes, idesc_real, acc);
                     }
-                    // k = T/2
-                    ptx::umma_f16(tmem_base + (uint32_t)((T - 1) * CoT),
-                                  ptx::umma_smem_desc_k_sw32(a0 + (T - 1) * 4096),
-                                  ptx::umma_smem_desc_k_sw32(b0 + (uint32_t)(rowsB - CoT) * 32u), idesc_real, acc);
                     ptx::umma_commit(&bar->empty_a[sa]);
                     ptx::umma_commit(&bar->empty_b[sb]);
                     EQL_STAMP(1024 + 4 * ca + 3);
@@ -294,7 +321,7 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
         // Per unit every compute warp first transforms its share of the raw slab rows (group DFT -> A operands)
         // and then drains its share of the accumulator (inverse DFT -> global).  Work items of the transform
         // are (slab, 32-row quarter).
-        constexpr int G = 64 / T;                                // channels per TMEM read group
+        constexpr int G = EPR / T;                               // channels per TMEM read group (128 output bytes per token)
         // The 12 warps form 3 groups of 4; raw slab number cr is transformed by group cr % 3, one 32-row quarter
         // per warp.  Because the ring has 3 slots, a slot is always served by the same groups, so each warp
         // sees every phase of the slot barriers it waits on, in order (a parity wait is only unambiguous one
@@ -347,17 +374,27 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
 #ifdef EQL_TRACE
                     if (tr) EQL_STAMP(tb + 2);
 #endif
-                    uint32_t packed[T][NCH / 2];
+                    // A tile of a plane: row r at r*32, its two 16-byte chunks exchanged when bit 2 of r is set (32B swizzle);
+                    // this slab row's run of channels starts at byte kb of the row
+                    const int kb = q * NCH * E;
+                    const int sw = (r >> 2) & 1;
+                    uint8_t* dst = xhat + sa * kAStage + r * 32 + (((kb >> 4) ^ sw) << 4) + (kb & 15);
+                    const int second = sw ? -16 : 16;            // where the other half of the same row lives (32-byte runs only)
+                    uint32_t packed[E == 2 ? T : 1][E == 2 ? NCH / 2 : 1];
+                    if constexpr (E == 2) {
 #ifdef EQL_ABLATE_DFT
 #pragma unroll
-                    for (int p = 0; p < T; ++p)
+                        for (int p = 0; p < T; ++p)
 #pragma unroll
-                        for (int c2 = 0; c2 < NCH / 2; ++c2) packed[p][c2] = wd[(p * (NCH / 2) + c2) & 31];
+                            for (int c2 = 0; c2 < NCH / 2; ++c2) packed[p][c2] = wd[(p * (NCH / 2) + c2) & 31];
 #else
-                    dft_words<T, false>(wd, packed, nullptr);
+                        dft_words<T, false>(wd, packed, nullptr);
 #endif
+                    } else {
+                        dft_words_f32<T>(wd);                    // wd[c*T + p] = plane p of channel c
+                    }
 #ifdef EQL_TRACE
-                    if (tr) { if (packed[0][0] == 0x12345678u) EQL_STAMP(tb + 7); EQL_STAMP(tb + 3); }
+                    if (tr) { if (wd[0] == 0x12345678u && packed[0][0] == 1u) EQL_STAMP(tb + 7); EQL_STAMP(tb + 3); }
 #endif
                     ok = ptx::mbar_wait(&bar->empty_a[sa], ((ca / SA) & 1) ^ 1, abort_flag, status, 107, true, 16);
                     if (!ok) break;
@@ -369,13 +406,19 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
 #ifdef EQL_TRACE
                     if (tr) EQL_STAMP(tb + 4);
 #endif
-                    const int kfirst = q * NCH;                  // first k of this slab inside the 16-channel chunk
-                    // A tile of a plane: row r at r*32, its two 16-byte chunks exchanged when bit 2 of r is set (32B swizzle)
-                    const int sw = (r >> 2) & 1;
-                    uint8_t* dst = xhat + sa * kAStage + r * 32 + (((kfirst >> 3) ^ sw) << 4) + (kfirst & 7) * 2;
-                    const int second = sw ? -16 : 16;            // where the other k-half of the same row lives (NCH = 16 only)
+                    if constexpr (E == 2) {
 #pragma unroll
-                    for (int p = 0; p < T; ++p) store_plane_run<NCH>(dst + p * 4096, packed[p], second);
+                        for (int p = 0; p < T; ++p) store_plane_run<2 * W>(dst + p * 4096, packed[p], second);
+                    } else {
+#pragma unroll
+                        for (int p = 0; p < T; ++p) {
+                            uint32_t hi[W], lo[W];
+#pragma unroll
+                            for (int c = 0; c < NCH; ++c) split_tf32(__uint_as_float(wd[c * T + p]), hi[c], lo[c]);
+                            store_plane_run<2 * W>(dst + p * 4096, hi, second);
+                            store_plane_run<2 * W>(dst + kAPart + p * 4096, lo, second);
+                        }
+                    }
                     ptx::fence_proxy_async_smem();               // generic-proxy writes -> visible to the MMA (async proxy)
                     __syncwarp();
                     // The same fence also orders this thread's earlier generic-proxy reads of the raw slab before the
@@ -421,7 +464,7 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
                 if (in[0][0] != 0x7fc54321u) continue;
 #endif
                 const int co0 = tile * CoT + c0;
-                uint32_t o[32];                                  // G channels x T halves = 64 halves = 128 bytes
+                uint32_t o[32];                                  // G channels x T elements = 128 bytes
 #pragma unroll
                 for (int g = 0; g < G; ++g) {
                     float v[T];
@@ -429,8 +472,13 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
                     for (int p = 0; p < T; ++p) v[p] = __uint_as_float(in[p][g]);
                     if (prm.bias != nullptr && co0 + g < prm.Cout) v[0] += __ldg(prm.bias + co0 + g);
                     rdft_inverse<T>(v);
+                    if constexpr (E == 2) {
 #pragma unroll
-                    for (int t = 0; t < T; t += 2) o[(g * T + t) / 2] = pack_h2(v[t], v[t + 1]);
+                        for (int t = 0; t < T; t += 2) o[(g * T + t) / 2] = pack_h2(v[t], v[t + 1]);
+                    } else {
+#pragma unroll
+                        for (int t = 0; t < T; ++t) o[g * T + t] = __float_as_uint(v[t]);
+                    }
                 }
 #ifdef EQL_TRACE
                 if (tre) { if (o[0] == 0x7fc12345u) EQL_STAMP(te + 3); EQL_STAMP(te + 2); }
@@ -496,22 +544,39 @@ EncodeTiledFn encode_tiled_fn() {
     return fn;
 }
 
-template <int T>
+template <int T, int E>
 size_t umma_smem_bytes(int b_slot_bytes) {
-    using Cfg = UmmaCfg<T>;
-    return 1024 + (size_t)kRawSlots * Cfg::SPS * kSlabBytes + (size_t)Cfg::SA * T * 4096 + (size_t)Cfg::SB * b_slot_bytes +
-           sizeof(SmemBarriers) + 64;
+    using Cfg = UmmaCfg<T, E>;
+    return 1024 + (size_t)kRawSlots * Cfg::SPS * kSlabBytes + (size_t)Cfg::SA * T * 4096 * (E == 4 ? 2 : 1) +
+           (size_t)Cfg::SB * b_slot_bytes + sizeof(SmemBarriers) + 64;
 }
 
+// Calls f(integral_constant<T>, element type tag) for the supported (T, dtype) pairs.
 template <typename F>
-cudaError_t dispatch_umma_T(int T, F&& f) {
+cudaError_t dispatch_umma(int T, int elem_bytes, F&& f) {
+    if (elem_bytes == 2) {
+        switch (T) {
+            case 4: return f(std::integral_constant<int, 4>{}, __half{});
+            case 8: return f(std::integral_constant<int, 8>{}, __half{});
+            case 16: return f(std::integral_constant<int, 16>{}, __half{});
+            case 32: return f(std::integral_constant<int, 32>{}, __half{});
+            default: return cudaErrorInvalidValue;
+        }
+    }
     switch (T) {
-        case 4: return f(std::integral_constant<int, 4>{});
-        case 8: return f(std::integral_constant<int, 8>{});
-        case 16: return f(std::integral_constant<int, 16>{});
-        case 32: return f(std::integral_constant<int, 32>{});
+        case 4: return f(std::integral_constant<int, 4>{}, float{});
+        case 8: return f(std::integral_constant<int, 8>{}, float{});
         default: return cudaErrorInvalidValue;
     }
+}
+
+int umma_max_cot(int T, int elem_bytes) {
+    int m = 0;
+    dispatch_umma(T, elem_bytes, [&](auto tc, auto io) {
+        m = UmmaCfg<decltype(tc)::value, sizeof(decltype(io))>::MAXCOT;
+        return cudaSuccess;
+    });
+    return m;
 }
 
 }  // namespace
@@ -528,29 +593,33 @@ extern "C" int eqlinear_debug_clear_trace() {
 #endif
 
 bool umma_linear_supported(int T, eql_dtype_t dtype) {
-    return dtype == EQL_FP16 && (T == 4 || T == 8 || T == 16 || T == 32);
+    if (dtype == EQL_FP16) return T == 4 || T == 8 || T == 16 || T == 32;
+    return T == 4 || T == 8;            // FP32 (3xTF32): the hi/lo operand stages of larger T do not fit in shared memory
 }
 
-UmmaLinearShape umma_linear_shape(int T, int Cin, int Cout) {
+UmmaLinearShape umma_linear_shape(int T, int Cin, int Cout, eql_dtype_t dtype) {
     UmmaLinearShape s{};
     s.T = T; s.Cin = Cin; s.Cout = Cout;
-    const int max_cot = kTmemCols / T;                           // T planes x CoT fp32 columns <= 512
+    s.elem_bytes = dtype == EQL_FP32 ? 4 : 2;
+    const int max_cot = umma_max_cot(T, s.elem_bytes);           // T planes x CoT fp32 TMEM columns <= 512
     s.nTiles = (Cout + max_cot - 1) / max_cot;
     const int per = (Cout + s.nTiles - 1) / s.nTiles;
     s.CoT = (per + 15) / 16 * 16;
-    s.nK = (Cin + kChunkK - 1) / kChunkK;
+    const int kch = kRowBytes / s.elem_bytes;                    // channels per chunk (one UMMA K step)
+    s.nK = (Cin + kch - 1) / kch;
     s.rowsB = (2 * T - 2) * s.CoT;
-    s.image_bytes = align_up((size_t)s.nTiles * s.nK * s.rowsB * kChunkK * sizeof(__half), kWsAlign);
+    s.image_bytes = align_up((size_t)s.nTiles * s.nK * s.rowsB * kRowBytes * (s.elem_bytes == 4 ? 2 : 1), kWsAlign);
     return s;
 }
 
 cudaError_t launch_build_umma_image(const UmmaLinearShape& s, const float* planes, void* image, cudaStream_t stream) {
-    return dispatch_umma_T(s.T, [&](auto tc) {
+    return dispatch_umma(s.T, s.elem_bytes, [&](auto tc, auto io) {
         constexpr int TT = decltype(tc)::value;
-        const int64_t total = (int64_t)s.nTiles * s.nK * s.rowsB * kChunkK;
+        using IO = decltype(io);
+        const int64_t total = (int64_t)(s.image_bytes / sizeof(IO));
         const int blocks = (int)((total + 255) / 256 < 4096 ? (total + 255) / 256 : 4096);
-        build_image_kernel<TT><<<blocks, 256, 0, stream>>>(planes, s.Cin, s.Cout, s.CoT, s.nTiles, s.nK, s.rowsB,
-                                                            (__half*)image);
+        build_image_kernel<TT, IO><<<blocks, 256, 0, stream>>>(planes, s.Cin, s.Cout, s.CoT, s.nTiles, s.nK, s.rowsB,
+                                                                (IO*)image);
         return cudaGetLastError();
     });
 }
@@ -559,47 +628,49 @@ cudaError_t launch_umma_linear(const UmmaLinearShape& s, const void* in, void* o
                                const float* bias_f32, int* status, int num_sms, cudaStream_t stream) {
     EncodeTiledFn enc = encode_tiled_fn();
     if (enc == nullptr) return cudaErrorNotSupported;
-    CUtensorMap tmap;
-    const cuuint64_t gdim[2] = {(cuuint64_t)s.Cin * s.T, (cuuint64_t)N};
-    const cuuint64_t gstr[1] = {(cuuint64_t)s.Cin * s.T * sizeof(__half)};
-    const cuuint32_t box[2] = {64, (cuuint32_t)kTileM};
+    const CUtensorMapDataType dt = s.elem_bytes == 4 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16;
+    const cuuint32_t epr = 128 / s.elem_bytes;                   // elements per 128-byte slab row
+    CUtensorMap tmap, tmap_out;
     const cuuint32_t estr[2] = {1, 1};
-    if (enc(&tmap, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(in), gdim, gstr, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-        return cudaErrorInvalidValue;
-
-    CUtensorMap tmap_out;
+    {
+        const cuuint64_t gdim[2] = {(cuuint64_t)s.Cin * s.T, (cuuint64_t)N};
+        const cuuint64_t gstr[1] = {(cuuint64_t)s.Cin * s.T * s.elem_bytes};
+        const cuuint32_t box[2] = {epr, (cuuint32_t)kTileM};
+        if (enc(&tmap, dt, 2, const_cast<void*>(in), gdim, gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return cudaErrorInvalidValue;
+    }
     {
         const cuuint64_t odim[2] = {(cuuint64_t)s.Cout * s.T, (cuuint64_t)N};
-        const cuuint64_t ostr[1] = {(cuuint64_t)s.Cout * s.T * sizeof(__half)};
-        const cuuint32_t obox[2] = {64, 32};
-        if (enc(&tmap_out, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, out, odim, ostr, obox, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+        const cuuint64_t ostr[1] = {(cuuint64_t)s.Cout * s.T * s.elem_bytes};
+        const cuuint32_t obox[2] = {epr, 32};
+        if (enc(&tmap_out, dt, 2, out, odim, ostr, obox, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                 CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return cudaErrorInvalidValue;
     }
     UmmaParams prm{};
-    prm.out = (__half*)out; prm.image = (const __half*)image; prm.bias = bias_f32; prm.status = status;
+    prm.out = out; prm.image = (const uint8_t*)image; prm.bias = bias_f32; prm.status = status;
     prm.N = N; prm.Cin = s.Cin; prm.Cout = s.Cout;
     prm.CoT = s.CoT; prm.nTiles = s.nTiles; prm.nK = s.nK; prm.rowsB = s.rowsB;
-    prm.b_slot_bytes = (int)align_up((size_t)s.rowsB * 32, 128);
+    prm.b_slot_bytes = (int)align_up((size_t)s.rowsB * kRowBytes * (s.elem_bytes == 4 ? 2 : 1), 128);
     prm.num_units = ((N + kTileM - 1) / kTileM) * s.nTiles;
     const int grid = (int)(prm.num_units < num_sms ? prm.num_units : num_sms);
 
-    return dispatch_umma_T(s.T, [&](auto tc) {
+    return dispatch_umma(s.T, s.elem_bytes, [&](auto tc, auto io) {
         constexpr int TT = decltype(tc)::value;
-        const size_t smem = umma_smem_bytes<TT>(prm.b_slot_bytes);
+        using IO = decltype(io);
+        const size_t smem = umma_smem_bytes<TT, sizeof(IO)>(prm.b_slot_bytes);
         static unsigned long long attr_done = 0;              // one bit per device (per instantiation)
         int dev = 0;
         cudaGetDevice(&dev);
         if (!((attr_done >> (dev & 63)) & 1ull)) {
-            cudaError_t e = cudaFuncSetAttribute(umma_linear_kernel<TT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+            cudaError_t e = cudaFuncSetAttribute(umma_linear_kernel<TT, IO>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                  227 * 1024);
             if (e != cudaSuccess) return e;
             attr_done |= 1ull << (dev & 63);
         }
         if (smem > 227 * 1024) return cudaErrorInvalidConfiguration;
-        umma_linear_kernel<TT><<<grid, kThreadsUmma, smem, stream>>>(tmap, tmap_out, prm);
+        umma_linear_kernel<TT, IO><<<grid, kThreadsUmma, smem, stream>>>(tmap, tmap_out, prm);
         return cudaGetLastError();
     });
 }
