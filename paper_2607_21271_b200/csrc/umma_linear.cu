@@ -470,8 +470,10 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
                     float v[T];
 #pragma unroll
                     for (int p = 0; p < T; ++p) v[p] = __uint_as_float(in[p][g]);
+#ifndef EQL_ABLATE_EPIMATH
                     if (prm.bias != nullptr && co0 + g < prm.Cout) v[0] += __ldg(prm.bias + co0 + g);
                     rdft_inverse<T>(v);
+#endif
                     if constexpr (E == 2) {
 #pragma unroll
                         for (int t = 0; t < T; t += 2) o[(g * T + t) / 2] = pack_h2(v[t], v[t + 1]);
