@@ -36,8 +36,8 @@ FALLBACK_BF16_TFLOPS = 1590.0
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per launch from the committed ncu capture
 # profiles/umma_kernels_fp16_vit_b_fc1.md (None = not captured for that workload / kernel).
 NCU_TRAFFIC_BYTES = {
-    ("vit_b_fc1_fp16", "fwd"): 39.8e6 + 101.1e6,
-    ("vit_b_fc1_fp16", "bwd_data"): 156.3e6 + 17.9e6,
+    ("vit_b_fc1_fp16", "fwd"): 39.8e6 + 94.7e6,
+    ("vit_b_fc1_fp16", "bwd_data"): 156.3e6 + 18.5e6,
     ("vit_b_fc1_fp16", "bwd_weight"): 193.7e6 + 3.8e6,
 }
 
@@ -66,7 +66,7 @@ class ClockSampler:
         try:
             self.fh = open(self.path, "w")
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "20"],
                                          stdout=self.fh, stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
@@ -183,7 +183,7 @@ def metric_name(wl):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
