@@ -60,13 +60,18 @@ enum {
      * conjugated when the plan is built). */
     EQL_FLAG_CORRELATION = 1u,
     /* Force the CUDA-core (FFMA) kernels even where a tensor-core kernel exists. */
-    EQL_FLAG_FORCE_SIMT = 2u
+    EQL_FLAG_FORCE_SIMT = 2u,
+    /* Among the tensor-core kernels, always take the streaming one (activations transformed per
+     * output-channel tile) even where the kernel that keeps the transformed activations of a token
+     * tile resident in shared memory applies.  For comparisons and tests. */
+    EQL_FLAG_FORCE_STREAMING = 4u
 };
 
 typedef struct {
     int32_t T, C_in, C_out, dtype;
     uint32_t flags;
-    int32_t fwd_kernel;           /* 0 = CUDA-core FFMA kernel, 1 = tcgen05 tensor-core kernel */
+    int32_t fwd_kernel;           /* 0 = CUDA-core FFMA kernel, 1 = tcgen05 streaming kernel,
+                                     2 = tcgen05 kernel with resident transformed activations */
     int32_t bwd_data_kernel;
     int32_t bwd_weight_kernel;
     int64_t macs_per_token;       /* Step-2 multiply-accumulates of Algorithm 1 per token, exact count */

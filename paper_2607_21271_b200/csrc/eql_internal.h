@@ -71,6 +71,22 @@ cudaError_t launch_build_umma_image(const UmmaLinearShape& s, const float* plane
 cudaError_t launch_umma_linear(const UmmaLinearShape& s, const void* in, void* out, int64_t N, const void* image,
                                const float* bias_f32, int* status, int num_sms, cudaStream_t stream);
 
+// ---- tcgen05 kernel with resident transformed activations (FP16, T = 4 or 8), umma_linear_res.cu -----
+struct UmmaResShape {
+    int T, Cin, Cout;
+    int nTok;           // tokens per tile = 512 / T
+    int nK;             // 16-channel chunks of the reduction dimension, all resident in shared memory
+    int nCT;            // tiles of 128 output channels
+    int w_slots, n_tw;  // weight-ring slots, transform warps
+    bool fits;          // the spectrum of one token tile plus the rings fit in shared memory
+    size_t image_bytes;
+};
+bool umma_res_supported(int T, eql_dtype_t dtype);
+UmmaResShape umma_res_shape(int T, int Cin, int Cout);
+cudaError_t launch_build_umma_res_image(const UmmaResShape& s, const float* planes, void* image, cudaStream_t stream);
+cudaError_t launch_umma_linear_res(const UmmaResShape& s, const void* in, void* out, int64_t N, const void* image,
+                                   const float* bias_f32, int* status, int num_sms, cudaStream_t stream);
+
 // ---- tcgen05 weight-gradient kernel (FP16 inputs), umma_bwd_weight.cu --------------------------------
 struct UmmaBwdWeightShape {
     int T, Ci, Co;
@@ -104,4 +120,5 @@ struct eqlinear_plan_s {
     int fwd_kernel, bwd_data_kernel, bwd_weight_kernel;
     int num_sms;
     eql::UmmaLinearShape umma_fwd, umma_bwd;
+    eql::UmmaResShape res_fwd, res_bwd;   // used when the kernel id is 2
 };

@@ -20,6 +20,11 @@ WorkspaceLayout workspace_layout(int T, int Ci, int Co, eql_dtype_t dtype) {
     if (umma_linear_supported(T, dtype)) {
         l.umma_fwd_bytes = umma_linear_shape(T, Ci, Co, dtype).image_bytes;
         l.umma_bwd_bytes = umma_linear_shape(T, Co, Ci, dtype).image_bytes;
+        if (umma_res_supported(T, dtype)) {          // one region serves whichever tensor-core kernel the plan selects
+            const size_t rf = umma_res_shape(T, Ci, Co).image_bytes, rb = umma_res_shape(T, Co, Ci).image_bytes;
+            if (rf > l.umma_fwd_bytes) l.umma_fwd_bytes = rf;
+            if (rb > l.umma_bwd_bytes) l.umma_bwd_bytes = rb;
+        }
         l.umma_fwd = off;  off += l.umma_fwd_bytes;
         l.umma_bwd = off;  off += l.umma_bwd_bytes;
     }
@@ -63,6 +68,14 @@ eql_status_t build_weights(eqlinear_plan_t p, const void* w, const void* bias, c
     }
     if (p->bwd_data_kernel == 1) {
         e = launch_build_umma_image(p->umma_bwd, (const float*)(p->ws + p->lay.planes_bwd), p->ws + p->lay.umma_bwd, s);
+        if (e != cudaSuccess) return EQL_ERR_CUDA;
+    }
+    if (p->fwd_kernel == 2) {
+        e = launch_build_umma_res_image(p->res_fwd, (const float*)(p->ws + p->lay.planes_fwd), p->ws + p->lay.umma_fwd, s);
+        if (e != cudaSuccess) return EQL_ERR_CUDA;
+    }
+    if (p->bwd_data_kernel == 2) {
+        e = launch_build_umma_res_image(p->res_bwd, (const float*)(p->ws + p->lay.planes_bwd), p->ws + p->lay.umma_bwd, s);
         if (e != cudaSuccess) return EQL_ERR_CUDA;
     }
     return EQL_OK;
@@ -110,7 +123,7 @@ eql_status_t eqlinear_plan(eqlinear_plan_t* plan, int T, int C_in, int C_out, eq
     eql_status_t st = check_shape(T, C_in, C_out, dtype);
     if (st != EQL_OK) return st;
     if (!w || !workspace) return EQL_ERR_INVALID_ARG;
-    if (flags & ~(unsigned)(EQL_FLAG_CORRELATION | EQL_FLAG_FORCE_SIMT)) return EQL_ERR_INVALID_ARG;
+    if (flags & ~(unsigned)(EQL_FLAG_CORRELATION | EQL_FLAG_FORCE_SIMT | EQL_FLAG_FORCE_STREAMING)) return EQL_ERR_INVALID_ARG;
     if (!aligned16(w) || (bias && !aligned16(bias))) return EQL_ERR_ALIGNMENT;
     if (reinterpret_cast<uintptr_t>(workspace) % kWsAlign != 0) return EQL_ERR_ALIGNMENT;
     WorkspaceLayout lay = workspace_layout(T, C_in, C_out, dtype);
@@ -138,6 +151,17 @@ eql_status_t eqlinear_plan(eqlinear_plan_t* plan, int T, int C_in, int C_out, eq
         p->umma_fwd = umma_linear_shape(T, C_in, C_out, dtype);
         p->umma_bwd = umma_linear_shape(T, C_out, C_in, dtype);
         if (umma_bwd_weight_supported(T, dtype)) p->bwd_weight_kernel = 1;
+        // Layers with few input channels: keep the transformed activations of a token tile resident and reuse them
+        // for every output-channel tile (needs a deep weight ring and reasonably full 128-channel tiles).
+        if (umma_res_supported(T, dtype) && !(flags & EQL_FLAG_FORCE_STREAMING)) {
+            auto prefer = [](const UmmaResShape& r) {
+                return r.fits && r.w_slots >= 3 && 2 * r.Cout >= 128 * r.nCT;
+            };
+            p->res_fwd = umma_res_shape(T, C_in, C_out);
+            p->res_bwd = umma_res_shape(T, C_out, C_in);
+            if (prefer(p->res_fwd)) p->fwd_kernel = 2;
+            if (prefer(p->res_bwd)) p->bwd_data_kernel = 2;
+        }
     }
 
     cudaStream_t s = (cudaStream_t)stream;
@@ -194,6 +218,11 @@ eql_status_t eqlinear_fwd(eqlinear_plan_t plan, const void* x, void* y, int64_t 
     if (!x || !y || x == y) return EQL_ERR_INVALID_ARG;
     if (!aligned16(x) || !aligned16(y)) return EQL_ERR_ALIGNMENT;
     const float* bias = plan->has_bias ? (const float*)(plan->ws + plan->lay.bias) : nullptr;
+    if (plan->fwd_kernel == 2) {
+        cudaError_t e = launch_umma_linear_res(plan->res_fwd, x, y, N, plan->ws + plan->lay.umma_fwd, bias,
+                                               (int*)(plan->ws + plan->lay.status), plan->num_sms, (cudaStream_t)stream);
+        return e == cudaSuccess ? EQL_OK : EQL_ERR_CUDA;
+    }
     if (plan->fwd_kernel == 1) {
         cudaError_t e = launch_umma_linear(plan->umma_fwd, x, y, N, plan->ws + plan->lay.umma_fwd, bias,
                                            (int*)(plan->ws + plan->lay.status), plan->num_sms, (cudaStream_t)stream);
@@ -211,6 +240,11 @@ eql_status_t eqlinear_bwd_data(eqlinear_plan_t plan, const void* dy, void* dx, i
     if (N == 0) return EQL_OK;
     if (!dy || !dx || dy == dx) return EQL_ERR_INVALID_ARG;
     if (!aligned16(dy) || !aligned16(dx)) return EQL_ERR_ALIGNMENT;
+    if (plan->bwd_data_kernel == 2) {
+        cudaError_t e = launch_umma_linear_res(plan->res_bwd, dy, dx, N, plan->ws + plan->lay.umma_bwd, nullptr,
+                                               (int*)(plan->ws + plan->lay.status), plan->num_sms, (cudaStream_t)stream);
+        return e == cudaSuccess ? EQL_OK : EQL_ERR_CUDA;
+    }
     if (plan->bwd_data_kernel == 1) {
         cudaError_t e = launch_umma_linear(plan->umma_bwd, dy, dx, N, plan->ws + plan->lay.umma_bwd, nullptr,
                                            (int*)(plan->ws + plan->lay.status), plan->num_sms, (cudaStream_t)stream);

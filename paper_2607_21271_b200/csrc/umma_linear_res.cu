@@ -1,0 +1,502 @@
+// Fused EQ-Linear forward / data-gradient with the transformed activations RESIDENT in shared memory (FP16 I/O,
+// FP32 accumulation in TMEM, T = 4 or 8).  Used where the spectrum of one token tile fits on chip
+// (C_in * T * 2 bytes * 512/T tokens <= ~150 KB), i.e. the layers with few input channels.
+//
+// Compared with the streaming kernel (umma_linear.cu) the roles of the two operands are exchanged: the
+// accumulator holds OUTPUT CHANNELS on the 128 TMEM lanes and (plane, token) on the columns,
+//     D_p[o, n] = sum_i w^_p[o, i] x^_p[n, i]          A = spectral weight tile [128 channels x 16], B = x^ tile [tokens x 16].
+// A work unit is (tile of 512/T tokens, tile of 128 output channels); a CTA owns a contiguous range of units in
+// token-major order, so the group DFT (Eq. 4) of a token tile is computed once and reused by all of its
+// output-channel tiles, and only the spectral weights stream through a ring.
+//
+//   TMA (2-D, 128B swizzle)     raw rows of x, 32 tokens x 128 B per item         -> one ring slot per transform warp
+//   transform warps             group DFT in registers, planes rounded to fp16    -> resident x^ tiles (K-major, 32B swizzle)
+//   TMA (1-D bulk)              spectral-weight image of (channel tile, 16-channel chunk) -> weight ring
+//   1 thread                    tcgen05.mma kind::f16; complex frequency (Eq. 5) as
+//                                   [Re|Im] += Wr [Xr|Xi],   Re += (-Wi) Xi (A negated by the instruction),   Im += Wi Xr
+//   12 warps                    tcgen05.ld, bias on plane k = 0, inverse DFT (Eq. 7), fp16 rounding; a thread owns one
+//                               output channel, so a warp writes 32 channels x T elements of a token as one contiguous run
+//
+// The transform of the next token tile runs while the MMAs of the current tile's last channel tile are in flight
+// (each x^ chunk is rewritten as soon as the MMAs that read it have retired).
+//
+// Every wait on an mbarrier is bounded: on a time-out the CTA raises an abort flag, records a status code for the
+// host, drains its outstanding copies and MMAs, frees its TMEM and returns.
+#include <cuda_fp16.h>
+
+#include <cstring>
+#include <mutex>
+
+#include "eql_internal.h"
+#include "ptx_sm100.cuh"
+#include "rdft.cuh"
+#include "umma_common.cuh"
+
+namespace eql {
+namespace {
+
+constexpr int kThreadsRes = 512;
+constexpr int kTmemColsRes = 512;
+constexpr int kResWarpTmaX = 0, kResWarpMma = 1, kResWarpTmaW = 2, kResWarpCompute0 = 4;
+constexpr int kResComputeWarps = 12;
+constexpr int kItemBytes = 4096;            // raw item: 32 token rows x 128 bytes
+constexpr int kWTileBytes = 4096;           // spectral-weight tile of one plane: [128 channels x 32 B]
+constexpr int kResMaxK = 12;                // resident chunks (barrier array size)
+constexpr int kResMaxWSlots = 4;
+constexpr uint32_t kResSpin = 256;
+constexpr uint32_t kIdescNegateA = 1u << 13;
+
+struct ResParams {
+    void* out;                   // [N, Cout*T] half
+    const uint8_t* image;        // [channel tile][chunk][plane][128 x 32 B], see build_image_res_kernel
+    const float* bias;           // [Cout] or nullptr
+    int* status;
+    int64_t N;
+    int Cin, Cout;
+    int nCT, nK;                 // output-channel tiles, 16-channel chunks
+    int w_slots, n_tw;           // weight-ring slots, transform warps (= raw ring slots)
+    int64_t num_units;           // token tiles x nCT
+};
+
+// Optional timeline instrumentation (compiled only with -DEQL_TRACE): CTA 0 records clock64() stamps.
+#ifdef EQL_TRACE
+__device__ unsigned long long g_trace_res[8192];
+#define RES_STAMP(slot) do { if (blockIdx.x == 0 && (slot) < 8192) g_trace_res[(slot)] = clock64(); } while (0)
+#else
+#define RES_STAMP(slot) do { } while (0)
+#endif
+
+struct ResBarriers {
+    uint64_t full_raw[kResComputeWarps], empty_raw[kResComputeWarps];
+    uint64_t full_x[kResMaxK], empty_x[kResMaxK];
+    uint64_t full_w[kResMaxWSlots], empty_w[kResMaxWSlots];
+    uint64_t full_d[2], empty_d[2], mma_done;
+    uint32_t tmem_base;
+    int abort_flag;
+};
+
+// Spectral-weight operand image: planes[p][cin][cout] (float, scaled, conjugated for the data gradient) ->
+// for every (channel tile ct, chunk kc, plane p) one [128 x 16] half tile in the canonical K-major layout with
+// 32-byte swizzle: byte b of row n lives at n*32 + (((b>>4) ^ ((n>>2)&1))<<4) + (b&15); row n = channel ct*128 + n.
+template <int T>
+__global__ void build_image_res_kernel(const float* __restrict__ planes, int Cin, int Cout, int nCT, int nK,
+                                       __half* __restrict__ image) {
+    const int64_t total = (int64_t)nCT * nK * T * 128 * 16;
+    for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
+         idx += (int64_t)gridDim.x * blockDim.x) {
+        const int within = (int)(idx % (128 * 16));
+        const int64_t tile = idx / (128 * 16);
+        const int p = (int)(tile % T);
+        const int kc = (int)((tile / T) % nK), ct = (int)(tile / ((int64_t)T * nK));
+        const int n = within / 16, c = (within % 16) / 8;
+        const int kk = (c ^ ((n >> 2) & 1)) * 8 + within % 8;
+        const int cin = kc * 16 + kk, cout = ct * 128 + n;
+        float v = 0.f;
+        if (cin < Cin && cout < Cout) v = planes[((size_t)p * Cin + cin) * Cout + cout];
+        image[idx] = __float2half_rn(v);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+template <int T, int NTOK>
+__global__ void __launch_bounds__(kThreadsRes, 1)
+umma_linear_res_kernel(const __grid_constant__ CUtensorMap tmap_in, const ResParams prm) {
+    // NTOK tokens per tile: the accumulator of a unit is T planes x NTOK fp32 TMEM columns.  With T * NTOK = 256 two
+    // accumulators alternate, so that the epilogue of a unit overlaps the MMAs of the next one.
+    constexpr int NBUF = 512 / (T * NTOK);
+    constexpr int kXChunkBytes = T * NTOK * 32; // x^ of one 16-channel chunk: T plane tiles of [NTOK tokens x 32 B]
+    constexpr int NCH = 64 / T;                 // channels per 128-byte raw row
+    constexpr int SPK = 16 / NCH;               // raw slabs (64 elements wide) per 16-channel chunk
+    constexpr int PARTS = NTOK / 32;            // 32-token items per slab
+    constexpr int IPC = SPK * PARTS;            // items per chunk (= 4 for T = 4 and T = 8)
+    constexpr int XT = NTOK * 32;               // bytes of one x^ plane tile [NTOK tokens x 16 channels]
+    constexpr int W = NCH / 2;                  // 32-bit words one raw row contributes to one plane
+    constexpr int kWSlot = T * kWTileBytes;
+    static_assert(T == 4 || T == 8, "resident kernel: T = 4 or 8");
+    static_assert(NBUF == 1 || NBUF == 2, "accumulator count");
+
+    extern __shared__ uint8_t smem_raw_base[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw_base) + 1023) & ~(uintptr_t)1023);
+    const int nK = prm.nK, nCT = prm.nCT, n_tw = prm.n_tw, w_slots = prm.w_slots;
+    uint8_t* raw = smem;                                         // n_tw items
+    uint8_t* xhat = raw + n_tw * kItemBytes;                     // nK chunks
+    uint8_t* wsm = xhat + nK * kXChunkBytes;                     // w_slots slots
+    ResBarriers* bar = reinterpret_cast<ResBarriers*>(wsm + w_slots * kWSlot);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    volatile int* abort_flag = &bar->abort_flag;
+    int* status = prm.status;
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < kResComputeWarps; ++i) { ptx::mbar_init(&bar->full_raw[i], 1); ptx::mbar_init(&bar->empty_raw[i], 1); }
+        for (int i = 0; i < kResMaxK; ++i) { ptx::mbar_init(&bar->full_x[i], IPC); ptx::mbar_init(&bar->empty_x[i], 1); }
+        for (int i = 0; i < kResMaxWSlots; ++i) { ptx::mbar_init(&bar->full_w[i], 1); ptx::mbar_init(&bar->empty_w[i], 1); }
+        for (int i = 0; i < 2; ++i) { ptx::mbar_init(&bar->full_d[i], 1); ptx::mbar_init(&bar->empty_d[i], kResComputeWarps); }
+        ptx::mbar_init(&bar->mma_done, 1);
+        bar->abort_flag = 0;
+        ptx::fence_mbar_init();
+        ptx::prefetch_tensormap(&tmap_in);
+    }
+    if (warp == kResWarpMma) {
+        ptx::tmem_alloc(&bar->tmem_base, kTmemColsRes);
+        ptx::tmem_relinquish();
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::tc_fence_after_sync();
+    const uint32_t tmem_base = bar->tmem_base;
+
+    // this CTA's contiguous range of units; unit u = token tile (u / nCT), channel tile (u % nCT)
+    const int64_t u0 = prm.num_units * (int64_t)blockIdx.x / gridDim.x;
+    const int64_t u1 = prm.num_units * ((int64_t)blockIdx.x + 1) / gridDim.x;
+    auto first_of_tile = [&](int64_t u) { return u == u0 || u % nCT == 0; };
+    auto last_of_tile = [&](int64_t u) { return u == u1 - 1 || u % nCT == nCT - 1; };
+    const int items_per_tile = IPC * nK;
+
+    if (warp == kResWarpTmaX) {
+        // ---------------------------------------------------------------- raw activation rows via TMA
+        if (lane == 0) {
+            uint32_t gi = 0;                                     // running item counter; item gi lives in slot gi % n_tw
+            int slot = 0;
+            uint32_t eph = 1;
+            bool ok = true;
+            for (int64_t u = u0; u < u1 && ok; ++u) {
+                if (!first_of_tile(u)) continue;
+                const int row0 = (int)(u / nCT) * NTOK;
+                for (int i = 0; i < items_per_tile; ++i, ++gi) {
+                    ok = ptx::mbar_wait(&bar->empty_raw[slot], eph, abort_flag, status, 301, true, kResSpin);
+                    if (!ok) break;
+                    ptx::mbar_arrive_expect_tx(&bar->full_raw[slot], kItemBytes);
+                    const int s = i / PARTS, h = i % PARTS;      // slab (64 elements of the row), 32-token part
+                    ptx::tma_load_2d(raw + slot * kItemBytes, &tmap_in, s * 64, row0 + h * 32, &bar->full_raw[slot]);
+                    if (++slot == n_tw) { slot = 0; eph ^= 1u; }
+                }
+            }
+            // drain: every copy this thread issued must have landed before the CTA may exit
+            const uint32_t lo = gi > (uint32_t)n_tw ? gi - n_tw : 0;
+            for (uint32_t c = lo; c < gi; ++c)
+                ptx::mbar_wait(&bar->full_raw[c % n_tw], (c / n_tw) & 1, abort_flag, status, 311, false);
+        }
+    } else if (warp == kResWarpTmaW) {
+        // ---------------------------------------------------------------- spectral-weight tiles via bulk copy
+        if (lane == 0) {
+            uint32_t cw = 0;
+            int slot = 0;
+            uint32_t eph = 1;                                    // parity to wait for on the slot's "empty" barrier
+            bool ok = true;
+            for (int64_t u = u0; u < u1 && ok; ++u) {
+                const int ct = (int)(u % nCT);
+                for (int kc = 0; kc < nK; ++kc, ++cw) {
+                    ok = ptx::mbar_wait(&bar->empty_w[slot], eph, abort_flag, status, 302, true, kResSpin);
+                    if (!ok) break;
+                    ptx::mbar_arrive_expect_tx(&bar->full_w[slot], kWSlot);
+                    ptx::bulk_load_1d(wsm + slot * kWSlot, prm.image + ((size_t)ct * nK + kc) * (size_t)kWSlot, kWSlot,
+                                      &bar->full_w[slot]);
+                    if (++slot == w_slots) { slot = 0; eph ^= 1u; }
+                }
+            }
+            const uint32_t lo = cw > (uint32_t)w_slots ? cw - w_slots : 0;
+            for (uint32_t c = lo; c < cw; ++c)
+                ptx::mbar_wait(&bar->full_w[c % w_slots], (c / w_slots) & 1, abort_flag, status, 312, false);
+        }
+    } else if (warp == kResWarpMma) {
+        // ---------------------------------------------------------------- tensor-core issue (one thread)
+        if (lane == 0) {
+            uint32_t cu = 0, tc = 0;
+            int slot = 0;                                        // weight-ring slot of the current chunk
+            uint32_t wph = 0;                                    // its phase parity
+            bool ok = true;
+            const uint32_t idesc1 = ptx::umma_idesc_f16_f32(128, NTOK);          // one plane of tokens
+            const uint32_t idesc2 = ptx::umma_idesc_f16_f32(128, 2 * NTOK);      // [Re | Im] planes of a complex frequency
+            auto mma = [](uint32_t d, uint32_t a_addr, uint32_t b_addr, uint32_t idesc, uint32_t accumulate) {
+                ptx::umma_f16(d, ptx::umma_smem_desc_k_sw32(a_addr), ptx::umma_smem_desc_k_sw32(b_addr), idesc, accumulate);
+            };
+            for (int64_t u = u0; u < u1 && ok; ++u, ++cu) {
+                const bool first = first_of_tile(u), last = last_of_tile(u);
+                if (first && u != u0) ++tc;
+                RES_STAMP(512 + 2 * cu);
+                const uint32_t buf = cu % NBUF;
+                const uint32_t dbase = tmem_base + buf * (uint32_t)(T * NTOK);
+                ok = ptx::mbar_wait(&bar->empty_d[buf], ((cu / NBUF) & 1) ^ 1, abort_flag, status, 303, true, kResSpin);
+                RES_STAMP(512 + 2 * cu + 1);
+                if (!ok) break;
+                // operands of the unit's first chunk
+                if (first) ok = ptx::mbar_wait(&bar->full_x[0], tc & 1, abort_flag, status, 304, true, kResSpin);
+                ok = ok && ptx::mbar_wait(&bar->full_w[slot], wph, abort_flag, status, 305, true, kResSpin);
+                if (!ok) break;
+                for (int kc = 0; kc < nK; ++kc) {
+                    RES_STAMP(1024 + 4 * (cu * nK + kc));
+                    ptx::tc_fence_after_sync();
+                    const uint32_t a0 = ptx::smem_u32(wsm + slot * kWSlot);      // weight tiles, plane p at p * 4 KB
+                    const uint32_t b0 = ptx::smem_u32(xhat + kc * kXChunkBytes); // x^ tiles, plane p at p * XT
+                    const uint32_t acc = kc > 0 ? 1u : 0u;
+                    int nslot = slot + 1;
+                    uint32_t nwph = wph;
+                    if (nslot == w_slots) { nslot = 0; nwph ^= 1u; }
+                    mma(dbase, a0, b0, idesc1, acc);                                                      // k = 0
+#pragma unroll
+                    for (int f = 1; f < T / 2; ++f) {
+                        const uint32_t dre = dbase + (uint32_t)((2 * f - 1) * NTOK), dim = dre + NTOK;
+                        const uint32_t wr = a0 + (2 * f - 1) * kWTileBytes, wi = wr + kWTileBytes;
+                        const uint32_t xr = b0 + (2 * f - 1) * XT, xi = xr + XT;
+                        mma(dre, wr, xr, idesc2, acc);                                                    // [Re|Im] += Wr [Xr|Xi]
+                        mma(dre, wi, xi, idesc1 | kIdescNegateA, 1u);                                     //  Re     -= Wi Xi
+                        mma(dim, wi, xr, idesc1, 1u);                                                     //  Im     += Wi Xr
+                        if (f == 1 && kc + 1 < nK) {
+                            // The next chunk's operands are checked here, while the tensor pipe still has this chunk's
+                            // MMAs queued, so that the issue stream has no gap between chunks.
+                            RES_STAMP(1024 + 4 * (cu * nK + kc) + 1);
+                            if (first) ok = ptx::mbar_wait(&bar->full_x[kc + 1], tc & 1, abort_flag, status, 304, true, kResSpin);
+                            ok = ok && ptx::mbar_wait(&bar->full_w[nslot], nwph, abort_flag, status, 305, true, kResSpin);
+                            RES_STAMP(1024 + 4 * (cu * nK + kc) + 2);
+                        }
+                    }
+                    mma(dbase + (uint32_t)((T - 1) * NTOK), a0 + (T - 1) * kWTileBytes, b0 + (T - 1) * XT, idesc1, acc);  // k = T/2
+                    ptx::umma_commit(&bar->empty_w[slot]);
+                    if (last) ptx::umma_commit(&bar->empty_x[kc]);  // the tile's x^ chunk may be overwritten once these MMAs retire
+                    RES_STAMP(1024 + 4 * (cu * nK + kc) + 3);
+                    slot = nslot; wph = nwph;
+                    if (!ok) break;
+                }
+                if (ok) ptx::umma_commit(&bar->full_d[buf]);
+            }
+            // all MMAs issued by this thread must have retired before shared memory and TMEM go away
+            ptx::umma_commit(&bar->mma_done);
+            ptx::mbar_wait(&bar->mma_done, 0, abort_flag, status, 313, false);
+        }
+    } else if (warp >= kResWarpCompute0) {
+        // ---------------------------------------------------------------- compute warps: transform and epilogue
+        const int cw = warp - kResWarpCompute0;
+        const int quad = warp & 3;                               // TMEM lane quadrant this warp may read
+        const int third = cw >> 2;                               // share of the token column groups
+        const uint32_t lane_base = tmem_base + ((uint32_t)(quad * 32) << 16);
+        bool ok = true;
+
+        // Group DFT of this warp's items of token tile number tc (the tc-th tile of this CTA).  Items are dealt
+        // round-robin over the transform warps by their running number, so warp cw always reads ring slot cw.
+        uint32_t my_items = 0;                                   // items this warp has taken from its ring slot
+        auto transform_tile = [&](uint32_t tc) {
+            if (cw >= n_tw) return;
+            const uint32_t base = tc * (uint32_t)items_per_tile;
+            // this warp's items of the tile: running numbers congruent to cw modulo n_tw
+            for (int i = (int)((cw + n_tw - base % n_tw) % n_tw); i < items_per_tile && ok; i += n_tw, ++my_items) {
+                ok = ptx::mbar_wait(&bar->full_raw[cw], my_items & 1, abort_flag, status, 306, true, 16);
+                if (!ok) break;
+                uint32_t wd[32];
+                load_slab_row(raw + cw * kItemBytes + lane * 128, lane, wd);
+                // The row is in registers: order these generic-proxy reads before the async-proxy (TMA) refill of
+                // the slot, then release it so that the refill overlaps the transform.
+                ptx::fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(&bar->empty_raw[cw]);
+                uint32_t packed[T][W];
+                dft_words<T, false>(wd, packed, nullptr);
+                const int s = i / PARTS, h = i % PARTS;
+                const int kc = s / SPK, q = s % SPK;
+                const int r = h * 32 + lane;                     // token row inside the tile
+                // the MMAs that read the previous tile's chunk kc must have retired
+                if (tc > 0) {
+                    ok = ptx::mbar_wait(&bar->empty_x[kc], (tc - 1) & 1, abort_flag, status, 307, true, 16);
+                    if (!ok) break;
+                }
+                // x^ plane tile: row r at r*32, its two 16-byte chunks exchanged when bit 2 of r is set (32B swizzle);
+                // this raw row's run of channels starts at byte kb of the row
+                const int kb = q * NCH * 2;
+                const int sw = (r >> 2) & 1;
+                uint8_t* dst = xhat + kc * kXChunkBytes + r * 32 + (((kb >> 4) ^ sw) << 4) + (kb & 15);
+                const int second = sw ? -16 : 16;
+#pragma unroll
+                for (int p = 0; p < T; ++p) store_plane_run<2 * W>(dst + p * XT, packed[p], second);
+                ptx::fence_proxy_async_smem();                   // generic-proxy writes -> visible to the MMA (async proxy)
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(&bar->full_x[kc]);
+            }
+        };
+
+        uint32_t tc = 0, cu = 0;
+        if (u0 < u1) transform_tile(0);
+        for (int64_t u = u0; u < u1 && ok; ++u, ++cu) {
+            // the next token tile is transformed while the MMAs of this tile's last channel tile are in flight
+            if (cw == 0 && lane == 0) RES_STAMP(8 * cu);
+            if (last_of_tile(u) && u + 1 < u1) {
+                ++tc;
+                transform_tile(tc);
+                if (!ok) break;
+            }
+            if (cw == 0 && lane == 0) RES_STAMP(8 * cu + 1);
+            // ---- epilogue of unit u: thread = output channel, columns = (plane, token)
+            const int ct = (int)(u % nCT);
+            const int64_t row0 = (u / nCT) * NTOK;
+            const int o = ct * 128 + quad * 32 + lane;
+            const bool o_ok = o < prm.Cout;
+            const float bias_v = (prm.bias != nullptr && o_ok) ? __ldg(prm.bias + o) : 0.f;
+            const size_t pitch = (size_t)prm.Cout * T * sizeof(__half);
+            uint8_t* out_o = reinterpret_cast<uint8_t*>(prm.out) + (size_t)o * T * sizeof(__half);
+            const uint32_t buf = cu % NBUF;
+            const uint32_t acc_base = lane_base + buf * (uint32_t)(T * NTOK);
+            ok = ptx::mbar_wait(&bar->full_d[buf], (cu / NBUF) & 1, abort_flag, status, 308, true, 16);
+            if (!ok) break;
+            if (cw == 0 && lane == 0) RES_STAMP(8 * cu + 2);
+            ptx::tc_fence_after_sync();
+            constexpr int NG = NTOK / 8;                         // groups of 8 tokens
+            for (int g = third; g < NG; g += 3) {
+                const int n0 = g * 8;
+                uint32_t in[T][8];
+#pragma unroll
+                for (int p = 0; p < T; ++p) ptx::tmem_ld<8>(acc_base + (uint32_t)(p * NTOK + n0), in[p]);
+                ptx::tmem_ld_wait();
+                if (g + 3 >= NG) {                               // this warp's last read of the accumulator
+                    ptx::tc_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) ptx::mbar_arrive(&bar->empty_d[buf]);
+                }
+                uint8_t* dst = out_o + (size_t)(row0 + n0) * pitch;
+                const int rows_left = (int)(prm.N - (row0 + n0) < 8 ? prm.N - (row0 + n0) : 8);   // may be <= 0
+#pragma unroll
+                for (int j = 0; j < 8; ++j, dst += pitch) {
+                    float v[T];
+#pragma unroll
+                    for (int p = 0; p < T; ++p) v[p] = __uint_as_float(in[p][j]);
+                    v[0] += bias_v;
+                    rdft_inverse<T>(v);
+                    if (o_ok && j < rows_left) {
+                        if constexpr (T == 8)
+                            *reinterpret_cast<uint4*>(dst) = make_uint4(pack_h2(v[0], v[1]), pack_h2(v[2], v[3]),
+                                                                        pack_h2(v[4], v[5]), pack_h2(v[6], v[7]));
+                        else
+                            *reinterpret_cast<uint2*>(dst) = make_uint2(pack_h2(v[0], v[1]), pack_h2(v[2], v[3]));
+                    }
+                }
+            }
+            if (cw == 0 && lane == 0) RES_STAMP(8 * cu + 4);
+        }
+    }
+
+    // ---------------------------------------------------------------- teardown (reached by every thread)
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    if (warp == kResWarpMma) {
+        ptx::tc_fence_after_sync();
+        ptx::tmem_dealloc(tmem_base, kTmemColsRes);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------ host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_res_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    });
+    return fn;
+}
+
+constexpr size_t kResSmemLimit = 227 * 1024;
+
+size_t res_smem_bytes(int T, int nTok, int nK, int w_slots, int n_tw) {
+    return 1024 + (size_t)n_tw * kItemBytes + (size_t)nK * T * nTok * 32 + (size_t)w_slots * T * kWTileBytes +
+           sizeof(ResBarriers) + 64;
+}
+
+}  // namespace
+
+#ifdef EQL_TRACE
+extern "C" int eqlinear_debug_read_trace_res(unsigned long long* dst, int n) {
+    cudaDeviceSynchronize();
+    return (int)cudaMemcpyFromSymbol(dst, g_trace_res, sizeof(unsigned long long) * (n < 8192 ? n : 8192));
+}
+extern "C" int eqlinear_debug_clear_trace_res() {
+    static unsigned long long zeros[8192];
+    return (int)cudaMemcpyToSymbol(g_trace_res, zeros, sizeof(zeros));
+}
+#endif
+
+bool umma_res_supported(int T, eql_dtype_t dtype) { return dtype == EQL_FP16 && (T == 4 || T == 8); }
+
+UmmaResShape umma_res_shape(int T, int Cin, int Cout) {
+    UmmaResShape s{};
+    s.T = T; s.Cin = Cin; s.Cout = Cout;
+    s.nTok = 512 / T;                                            // one accumulator filling the 512 TMEM columns
+    s.nK = (Cin + 15) / 16;
+    s.nCT = (Cout + 127) / 128;
+    s.image_bytes = align_up((size_t)s.nCT * s.nK * T * kWTileBytes, kWsAlign);
+    s.fits = false;
+    if (s.nK > kResMaxK) return s;
+    // ring depths in order of preference: the weight stream paces the main loop (3 chunks cover its latency), then
+    // as many transform warps as shared memory allows
+    static const int cand[][2] = {{3, 12}, {3, 8}, {2, 12}, {2, 8}, {2, 4}};
+    for (const auto& c : cand) {
+        if (res_smem_bytes(T, s.nTok, s.nK, c[0], c[1]) <= kResSmemLimit) {
+            s.w_slots = c[0]; s.n_tw = c[1]; s.fits = true;
+            break;
+        }
+    }
+    if (s.fits && s.w_slots == 3 && res_smem_bytes(T, s.nTok, s.nK, 4, s.n_tw) <= kResSmemLimit) s.w_slots = 4;
+    return s;
+}
+
+cudaError_t launch_build_umma_res_image(const UmmaResShape& s, const float* planes, void* image, cudaStream_t stream) {
+    const int64_t total = (int64_t)s.nCT * s.nK * s.T * 128 * 16;
+    const int blocks = (int)((total + 255) / 256 < 4096 ? (total + 255) / 256 : 4096);
+    if (s.T == 4)
+        build_image_res_kernel<4><<<blocks, 256, 0, stream>>>(planes, s.Cin, s.Cout, s.nCT, s.nK, (__half*)image);
+    else if (s.T == 8)
+        build_image_res_kernel<8><<<blocks, 256, 0, stream>>>(planes, s.Cin, s.Cout, s.nCT, s.nK, (__half*)image);
+    else
+        return cudaErrorInvalidValue;
+    return cudaGetLastError();
+}
+
+cudaError_t launch_umma_linear_res(const UmmaResShape& s, const void* in, void* out, int64_t N, const void* image,
+                                   const float* bias_f32, int* status, int num_sms, cudaStream_t stream) {
+    if (!s.fits) return cudaErrorInvalidConfiguration;
+    EncodeTiledFn enc = encode_tiled_res_fn();
+    if (enc == nullptr) return cudaErrorNotSupported;
+    CUtensorMap tmap;
+    {
+        const cuuint64_t gdim[2] = {(cuuint64_t)s.Cin * s.T, (cuuint64_t)N};
+        const cuuint64_t gstr[1] = {(cuuint64_t)s.Cin * s.T * sizeof(__half)};
+        const cuuint32_t box[2] = {64, 32};
+        const cuuint32_t estr[2] = {1, 1};
+        if (enc(&tmap, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(in), gdim, gstr, box, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return cudaErrorInvalidValue;
+    }
+    ResParams prm{};
+    prm.out = out; prm.image = (const uint8_t*)image; prm.bias = bias_f32; prm.status = status;
+    prm.N = N; prm.Cin = s.Cin; prm.Cout = s.Cout; prm.nCT = s.nCT; prm.nK = s.nK;
+    prm.w_slots = s.w_slots; prm.n_tw = s.n_tw;
+    prm.num_units = ((N + s.nTok - 1) / s.nTok) * s.nCT;
+    const int grid = (int)(prm.num_units < num_sms ? prm.num_units : num_sms);
+    const size_t smem = res_smem_bytes(s.T, s.nTok, s.nK, s.w_slots, s.n_tw);
+
+    auto go = [&](auto tc, auto nt) -> cudaError_t {
+        constexpr int TT = decltype(tc)::value, NT = decltype(nt)::value;
+        static unsigned long long attr_done = 0;
+        int dev = 0;
+        cudaGetDevice(&dev);
+        if (!((attr_done >> (dev & 63)) & 1ull)) {
+            cudaError_t e = cudaFuncSetAttribute(umma_linear_res_kernel<TT, NT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                 (int)kResSmemLimit);
+            if (e != cudaSuccess) return e;
+            attr_done |= 1ull << (dev & 63);
+        }
+        umma_linear_res_kernel<TT, NT><<<grid, kThreadsRes, smem, stream>>>(tmap, prm);
+        return cudaGetLastError();
+    };
+    if (s.T == 4 && s.nTok == 128) return go(std::integral_constant<int, 4>{}, std::integral_constant<int, 128>{});
+    if (s.T == 4 && s.nTok == 64) return go(std::integral_constant<int, 4>{}, std::integral_constant<int, 64>{});
+    if (s.T == 8 && s.nTok == 64) return go(std::integral_constant<int, 8>{}, std::integral_constant<int, 64>{});
+    return cudaErrorInvalidValue;
+}
+
+}  // namespace eql
