@@ -65,6 +65,28 @@ def test_shapes(dtype, T, Ci, Co):
         assert v <= TOL[dtype], f"T={T} Ci={Ci} Co={Co} {dtype}: {k} error {v:.3e}"
 
 
+# ------------------------------------------------------------------ the two tensor-core kernels of fwd / bwd_data
+@pytest.mark.parametrize("T,Ci,Co,N,ids", [(8, 96, 384, 1000, (2, 1)), (8, 24, 200, 777, (2, 1)), (8, 10, 64, 130, (2, 1)),
+                                             (8, 16, 520, 6500, (2, 1)), (8, 64, 64, 900, (2, 2)), (4, 24, 96, 1111, (2, 1)),
+                                             (4, 100, 130, 515, (2, 2)), (4, 8, 300, 20000, (2, 1))])
+def test_resident_and_streaming_kernels_agree_with_oracle(T, Ci, Co, N, ids):
+    """Layers with few input channels run the kernel that keeps a token tile's spectrum in shared memory (id 2);
+    EQL_FLAG_FORCE_STREAMING selects the streaming kernel (id 1) for the same plan shape.  Both must meet the bar,
+    on channel counts that are not multiples of the 128-channel / 16-channel tiles, ragged token counts, and token
+    counts large enough that a CTA's range of work starts and ends in the middle of a token tile."""
+    wl = Workload("res", "fp16", T, Ci, Co, N, "normal", ("fwd", "bwd_data"), 21)
+    data = eq.workloads.generate(wl)
+    for flags, want in ((0, ids), (eq.EQL_FLAG_FORCE_STREAMING, (1, 1))):
+        layer = GpuLayer(T, Ci, Co, "fp16", data["w"], data["bias"], flags)
+        try:
+            info = eq.eqlinear_plan_info(layer.plan)
+            assert (info.fwd_kernel, info.bwd_data_kernel) == want
+        finally:
+            layer.close()
+        for k, v in check_workload(wl, flags=flags, data=data).items():
+            assert v <= TOL["fp16"], f"T={T} Ci={Ci} Co={Co} N={N} flags={flags}: {k} error {v:.3e}"
+
+
 @pytest.mark.parametrize("dtype", ["fp32", "fp16"])
 def test_paper_parity_shape(dtype):
     """The shape of the paper's numerical-equivalence table (Table 4): (B, N, c, T) = (32, 1024, 64, 4)."""
