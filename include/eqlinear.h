@@ -188,10 +188,15 @@ eql_status_t eqlinear_bwd_weight_static(eqlinear_plan_t plan, const void* x, con
 
 /* ---- host-buffer variants (end-to-end measurement, small-batch convenience) ------------------ */
 /* Same operations with HOST input/output buffers (pinned memory recommended).  Each call copies
- * its inputs into the caller's device staging buffers on `stream`, runs the kernels above and
- * copies the results back, all asynchronously on `stream`; the host buffers may be read once the
- * stream has been synchronised.  Staging buffers are device memory with the sizes of the
- * corresponding device-variant tensors. */
+ * its inputs into the caller's device staging buffers, runs the kernels above and copies the
+ * results back, all asynchronously; the host buffers may be read once `stream` has been
+ * synchronised.  Staging buffers are device memory with the sizes of the corresponding
+ * device-variant tensors.
+ * eqlinear_fwd_host and eqlinear_step_host move batches of 8192 tokens or more in up to eight token
+ * chunks through a three-stream pipeline (host -> device copies, kernels on `stream`, device -> host
+ * copies), so that both copy directions and the kernels overlap; `stream` waits for the last copy
+ * before the call's remaining work.  The two extra streams and their events belong to the plan:
+ * created at the first such call, destroyed by eqlinear_plan_destroy (no device memory). */
 eql_status_t eqlinear_fwd_host(eqlinear_plan_t plan, const void* x_host, void* y_host, int64_t N,
                                void* x_staging, void* y_staging, void* stream);
 eql_status_t eqlinear_bwd_data_host(eqlinear_plan_t plan, const void* dy_host, void* dx_host, int64_t N,

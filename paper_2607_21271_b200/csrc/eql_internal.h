@@ -108,6 +108,16 @@ cudaError_t launch_bwd_weight_finalize(int T, bool correlation, const float* scr
 
 }  // namespace eql
 
+// Copy pipeline of the host-buffer entry points: token chunks travel host -> device on one stream, are computed on
+// the caller's stream and travel back on a third, so that the two copy directions and the kernels overlap.
+// Created on first use, destroyed with the plan (streams and events only: no device memory).
+constexpr int kHostChunks = 8;
+struct HostPipe {
+    cudaStream_t in = nullptr, out = nullptr;
+    cudaEvent_t start = nullptr, out_done = nullptr;
+    cudaEvent_t in_done[kHostChunks] = {}, out_ready[kHostChunks] = {};
+};
+
 // The host object behind eqlinear_plan_t.
 struct eqlinear_plan_s {
     int T, Ci, Co;
@@ -121,4 +131,5 @@ struct eqlinear_plan_s {
     int num_sms;
     eql::UmmaLinearShape umma_fwd, umma_bwd;
     eql::UmmaResShape res_fwd, res_bwd;   // used when the kernel id is 2
+    HostPipe* pipe = nullptr;
 };

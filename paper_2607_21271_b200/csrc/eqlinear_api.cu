@@ -81,6 +81,87 @@ eql_status_t build_weights(eqlinear_plan_t p, const void* w, const void* bias, c
     return EQL_OK;
 }
 
+void destroy_pipe(HostPipe* hp) {
+    if (!hp) return;
+    if (hp->in) cudaStreamDestroy(hp->in);
+    if (hp->out) cudaStreamDestroy(hp->out);
+    if (hp->start) cudaEventDestroy(hp->start);
+    if (hp->out_done) cudaEventDestroy(hp->out_done);
+    for (int i = 0; i < kHostChunks; ++i) {
+        if (hp->in_done[i]) cudaEventDestroy(hp->in_done[i]);
+        if (hp->out_ready[i]) cudaEventDestroy(hp->out_ready[i]);
+    }
+    delete hp;
+}
+
+HostPipe* get_pipe(eqlinear_plan_t p) {
+    if (p->pipe) return p->pipe;
+    HostPipe* hp = new (std::nothrow) HostPipe();
+    if (!hp) return nullptr;
+    bool ok = cudaStreamCreateWithFlags(&hp->in, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaStreamCreateWithFlags(&hp->out, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaEventCreateWithFlags(&hp->start, cudaEventDisableTiming) == cudaSuccess &&
+              cudaEventCreateWithFlags(&hp->out_done, cudaEventDisableTiming) == cudaSuccess;
+    for (int i = 0; i < kHostChunks && ok; ++i)
+        ok = cudaEventCreateWithFlags(&hp->in_done[i], cudaEventDisableTiming) == cudaSuccess &&
+             cudaEventCreateWithFlags(&hp->out_ready[i], cudaEventDisableTiming) == cudaSuccess;
+    if (!ok) { destroy_pipe(hp); return nullptr; }
+    p->pipe = hp;
+    return hp;
+}
+
+// Tokens per chunk of the copy pipeline: whole 128-token tiles, at most kHostChunks chunks; small batches travel whole.
+int64_t host_chunk_tokens(int64_t N) {
+    if (N < 8192) return N;
+    const int64_t per = (N + kHostChunks - 1) / kHostChunks;
+    return (per + 127) / 128 * 128;
+}
+
+// fwd (and, with dy/dx, the data gradient) of N tokens from host buffers through the three-stream pipeline.
+// On return every copy and kernel has been enqueued and `s` waits for the last device -> host copy.
+eql_status_t pipelined_host(eqlinear_plan_t plan, const void* x_host, const void* dy_host, void* y_host, void* dx_host,
+                            int64_t N, void* x_staging, void* dy_staging, void* y_staging, void* dx_staging,
+                            cudaStream_t s) {
+    HostPipe* hp = get_pipe(plan);
+    if (!hp) return EQL_ERR_CUDA;
+    const size_t e = elem_size(plan->dtype);
+    const size_t xrow = (size_t)plan->Ci * plan->T * e, yrow = (size_t)plan->Co * plan->T * e;
+    const int64_t chunk = host_chunk_tokens(N);
+    // the copy streams start after whatever the caller's stream did before (earlier users of the staging buffers)
+    if (cudaEventRecord(hp->start, s) != cudaSuccess) return EQL_ERR_CUDA;
+    if (cudaStreamWaitEvent(hp->in, hp->start, 0) != cudaSuccess) return EQL_ERR_CUDA;
+    if (cudaStreamWaitEvent(hp->out, hp->start, 0) != cudaSuccess) return EQL_ERR_CUDA;
+    int c = 0;
+    for (int64_t n0 = 0; n0 < N; n0 += chunk, ++c) {
+        const int64_t n = N - n0 < chunk ? N - n0 : chunk;
+        const char* xh = (const char*)x_host + n0 * xrow;
+        char* xs = (char*)x_staging + n0 * xrow;
+        char* ys = (char*)y_staging + n0 * yrow;
+        if (cudaMemcpyAsync(xs, xh, n * xrow, cudaMemcpyHostToDevice, hp->in) != cudaSuccess) return EQL_ERR_CUDA;
+        if (dy_host &&
+            cudaMemcpyAsync((char*)dy_staging + n0 * yrow, (const char*)dy_host + n0 * yrow, n * yrow,
+                            cudaMemcpyHostToDevice, hp->in) != cudaSuccess) return EQL_ERR_CUDA;
+        if (cudaEventRecord(hp->in_done[c], hp->in) != cudaSuccess) return EQL_ERR_CUDA;
+        if (cudaStreamWaitEvent(s, hp->in_done[c], 0) != cudaSuccess) return EQL_ERR_CUDA;
+        eql_status_t st = eqlinear_fwd(plan, xs, ys, n, s);
+        if (st != EQL_OK) return st;
+        if (dy_host) {
+            st = eqlinear_bwd_data(plan, (char*)dy_staging + n0 * yrow, (char*)dx_staging + n0 * xrow, n, s);
+            if (st != EQL_OK) return st;
+        }
+        if (cudaEventRecord(hp->out_ready[c], s) != cudaSuccess) return EQL_ERR_CUDA;
+        if (cudaStreamWaitEvent(hp->out, hp->out_ready[c], 0) != cudaSuccess) return EQL_ERR_CUDA;
+        if (cudaMemcpyAsync((char*)y_host + n0 * yrow, ys, n * yrow, cudaMemcpyDeviceToHost, hp->out) != cudaSuccess)
+            return EQL_ERR_CUDA;
+        if (dy_host &&
+            cudaMemcpyAsync((char*)dx_host + n0 * xrow, (char*)dx_staging + n0 * xrow, n * xrow, cudaMemcpyDeviceToHost,
+                            hp->out) != cudaSuccess) return EQL_ERR_CUDA;
+    }
+    if (cudaEventRecord(hp->out_done, hp->out) != cudaSuccess) return EQL_ERR_CUDA;
+    if (cudaStreamWaitEvent(s, hp->out_done, 0) != cudaSuccess) return EQL_ERR_CUDA;
+    return EQL_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -206,6 +287,7 @@ eql_status_t eqlinear_plan_device_status(eqlinear_plan_t plan, void* stream) {
 }
 
 eql_status_t eqlinear_plan_destroy(eqlinear_plan_t plan) {
+    if (plan) destroy_pipe(plan->pipe);
     delete plan;
     return EQL_OK;
 }
@@ -306,14 +388,8 @@ eql_status_t eqlinear_fwd_host(eqlinear_plan_t plan, const void* x_host, void* y
     if (st != EQL_OK) return st;
     if (N == 0) return EQL_OK;
     if (!x_host || !y_host || !x_staging || !y_staging) return EQL_ERR_INVALID_ARG;
-    cudaStream_t s = (cudaStream_t)stream;
-    const size_t e = elem_size(plan->dtype);
-    const size_t xb = (size_t)N * plan->Ci * plan->T * e, yb = (size_t)N * plan->Co * plan->T * e;
-    if (cudaMemcpyAsync(x_staging, x_host, xb, cudaMemcpyHostToDevice, s) != cudaSuccess) return EQL_ERR_CUDA;
-    st = eqlinear_fwd(plan, x_staging, y_staging, N, stream);
-    if (st != EQL_OK) return st;
-    if (cudaMemcpyAsync(y_host, y_staging, yb, cudaMemcpyDeviceToHost, s) != cudaSuccess) return EQL_ERR_CUDA;
-    return EQL_OK;
+    return pipelined_host(plan, x_host, nullptr, y_host, nullptr, N, x_staging, nullptr, y_staging, nullptr,
+                          (cudaStream_t)stream);
 }
 
 eql_status_t eqlinear_bwd_data_host(eqlinear_plan_t plan, const void* dy_host, void* dx_host, int64_t N,
@@ -370,14 +446,10 @@ eql_status_t eqlinear_step_host(eqlinear_plan_t plan, const void* x_host, const 
     if (!x_staging || !dy_staging || !y_staging || !dx_staging || !dw_staging) return EQL_ERR_INVALID_ARG;
     if ((db_host != nullptr) != (db_staging != nullptr)) return EQL_ERR_INVALID_ARG;
     cudaStream_t s = (cudaStream_t)stream;
-    const size_t e = elem_size(plan->dtype);
-    const size_t xb = (size_t)N * plan->Ci * plan->T * e, yb = (size_t)N * plan->Co * plan->T * e;
-    if (cudaMemcpyAsync(x_staging, x_host, xb, cudaMemcpyHostToDevice, s) != cudaSuccess) return EQL_ERR_CUDA;
-    if (cudaMemcpyAsync(dy_staging, dy_host, yb, cudaMemcpyHostToDevice, s) != cudaSuccess) return EQL_ERR_CUDA;
-    if ((st = eqlinear_fwd(plan, x_staging, y_staging, N, stream)) != EQL_OK) return st;
-    if (cudaMemcpyAsync(y_host, y_staging, yb, cudaMemcpyDeviceToHost, s) != cudaSuccess) return EQL_ERR_CUDA;
-    if ((st = eqlinear_bwd_data(plan, dy_staging, dx_staging, N, stream)) != EQL_OK) return st;
-    if (cudaMemcpyAsync(dx_host, dx_staging, xb, cudaMemcpyDeviceToHost, s) != cudaSuccess) return EQL_ERR_CUDA;
+    // forward and data gradient chunk by chunk while the copies of the neighbouring chunks are in flight; the weight
+    // gradient reduces over all tokens and runs once every chunk has arrived
+    st = pipelined_host(plan, x_host, dy_host, y_host, dx_host, N, x_staging, dy_staging, y_staging, dx_staging, s);
+    if (st != EQL_OK) return st;
     if ((st = eqlinear_bwd_weight(plan, x_staging, dy_staging, dw_staging, db_staging, N, scratch, scratch_bytes,
                                   stream)) != EQL_OK) return st;
     if (cudaMemcpyAsync(dw_host, dw_staging, (size_t)plan->Co * plan->Ci * plan->T * sizeof(float),

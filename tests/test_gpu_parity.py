@@ -207,8 +207,10 @@ def test_gpu_equivariance_and_adjoint(dtype, T):
 
 
 # ------------------------------------------------------------------ host-buffer variants
-def test_host_buffer_variants():
-    wl = Workload("host", "fp16", 8, 24, 40, 700, "normal", ("fwd", "bwd_data", "bwd_weight"), 20)
+@pytest.mark.parametrize("N", [700, 9001])
+def test_host_buffer_variants(N):
+    """N = 9001 goes through the chunked three-stream copy pipeline (eight chunks, the last one ragged)."""
+    wl = Workload("host", "fp16", 8, 24, 40, N, "normal", ("fwd", "bwd_data", "bwd_weight"), 20)
     d = generate(wl)
     layer = GpuLayer(wl.T, wl.Ci, wl.Co, wl.dtype, d["w"], d["bias"])
     try:
@@ -227,10 +229,21 @@ def test_host_buffer_variants():
         eq.eqlinear_bwd_data_host(layer.plan, dyh, dxh, N, dys, dxs, layer.stream)
         eq.eqlinear_bwd_weight_host(layer.plan, xh, dyh, dwh, dbh, N, xs, dys, dws, dbs, sc, sb, layer.stream)
         torch.cuda.synchronize()
-        assert rel_max_err(yh.numpy(), orc.fwd(d["x"], d["w"], d["bias"])) <= TOL["fp16"]
-        assert rel_max_err(dxh.numpy(), orc.bwd_data(d["dy"], d["w"])) <= TOL["fp16"]
+        ry, rdx = orc.fwd(d["x"], d["w"], d["bias"]), orc.bwd_data(d["dy"], d["w"])
         rdw, rdb = orc.bwd_weight(d["x"], d["dy"], wl.T)
+        assert rel_max_err(yh.numpy(), ry) <= TOL["fp16"]
+        assert rel_max_err(dxh.numpy(), rdx) <= TOL["fp16"]
         assert rel_max_err(dwh.numpy(), rdw) <= TOL["fp16"]
         assert rel_max_err(dbh.numpy(), rdb) <= TOL["fp16"]
+        # the whole step in one call, twice in a row on the same buffers
+        for _ in range(2):
+            for t in (yh, dxh, dwh, dbh):
+                t.zero_()
+            eq.eqlinear_step_host(layer.plan, xh, dyh, yh, dxh, dwh, dbh, N, xs, dys, ys, dxs, dws, dbs, sc, sb, layer.stream)
+            torch.cuda.synchronize()
+            assert rel_max_err(yh.numpy(), ry) <= TOL["fp16"]
+            assert rel_max_err(dxh.numpy(), rdx) <= TOL["fp16"]
+            assert rel_max_err(dwh.numpy(), rdw) <= TOL["fp16"]
+            assert rel_max_err(dbh.numpy(), rdb) <= TOL["fp16"]
     finally:
         layer.close()
