@@ -11,7 +11,7 @@
 //   1 thread                  tcgen05.mma: A = x^ plane (M = input channels), B = dy^ planes
 //                             real k:     D_k          += X_k^T G_k
 //                             complex k: [Re | Im] dW^ += Xr^T [Gr | Gi] + Xi^T [Gi | -Gr]
-//   4 warps (after the loop)  tcgen05.ld -> partial spectra in scratch;  db partials from plane k = 0
+//   12 warps (after the loop) tcgen05.ld -> partial spectra in scratch;  db partials from plane k = 0
 //
 // All mbarrier waits are bounded (see ptx_sm100.cuh); on a time-out the CTA drains and returns.
 #include <cuda_fp16.h>
@@ -47,6 +47,14 @@ struct BwParams {
     int xhat_bytes, stage_bytes;
     int x3d, y3d;                // tensor maps are 3-D (64 elements, rows, slab index): one load per chunk and tensor
 };
+
+// Optional timeline instrumentation (compiled only with -DEQL_TRACE): CTA 0 records clock64() stamps.
+#ifdef EQL_TRACE
+__device__ unsigned long long g_trace_bw[8192];
+#define BW_STAMP(slot) do { if (blockIdx.x == 0 && (slot) < 8192) g_trace_bw[(slot)] = clock64(); } while (0)
+#else
+#define BW_STAMP(slot) do { } while (0)
+#endif
 
 struct BwBarriers {
     uint64_t full_raw[kRawSlots], empty_raw[kRawSlots];
@@ -111,6 +119,7 @@ umma_bwd_weight_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
                 const int slot = (int)(c % kRawSlots);
                 ok = ptx::mbar_wait(&bar->empty_raw[slot], (uint32_t)((c / kRawSlots) & 1) ^ 1, abort_flag, status, 201);
                 if (!ok) break;
+                BW_STAMP(3000 + (int)c);
                 ptx::mbar_arrive_expect_tx(&bar->full_raw[slot], bytes);
                 const int row = (int)((chunk0 + c) * kChunkTok);
                 uint8_t* dst = raw + slot * kRawSlot;
@@ -144,7 +153,9 @@ umma_bwd_weight_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
             const uint32_t a_plane = (uint32_t)CiT * 32u, b_tile = (uint32_t)CoT * 32u;
             for (int64_t c = 0; c < nchunks; ++c) {
                 const int st = (int)(c % kStages);
+                BW_STAMP(1000 + 3 * (int)c);
                 ok = ptx::mbar_wait(&bar->full_ab[st], (uint32_t)((c / kStages) & 1), abort_flag, status, 202);
+                BW_STAMP(1000 + 3 * (int)c + 1);
                 if (!ok) break;
                 ptx::tc_fence_after_sync();
                 const uint32_t a0 = ptx::smem_u32(stages + st * prm.stage_bytes);
@@ -164,6 +175,7 @@ umma_bwd_weight_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
                 ptx::umma_f16(tmem_base + (uint32_t)((T - 1) * CoT), ptx::umma_smem_desc(a0 + (T - 1) * a_plane, 128, 256),
                               ptx::umma_smem_desc(b0 + (uint32_t)(1 + 3 * (T / 2 - 1)) * b_tile, 128, 256), idesc_real, acc);
                 ptx::umma_commit(&bar->empty_ab[st]);
+                BW_STAMP(1000 + 3 * (int)c + 2);
             }
             if (ok) ptx::umma_commit(&bar->full_d);
             ptx::umma_commit(&bar->mma_done);
@@ -182,8 +194,19 @@ umma_bwd_weight_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
         bool ok = true;
         for (int64_t c = 0; c < nchunks; ++c) {
             const int slot = (int)(c % kRawSlots), st = (int)(c % kStages);
-            ok = ptx::mbar_wait(&bar->full_raw[slot], (uint32_t)((c / kRawSlots) & 1), abort_flag, status, 203) &&
-                 ptx::mbar_wait(&bar->empty_ab[st], (uint32_t)((c / kStages) & 1) ^ 1, abort_flag, status, 204);
+#ifdef EQL_TRACE
+            const bool tr = lane == 0 && (warp == kWarpDftX0 || warp == kWarpDftY0);
+            const int tb = (warp == kWarpDftX0 ? 4000 : 5000) + 6 * (int)c;
+            if (tr) BW_STAMP(tb);
+#endif
+            ok = ptx::mbar_wait(&bar->full_raw[slot], (uint32_t)((c / kRawSlots) & 1), abort_flag, status, 203);
+#ifdef EQL_TRACE
+            if (tr) BW_STAMP(tb + 1);
+#endif
+            ok = ok && ptx::mbar_wait(&bar->empty_ab[st], (uint32_t)((c / kStages) & 1) ^ 1, abort_flag, status, 204);
+#ifdef EQL_TRACE
+            if (tr) BW_STAMP(tb + 2);
+#endif
             if (!ok) break;
             uint32_t wd[32];
             if (active)
@@ -232,6 +255,9 @@ umma_bwd_weight_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
             ptx::fence_proxy_async_smem();
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(&bar->full_ab[st]);
+#ifdef EQL_TRACE
+            if (tr) BW_STAMP(tb + 3);
+#endif
         }
         // db partial of this token range: sum over the 16 token rows of each half warp
         if (is_y) {
@@ -247,9 +273,11 @@ umma_bwd_weight_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
                     prm.db_part[(size_t)split * prm.Co + co] = v;
             }
         }
-        // ------------------------------------------------------------ epilogue: TMEM -> partial spectra (warps 4..7)
-        if (ok && warp < kWarpDftX0 + 4) {
+        // ------------------------------------------------------------ epilogue: TMEM -> partial spectra
+        // all 12 warps: a warp reads the TMEM lane quadrant (warp & 3) and every third group of 16 columns
+        if (ok) {
             const int quad = warp & 3;
+            const int third = (warp - kWarpDftX0) >> 2;
             const int ci_local = quad * 32 + lane;
             const int ci = ci_tile * CiT + ci_local;
             const bool lane_ok = ci_local < CiT && ci < prm.Ci;
@@ -259,7 +287,7 @@ umma_bwd_weight_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
                 const uint32_t lane_base = tmem_base + ((uint32_t)(quad * 32) << 16);
                 const size_t plane_stride = (size_t)prm.Co * prm.Ci;
                 float* dst = prm.part + (size_t)split * T * plane_stride;
-                for (int col = 0; col < T * CoT; col += 16) {
+                for (int col = third * 16; col < T * CoT; col += 48) {
                     uint32_t v[16];
                     if (nchunks > 0) {
                         ptx::tmem_ld<16>(lane_base + (uint32_t)col, v);
@@ -334,6 +362,13 @@ int balanced_tile(int C, int max_tile, int round) {
 }
 
 }  // namespace
+
+#ifdef EQL_TRACE
+extern "C" int eqlinear_debug_read_trace_bw(unsigned long long* dst, int n) {
+    cudaDeviceSynchronize();
+    return (int)cudaMemcpyFromSymbol(dst, g_trace_bw, sizeof(unsigned long long) * (n < 8192 ? n : 8192));
+}
+#endif
 
 bool umma_bwd_weight_supported(int T, eql_dtype_t dtype) {
     return dtype == EQL_FP16 && (T == 4 || T == 8 || T == 16 || T == 32);
