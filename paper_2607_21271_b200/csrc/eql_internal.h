@@ -75,10 +75,12 @@ cudaError_t launch_umma_linear(const UmmaLinearShape& s, const void* in, void* o
 struct UmmaResShape {
     int T, Cin, Cout;
     int nTok;           // tokens per tile = 512 / T
-    int nK;             // 16-channel chunks of the reduction dimension, all resident in shared memory
+    int nK;             // 16-channel chunks of the reduction dimension
+    int x_slots;        // x^ chunk buffers in shared memory: nK (token tile resident) or a ring of 3 (one channel tile)
     int nCT;            // tiles of 128 output channels
     int w_slots, n_tw;  // weight-ring slots, transform warps
     bool fits;          // the spectrum of one token tile plus the rings fit in shared memory
+    bool paired;        // x^ also keeps -Re of the complex frequencies: two MMAs per complex frequency instead of three
     size_t image_bytes;
 };
 bool umma_res_supported(int T, eql_dtype_t dtype);

@@ -55,6 +55,7 @@ struct ResParams {
     int Cin, Cout;
     int nCT, nK;                 // output-channel tiles, 16-channel chunks
     int w_slots, n_tw;           // weight-ring slots, transform warps (= raw ring slots)
+    int x_slots;                 // x^ chunk buffers: nK (a whole token tile resident) or, with one channel tile, a ring of 3
     int64_t num_units;           // token tiles x nCT
 };
 
@@ -98,13 +99,18 @@ __global__ void build_image_res_kernel(const float* __restrict__ planes, int Cin
 }
 
 // ------------------------------------------------------------------------------------------------
-template <int T, int NTOK>
+// PF ("paired form"): x^ additionally keeps -Re x^ of every complex frequency, stored as tiles [Re | Im | -Re], so that a
+// complex frequency takes two MMAs of width 2 NTOK ([Re|Im] += Wr [Xr|Xi] and, with A negated, += (-Wi) [Xi|-Xr])
+// instead of three; an MMA costs about the same whatever its width, so this shortens the main loop where the larger
+// x^ buffers fit.
+template <int T, int NTOK, bool PF>
 __global__ void __launch_bounds__(kThreadsRes, 1)
 umma_linear_res_kernel(const __grid_constant__ CUtensorMap tmap_in, const ResParams prm) {
     // NTOK tokens per tile: the accumulator of a unit is T planes x NTOK fp32 TMEM columns.  With T * NTOK = 256 two
     // accumulators alternate, so that the epilogue of a unit overlaps the MMAs of the next one.
     constexpr int NBUF = 512 / (T * NTOK);
-    constexpr int kXChunkBytes = T * NTOK * 32; // x^ of one 16-channel chunk: T plane tiles of [NTOK tokens x 32 B]
+    constexpr int XTILES = PF ? 2 + 3 * (T / 2 - 1) : T;   // plane tiles per chunk
+    constexpr int kXChunkBytes = XTILES * NTOK * 32;       // x^ of one 16-channel chunk: tiles of [NTOK tokens x 32 B]
     constexpr int NCH = 64 / T;                 // channels per 128-byte raw row
     constexpr int SPK = 16 / NCH;               // raw slabs (64 elements wide) per 16-channel chunk
     constexpr int PARTS = NTOK / 32;            // 32-token items per slab
@@ -117,10 +123,10 @@ umma_linear_res_kernel(const __grid_constant__ CUtensorMap tmap_in, const ResPar
 
     extern __shared__ uint8_t smem_raw_base[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw_base) + 1023) & ~(uintptr_t)1023);
-    const int nK = prm.nK, nCT = prm.nCT, n_tw = prm.n_tw, w_slots = prm.w_slots;
+    const int nK = prm.nK, nCT = prm.nCT, n_tw = prm.n_tw, w_slots = prm.w_slots, XR = prm.x_slots;
     uint8_t* raw = smem;                                         // n_tw items
-    uint8_t* xhat = raw + n_tw * kItemBytes;                     // nK chunks
-    uint8_t* wsm = xhat + nK * kXChunkBytes;                     // w_slots slots
+    uint8_t* xhat = raw + n_tw * kItemBytes;                     // XR chunk buffers
+    uint8_t* wsm = xhat + XR * kXChunkBytes;                     // w_slots slots
     ResBarriers* bar = reinterpret_cast<ResBarriers*>(wsm + w_slots * kWSlot);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -149,8 +155,11 @@ umma_linear_res_kernel(const __grid_constant__ CUtensorMap tmap_in, const ResPar
     // this CTA's contiguous range of units; unit u = token tile (u / nCT), channel tile (u % nCT)
     const int64_t u0 = prm.num_units * (int64_t)blockIdx.x / gridDim.x;
     const int64_t u1 = prm.num_units * ((int64_t)blockIdx.x + 1) / gridDim.x;
-    auto first_of_tile = [&](int64_t u) { return u == u0 || u % nCT == 0; };
-    auto last_of_tile = [&](int64_t u) { return u == u1 - 1 || u % nCT == nCT - 1; };
+    // every role walks the units with a running (token tile, channel tile) pair instead of dividing per unit
+    const int ct0 = (int)(u0 % nCT);
+    const int64_t tt0 = u0 / nCT;
+    auto first_of_tile = [&](int64_t u, int ct) { return u == u0 || ct == 0; };
+    auto last_of_tile = [&](int64_t u, int ct) { return u == u1 - 1 || ct == nCT - 1; };
     const int items_per_tile = IPC * nK;
 
     if (warp == kResWarpTmaX) {
@@ -160,9 +169,12 @@ umma_linear_res_kernel(const __grid_constant__ CUtensorMap tmap_in, const ResPar
             int slot = 0;
             uint32_t eph = 1;
             bool ok = true;
-            for (int64_t u = u0; u < u1 && ok; ++u) {
-                if (!first_of_tile(u)) continue;
-                const int row0 = (int)(u / nCT) * NTOK;
+            int ct = ct0;
+            int64_t tt = tt0;
+            for (int64_t u = u0; u < u1 && ok; ++u, ++ct) {
+                if (ct == nCT) { ct = 0; ++tt; }
+                if (!first_of_tile(u, ct)) continue;
+                const int row0 = (int)tt * NTOK;
                 for (int i = 0; i < items_per_tile; ++i, ++gi) {
                     ok = ptx::mbar_wait(&bar->empty_raw[slot], eph, abort_flag, status, 301, true, kResSpin);
                     if (!ok) break;
@@ -184,8 +196,9 @@ umma_linear_res_kernel(const __grid_constant__ CUtensorMap tmap_in, const ResPar
             int slot = 0;
             uint32_t eph = 1;                                    // parity to wait for on the slot's "empty" barrier
             bool ok = true;
-            for (int64_t u = u0; u < u1 && ok; ++u) {
-                const int ct = (int)(u % nCT);
+            int ct = ct0;
+            for (int64_t u = u0; u < u1 && ok; ++u, ++ct) {
+                if (ct == nCT) ct = 0;
                 for (int kc = 0; kc < nK; ++kc, ++cw) {
                     ok = ptx::mbar_wait(&bar->empty_w[slot], eph, abort_flag, status, 302, true, kResSpin);
                     if (!ok) break;
@@ -211,8 +224,10 @@ umma_linear_res_kernel(const __grid_constant__ CUtensorMap tmap_in, const ResPar
             auto mma = [](uint32_t d, uint32_t a_addr, uint32_t b_addr, uint32_t idesc, uint32_t accumulate) {
                 ptx::umma_f16(d, ptx::umma_smem_desc_k_sw32(a_addr), ptx::umma_smem_desc_k_sw32(b_addr), idesc, accumulate);
             };
-            for (int64_t u = u0; u < u1 && ok; ++u, ++cu) {
-                const bool first = first_of_tile(u), last = last_of_tile(u);
+            int ct = ct0;
+            for (int64_t u = u0; u < u1 && ok; ++u, ++cu, ++ct) {
+                if (ct == nCT) ct = 0;
+                const bool first = first_of_tile(u, ct), last = last_of_tile(u, ct);
                 if (first && u != u0) ++tc;
                 RES_STAMP(512 + 2 * cu);
                 const uint32_t buf = cu % NBUF;
@@ -220,42 +235,55 @@ umma_linear_res_kernel(const __grid_constant__ CUtensorMap tmap_in, const ResPar
                 ok = ptx::mbar_wait(&bar->empty_d[buf], ((cu / NBUF) & 1) ^ 1, abort_flag, status, 303, true, kResSpin);
                 RES_STAMP(512 + 2 * cu + 1);
                 if (!ok) break;
+                // x^ buffer and phase of the tile's chunk 0: chunk kc of the CTA's tc-th tile has running number tc*nK + kc
+                int xs = (int)((tc * (uint32_t)nK) % (uint32_t)XR);
+                uint32_t xph = ((tc * (uint32_t)nK) / (uint32_t)XR) & 1u;
                 // operands of the unit's first chunk
-                if (first) ok = ptx::mbar_wait(&bar->full_x[0], tc & 1, abort_flag, status, 304, true, kResSpin);
+                if (first) ok = ptx::mbar_wait(&bar->full_x[xs], xph, abort_flag, status, 304, true, kResSpin);
                 ok = ok && ptx::mbar_wait(&bar->full_w[slot], wph, abort_flag, status, 305, true, kResSpin);
                 if (!ok) break;
                 for (int kc = 0; kc < nK; ++kc) {
                     RES_STAMP(1024 + 4 * (cu * nK + kc));
                     ptx::tc_fence_after_sync();
                     const uint32_t a0 = ptx::smem_u32(wsm + slot * kWSlot);      // weight tiles, plane p at p * 4 KB
-                    const uint32_t b0 = ptx::smem_u32(xhat + kc * kXChunkBytes); // x^ tiles, plane p at p * XT
+                    const uint32_t b0 = ptx::smem_u32(xhat + xs * kXChunkBytes); // x^ tiles, plane p at p * XT
                     const uint32_t acc = kc > 0 ? 1u : 0u;
                     int nslot = slot + 1;
                     uint32_t nwph = wph;
                     if (nslot == w_slots) { nslot = 0; nwph ^= 1u; }
+                    int nxs = xs + 1;
+                    uint32_t nxph = xph;
+                    if (nxs == XR) { nxs = 0; nxph ^= 1u; }
                     mma(dbase, a0, b0, idesc1, acc);                                                      // k = 0
 #pragma unroll
                     for (int f = 1; f < T / 2; ++f) {
                         const uint32_t dre = dbase + (uint32_t)((2 * f - 1) * NTOK), dim = dre + NTOK;
                         const uint32_t wr = a0 + (2 * f - 1) * kWTileBytes, wi = wr + kWTileBytes;
-                        const uint32_t xr = b0 + (2 * f - 1) * XT, xi = xr + XT;
-                        mma(dre, wr, xr, idesc2, acc);                                                    // [Re|Im] += Wr [Xr|Xi]
-                        mma(dre, wi, xi, idesc1 | kIdescNegateA, 1u);                                     //  Re     -= Wi Xi
-                        mma(dim, wi, xr, idesc1, 1u);                                                     //  Im     += Wi Xr
+                        if constexpr (PF) {
+                            const uint32_t xr = b0 + (1 + 3 * (f - 1)) * XT, xi = xr + XT;            // tiles Re | Im | -Re
+                            mma(dre, wr, xr, idesc2, acc);                                                // [Re|Im] += Wr [Xr|Xi]
+                            mma(dre, wi, xi, idesc2 | kIdescNegateA, 1u);                                 // [Re|Im] -= Wi [Xi|-Xr]
+                        } else {
+                            const uint32_t xr = b0 + (2 * f - 1) * XT, xi = xr + XT;
+                            mma(dre, wr, xr, idesc2, acc);                                                // [Re|Im] += Wr [Xr|Xi]
+                            mma(dre, wi, xi, idesc1 | kIdescNegateA, 1u);                                 //  Re     -= Wi Xi
+                            mma(dim, wi, xr, idesc1, 1u);                                                 //  Im     += Wi Xr
+                        }
                         if (f == 1 && kc + 1 < nK) {
                             // The next chunk's operands are checked here, while the tensor pipe still has this chunk's
                             // MMAs queued, so that the issue stream has no gap between chunks.
                             RES_STAMP(1024 + 4 * (cu * nK + kc) + 1);
-                            if (first) ok = ptx::mbar_wait(&bar->full_x[kc + 1], tc & 1, abort_flag, status, 304, true, kResSpin);
+                            if (first) ok = ptx::mbar_wait(&bar->full_x[nxs], nxph, abort_flag, status, 304, true, kResSpin);
                             ok = ok && ptx::mbar_wait(&bar->full_w[nslot], nwph, abort_flag, status, 305, true, kResSpin);
                             RES_STAMP(1024 + 4 * (cu * nK + kc) + 2);
                         }
                     }
-                    mma(dbase + (uint32_t)((T - 1) * NTOK), a0 + (T - 1) * kWTileBytes, b0 + (T - 1) * XT, idesc1, acc);  // k = T/2
+                    mma(dbase + (uint32_t)((T - 1) * NTOK), a0 + (T - 1) * kWTileBytes, b0 + (XTILES - 1) * XT, idesc1, acc);  // k = T/2
                     ptx::umma_commit(&bar->empty_w[slot]);
-                    if (last) ptx::umma_commit(&bar->empty_x[kc]);  // the tile's x^ chunk may be overwritten once these MMAs retire
+                    if (last) ptx::umma_commit(&bar->empty_x[xs]);  // the x^ buffer may be overwritten once these MMAs retire
                     RES_STAMP(1024 + 4 * (cu * nK + kc) + 3);
                     slot = nslot; wph = nwph;
+                    xs = nxs; xph = nxph;
                     if (!ok) break;
                 }
                 if (ok) ptx::umma_commit(&bar->full_d[buf]);
@@ -275,11 +303,15 @@ umma_linear_res_kernel(const __grid_constant__ CUtensorMap tmap_in, const ResPar
         // Group DFT of this warp's items of token tile number tc (the tc-th tile of this CTA).  Items are dealt
         // round-robin over the transform warps by their running number, so warp cw always reads ring slot cw.
         uint32_t my_items = 0;                                   // items this warp has taken from its ring slot
-        auto transform_tile = [&](uint32_t tc) {
-            if (cw >= n_tw) return;
+        // Chunks [c_lo, c_hi) of the tile only: with a ring of x^ buffers the first XR chunks are transformed before the
+        // previous unit's epilogue and the rest after it, while the MMAs of the tile consume them.
+        auto transform_tile = [&](uint32_t tc, int c_lo, int c_hi) {
+            if (cw >= n_tw || c_lo >= c_hi) return;
             const uint32_t base = tc * (uint32_t)items_per_tile;
+            const int lo = c_lo * IPC, hi = c_hi * IPC;
             // this warp's items of the tile: running numbers congruent to cw modulo n_tw
-            for (int i = (int)((cw + n_tw - base % n_tw) % n_tw); i < items_per_tile && ok; i += n_tw, ++my_items) {
+            const int i0 = lo + (int)(((uint32_t)cw + 4u * (uint32_t)n_tw - (base + (uint32_t)lo) % (uint32_t)n_tw) % (uint32_t)n_tw);
+            for (int i = i0; i < hi && ok; i += n_tw, ++my_items) {
                 ok = ptx::mbar_wait(&bar->full_raw[cw], my_items & 1, abort_flag, status, 306, true, 16);
                 if (!ok) break;
                 uint32_t wd[32];
@@ -294,39 +326,62 @@ umma_linear_res_kernel(const __grid_constant__ CUtensorMap tmap_in, const ResPar
                 const int s = i / PARTS, h = i % PARTS;
                 const int kc = s / SPK, q = s % SPK;
                 const int r = h * 32 + lane;                     // token row inside the tile
-                // the MMAs that read the previous tile's chunk kc must have retired
-                if (tc > 0) {
-                    ok = ptx::mbar_wait(&bar->empty_x[kc], (tc - 1) & 1, abort_flag, status, 307, true, 16);
+                // buffer of this chunk (running number qn); the MMAs that read the buffer's previous contents must have retired
+                const uint32_t qn = tc * (uint32_t)nK + (uint32_t)kc;
+                const int xsl = (int)(qn % (uint32_t)XR);
+                const uint32_t use = qn / (uint32_t)XR;
+                if (use > 0) {
+                    ok = ptx::mbar_wait(&bar->empty_x[xsl], (use - 1) & 1, abort_flag, status, 307, true, 16);
                     if (!ok) break;
                 }
                 // x^ plane tile: row r at r*32, its two 16-byte chunks exchanged when bit 2 of r is set (32B swizzle);
                 // this raw row's run of channels starts at byte kb of the row
                 const int kb = q * NCH * 2;
                 const int sw = (r >> 2) & 1;
-                uint8_t* dst = xhat + kc * kXChunkBytes + r * 32 + (((kb >> 4) ^ sw) << 4) + (kb & 15);
+                uint8_t* dst = xhat + xsl * kXChunkBytes + r * 32 + (((kb >> 4) ^ sw) << 4) + (kb & 15);
                 const int second = sw ? -16 : 16;
+                if constexpr (PF) {
+                    store_plane_run<2 * W>(dst, packed[0], second);
 #pragma unroll
-                for (int p = 0; p < T; ++p) store_plane_run<2 * W>(dst + p * XT, packed[p], second);
+                    for (int f = 1; f < T / 2; ++f) {
+                        uint8_t* t0 = dst + (1 + 3 * (f - 1)) * XT;
+                        store_plane_run<2 * W>(t0, packed[2 * f - 1], second);                      // Re
+                        store_plane_run<2 * W>(t0 + XT, packed[2 * f], second);                     // Im
+                        store_plane_run<2 * W>(t0 + 2 * XT, packed[2 * f - 1], second, 0x80008000u); // -Re
+                    }
+                    store_plane_run<2 * W>(dst + (XTILES - 1) * XT, packed[T - 1], second);
+                } else {
+#pragma unroll
+                    for (int p = 0; p < T; ++p) store_plane_run<2 * W>(dst + p * XT, packed[p], second);
+                }
                 ptx::fence_proxy_async_smem();                   // generic-proxy writes -> visible to the MMA (async proxy)
                 __syncwarp();
-                if (lane == 0) ptx::mbar_arrive(&bar->full_x[kc]);
+                if (lane == 0) ptx::mbar_arrive(&bar->full_x[xsl]);
             }
         };
 
         uint32_t tc = 0, cu = 0;
-        if (u0 < u1) transform_tile(0);
-        for (int64_t u = u0; u < u1 && ok; ++u, ++cu) {
-            // the next token tile is transformed while the MMAs of this tile's last channel tile are in flight
+        const int pre = XR < nK ? XR : nK;                       // chunks of a tile that fit before its MMAs start freeing buffers
+        if (u0 < u1) transform_tile(0, 0, pre);
+        int ct = ct0;
+        int64_t tt = tt0;
+        for (int64_t u = u0; u < u1 && ok; ++u, ++cu, ++ct) {
+            if (ct == nCT) { ct = 0; ++tt; }
             if (cw == 0 && lane == 0) RES_STAMP(8 * cu);
-            if (last_of_tile(u) && u + 1 < u1) {
+            // ring of x^ buffers (one channel tile): the rest of this tile's chunks, consumed by its MMAs as they arrive
+            if (first_of_tile(u, ct)) {
+                transform_tile(tc, pre, nK);
+                if (!ok) break;
+            }
+            // the next token tile is transformed while the MMAs of this tile's last channel tile are in flight
+            if (last_of_tile(u, ct) && u + 1 < u1) {
                 ++tc;
-                transform_tile(tc);
+                transform_tile(tc, 0, pre);
                 if (!ok) break;
             }
             if (cw == 0 && lane == 0) RES_STAMP(8 * cu + 1);
             // ---- epilogue of unit u: thread = output channel, columns = (plane, token)
-            const int ct = (int)(u % nCT);
-            const int64_t row0 = (u / nCT) * NTOK;
+            const int64_t row0 = tt * NTOK;
             const int o = ct * 128 + quad * 32 + lane;
             const bool o_ok = o < prm.Cout;
             const float bias_v = (prm.bias != nullptr && o_ok) ? __ldg(prm.bias + o) : 0.f;
@@ -401,8 +456,9 @@ EncodeTiledFn encode_tiled_res_fn() {
 
 constexpr size_t kResSmemLimit = 227 * 1024;
 
-size_t res_smem_bytes(int T, int nTok, int nK, int w_slots, int n_tw) {
-    return 1024 + (size_t)n_tw * kItemBytes + (size_t)nK * T * nTok * 32 + (size_t)w_slots * T * kWTileBytes +
+size_t res_smem_bytes(int T, int nTok, bool paired, int x_slots, int w_slots, int n_tw) {
+    const int tiles = paired ? 2 + 3 * (T / 2 - 1) : T;
+    return 1024 + (size_t)n_tw * kItemBytes + (size_t)x_slots * tiles * nTok * 32 + (size_t)w_slots * T * kWTileBytes +
            sizeof(ResBarriers) + 64;
 }
 
@@ -429,17 +485,32 @@ UmmaResShape umma_res_shape(int T, int Cin, int Cout) {
     s.nCT = (Cout + 127) / 128;
     s.image_bytes = align_up((size_t)s.nCT * s.nK * T * kWTileBytes, kWsAlign);
     s.fits = false;
-    if (s.nK > kResMaxK) return s;
+    s.paired = false;
     // ring depths in order of preference: the weight stream paces the main loop (3 chunks cover its latency), then
     // as many transform warps as shared memory allows
     static const int cand[][2] = {{3, 12}, {3, 8}, {2, 12}, {2, 8}, {2, 4}};
-    for (const auto& c : cand) {
-        if (res_smem_bytes(T, s.nTok, s.nK, c[0], c[1]) <= kResSmemLimit) {
-            s.w_slots = c[0]; s.n_tw = c[1]; s.fits = true;
-            break;
+    if (s.nK <= kResMaxK) {                                      // the whole token tile resident: x^ buffers = chunks
+        s.x_slots = s.nK;
+        for (const auto& c : cand) {
+            if (res_smem_bytes(T, s.nTok, false, s.x_slots, c[0], c[1]) <= kResSmemLimit) {
+                s.w_slots = c[0]; s.n_tw = c[1]; s.fits = true;
+                break;
+            }
         }
     }
-    if (s.fits && s.w_slots == 3 && res_smem_bytes(T, s.nTok, s.nK, 4, s.n_tw) <= kResSmemLimit) s.w_slots = 4;
+    // One channel tile: nothing is reused across units, so three x^ buffers used as a ring are enough.  The ring
+    // needs all 12 transform warps (chunk q is then always transformed by warps 4 (q % 3) .. 4 (q % 3) + 3, which
+    // therefore see every phase of the buffer barriers they wait on).
+    if (s.nCT == 1 && !(s.fits && s.w_slots >= 3) && s.nK > 3 &&
+        res_smem_bytes(T, s.nTok, false, 3, 3, 12) <= kResSmemLimit) {
+        s.x_slots = 3; s.w_slots = 3; s.n_tw = 12; s.fits = true;
+    }
+    // paired form where the larger x^ buffers still leave a deep weight ring
+    if (s.fits && s.w_slots >= 3 && res_smem_bytes(T, s.nTok, true, s.x_slots, 3, s.n_tw) <= kResSmemLimit) {
+        s.paired = true;
+        s.w_slots = 3;
+    }
+    if (s.fits && s.w_slots == 3 && res_smem_bytes(T, s.nTok, s.paired, s.x_slots, 4, s.n_tw) <= kResSmemLimit) s.w_slots = 4;
     return s;
 }
 
@@ -474,28 +545,32 @@ cudaError_t launch_umma_linear_res(const UmmaResShape& s, const void* in, void* 
     ResParams prm{};
     prm.out = out; prm.image = (const uint8_t*)image; prm.bias = bias_f32; prm.status = status;
     prm.N = N; prm.Cin = s.Cin; prm.Cout = s.Cout; prm.nCT = s.nCT; prm.nK = s.nK;
-    prm.w_slots = s.w_slots; prm.n_tw = s.n_tw;
+    prm.w_slots = s.w_slots; prm.n_tw = s.n_tw; prm.x_slots = s.x_slots;
     prm.num_units = ((N + s.nTok - 1) / s.nTok) * s.nCT;
     const int grid = (int)(prm.num_units < num_sms ? prm.num_units : num_sms);
-    const size_t smem = res_smem_bytes(s.T, s.nTok, s.nK, s.w_slots, s.n_tw);
+    const size_t smem = res_smem_bytes(s.T, s.nTok, s.paired, s.x_slots, s.w_slots, s.n_tw);
 
-    auto go = [&](auto tc, auto nt) -> cudaError_t {
+    auto go = [&](auto tc, auto nt, auto pf) -> cudaError_t {
         constexpr int TT = decltype(tc)::value, NT = decltype(nt)::value;
+        constexpr bool PF = decltype(pf)::value;
         static unsigned long long attr_done = 0;
         int dev = 0;
         cudaGetDevice(&dev);
         if (!((attr_done >> (dev & 63)) & 1ull)) {
-            cudaError_t e = cudaFuncSetAttribute(umma_linear_res_kernel<TT, NT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+            cudaError_t e = cudaFuncSetAttribute(umma_linear_res_kernel<TT, NT, PF>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                  (int)kResSmemLimit);
             if (e != cudaSuccess) return e;
             attr_done |= 1ull << (dev & 63);
         }
-        umma_linear_res_kernel<TT, NT><<<grid, kThreadsRes, smem, stream>>>(tmap, prm);
+        umma_linear_res_kernel<TT, NT, PF><<<grid, kThreadsRes, smem, stream>>>(tmap, prm);
         return cudaGetLastError();
     };
-    if (s.T == 4 && s.nTok == 128) return go(std::integral_constant<int, 4>{}, std::integral_constant<int, 128>{});
-    if (s.T == 4 && s.nTok == 64) return go(std::integral_constant<int, 4>{}, std::integral_constant<int, 64>{});
-    if (s.T == 8 && s.nTok == 64) return go(std::integral_constant<int, 8>{}, std::integral_constant<int, 64>{});
+    using I4 = std::integral_constant<int, 4>;
+    using I8 = std::integral_constant<int, 8>;
+    using I64 = std::integral_constant<int, 64>;
+    using I128 = std::integral_constant<int, 128>;
+    if (s.T == 4 && s.nTok == 128) return s.paired ? go(I4{}, I128{}, std::true_type{}) : go(I4{}, I128{}, std::false_type{});
+    if (s.T == 8 && s.nTok == 64) return s.paired ? go(I8{}, I64{}, std::true_type{}) : go(I8{}, I64{}, std::false_type{});
     return cudaErrorInvalidValue;
 }
 

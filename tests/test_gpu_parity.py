@@ -66,14 +66,17 @@ def test_shapes(dtype, T, Ci, Co):
 
 
 # ------------------------------------------------------------------ the two tensor-core kernels of fwd / bwd_data
-@pytest.mark.parametrize("T,Ci,Co,N,ids", [(8, 96, 384, 1000, (2, 1)), (8, 24, 200, 777, (2, 1)), (8, 10, 64, 130, (2, 1)),
+@pytest.mark.parametrize("T,Ci,Co,N,ids", [(8, 96, 384, 1000, (2, 2)), (8, 24, 200, 777, (2, 1)), (8, 10, 64, 130, (2, 1)),
                                              (8, 16, 520, 6500, (2, 1)), (8, 64, 64, 900, (2, 2)), (4, 24, 96, 1111, (2, 1)),
-                                             (4, 100, 130, 515, (2, 2)), (4, 8, 300, 20000, (2, 1))])
+                                             (4, 100, 130, 515, (2, 2)), (4, 8, 300, 20000, (2, 1)),
+                                             (8, 384, 96, 12000, (2, 2)), (4, 320, 100, 600, (2, 2)), (8, 200, 100, 3333, (2, 1))])
 def test_resident_and_streaming_kernels_agree_with_oracle(T, Ci, Co, N, ids):
-    """Layers with few input channels run the kernel that keeps a token tile's spectrum in shared memory (id 2);
-    EQL_FLAG_FORCE_STREAMING selects the streaming kernel (id 1) for the same plan shape.  Both must meet the bar,
-    on channel counts that are not multiples of the 128-channel / 16-channel tiles, ragged token counts, and token
-    counts large enough that a CTA's range of work starts and ends in the middle of a token tile."""
+    """Layers with few input channels run the kernel that keeps a token tile's spectrum in shared memory (id 2), and so
+    do layers with at most 128 output channels (one channel tile: the spectrum then streams through a ring of three
+    chunk buffers, e.g. 384 -> 96 channels); EQL_FLAG_FORCE_STREAMING selects the streaming kernel (id 1) for the same
+    plan shape.  Both must meet the bar, on channel counts that are not multiples of the 128-channel / 16-channel
+    tiles, ragged token counts, and token counts large enough that a CTA's range of work starts and ends in the
+    middle of a token tile and covers several units."""
     wl = Workload("res", "fp16", T, Ci, Co, N, "normal", ("fwd", "bwd_data"), 21)
     data = eq.workloads.generate(wl)
     for flags, want in ((0, ids), (eq.EQL_FLAG_FORCE_STREAMING, (1, 1))):
