@@ -408,7 +408,7 @@ BwdWeightSplit direct_bwd_weight_split(int T, int Ci, int Co, int64_t N) {
         default: TO = 2; TI = 2; BK = 4; break;
     }
     const int64_t tiles = (int64_t)((Co + 16 * TO - 1) / (16 * TO)) * ((Ci + 16 * TI - 1) / (16 * TI));
-    int64_t want = (2 * kNumSMs + tiles - 1) / tiles;            // about two blocks per SM in flight
+    int64_t want = (kNumSMs + tiles - 1) / tiles;                // about one block per SM: fewer partial spectra to write and re-read
     const int64_t chunks = (N + BK - 1) / BK;
     if (want > chunks) want = chunks;
     if (want < 1) want = 1;

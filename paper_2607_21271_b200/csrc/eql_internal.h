@@ -89,9 +89,10 @@ cudaError_t launch_build_umma_res_image(const UmmaResShape& s, const float* plan
 cudaError_t launch_umma_linear_res(const UmmaResShape& s, const void* in, void* out, int64_t N, const void* image,
                                    const float* bias_f32, int* status, int num_sms, cudaStream_t stream);
 
-// ---- tcgen05 weight-gradient kernel (FP16 inputs), umma_bwd_weight.cu --------------------------------
+// ---- tcgen05 weight-gradient kernel (FP16 inputs; FP32 inputs with the 3xTF32 split), umma_bwd_weight.cu --------------------------------
 struct UmmaBwdWeightShape {
     int T, Ci, Co;
+    int elem_bytes;             // 2: half inputs (kind::f16), 4: float inputs (kind::tf32, 3xTF32 split)
     int CiT, nCiTiles;          // input-channel tile (UMMA M side, <= 128 lanes, CiT*T <= 1024)
     int CoT, nCoTiles;          // output-channel tile (UMMA N side, T*CoT <= 512 TMEM columns)
     int nXs, nYs;               // 64-element raw slabs of x / dy per 16-token chunk
@@ -100,7 +101,7 @@ struct UmmaBwdWeightShape {
     size_t scratch_bytes;       // splits * (T*Co*Ci + Co) floats
 };
 bool umma_bwd_weight_supported(int T, eql_dtype_t dtype);
-UmmaBwdWeightShape umma_bwd_weight_shape(int T, int Ci, int Co, int64_t N, int num_sms);
+UmmaBwdWeightShape umma_bwd_weight_shape(int T, int Ci, int Co, eql_dtype_t dtype, int64_t N, int num_sms);
 // Phase 1 only: partial spectra + db partials into scratch (same layout as the CUDA-core kernel's).
 cudaError_t launch_umma_bwd_weight(const UmmaBwdWeightShape& s, const void* x, const void* dy, int64_t N,
                                    float* scratch, int* status, cudaStream_t stream);

@@ -342,7 +342,7 @@ eql_status_t eqlinear_bwd_weight_scratch_bytes(eqlinear_plan_t plan, int64_t N, 
     eql_status_t st = check_tokens(N);
     if (st != EQL_OK) return st;
     if (plan->bwd_weight_kernel == 1)
-        *bytes = umma_bwd_weight_shape(plan->T, plan->Ci, plan->Co, N > 0 ? N : 1, plan->num_sms).scratch_bytes;
+        *bytes = umma_bwd_weight_shape(plan->T, plan->Ci, plan->Co, plan->dtype, N > 0 ? N : 1, plan->num_sms).scratch_bytes;
     else
         *bytes = direct_bwd_weight_split(plan->T, plan->Ci, plan->Co, N > 0 ? N : 1).scratch_bytes;
     return EQL_OK;
@@ -365,7 +365,7 @@ eql_status_t eqlinear_bwd_weight(eqlinear_plan_t plan, const void* x, const void
     if (!aligned16(x) || !aligned16(dy)) return EQL_ERR_ALIGNMENT;
     if (reinterpret_cast<uintptr_t>(scratch) % kWsAlign != 0) return EQL_ERR_ALIGNMENT;
     if (plan->bwd_weight_kernel == 1) {
-        UmmaBwdWeightShape bs = umma_bwd_weight_shape(plan->T, plan->Ci, plan->Co, N, plan->num_sms);
+        UmmaBwdWeightShape bs = umma_bwd_weight_shape(plan->T, plan->Ci, plan->Co, plan->dtype, N, plan->num_sms);
         if (scratch_bytes < bs.scratch_bytes) return EQL_ERR_WORKSPACE;
         cudaError_t e = launch_umma_bwd_weight(bs, x, dy, N, (float*)scratch, (int*)(plan->ws + plan->lay.status), s);
         if (e != cudaSuccess) return EQL_ERR_CUDA;

@@ -1,4 +1,5 @@
-// Weight gradient on the tcgen05 tensor cores (FP16 inputs, FP32 accumulation in TMEM):
+// Weight gradient on the tcgen05 tensor cores (FP32 accumulation in TMEM; FP16 inputs with kind::f16, FP32 inputs
+// with kind::tf32 and the 3xTF32 hi/lo split: hi*hi + hi*lo + lo*hi):
 //   dW^_k[o, i] = sum_n dY^_k[n, o] * conj(X^_k[n, i])     for every retained frequency k,
 // a GEMM whose reduction dimension is the token index.  One CTA owns an (input-channel tile,
 // output-channel tile) block of all T real-packed planes for one token range; the per-range partial
@@ -45,6 +46,8 @@ struct BwParams {
     int splits;
     int64_t chunks_per_split;    // 16-token chunks per token range
     int xhat_bytes, stage_bytes;
+    int x_part_bytes, y_part_bytes;   // FP32: bytes of the TF32 "hi" copy of x^ / dy^ inside a stage; the "lo" copy follows it
+    int stages;                  // operand stages (2; 1 where the hi/lo copies of FP32 leave no room for two)
     int x3d, y3d;                // tensor maps are 3-D (64 elements, rows, slab index): one load per chunk and tensor
 };
 
@@ -64,16 +67,26 @@ struct BwBarriers {
     int abort_flag;
 };
 
-template <int T>
+template <int T, typename IO>
 __global__ void __launch_bounds__(kThreadsBw, 1)
 umma_bwd_weight_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_dy,
                        const BwParams prm) {
-    constexpr int NCH = 64 / T;
+    constexpr int E = sizeof(IO);                 // 2: half inputs, 4: float inputs (3xTF32)
+    constexpr int EPR = 128 / E;                  // elements per 128-byte raw row
+    constexpr int NCH = EPR / T;                  // channels per raw row
+    // Operand tiles of a 16-token chunk.  FP16: MN-major (channels contiguous, as they come out of the transform),
+    // 32 bytes per channel.  FP32: the tensor core transposes 32-bit operands only in a swizzle mode of its own, so
+    // the TF32 tiles are written K-major (tokens contiguous): core matrix = 8 channels x 4 tokens (128 B), the four
+    // core matrices of a channel group kF32Lbo = 144 bytes apart (16 bytes of padding keep the scattered 4-byte
+    // stores of a half warp on distinct banks), channel groups kF32Sbo = 576 bytes apart: 72 bytes per channel.
+    constexpr int kF32Lbo = 144, kF32Sbo = 4 * kF32Lbo;
+    constexpr int TOKB = E == 2 ? kChunkTok * E : kF32Sbo / 8;   // bytes per channel of one tile
     extern __shared__ uint8_t smem_raw_base[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw_base) + 1023) & ~(uintptr_t)1023);
     BwBarriers* bar = reinterpret_cast<BwBarriers*>(smem);
     uint8_t* raw = smem + 1024;                                  // kRawSlots x 48 KB
-    uint8_t* stages = raw + kRawSlots * kRawSlot;                // kStages x stage_bytes (+ 4 KB slack after the last)
+    uint8_t* stages = raw + kRawSlots * kRawSlot;                // prm.stages x stage_bytes (+ 8 KB slack after the last)
+    const int NST = prm.stages;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     volatile int* abort_flag = &bar->abort_flag;
@@ -126,16 +139,16 @@ umma_bwd_weight_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
                 // One 3-D box [slab][16 rows][64 elements] per tensor where the row length is a whole number of
                 // slabs; otherwise one 2-D box per slab (the same shared-memory layout either way).
                 if (prm.x3d) {
-                    ptx::tma_load_3d(dst, &tmap_x, 0, row, ci_tile * CiT * T / 64, &bar->full_raw[slot]);
+                    ptx::tma_load_3d(dst, &tmap_x, 0, row, ci_tile * CiT * T / EPR, &bar->full_raw[slot]);
                 } else {
                     for (int s = 0; s < prm.nXs; ++s)
-                        ptx::tma_load_2d(dst + s * kSlab, &tmap_x, ci_tile * CiT * T + s * 64, row, &bar->full_raw[slot]);
+                        ptx::tma_load_2d(dst + s * kSlab, &tmap_x, ci_tile * CiT * T + s * EPR, row, &bar->full_raw[slot]);
                 }
                 if (prm.y3d) {
-                    ptx::tma_load_3d(dst + kMaxXSlabs * kSlab, &tmap_dy, 0, row, co_tile * CoT * T / 64, &bar->full_raw[slot]);
+                    ptx::tma_load_3d(dst + kMaxXSlabs * kSlab, &tmap_dy, 0, row, co_tile * CoT * T / EPR, &bar->full_raw[slot]);
                 } else {
                     for (int s = 0; s < prm.nYs; ++s)
-                        ptx::tma_load_2d(dst + (kMaxXSlabs + s) * kSlab, &tmap_dy, co_tile * CoT * T + s * 64, row,
+                        ptx::tma_load_2d(dst + (kMaxXSlabs + s) * kSlab, &tmap_dy, co_tile * CoT * T + s * EPR, row,
                                          &bar->full_raw[slot]);
                 }
             }
@@ -148,34 +161,46 @@ umma_bwd_weight_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
     } else if (warp == kWarpMmaBw) {
         if (lane == 0) {
             bool ok = true;
-            const uint32_t idesc_real = ptx::umma_idesc_f16_f32_mn_major(128, CoT);
-            const uint32_t idesc_cplx = ptx::umma_idesc_f16_f32_mn_major(128, 2 * CoT);
-            const uint32_t a_plane = (uint32_t)CiT * 32u, b_tile = (uint32_t)CoT * 32u;
+            constexpr uint32_t kMnMajor = (1u << 15) | (1u << 16);       // both operands MN-major
+            const uint32_t idesc_real = E == 2 ? (ptx::umma_idesc_f16_f32(128, CoT) | kMnMajor) : ptx::umma_idesc_tf32_f32(128, CoT);
+            const uint32_t idesc_cplx = E == 2 ? (ptx::umma_idesc_f16_f32(128, 2 * CoT) | kMnMajor) : ptx::umma_idesc_tf32_f32(128, 2 * CoT);
+            const uint32_t a_plane = (uint32_t)CiT * TOKB, b_tile = (uint32_t)CoT * TOKB;
+            // FP16, MN-major no-swizzle tiles: lbo = stride between 8-token groups (128 B), sbo = stride between 8-channel groups
+            // (256 B).  FP32, K-major no-swizzle tiles: lbo = stride between 4-token core matrices, sbo = between 8-channel groups.
+            auto mma = [](uint32_t d, uint32_t a_addr, uint32_t b_addr, uint32_t idesc, uint32_t accumulate) {
+                if constexpr (E == 2)
+                    ptx::umma_f16(d, ptx::umma_smem_desc(a_addr, 128, 256), ptx::umma_smem_desc(b_addr, 128, 256), idesc, accumulate);
+                else
+                    ptx::umma_tf32(d, ptx::umma_smem_desc(a_addr, kF32Lbo, kF32Sbo), ptx::umma_smem_desc(b_addr, kF32Lbo, kF32Sbo), idesc, accumulate);
+            };
+            constexpr int KSTEPS = E == 2 ? 1 : 2;                       // a 16-token chunk is one K step of halves, two of TF32
+            constexpr int PASSES = E == 2 ? 1 : 3;                       // 3xTF32: hi*hi, hi*lo, lo*hi
             for (int64_t c = 0; c < nchunks; ++c) {
-                const int st = (int)(c % kStages);
-                BW_STAMP(1000 + 3 * (int)c);
-                ok = ptx::mbar_wait(&bar->full_ab[st], (uint32_t)((c / kStages) & 1), abort_flag, status, 202);
-                BW_STAMP(1000 + 3 * (int)c + 1);
+                const int st = (int)(c % NST);
+                ok = ptx::mbar_wait(&bar->full_ab[st], (uint32_t)((c / NST) & 1), abort_flag, status, 202);
                 if (!ok) break;
                 ptx::tc_fence_after_sync();
-                const uint32_t a0 = ptx::smem_u32(stages + st * prm.stage_bytes);
-                const uint32_t b0 = a0 + prm.xhat_bytes;
-                const uint32_t acc = c > 0 ? 1u : 0u;
-                // MN-major no-swizzle: lbo = stride between 8-token groups (128 B), sbo = stride between 8-channel groups (256 B)
-                ptx::umma_f16(tmem_base, ptx::umma_smem_desc(a0, 128, 256), ptx::umma_smem_desc(b0, 128, 256), idesc_real, acc);
+                const uint32_t stage0 = ptx::smem_u32(stages + st * prm.stage_bytes);
 #pragma unroll
-                for (int f = 1; f < T / 2; ++f) {
-                    const uint32_t d = tmem_base + (uint32_t)((2 * f - 1) * CoT);
-                    const uint32_t bt = b0 + (uint32_t)(1 + 3 * (f - 1)) * b_tile;          // tiles Gr | Gi | -Gr
-                    ptx::umma_f16(d, ptx::umma_smem_desc(a0 + (2 * f - 1) * a_plane, 128, 256),
-                                  ptx::umma_smem_desc(bt, 128, 256), idesc_cplx, acc);       // Xr^T [Gr | Gi]
-                    ptx::umma_f16(d, ptx::umma_smem_desc(a0 + (2 * f) * a_plane, 128, 256),
-                                  ptx::umma_smem_desc(bt + b_tile, 128, 256), idesc_cplx, 1u);  // Xi^T [Gi | -Gr]
+                for (int ks = 0; ks < KSTEPS; ++ks) {
+#pragma unroll
+                    for (int pass = 0; pass < PASSES; ++pass) {
+                        const uint32_t a0 = stage0 + (pass == 2 ? prm.x_part_bytes : 0) + ks * 2 * kF32Lbo;   // 8 tokens = 2 core matrices
+                        const uint32_t b0 = stage0 + prm.xhat_bytes + (pass == 1 ? prm.y_part_bytes : 0) + ks * 2 * kF32Lbo;
+                        const uint32_t acc = (c > 0 || ks > 0 || pass > 0) ? 1u : 0u;
+                        mma(tmem_base, a0, b0, idesc_real, acc);
+#pragma unroll
+                        for (int f = 1; f < T / 2; ++f) {
+                            const uint32_t d = tmem_base + (uint32_t)((2 * f - 1) * CoT);
+                            const uint32_t bt = b0 + (uint32_t)(1 + 3 * (f - 1)) * b_tile;      // tiles Gr | Gi | -Gr
+                            mma(d, a0 + (2 * f - 1) * a_plane, bt, idesc_cplx, acc);             // Xr^T [Gr | Gi]
+                            mma(d, a0 + (2 * f) * a_plane, bt + b_tile, idesc_cplx, 1u);         // Xi^T [Gi | -Gr]
+                        }
+                        mma(tmem_base + (uint32_t)((T - 1) * CoT), a0 + (T - 1) * a_plane,
+                            b0 + (uint32_t)(1 + 3 * (T / 2 - 1)) * b_tile, idesc_real, acc);
+                    }
                 }
-                ptx::umma_f16(tmem_base + (uint32_t)((T - 1) * CoT), ptx::umma_smem_desc(a0 + (T - 1) * a_plane, 128, 256),
-                              ptx::umma_smem_desc(b0 + (uint32_t)(1 + 3 * (T / 2 - 1)) * b_tile, 128, 256), idesc_real, acc);
                 ptx::umma_commit(&bar->empty_ab[st]);
-                BW_STAMP(1000 + 3 * (int)c + 2);
             }
             if (ok) ptx::umma_commit(&bar->full_d);
             ptx::umma_commit(&bar->mma_done);
@@ -193,7 +218,7 @@ umma_bwd_weight_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
         for (int i = 0; i < NCH; ++i) dbacc[i] = 0.f;
         bool ok = true;
         for (int64_t c = 0; c < nchunks; ++c) {
-            const int slot = (int)(c % kRawSlots), st = (int)(c % kStages);
+            const int slot = (int)(c % kRawSlots), st = (int)(c % NST);
 #ifdef EQL_TRACE
             const bool tr = lane == 0 && (warp == kWarpDftX0 || warp == kWarpDftY0);
             const int tb = (warp == kWarpDftX0 ? 4000 : 5000) + 6 * (int)c;
@@ -203,7 +228,7 @@ umma_bwd_weight_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
 #ifdef EQL_TRACE
             if (tr) BW_STAMP(tb + 1);
 #endif
-            ok = ok && ptx::mbar_wait(&bar->empty_ab[st], (uint32_t)((c / kStages) & 1) ^ 1, abort_flag, status, 204);
+            ok = ok && ptx::mbar_wait(&bar->empty_ab[st], (uint32_t)((c / NST) & 1) ^ 1, abort_flag, status, 204);
 #ifdef EQL_TRACE
             if (tr) BW_STAMP(tb + 2);
 #endif
@@ -217,39 +242,75 @@ umma_bwd_weight_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(&bar->empty_raw[slot]);
             if (active) {
-                uint32_t packed[T][NCH / 2];
-                float p0[NCH];
+                const int mn0 = slab * NCH;                      // first channel of this slab inside the tile
+                // FP16, MN-major tile: (channel mn, token k) at (mn/8)*256 + (k/8)*128 + (k%8)*16 + (mn%8)*2
+                // FP32, K-major tile:  (channel mn, token k) at (mn/8)*576 + (k/4)*144 + (mn%8)*16 + (k%4)*4
+                const int off = E == 2 ? (mn0 >> 3) * 256 + (row >> 3) * 128 + (row & 7) * 16 + (mn0 & 7) * 2
+                                       : (row >> 2) * kF32Lbo + (row & 3) * 4;
+                uint8_t* stage = stages + st * prm.stage_bytes;
+                const int a_plane = CiT * TOKB, tb = CoT * TOKB;
+                if constexpr (E == 2) {
+                    uint32_t packed[T][NCH / 2];
+                    float p0[NCH];
 #ifdef EQL_ABLATE_DFT
 #pragma unroll
-                for (int p = 0; p < T; ++p)
+                    for (int p = 0; p < T; ++p)
 #pragma unroll
-                    for (int c2 = 0; c2 < NCH / 2; ++c2) packed[p][c2] = wd[(p * (NCH / 2) + c2) & 31];
+                        for (int c2 = 0; c2 < NCH / 2; ++c2) packed[p][c2] = wd[(p * (NCH / 2) + c2) & 31];
 #pragma unroll
-                for (int i = 0; i < NCH; ++i) p0[i] = 0.f;
+                    for (int i = 0; i < NCH; ++i) p0[i] = 0.f;
 #else
-                dft_words<T, true>(wd, packed, p0);
+                    dft_words<T, true>(wd, packed, p0);
 #endif
-                const int mn0 = slab * NCH;                      // first channel of this slab inside the tile
-                // MN-major tile: (channel mn, token k) at (mn/8)*256 + (k/8)*128 + (k%8)*16 + (mn%8)*2
-                const int off = (mn0 >> 3) * 256 + (row >> 3) * 128 + (row & 7) * 16 + (mn0 & 7) * 2;
-                uint8_t* stage = stages + st * prm.stage_bytes;
-                if (!is_y) {
+                    if (!is_y) {
 #pragma unroll
-                    for (int p = 0; p < T; ++p) store_plane_run<NCH>(stage + p * CiT * 32 + off, packed[p], 256);
-                } else {
+                        for (int p = 0; p < T; ++p) store_plane_run<NCH>(stage + p * a_plane + off, packed[p], 256);
+                    } else {
 #pragma unroll
-                    for (int i = 0; i < NCH; ++i) dbacc[i] += p0[i];
-                    uint8_t* yb = stage + prm.xhat_bytes + off;
-                    const int tb = CoT * 32;
-                    store_plane_run<NCH>(yb, packed[0], 256);
+                        for (int i = 0; i < NCH; ++i) dbacc[i] += p0[i];
+                        uint8_t* yb = stage + prm.xhat_bytes + off;
+                        store_plane_run<NCH>(yb, packed[0], 256);
 #pragma unroll
-                    for (int f = 1; f < T / 2; ++f) {
-                        uint8_t* t0 = yb + (1 + 3 * (f - 1)) * tb;
-                        store_plane_run<NCH>(t0, packed[2 * f - 1], 256);                    // Gr
-                        store_plane_run<NCH>(t0 + tb, packed[2 * f], 256);                   // Gi
-                        store_plane_run<NCH>(t0 + 2 * tb, packed[2 * f - 1], 256, 0x80008000u);   // -Gr
+                        for (int f = 1; f < T / 2; ++f) {
+                            uint8_t* t0 = yb + (1 + 3 * (f - 1)) * tb;
+                            store_plane_run<NCH>(t0, packed[2 * f - 1], 256);                    // Gr
+                            store_plane_run<NCH>(t0 + tb, packed[2 * f], 256);                   // Gi
+                            store_plane_run<NCH>(t0 + 2 * tb, packed[2 * f - 1], 256, 0x80008000u);   // -Gr
+                        }
+                        store_plane_run<NCH>(yb + (1 + 3 * (T / 2 - 1)) * tb, packed[T - 1], 256);
                     }
-                    store_plane_run<NCH>(yb + (1 + 3 * (T / 2 - 1)) * tb, packed[T - 1], 256);
+                } else {
+                    // FP32: group DFT in place (wd[c*T + p] = plane p of channel c), then every plane goes out twice:
+                    // rounded to TF32 ("hi") and the TF32-rounded remainder ("lo"), one stage part after the other
+                    dft_words_f32<T>(wd);
+                    auto put = [&](uint8_t* dst, int part_bytes, int p, uint32_t sign) {
+#pragma unroll
+                        for (int c2 = 0; c2 < NCH; ++c2) {
+                            uint32_t hi, lo;
+                            split_tf32(__uint_as_float(wd[c2 * T + p] ^ sign), hi, lo);
+                            const int mn = mn0 + c2;
+                            uint8_t* e = dst + (mn >> 3) * kF32Sbo + (mn & 7) * 16;
+                            *reinterpret_cast<uint32_t*>(e) = hi;
+                            *reinterpret_cast<uint32_t*>(e + part_bytes) = lo;
+                        }
+                    };
+                    if (!is_y) {
+#pragma unroll
+                        for (int p = 0; p < T; ++p) put(stage + p * a_plane + off, prm.x_part_bytes, p, 0u);
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < NCH; ++i) dbacc[i] += __uint_as_float(wd[i * T]);
+                        uint8_t* yb = stage + prm.xhat_bytes + off;
+                        put(yb, prm.y_part_bytes, 0, 0u);
+#pragma unroll
+                        for (int f = 1; f < T / 2; ++f) {
+                            uint8_t* t0 = yb + (1 + 3 * (f - 1)) * tb;
+                            put(t0, prm.y_part_bytes, 2 * f - 1, 0u);                            // Gr
+                            put(t0 + tb, prm.y_part_bytes, 2 * f, 0u);                           // Gi
+                            put(t0 + 2 * tb, prm.y_part_bytes, 2 * f - 1, 0x80000000u);          // -Gr
+                        }
+                        put(yb + (1 + 3 * (T / 2 - 1)) * tb, prm.y_part_bytes, T - 1, 0u);
+                    }
                 }
             }
             ptx::fence_proxy_async_smem();
@@ -332,27 +393,44 @@ EncodeTiledFn encode_fn() {
     return fn;
 }
 
-bool encode_rows16(EncodeTiledFn enc, CUtensorMap* map, const void* base, int64_t cols, int64_t rows) {
+bool encode_rows16(EncodeTiledFn enc, CUtensorMap* map, const void* base, int64_t cols, int64_t rows, int elem_bytes) {
     const cuuint64_t gdim[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
-    const cuuint64_t gstr[1] = {(cuuint64_t)cols * sizeof(__half)};
-    const cuuint32_t box[2] = {64, (cuuint32_t)kChunkTok};
+    const cuuint64_t gstr[1] = {(cuuint64_t)cols * elem_bytes};
+    const cuuint32_t box[2] = {(cuuint32_t)(128 / elem_bytes), (cuuint32_t)kChunkTok};
     const cuuint32_t estr[2] = {1, 1};
-    return enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(base), gdim, gstr, box, estr,
-               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    return enc(map, elem_bytes == 4 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2,
+               const_cast<void*>(base), gdim, gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+               CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// 3-D view of a [rows, cols] half tensor whose row length is a multiple of 64 elements:
-// dim0 = 64 contiguous elements, dim1 = rows (stride = row pitch), dim2 = slab index (stride = 128 bytes).
-// A box [64, 16, nslabs] lands in shared memory as nslabs consecutive [16 x 128 B] slabs.
-bool encode_slabs3d(EncodeTiledFn enc, CUtensorMap* map, const void* base, int64_t cols, int64_t rows, int nslabs) {
-    const cuuint64_t gdim[3] = {64, (cuuint64_t)rows, (cuuint64_t)(cols / 64)};
-    const cuuint64_t gstr[2] = {(cuuint64_t)cols * sizeof(__half), 128};
-    const cuuint32_t box[3] = {64, (cuuint32_t)kChunkTok, (cuuint32_t)nslabs};
+// 3-D view of a [rows, cols] tensor whose row length is a multiple of 128 bytes:
+// dim0 = 128 contiguous bytes of elements, dim1 = rows (stride = row pitch), dim2 = slab index (stride = 128 bytes).
+// A box [128 B, 16, nslabs] lands in shared memory as nslabs consecutive [16 x 128 B] slabs.
+bool encode_slabs3d(EncodeTiledFn enc, CUtensorMap* map, const void* base, int64_t cols, int64_t rows, int nslabs,
+                    int elem_bytes) {
+    const cuuint32_t epr = (cuuint32_t)(128 / elem_bytes);
+    const cuuint64_t gdim[3] = {epr, (cuuint64_t)rows, (cuuint64_t)(cols / epr)};
+    const cuuint64_t gstr[2] = {(cuuint64_t)cols * elem_bytes, 128};
+    const cuuint32_t box[3] = {epr, (cuuint32_t)kChunkTok, (cuuint32_t)nslabs};
     const cuuint32_t estr[3] = {1, 1, 1};
-    return enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, const_cast<void*>(base), gdim, gstr, box, estr,
-               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    return enc(map, elem_bytes == 4 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3,
+               const_cast<void*>(base), gdim, gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+               CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Shared memory outside the operand stages: barriers, alignment, two raw slots, and 8 KB of slack after the last stage
+// (the UMMA reads 128 rows of every plane although only CiT are valid).
+constexpr size_t kBwFixedSmem = 1024 + 1024 + (size_t)kRawSlots * kRawSlot + 8192;
+
+// Bytes per channel of one operand tile of a 16-token chunk: FP16 MN-major 32; FP32 K-major with padded cores 72.
+int bw_chan_bytes(int elem_bytes) { return elem_bytes == 2 ? kChunkTok * 2 : 72; }
+
+size_t bw_stage_bytes(int T, int CiT, int CoT, int elem_bytes) {
+    const int copies = elem_bytes == 4 ? 2 : 1;
+    const int ytiles = 2 + 3 * (T / 2 - 1);
+    const size_t x_part = (size_t)T * ((CiT + 7) / 8 * 8) * bw_chan_bytes(elem_bytes);
+    const size_t y_part = (size_t)ytiles * CoT * bw_chan_bytes(elem_bytes);
+    return align_up(copies * (x_part + y_part), 1024);
 }
 
 int balanced_tile(int C, int max_tile, int round) {
@@ -371,20 +449,30 @@ extern "C" int eqlinear_debug_read_trace_bw(unsigned long long* dst, int n) {
 #endif
 
 bool umma_bwd_weight_supported(int T, eql_dtype_t dtype) {
-    return dtype == EQL_FP16 && (T == 4 || T == 8 || T == 16 || T == 32);
+    if (dtype == EQL_FP16) return T == 4 || T == 8 || T == 16 || T == 32;
+    return T == 4 || T == 8;            // FP32 (3xTF32): larger T leaves too few channels per tile
 }
 
-UmmaBwdWeightShape umma_bwd_weight_shape(int T, int Ci, int Co, int64_t N, int num_sms) {
+UmmaBwdWeightShape umma_bwd_weight_shape(int T, int Ci, int Co, eql_dtype_t dtype, int64_t N, int num_sms) {
     UmmaBwdWeightShape s{};
     s.T = T; s.Ci = Ci; s.Co = Co;
-    int max_cit = 1024 / T;                                      // at most 16 raw slabs of x per chunk
+    s.elem_bytes = dtype == EQL_FP32 ? 4 : 2;
+    const int epr = 128 / s.elem_bytes;                          // elements per raw slab row
+    int max_cit = kMaxXSlabs * epr / T;                          // at most 16 raw slabs of x per chunk
     if (max_cit > 128) max_cit = 128;                            // UMMA M = 128 TMEM lanes
-    s.CiT = balanced_tile(Ci, max_cit, T == 4 ? 16 : 8);
-    s.nCiTiles = (Ci + s.CiT - 1) / s.CiT;
-    s.CoT = balanced_tile(Co, kTmemColsBw / T, 16);
+    int max_cot = kMaxYSlabs * epr / T;                          // at most 8 raw slabs of dy per chunk
+    if (max_cot > kTmemColsBw / T) max_cot = kTmemColsBw / T;    // T planes x CoT fp32 TMEM columns
+    s.CoT = balanced_tile(Co, max_cot, 16);
     s.nCoTiles = (Co + s.CoT - 1) / s.CoT;
-    s.nXs = s.CiT * T / 64;
-    s.nYs = s.CoT * T / 64;
+    s.CiT = balanced_tile(Ci, max_cit, T == 4 ? 16 : 8);
+    // FP32 keeps two copies (hi, lo) of every operand tile: shrink the input-channel tile until one stage fits
+    while (kBwFixedSmem + bw_stage_bytes(T, s.CiT, s.CoT, s.elem_bytes) > 227 * 1024 && max_cit > 16) {
+        max_cit -= 8;
+        s.CiT = balanced_tile(Ci, max_cit, T == 4 ? 16 : 8);
+    }
+    s.nCiTiles = (Ci + s.CiT - 1) / s.CiT;
+    s.nXs = (s.CiT * T + epr - 1) / epr;
+    s.nYs = (s.CoT * T + epr - 1) / epr;
     const int64_t tiles = (int64_t)s.nCiTiles * s.nCoTiles;
     const int64_t chunks = N > 0 ? (N + kChunkTok - 1) / kChunkTok : 1;
     int64_t want = num_sms / tiles;
@@ -401,11 +489,12 @@ cudaError_t launch_umma_bwd_weight(const UmmaBwdWeightShape& s, const void* x, c
     EncodeTiledFn enc = encode_fn();
     if (enc == nullptr) return cudaErrorNotSupported;
     CUtensorMap mx, my;
+    const int E = s.elem_bytes, epr = 128 / E, nsplit = E == 4 ? 2 : 1;
     const int64_t xcols = (int64_t)s.Ci * s.T, ycols = (int64_t)s.Co * s.T;
-    const bool x3d = (xcols % 64 == 0) && encode_slabs3d(enc, &mx, x, xcols, N, s.nXs);
-    const bool y3d = (ycols % 64 == 0) && encode_slabs3d(enc, &my, dy, ycols, N, s.nYs);
-    if (!x3d && !encode_rows16(enc, &mx, x, xcols, N)) return cudaErrorInvalidValue;
-    if (!y3d && !encode_rows16(enc, &my, dy, ycols, N)) return cudaErrorInvalidValue;
+    const bool x3d = (xcols % epr == 0) && encode_slabs3d(enc, &mx, x, xcols, N, s.nXs, E);
+    const bool y3d = (ycols % epr == 0) && encode_slabs3d(enc, &my, dy, ycols, N, s.nYs, E);
+    if (!x3d && !encode_rows16(enc, &mx, x, xcols, N, E)) return cudaErrorInvalidValue;
+    if (!y3d && !encode_rows16(enc, &my, dy, ycols, N, E)) return cudaErrorInvalidValue;
     BwParams prm{};
     prm.x3d = x3d; prm.y3d = y3d;
     prm.part = scratch;
@@ -414,31 +503,41 @@ cudaError_t launch_umma_bwd_weight(const UmmaBwdWeightShape& s, const void* x, c
     prm.N = N; prm.Ci = s.Ci; prm.Co = s.Co; prm.CiT = s.CiT; prm.CoT = s.CoT;
     prm.nCiTiles = s.nCiTiles; prm.nCoTiles = s.nCoTiles; prm.nXs = s.nXs; prm.nYs = s.nYs;
     prm.splits = s.splits; prm.chunks_per_split = s.chunks_per_split;
-    prm.xhat_bytes = s.T * s.CiT * 32;
     const int ytiles = 2 + 3 * (s.T / 2 - 1);
-    prm.stage_bytes = (int)align_up((size_t)prm.xhat_bytes + (size_t)ytiles * s.CoT * 32, 1024);
-    const size_t smem = 1024 + 1024 + (size_t)kRawSlots * kRawSlot + (size_t)kStages * prm.stage_bytes + 4096;
+    const int chan_bytes = bw_chan_bytes(E);
+    prm.x_part_bytes = s.T * ((s.CiT + 7) / 8 * 8) * chan_bytes;  // one copy of the x^ planes
+    prm.y_part_bytes = ytiles * s.CoT * chan_bytes;              // one copy of the dy^ tiles
+    prm.xhat_bytes = nsplit * prm.x_part_bytes;
+    prm.stage_bytes = (int)bw_stage_bytes(s.T, s.CiT, s.CoT, E);
+    prm.stages = kBwFixedSmem + 2 * (size_t)prm.stage_bytes <= 227 * 1024 ? 2 : 1;
+    const size_t smem = kBwFixedSmem + (size_t)prm.stages * prm.stage_bytes;
     if (smem > 227 * 1024) return cudaErrorInvalidConfiguration;
     const int grid = s.splits * s.nCiTiles * s.nCoTiles;
 
-    auto go = [&](auto tc) -> cudaError_t {
+    auto go = [&](auto tc, auto io) -> cudaError_t {
         constexpr int TT = decltype(tc)::value;
+        using IO = decltype(io);
         static unsigned long long attr_done = 0;
         int dev = 0;
         cudaGetDevice(&dev);
         if (!((attr_done >> (dev & 63)) & 1ull)) {
-            cudaError_t e = cudaFuncSetAttribute(umma_bwd_weight_kernel<TT>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+            cudaError_t e = cudaFuncSetAttribute(umma_bwd_weight_kernel<TT, IO>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
             if (e != cudaSuccess) return e;
             attr_done |= 1ull << (dev & 63);
         }
-        umma_bwd_weight_kernel<TT><<<grid, kThreadsBw, smem, stream>>>(mx, my, prm);
+        umma_bwd_weight_kernel<TT, IO><<<grid, kThreadsBw, smem, stream>>>(mx, my, prm);
         return cudaGetLastError();
     };
+    if (E == 4) {
+        if (s.T == 4) return go(std::integral_constant<int, 4>{}, float{});
+        if (s.T == 8) return go(std::integral_constant<int, 8>{}, float{});
+        return cudaErrorInvalidValue;
+    }
     switch (s.T) {
-        case 4: return go(std::integral_constant<int, 4>{});
-        case 8: return go(std::integral_constant<int, 8>{});
-        case 16: return go(std::integral_constant<int, 16>{});
-        case 32: return go(std::integral_constant<int, 32>{});
+        case 4: return go(std::integral_constant<int, 4>{}, __half{});
+        case 8: return go(std::integral_constant<int, 8>{}, __half{});
+        case 16: return go(std::integral_constant<int, 16>{}, __half{});
+        case 32: return go(std::integral_constant<int, 32>{}, __half{});
         default: return cudaErrorInvalidValue;
     }
 }
