@@ -176,8 +176,10 @@ umma_bwd_weight_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
             constexpr int KSTEPS = E == 2 ? 1 : 2;                       // a 16-token chunk is one K step of halves, two of TF32
             constexpr int PASSES = E == 2 ? 1 : 3;                       // 3xTF32: hi*hi, hi*lo, lo*hi
             for (int64_t c = 0; c < nchunks; ++c) {
-                const int st = (int)(c % NST);
-                ok = ptx::mbar_wait(&bar->full_ab[st], (uint32_t)((c / NST) & 1), abort_flag, status, 202);
+                // NST is 1 or 2: stage and phase parity without a division
+                const int st = NST == 2 ? (int)(c & 1) : 0;
+                const uint32_t sph = (uint32_t)((NST == 2 ? (c >> 1) : c) & 1);
+                ok = ptx::mbar_wait(&bar->full_ab[st], sph, abort_flag, status, 202);
                 if (!ok) break;
                 ptx::tc_fence_after_sync();
                 const uint32_t stage0 = ptx::smem_u32(stages + st * prm.stage_bytes);
@@ -218,7 +220,8 @@ umma_bwd_weight_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
         for (int i = 0; i < NCH; ++i) dbacc[i] = 0.f;
         bool ok = true;
         for (int64_t c = 0; c < nchunks; ++c) {
-            const int slot = (int)(c % kRawSlots), st = (int)(c % NST);
+            const int slot = (int)(c % kRawSlots), st = NST == 2 ? (int)(c & 1) : 0;
+            const uint32_t sph = (uint32_t)((NST == 2 ? (c >> 1) : c) & 1);
 #ifdef EQL_TRACE
             const bool tr = lane == 0 && (warp == kWarpDftX0 || warp == kWarpDftY0);
             const int tb = (warp == kWarpDftX0 ? 4000 : 5000) + 6 * (int)c;
@@ -228,7 +231,7 @@ umma_bwd_weight_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
 #ifdef EQL_TRACE
             if (tr) BW_STAMP(tb + 1);
 #endif
-            ok = ok && ptx::mbar_wait(&bar->empty_ab[st], (uint32_t)((c / NST) & 1) ^ 1, abort_flag, status, 204);
+            ok = ok && ptx::mbar_wait(&bar->empty_ab[st], sph ^ 1, abort_flag, status, 204);
 #ifdef EQL_TRACE
             if (tr) BW_STAMP(tb + 2);
 #endif
