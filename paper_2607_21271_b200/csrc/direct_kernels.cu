@@ -325,8 +325,21 @@ bwd_weight_finalize_kernel(const float* __restrict__ part, const float* __restri
     }
     float acc = 0.f;
     if (idx < Ci * Co) {
+        // four running sums (split index mod 4), combined in a fixed order: the result does not depend on timing, and
+        // eight loads are in flight per thread instead of one dependent chain
         const float* src = part + (size_t)p * plane_stride + idx;
-        for (int sp = 0; sp < splits; ++sp) acc += src[(size_t)sp * T * plane_stride];
+        const size_t step = (size_t)T * plane_stride;
+        float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+        int sp = 0;
+#pragma unroll 2
+        for (; sp + 4 <= splits; sp += 4) {
+            a0 += __ldg(src + (size_t)sp * step);
+            a1 += __ldg(src + (size_t)(sp + 1) * step);
+            a2 += __ldg(src + (size_t)(sp + 2) * step);
+            a3 += __ldg(src + (size_t)(sp + 3) * step);
+        }
+        for (; sp < splits; ++sp) a0 += __ldg(src + (size_t)sp * step);
+        acc = (a0 + a1) + (a2 + a3);
     }
     const bool imag = (p != 0) && (p != T - 1) && ((p & 1) == 0);
     acc *= plane_inverse_scale<T>(p);

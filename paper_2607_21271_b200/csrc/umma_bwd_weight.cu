@@ -49,6 +49,7 @@ struct BwParams {
     int x_part_bytes, y_part_bytes;   // FP32: bytes of the TF32 "hi" copy of x^ / dy^ inside a stage; the "lo" copy follows it
     int stages;                  // operand stages (2; 1 where the hi/lo copies of FP32 leave no room for two)
     int x3d, y3d;                // tensor maps are 3-D (64 elements, rows, slab index): one load per chunk and tensor
+    int part_tma;                // the partial spectra can be written with TMA tensor stores (row pitch a multiple of 16 bytes)
 };
 
 // Optional timeline instrumentation (compiled only with -DEQL_TRACE): CTA 0 records clock64() stamps.
@@ -70,7 +71,7 @@ struct BwBarriers {
 template <int T, typename IO>
 __global__ void __launch_bounds__(kThreadsBw, 1)
 umma_bwd_weight_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_dy,
-                       const BwParams prm) {
+                       const __grid_constant__ CUtensorMap tmap_part, const BwParams prm) {
     constexpr int E = sizeof(IO);                 // 2: half inputs, 4: float inputs (3xTF32)
     constexpr int EPR = 128 / E;                  // elements per 128-byte raw row
     constexpr int NCH = EPR / T;                  // channels per raw row
@@ -351,7 +352,14 @@ umma_bwd_weight_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
                 const uint32_t lane_base = tmem_base + ((uint32_t)(quad * 32) << 16);
                 const size_t plane_stride = (size_t)prm.Co * prm.Ci;
                 float* dst = prm.part + (size_t)split * T * plane_stride;
-                for (int col = third * 16; col < T * CoT; col += 48) {
+                // A quad whose 32 rows all belong to this input-channel tile goes out through shared memory and TMA
+                // tensor stores ([16 output channels x 32 input channels] floats per store, two staging buffers per
+                // warp in the idle raw slots; channels beyond C_in / C_out are clipped by the hardware).  Other quads
+                // write their valid lanes directly.
+                const bool via_tma = prm.part_tma != 0 && quad * 32 + 32 <= CiT;
+                float* stg = reinterpret_cast<float*>(raw + (warp - kWarpDftX0) * 4096);
+                int it = 0;
+                for (int col = third * 16; col < T * CoT; col += 48, ++it) {
                     uint32_t v[16];
                     if (nchunks > 0) {
                         ptx::tmem_ld<16>(lane_base + (uint32_t)col, v);
@@ -361,12 +369,25 @@ umma_bwd_weight_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
                         for (int j = 0; j < 16; ++j) v[j] = 0u;
                     }
                     const int p = col / CoT, o0 = co_tile * CoT + col % CoT;
-                    if (lane_ok) {
+                    if (via_tma) {
+                        float* buf = stg + (it & 1) * 512;
+                        if (lane == 0) ptx::bulk_wait_group_read1();     // the store issued two iterations ago has read this buffer
+                        __syncwarp();
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) buf[j * 32 + lane] = __uint_as_float(v[j]);
+                        ptx::fence_proxy_async_smem();
+                        __syncwarp();
+                        if (lane == 0 && o0 < prm.Co) {
+                            ptx::tma_store_3d(&tmap_part, ci_tile * CiT + quad * 32, o0, split * T + p, buf);
+                            ptx::bulk_commit_group();
+                        }
+                    } else if (lane_ok) {
 #pragma unroll
                         for (int j = 0; j < 16; ++j)
                             if (o0 + j < prm.Co) dst[p * plane_stride + (size_t)(o0 + j) * prm.Ci + ci] = __uint_as_float(v[j]);
                     }
                 }
+                if (via_tma && lane == 0) ptx::bulk_wait_group_read0();
             }
         }
     }
@@ -498,8 +519,20 @@ cudaError_t launch_umma_bwd_weight(const UmmaBwdWeightShape& s, const void* x, c
     const bool y3d = (ycols % epr == 0) && encode_slabs3d(enc, &my, dy, ycols, N, s.nYs, E);
     if (!x3d && !encode_rows16(enc, &mx, x, xcols, N, E)) return cudaErrorInvalidValue;
     if (!y3d && !encode_rows16(enc, &my, dy, ycols, N, E)) return cudaErrorInvalidValue;
+    // partial spectra [splits*T][Co][Ci] floats as a 3-D tensor for the epilogue's TMA stores (box 32 x 16 x 1)
+    CUtensorMap mp;
+    bool part_tma = (s.Ci % 4 == 0) && (reinterpret_cast<uintptr_t>(scratch) % 16 == 0);
+    if (part_tma) {
+        const cuuint64_t gdim[3] = {(cuuint64_t)s.Ci, (cuuint64_t)s.Co, (cuuint64_t)s.splits * s.T};
+        const cuuint64_t gstr[2] = {(cuuint64_t)s.Ci * sizeof(float), (cuuint64_t)s.Ci * s.Co * sizeof(float)};
+        const cuuint32_t box[3] = {32, 16, 1};
+        const cuuint32_t estr[3] = {1, 1, 1};
+        part_tma = enc(&mp, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, scratch, gdim, gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                       CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    }
+    if (!part_tma) mp = mx;                                     // unused by the kernel then; any valid map will do
     BwParams prm{};
-    prm.x3d = x3d; prm.y3d = y3d;
+    prm.x3d = x3d; prm.y3d = y3d; prm.part_tma = part_tma;
     prm.part = scratch;
     prm.db_part = scratch + (size_t)s.splits * s.T * s.Co * s.Ci;
     prm.status = status;
@@ -528,7 +561,7 @@ cudaError_t launch_umma_bwd_weight(const UmmaBwdWeightShape& s, const void* x, c
             if (e != cudaSuccess) return e;
             attr_done |= 1ull << (dev & 63);
         }
-        umma_bwd_weight_kernel<TT, IO><<<grid, kThreadsBw, smem, stream>>>(mx, my, prm);
+        umma_bwd_weight_kernel<TT, IO><<<grid, kThreadsBw, smem, stream>>>(mx, my, mp, prm);
         return cudaGetLastError();
     };
     if (E == 4) {
