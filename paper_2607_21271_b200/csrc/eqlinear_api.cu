@@ -118,10 +118,10 @@ int64_t host_chunk_tokens(int64_t N) {
 }
 
 // fwd (and, with dy/dx, the data gradient) of N tokens from host buffers through the three-stream pipeline.
-// On return every copy and kernel has been enqueued and `s` waits for the last device -> host copy.
+// On return every copy and kernel has been enqueued; with join, `s` also waits for the last device -> host copy.
 eql_status_t pipelined_host(eqlinear_plan_t plan, const void* x_host, const void* dy_host, void* y_host, void* dx_host,
                             int64_t N, void* x_staging, void* dy_staging, void* y_staging, void* dx_staging,
-                            cudaStream_t s) {
+                            cudaStream_t s, bool join) {
     HostPipe* hp = get_pipe(plan);
     if (!hp) return EQL_ERR_CUDA;
     const size_t e = elem_size(plan->dtype);
@@ -158,8 +158,14 @@ eql_status_t pipelined_host(eqlinear_plan_t plan, const void* x_host, const void
                             hp->out) != cudaSuccess) return EQL_ERR_CUDA;
     }
     if (cudaEventRecord(hp->out_done, hp->out) != cudaSuccess) return EQL_ERR_CUDA;
-    if (cudaStreamWaitEvent(s, hp->out_done, 0) != cudaSuccess) return EQL_ERR_CUDA;
+    if (join && cudaStreamWaitEvent(s, hp->out_done, 0) != cudaSuccess) return EQL_ERR_CUDA;
     return EQL_OK;
+}
+
+// Makes `s` wait for the last device -> host copy of the preceding pipelined_host(..., join = false).
+eql_status_t join_pipe(eqlinear_plan_t plan, cudaStream_t s) {
+    if (!plan->pipe) return EQL_OK;
+    return cudaStreamWaitEvent(s, plan->pipe->out_done, 0) == cudaSuccess ? EQL_OK : EQL_ERR_CUDA;
 }
 
 }  // namespace
@@ -389,7 +395,7 @@ eql_status_t eqlinear_fwd_host(eqlinear_plan_t plan, const void* x_host, void* y
     if (N == 0) return EQL_OK;
     if (!x_host || !y_host || !x_staging || !y_staging) return EQL_ERR_INVALID_ARG;
     return pipelined_host(plan, x_host, nullptr, y_host, nullptr, N, x_staging, nullptr, y_staging, nullptr,
-                          (cudaStream_t)stream);
+                          (cudaStream_t)stream, true);
 }
 
 eql_status_t eqlinear_bwd_data_host(eqlinear_plan_t plan, const void* dy_host, void* dx_host, int64_t N,
@@ -448,7 +454,7 @@ eql_status_t eqlinear_step_host(eqlinear_plan_t plan, const void* x_host, const 
     cudaStream_t s = (cudaStream_t)stream;
     // forward and data gradient chunk by chunk while the copies of the neighbouring chunks are in flight; the weight
     // gradient reduces over all tokens and runs once every chunk has arrived
-    st = pipelined_host(plan, x_host, dy_host, y_host, dx_host, N, x_staging, dy_staging, y_staging, dx_staging, s);
+    st = pipelined_host(plan, x_host, dy_host, y_host, dx_host, N, x_staging, dy_staging, y_staging, dx_staging, s, false);
     if (st != EQL_OK) return st;
     if ((st = eqlinear_bwd_weight(plan, x_staging, dy_staging, dw_staging, db_staging, N, scratch, scratch_bytes,
                                   stream)) != EQL_OK) return st;
@@ -456,7 +462,7 @@ eql_status_t eqlinear_step_host(eqlinear_plan_t plan, const void* x_host, const 
                         cudaMemcpyDeviceToHost, s) != cudaSuccess) return EQL_ERR_CUDA;
     if (db_host && cudaMemcpyAsync(db_host, db_staging, (size_t)plan->Co * sizeof(float), cudaMemcpyDeviceToHost, s) !=
                        cudaSuccess) return EQL_ERR_CUDA;
-    return EQL_OK;
+    return join_pipe(plan, s);                                   // the y / dx copies of the last chunks may still be in flight
 }
 
 }  // extern "C"
