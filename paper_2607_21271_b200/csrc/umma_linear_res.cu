@@ -158,8 +158,11 @@ umma_linear_res_kernel(const __grid_constant__ CUtensorMap tmap_in, const ResPar
     // every role walks the units with a running (token tile, channel tile) pair instead of dividing per unit
     const int ct0 = (int)(u0 % nCT);
     const int64_t tt0 = u0 / nCT;
-    auto first_of_tile = [&](int64_t u, int ct) { return u == u0 || ct == 0; };
-    auto last_of_tile = [&](int64_t u, int ct) { return u == u1 - 1 || ct == nCT - 1; };
+    // With a ring of x^ buffers (fewer buffers than chunks) nothing survives a unit: every unit transforms its token
+    // tile itself, i.e. is the first and the last of its tile.
+    const bool ring = XR < nK;
+    auto first_of_tile = [&](int64_t u, int ct) { return ring || u == u0 || ct == 0; };
+    auto last_of_tile = [&](int64_t u, int ct) { return ring || u == u1 - 1 || ct == nCT - 1; };
     const int items_per_tile = IPC * nK;
 
     if (warp == kResWarpTmaX) {
@@ -498,7 +501,9 @@ UmmaResShape umma_res_shape(int T, int Cin, int Cout) {
             }
         }
     }
-    // One channel tile: nothing is reused across units, so three x^ buffers used as a ring are enough.  The ring
+    // One channel tile: nothing is reused across units, so three x^ buffers used as a ring are enough (with two
+    // channel tiles, each repeating the transform, the streaming kernel measured faster: 104 vs 111 us on the
+    // D = 1024, T = 4 shape).  The ring
     // needs all 12 transform warps (chunk q is then always transformed by warps 4 (q % 3) .. 4 (q % 3) + 3, which
     // therefore see every phase of the buffer barriers they wait on).
     if (s.nCT == 1 && !(s.fits && s.w_slots >= 3) && s.nK > 3 &&
