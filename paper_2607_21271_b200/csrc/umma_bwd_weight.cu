@@ -180,7 +180,9 @@ umma_bwd_weight_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
                 // NST is 1 or 2: stage and phase parity without a division
                 const int st = NST == 2 ? (int)(c & 1) : 0;
                 const uint32_t sph = (uint32_t)((NST == 2 ? (c >> 1) : c) & 1);
+                BW_STAMP(1000 + 3 * (int)c);
                 ok = ptx::mbar_wait(&bar->full_ab[st], sph, abort_flag, status, 202);
+                BW_STAMP(1000 + 3 * (int)c + 1);
                 if (!ok) break;
                 ptx::tc_fence_after_sync();
                 const uint32_t stage0 = ptx::smem_u32(stages + st * prm.stage_bytes);
@@ -204,6 +206,7 @@ umma_bwd_weight_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
                     }
                 }
                 ptx::umma_commit(&bar->empty_ab[st]);
+                BW_STAMP(1000 + 3 * (int)c + 2);
             }
             if (ok) ptx::umma_commit(&bar->full_d);
             ptx::umma_commit(&bar->mma_done);
