@@ -192,7 +192,7 @@ eql_status_t eqlinear_bwd_weight_static(eqlinear_plan_t plan, const void* x, con
  * results back, all asynchronously; the host buffers may be read once `stream` has been
  * synchronised.  Staging buffers are device memory with the sizes of the corresponding
  * device-variant tensors.
- * eqlinear_fwd_host and eqlinear_step_host move batches of 8192 tokens or more in up to eight token
+ * eqlinear_fwd_host and eqlinear_step_host move batches of 8192 tokens or more in up to sixteen token
  * chunks through a three-stream pipeline (host -> device copies, kernels on `stream`, device -> host
  * copies), so that both copy directions and the kernels overlap; `stream` waits for the last copy
  * before the call's remaining work.  The two extra streams and their events belong to the plan:

@@ -114,7 +114,7 @@ cudaError_t launch_bwd_weight_finalize(int T, bool correlation, const float* scr
 // Copy pipeline of the host-buffer entry points: token chunks travel host -> device on one stream, are computed on
 // the caller's stream and travel back on a third, so that the two copy directions and the kernels overlap.
 // Created on first use, destroyed with the plan (streams and events only: no device memory).
-constexpr int kHostChunks = 8;
+constexpr int kHostChunks = 16;
 struct HostPipe {
     cudaStream_t in = nullptr, out = nullptr;
     cudaEvent_t start = nullptr, out_done = nullptr;

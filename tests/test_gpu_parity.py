@@ -212,7 +212,7 @@ def test_gpu_equivariance_and_adjoint(dtype, T):
 # ------------------------------------------------------------------ host-buffer variants
 @pytest.mark.parametrize("N", [700, 9001])
 def test_host_buffer_variants(N):
-    """N = 9001 goes through the chunked three-stream copy pipeline (eight chunks, the last one ragged)."""
+    """N = 9001 goes through the chunked three-stream copy pipeline (chunks of 640 tokens, the last one ragged)."""
     wl = Workload("host", "fp16", 8, 24, 40, N, "normal", ("fwd", "bwd_data", "bwd_weight"), 20)
     d = generate(wl)
     layer = GpuLayer(wl.T, wl.Ci, wl.Co, wl.dtype, d["w"], d["bias"])
