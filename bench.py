@@ -190,6 +190,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--force-simt", action="store_true", help="use the CUDA-core kernels (context numbers)")
+    ap.add_argument("--no-saved-spectrum", action="store_true",
+                    help="weight gradient from x (eqlinear_bwd_weight) instead of from the spectrum saved by the forward pass")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -251,18 +253,33 @@ def main():
     db = torch.empty(wl.Co, dtype=torch.float32, device=dev)
     sb = eq.eqlinear_bwd_weight_scratch_bytes(plan, wl.N) if has_bwd else 0
     scratch = torch.empty(max(sb, 256), dtype=torch.uint8, device=dev)
+    # Training with a saved spectrum: the forward kernel that transforms x once per token tile also writes x^ for
+    # the weight gradient (same step, same results within the same bars).  Used where that forward kernel runs and
+    # x is the small tensor of the layer (else writing x^ costs more than repeating the transform).
+    use_saved = (has_bwd and not args.no_saved_spectrum and wl.dtype == "fp16" and info.fwd_kernel == 2
+                 and info.bwd_weight_kernel == 1 and wl.Co >= 2 * wl.Ci)
+    spec_bytes = eq.eqlinear_spectrum_bytes(plan, wl.N) if use_saved else 0
+    if use_saved:
+        for s in sets:
+            s["spec"] = torch.empty(spec_bytes, dtype=torch.uint8, device=dev)
 
     def step(s, events=None):
         if events is not None:
             events[0].record()
-        eq.eqlinear_fwd(plan, s["x"], s["y"], wl.N, stream)
+        if use_saved:
+            eq.eqlinear_fwd_save_spectrum(plan, s["x"], s["y"], wl.N, s["spec"], spec_bytes, stream)
+        else:
+            eq.eqlinear_fwd(plan, s["x"], s["y"], wl.N, stream)
         if events is not None:
             events[1].record()
         if has_bwd:
             eq.eqlinear_bwd_data(plan, s["dy"], s["dx"], wl.N, stream)
             if events is not None:
                 events[2].record()
-            eq.eqlinear_bwd_weight(plan, s["x"], s["dy"], dw, db, wl.N, scratch, sb, stream)
+            if use_saved:
+                eq.eqlinear_bwd_weight_from_spectrum(plan, s["spec"], spec_bytes, s["dy"], dw, db, wl.N, scratch, sb, stream)
+            else:
+                eq.eqlinear_bwd_weight(plan, s["x"], s["dy"], dw, db, wl.N, scratch, sb, stream)
             if events is not None:
                 events[3].record()
             if world > 1:
@@ -387,7 +404,8 @@ def main():
                 "scaling": "weak", "vs_baseline": None, "dtype": "f16" if wl.dtype == "fp16" else "f32",
                 "data": "synthetic",
                 "config": workload_config(wl, n_gpus, {"l2": f"rotating {n_sets} buffer sets "
-                                                              f"({n_sets * bytes_per_set / 1e6:.0f} MB > 126 MB L2)"}),
+                                                              f"({n_sets * bytes_per_set / 1e6:.0f} MB > 126 MB L2)",
+                                                        "saved_spectrum": bool(use_saved)}),
                 "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
                 "roofline": roofline, "cpu_baseline": cpu_baseline}
         print(json.dumps(line))

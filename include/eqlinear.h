@@ -158,6 +158,31 @@ eql_status_t eqlinear_bwd_weight(eqlinear_plan_t plan, const void* x, const void
                                  void* dw, void* db, int64_t N,
                                  void* scratch, size_t scratch_bytes, void* stream);
 
+/* ---- training with a saved spectrum (FP16 plans whose weight gradient runs on the tensor cores) --
+ * Algorithm 1 transforms x once for the forward pass; the weight gradient needs the same spectrum
+ * x^ again, and computing it there is the largest share of that kernel's instructions (every
+ * output-channel tile repeats it).  These three calls let the forward pass save x^ -- rounded to
+ * fp16, in the operand layout of the weight-gradient kernel -- so that the weight gradient reads it
+ * back instead of x.  (The paper's kernels keep no frequency-domain tensor in global memory; this
+ * is an optional trade of N*C_in*T*2 bytes of device memory and one extra write of that size for a
+ * shorter backward pass.)  The buffer's layout is private to the library; it is valid for the plan
+ * and N it was written with. */
+
+/* Bytes of the saved-spectrum buffer for N tokens.  EQL_ERR_UNSUPPORTED for plans without this path
+ * (FP32 plans, EQL_FLAG_FORCE_SIMT). */
+eql_status_t eqlinear_spectrum_bytes(eqlinear_plan_t plan, int64_t N, size_t* bytes);
+
+/* eqlinear_fwd that also writes the spectrum of x.
+ *   spectrum: device, 256-byte aligned, >= eqlinear_spectrum_bytes(plan, N). */
+eql_status_t eqlinear_fwd_save_spectrum(eqlinear_plan_t plan, const void* x, void* y, int64_t N,
+                                        void* spectrum, size_t spectrum_bytes, void* stream);
+
+/* eqlinear_bwd_weight with the saved spectrum in place of x (same outputs, same scratch size, same
+ * fixed reduction order).  N must be the N of the eqlinear_fwd_save_spectrum call that wrote it. */
+eql_status_t eqlinear_bwd_weight_from_spectrum(eqlinear_plan_t plan, const void* spectrum, size_t spectrum_bytes,
+                                               const void* dy, void* dw, void* db, int64_t N,
+                                               void* scratch, size_t scratch_bytes, void* stream);
+
 /* Size of the scratch array that is built into the library for eqlinear_bwd_weight_static. */
 #define EQL_STATIC_SCRATCH_BYTES (32u << 20)
 

@@ -38,6 +38,7 @@ EXPORTED_SYMBOLS = (
     "eqlinear_plan_set_weight", "eqlinear_plan_info", "eqlinear_plan_device_status", "eqlinear_plan_destroy",
     "eqlinear_fwd", "eqlinear_bwd_data", "eqlinear_bwd_weight_scratch_bytes", "eqlinear_bwd_weight",
     "eqlinear_fwd_host", "eqlinear_bwd_data_host", "eqlinear_bwd_weight_host", "eqlinear_step_host", "eqlinear_bwd_weight_static",
+    "eqlinear_spectrum_bytes", "eqlinear_fwd_save_spectrum", "eqlinear_bwd_weight_from_spectrum",
 )
 
 
@@ -93,6 +94,9 @@ def load_library(path: str | None = None) -> ctypes.CDLL:
         "eqlinear_bwd_weight_host": [V, V, V, V, V, I64, V, V, V, V, V, SZ, V],
         "eqlinear_bwd_weight_static": [V, V, V, V, V, I64, V],
         "eqlinear_step_host": [V, V, V, V, V, V, V, I64, V, V, V, V, V, V, V, SZ, V],
+        "eqlinear_spectrum_bytes": [V, I64, POINTER(SZ)],
+        "eqlinear_fwd_save_spectrum": [V, V, V, I64, V, SZ, V],
+        "eqlinear_bwd_weight_from_spectrum": [V, V, SZ, V, V, V, I64, V, SZ, V],
     }
     for name, argtypes in sigs.items():
         fn = getattr(lib, name)
@@ -206,6 +210,24 @@ def eqlinear_step_host(plan, x_host, dy_host, y_host, dx_host, dw_host, db_host,
                                              _ptr(dw_host), _ptr(db_host), N, _ptr(x_staging), _ptr(dy_staging),
                                              _ptr(y_staging), _ptr(dx_staging), _ptr(dw_staging), _ptr(db_staging),
                                              _ptr(scratch), scratch_bytes, stream or None), "eqlinear_step_host")
+
+
+def eqlinear_spectrum_bytes(plan, N) -> int:
+    out = c_size_t(0)
+    _check(load_library().eqlinear_spectrum_bytes(plan, N, byref(out)), "eqlinear_spectrum_bytes")
+    return out.value
+
+
+def eqlinear_fwd_save_spectrum(plan, x, y, N, spectrum, spectrum_bytes, stream=0) -> None:
+    """eqlinear_fwd that also saves the fp16 spectrum of x for eqlinear_bwd_weight_from_spectrum."""
+    _check(load_library().eqlinear_fwd_save_spectrum(plan, _ptr(x), _ptr(y), N, _ptr(spectrum), spectrum_bytes,
+                                                     stream or None), "eqlinear_fwd_save_spectrum")
+
+
+def eqlinear_bwd_weight_from_spectrum(plan, spectrum, spectrum_bytes, dy, dw, db, N, scratch, scratch_bytes, stream=0) -> None:
+    _check(load_library().eqlinear_bwd_weight_from_spectrum(plan, _ptr(spectrum), spectrum_bytes, _ptr(dy), _ptr(dw),
+                                                            _ptr(db), N, _ptr(scratch), scratch_bytes, stream or None),
+           "eqlinear_bwd_weight_from_spectrum")
 
 
 def eqlinear_bwd_weight_static(plan, x, dy, dw, db, N, stream=0) -> None:

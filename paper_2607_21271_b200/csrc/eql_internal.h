@@ -86,8 +86,11 @@ struct UmmaResShape {
 bool umma_res_supported(int T, eql_dtype_t dtype);
 UmmaResShape umma_res_shape(int T, int Cin, int Cout);
 cudaError_t launch_build_umma_res_image(const UmmaResShape& s, const float* planes, void* image, cudaStream_t stream);
+struct UmmaBwdWeightShape;
+// stash (optional): also write the spectrum of `in` as the operand image of the saved-spectrum weight-gradient kernel
 cudaError_t launch_umma_linear_res(const UmmaResShape& s, const void* in, void* out, int64_t N, const void* image,
-                                   const float* bias_f32, int* status, int num_sms, cudaStream_t stream);
+                                   const float* bias_f32, int* status, int num_sms, cudaStream_t stream,
+                                   const UmmaBwdWeightShape* stash_shape = nullptr, void* stash = nullptr);
 
 // ---- tcgen05 weight-gradient kernel (FP16 inputs; FP32 inputs with the 3xTF32 split), umma_bwd_weight.cu --------------------------------
 struct UmmaBwdWeightShape {
@@ -99,12 +102,19 @@ struct UmmaBwdWeightShape {
     int splits;                 // token ranges
     int64_t chunks_per_split;   // 16-token chunks per range
     size_t scratch_bytes;       // splits * (T*Co*Ci + Co) floats
+    int64_t total_chunks;       // 16-token chunks in all
+    size_t stash_bytes;         // FP16: saved spectrum of x as operand image, nCiTiles * total_chunks * T*CiT*32 bytes (else 0)
 };
 bool umma_bwd_weight_supported(int T, eql_dtype_t dtype);
 UmmaBwdWeightShape umma_bwd_weight_shape(int T, int Ci, int Co, eql_dtype_t dtype, int64_t N, int num_sms);
 // Phase 1 only: partial spectra + db partials into scratch (same layout as the CUDA-core kernel's).
 cudaError_t launch_umma_bwd_weight(const UmmaBwdWeightShape& s, const void* x, const void* dy, int64_t N,
                                    float* scratch, int* status, cudaStream_t stream);
+// The same from a saved spectrum of x (umma_bwd_weight_saved.cu, FP16): the image written by the forward pass, or by
+// launch_xhat_image, replaces x.
+cudaError_t launch_xhat_image(const UmmaBwdWeightShape& s, const void* x, int64_t N, void* stash, cudaStream_t stream);
+cudaError_t launch_umma_bwd_weight_saved(const UmmaBwdWeightShape& s, const void* stash, const void* dy, int64_t N,
+                                         float* scratch, int* status, cudaStream_t stream);
 // Phase 2 (direct_kernels.cu): fixed-order sum over splits, 1/T, inverse DFT -> dw, db.
 cudaError_t launch_bwd_weight_finalize(int T, bool correlation, const float* scratch, int splits, int Ci, int Co,
                                        float* dw, float* db, cudaStream_t stream);

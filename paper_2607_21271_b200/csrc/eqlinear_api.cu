@@ -386,6 +386,72 @@ eql_status_t eqlinear_bwd_weight(eqlinear_plan_t plan, const void* x, const void
     return e == cudaSuccess ? EQL_OK : EQL_ERR_CUDA;
 }
 
+// ---- training with a saved spectrum ---------------------------------------------------------------
+eql_status_t eqlinear_spectrum_bytes(eqlinear_plan_t plan, int64_t N, size_t* bytes) {
+    if (!plan || !bytes) return EQL_ERR_INVALID_ARG;
+    eql_status_t st = check_tokens(N);
+    if (st != EQL_OK) return st;
+    if (plan->dtype != EQL_FP16 || plan->bwd_weight_kernel != 1) return EQL_ERR_UNSUPPORTED;
+    *bytes = umma_bwd_weight_shape(plan->T, plan->Ci, plan->Co, plan->dtype, N > 0 ? N : 1, plan->num_sms).stash_bytes;
+    return EQL_OK;
+}
+
+eql_status_t eqlinear_fwd_save_spectrum(eqlinear_plan_t plan, const void* x, void* y, int64_t N, void* spectrum,
+                                        size_t spectrum_bytes, void* stream) {
+    if (!plan) return EQL_ERR_INVALID_ARG;
+    size_t need = 0;
+    eql_status_t st = eqlinear_spectrum_bytes(plan, N, &need);
+    if (st != EQL_OK) return st;
+    if (N == 0) return EQL_OK;
+    if (!spectrum) return EQL_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(spectrum) % kWsAlign != 0) return EQL_ERR_ALIGNMENT;
+    if (spectrum_bytes < need) return EQL_ERR_WORKSPACE;
+    const UmmaBwdWeightShape bs = umma_bwd_weight_shape(plan->T, plan->Ci, plan->Co, plan->dtype, N, plan->num_sms);
+    if (plan->fwd_kernel == 2) {
+        // the resident-activation kernel writes the spectrum while it transforms x for its own use
+        if (!x || !y || x == y) return EQL_ERR_INVALID_ARG;
+        if (!aligned16(x) || !aligned16(y)) return EQL_ERR_ALIGNMENT;
+        const float* bias = plan->has_bias ? (const float*)(plan->ws + plan->lay.bias) : nullptr;
+        cudaError_t e = launch_umma_linear_res(plan->res_fwd, x, y, N, plan->ws + plan->lay.umma_fwd, bias,
+                                               (int*)(plan->ws + plan->lay.status), plan->num_sms, (cudaStream_t)stream,
+                                               &bs, spectrum);
+        return e == cudaSuccess ? EQL_OK : EQL_ERR_CUDA;
+    }
+    // other forward kernels: a pre-pass kernel transforms x once more
+    st = eqlinear_fwd(plan, x, y, N, stream);
+    if (st != EQL_OK) return st;
+    cudaError_t e = launch_xhat_image(bs, x, N, spectrum, (cudaStream_t)stream);
+    return e == cudaSuccess ? EQL_OK : EQL_ERR_CUDA;
+}
+
+eql_status_t eqlinear_bwd_weight_from_spectrum(eqlinear_plan_t plan, const void* spectrum, size_t spectrum_bytes,
+                                               const void* dy, void* dw, void* db, int64_t N, void* scratch,
+                                               size_t scratch_bytes, void* stream) {
+    if (!plan) return EQL_ERR_INVALID_ARG;
+    size_t need = 0;
+    eql_status_t st = eqlinear_spectrum_bytes(plan, N, &need);
+    if (st != EQL_OK) return st;
+    if (!dw) return EQL_ERR_INVALID_ARG;
+    if (!aligned16(dw) || (db && !aligned16(db))) return EQL_ERR_ALIGNMENT;
+    cudaStream_t s = (cudaStream_t)stream;
+    if (N == 0) {
+        if (cudaMemsetAsync(dw, 0, (size_t)plan->Co * plan->Ci * plan->T * sizeof(float), s) != cudaSuccess) return EQL_ERR_CUDA;
+        if (db && cudaMemsetAsync(db, 0, (size_t)plan->Co * sizeof(float), s) != cudaSuccess) return EQL_ERR_CUDA;
+        return EQL_OK;
+    }
+    if (!spectrum || !dy || !scratch) return EQL_ERR_INVALID_ARG;
+    if (!aligned16(dy) || reinterpret_cast<uintptr_t>(spectrum) % kWsAlign != 0 ||
+        reinterpret_cast<uintptr_t>(scratch) % kWsAlign != 0) return EQL_ERR_ALIGNMENT;
+    if (spectrum_bytes < need) return EQL_ERR_WORKSPACE;
+    const UmmaBwdWeightShape bs = umma_bwd_weight_shape(plan->T, plan->Ci, plan->Co, plan->dtype, N, plan->num_sms);
+    if (scratch_bytes < bs.scratch_bytes) return EQL_ERR_WORKSPACE;
+    cudaError_t e = launch_umma_bwd_weight_saved(bs, spectrum, dy, N, (float*)scratch, (int*)(plan->ws + plan->lay.status), s);
+    if (e != cudaSuccess) return EQL_ERR_CUDA;
+    e = launch_bwd_weight_finalize(plan->T, (plan->flags & EQL_FLAG_CORRELATION) != 0, (const float*)scratch, bs.splits,
+                                   plan->Ci, plan->Co, (float*)dw, (float*)db, s);
+    return e == cudaSuccess ? EQL_OK : EQL_ERR_CUDA;
+}
+
 // ---- host-buffer variants ---------------------------------------------------------------------
 eql_status_t eqlinear_fwd_host(eqlinear_plan_t plan, const void* x_host, void* y_host, int64_t N, void* x_staging,
                                void* y_staging, void* stream) {

@@ -514,6 +514,8 @@ UmmaBwdWeightShape umma_bwd_weight_shape(int T, int Ci, int Co, eql_dtype_t dtyp
     s.chunks_per_split = (chunks + want - 1) / want;
     s.splits = (int)((chunks + s.chunks_per_split - 1) / s.chunks_per_split);
     s.scratch_bytes = align_up((size_t)s.splits * ((size_t)T * Co * Ci + Co) * sizeof(float), kWsAlign);
+    s.total_chunks = chunks;
+    s.stash_bytes = s.elem_bytes == 2 ? align_up((size_t)s.nCiTiles * chunks * ((size_t)T * s.CiT * 32), kWsAlign) : 0;
     return s;
 }
 

@@ -57,6 +57,11 @@ struct ResParams {
     int w_slots, n_tw;           // weight-ring slots, transform warps (= raw ring slots)
     int x_slots;                 // x^ chunk buffers: nK (a whole token tile resident) or, with one channel tile, a ring of 3
     int64_t num_units;           // token tiles x nCT
+    // optional: also write the spectrum of the input in the operand layout of the weight-gradient kernel
+    // (umma_bwd_weight_saved.cu): blob (input-channel tile, 16-token chunk), T planes of MN-major [CiT x 16] tiles
+    uint8_t* stash;              // nullptr: off
+    int st_CiT, st_nCiTiles;     // the weight gradient's input-channel tiling
+    int64_t st_chunks;           // 16-token chunks in all
 };
 
 // Optional timeline instrumentation (compiled only with -DEQL_TRACE): CTA 0 records clock64() stamps.
@@ -308,7 +313,7 @@ umma_linear_res_kernel(const __grid_constant__ CUtensorMap tmap_in, const ResPar
         uint32_t my_items = 0;                                   // items this warp has taken from its ring slot
         // Chunks [c_lo, c_hi) of the tile only: with a ring of x^ buffers the first XR chunks are transformed before the
         // previous unit's epilogue and the rest after it, while the MMAs of the tile consume them.
-        auto transform_tile = [&](uint32_t tc, int c_lo, int c_hi) {
+        auto transform_tile = [&](uint32_t tc, int c_lo, int c_hi, int64_t tile_row0) {
             if (cw >= n_tw || c_lo >= c_hi) return;
             const uint32_t base = tc * (uint32_t)items_per_tile;
             const int lo = c_lo * IPC, hi = c_hi * IPC;
@@ -334,6 +339,20 @@ umma_linear_res_kernel(const __grid_constant__ CUtensorMap tmap_in, const ResPar
                 const int s = i / PARTS, h = i % PARTS;
                 const int kc = s / SPK, q = s % SPK;
                 const int r = h * 32 + lane;                     // token row inside the tile
+                if (prm.stash != nullptr) {
+                    // the same planes, for the weight gradient of this batch (rows past N and channels past C_in are
+                    // zero here, as the TMA load filled them, and are written as such)
+                    const int c0 = s * NCH;                      // first channel of this raw row's run
+                    const int64_t n = tile_row0 + r;
+                    if (c0 < prm.st_nCiTiles * prm.st_CiT && n < prm.st_chunks * 16) {
+                        const int cit = c0 / prm.st_CiT, mn0 = c0 - cit * prm.st_CiT;
+                        const int k = (int)(n & 15);
+                        uint8_t* g = prm.stash + ((size_t)cit * prm.st_chunks + (size_t)(n >> 4)) * ((size_t)T * prm.st_CiT * 32) +
+                                     (mn0 >> 3) * 256 + (k >> 3) * 128 + (k & 7) * 16;
+#pragma unroll
+                        for (int p = 0; p < T; ++p) store_plane_run<2 * W>(g + (size_t)p * prm.st_CiT * 32, packed[p], 256);
+                    }
+                }
                 // buffer of this chunk (running number qn); the MMAs that read the buffer's previous contents must have retired
                 const uint32_t qn = tc * (uint32_t)nK + (uint32_t)kc;
                 const int xsl = (int)(qn % (uint32_t)XR);
@@ -370,7 +389,7 @@ umma_linear_res_kernel(const __grid_constant__ CUtensorMap tmap_in, const ResPar
 
         uint32_t tc = 0, cu = 0;
         const int pre = XR < nK ? XR : nK;                       // chunks of a tile that fit before its MMAs start freeing buffers
-        if (u0 < u1) transform_tile(0, 0, pre);
+        if (u0 < u1) transform_tile(0, 0, pre, tt0 * NTOK);
         int ct = ct0;
         int64_t tt = tt0;
         for (int64_t u = u0; u < u1 && ok; ++u, ++cu, ++ct) {
@@ -378,13 +397,13 @@ umma_linear_res_kernel(const __grid_constant__ CUtensorMap tmap_in, const ResPar
             if (cw == 0 && lane == 0) RES_STAMP(8 * cu);
             // ring of x^ buffers (one channel tile): the rest of this tile's chunks, consumed by its MMAs as they arrive
             if (first_of_tile(u, ct)) {
-                transform_tile(tc, pre, nK);
+                transform_tile(tc, pre, nK, tt * NTOK);
                 if (!ok) break;
             }
             // the next token tile is transformed while the MMAs of this tile's last channel tile are in flight
             if (last_of_tile(u, ct) && u + 1 < u1) {
                 ++tc;
-                transform_tile(tc, 0, pre);
+                transform_tile(tc, 0, pre, (tt + 1) * NTOK);
                 if (!ok) break;
             }
             if (cw == 0 && lane == 0) RES_STAMP(8 * cu + 1);
@@ -537,7 +556,8 @@ cudaError_t launch_build_umma_res_image(const UmmaResShape& s, const float* plan
 }
 
 cudaError_t launch_umma_linear_res(const UmmaResShape& s, const void* in, void* out, int64_t N, const void* image,
-                                   const float* bias_f32, int* status, int num_sms, cudaStream_t stream) {
+                                   const float* bias_f32, int* status, int num_sms, cudaStream_t stream,
+                                   const UmmaBwdWeightShape* stash_shape, void* stash) {
     if (!s.fits) return cudaErrorInvalidConfiguration;
     EncodeTiledFn enc = encode_tiled_res_fn();
     if (enc == nullptr) return cudaErrorNotSupported;
@@ -557,6 +577,10 @@ cudaError_t launch_umma_linear_res(const UmmaResShape& s, const void* in, void* 
     prm.N = N; prm.Cin = s.Cin; prm.Cout = s.Cout; prm.nCT = s.nCT; prm.nK = s.nK;
     prm.w_slots = s.w_slots; prm.n_tw = s.n_tw; prm.x_slots = s.x_slots;
     prm.num_units = ((N + s.nTok - 1) / s.nTok) * s.nCT;
+    if (stash != nullptr && stash_shape != nullptr) {
+        prm.stash = (uint8_t*)stash;
+        prm.st_CiT = stash_shape->CiT; prm.st_nCiTiles = stash_shape->nCiTiles; prm.st_chunks = stash_shape->total_chunks;
+    }
     const int grid = (int)(prm.num_units < num_sms ? prm.num_units : num_sms);
     const size_t smem = res_smem_bytes(s.T, s.nTok, s.paired, s.x_slots, s.w_slots, s.n_tw);
 

@@ -90,6 +90,72 @@ def test_resident_and_streaming_kernels_agree_with_oracle(T, Ci, Co, N, ids):
             assert v <= TOL["fp16"], f"T={T} Ci={Ci} Co={Co} N={N} flags={flags}: {k} error {v:.3e}"
 
 
+# ------------------------------------------------------------------ training with a saved spectrum
+@pytest.mark.parametrize("T,Ci,Co,N", [(8, 96, 384, 1000), (8, 96, 384, 12000), (8, 10, 24, 77), (4, 24, 96, 1111),
+                                         (4, 256, 256, 700), (8, 384, 96, 640), (16, 17, 33, 333), (32, 32, 32, 500)])
+def test_saved_spectrum_path_matches_oracle(T, Ci, Co, N):
+    """eqlinear_fwd_save_spectrum + eqlinear_bwd_weight_from_spectrum: the forward result and the weight gradient
+    computed from the saved spectrum of x meet the same bars as the plain calls.  The shapes cover the forward kernel
+    that writes the spectrum itself (resident and ring mode), the pre-pass fallback behind the streaming kernel,
+    token counts that are not multiples of the 16-token chunk, and channel counts that are not multiples of a tile."""
+    wl = Workload("spec", "fp16", T, Ci, Co, N, "normal", ("fwd", "bwd_weight"), 23)
+    d = generate(wl)
+    layer = GpuLayer(T, Ci, Co, "fp16", d["w"], d["bias"])
+    try:
+        x = torch.from_numpy(d["x"]).cuda()
+        dy = torch.from_numpy(d["dy"]).cuda()
+        sb = eq.eqlinear_spectrum_bytes(layer.plan, N)
+        spec = torch.full((sb + 64,), 0x7F, dtype=torch.uint8, device="cuda")       # NaN pattern: nothing stale may be read
+        y = torch.empty(N, Co * T, dtype=torch.float16, device="cuda")
+        eq.eqlinear_fwd_save_spectrum(layer.plan, x, y, N, spec, sb, layer.stream)
+        scb = eq.eqlinear_bwd_weight_scratch_bytes(layer.plan, N)
+        sc = torch.empty(scb, dtype=torch.uint8, device="cuda")
+        outs = []
+        for _ in range(2):                                                          # twice: bit-identical results
+            dw = torch.full((Co, Ci, T), float("nan"), dtype=torch.float32, device="cuda")
+            db = torch.full((Co,), float("nan"), dtype=torch.float32, device="cuda")
+            eq.eqlinear_bwd_weight_from_spectrum(layer.plan, spec, sb, dy, dw, db, N, sc, scb, layer.stream)
+            torch.cuda.synchronize()
+            outs.append((dw.cpu().numpy(), db.cpu().numpy()))
+        assert layer.raw_status() == 0
+        assert bool((spec[sb:] == 0x7F).all().item()), "the spectrum write went past its buffer"
+        assert rel_max_err(y.cpu().numpy(), orc.fwd(d["x"], d["w"], d["bias"])) <= TOL["fp16"]
+        rdw, rdb = orc.bwd_weight(d["x"], d["dy"], T)
+        assert rel_max_err(outs[0][0], rdw) <= TOL["fp16"]
+        assert rel_max_err(outs[0][1], rdb) <= TOL["fp16"]
+        assert np.array_equal(outs[0][0], outs[1][0]) and np.array_equal(outs[0][1], outs[1][1])
+    finally:
+        layer.close()
+
+
+def test_saved_spectrum_argument_errors():
+    d = generate(Workload("spec", "fp32", 8, 16, 16, 64, "normal", ("fwd",), 24))
+    layer = GpuLayer(8, 16, 16, "fp32", d["w"], d["bias"])
+    try:
+        with pytest.raises(eq.EqlError) as e:                                        # FP32 plans have no such path
+            eq.eqlinear_spectrum_bytes(layer.plan, 64)
+        assert e.value.status == eq.binding.EQL_ERR_UNSUPPORTED
+    finally:
+        layer.close()
+    d = generate(Workload("spec", "fp16", 8, 16, 16, 64, "normal", ("fwd",), 24))
+    layer = GpuLayer(8, 16, 16, "fp16", d["w"], d["bias"])
+    try:
+        x = torch.from_numpy(d["x"]).cuda()
+        y = torch.empty(64, 128, dtype=torch.float16, device="cuda")
+        sb = eq.eqlinear_spectrum_bytes(layer.plan, 64)
+        spec = torch.empty(sb, dtype=torch.uint8, device="cuda")
+        with pytest.raises(eq.EqlError) as e:                                        # buffer too small
+            eq.eqlinear_fwd_save_spectrum(layer.plan, x, y, 64, spec, sb - 1, layer.stream)
+        assert e.value.status == eq.binding.EQL_ERR_WORKSPACE
+        eq.eqlinear_fwd_save_spectrum(layer.plan, x, y, 0, None, 0, layer.stream)   # N = 0: no-op
+        dw = torch.full((16, 16, 8), 1.0, dtype=torch.float32, device="cuda")
+        eq.eqlinear_bwd_weight_from_spectrum(layer.plan, None, 0, None, dw, None, 0, None, 0, layer.stream)
+        torch.cuda.synchronize()
+        assert float(dw.abs().max().item()) == 0.0                                   # N = 0: gradients are zero
+    finally:
+        layer.close()
+
+
 @pytest.mark.parametrize("dtype", ["fp32", "fp16"])
 def test_paper_parity_shape(dtype):
     """The shape of the paper's numerical-equivalence table (Table 4): (B, N, c, T) = (32, 1024, 64, 4)."""
