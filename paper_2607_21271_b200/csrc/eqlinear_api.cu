@@ -230,9 +230,10 @@ eql_status_t eqlinear_plan(eqlinear_plan_t* plan, int T, int C_in, int C_out, eq
     p->num_sms = kNumSMs;
     if (cudaDeviceGetAttribute(&p->num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) { delete p; return EQL_ERR_CUDA; }
     if (umma_linear_supported(T, dtype) && !(flags & EQL_FLAG_FORCE_SIMT)) {
-        // 3xTF32 accumulates ~1.3e-8 of relative error per reduced channel (measured); beyond 512 channels the FP32
-        // bar of 1e-5 is no longer safe and the FFMA kernel is used instead.
-        const int max_red = dtype == EQL_FP32 ? 512 : (1 << 30);
+        // 3xTF32 accumulates 1.4e-8 ... 1.6e-8 of relative error per reduced channel (measured: the tensor core adds
+        // into its FP32 accumulator with truncation); beyond 256 channels (4e-6) the margin to the FP32 bar of 1e-5
+        // gets thin and the FFMA kernel is used instead.
+        const int max_red = dtype == EQL_FP32 ? 256 : (1 << 30);
         p->fwd_kernel = C_in <= max_red ? 1 : 0;
         p->bwd_data_kernel = C_out <= max_red ? 1 : 0;
         p->umma_fwd = umma_linear_shape(T, C_in, C_out, dtype);

@@ -486,6 +486,8 @@ bool umma_bwd_weight_supported(int T, eql_dtype_t dtype) {
     return T == 4 || T == 8;            // FP32 (3xTF32): larger T leaves too few channels per tile
 }
 
+constexpr int64_t kMaxChunksPerSplitFp32 = 12;
+
 UmmaBwdWeightShape umma_bwd_weight_shape(int T, int Ci, int Co, eql_dtype_t dtype, int64_t N, int num_sms) {
     UmmaBwdWeightShape s{};
     s.T = T; s.Ci = Ci; s.Co = Co;
@@ -510,6 +512,16 @@ UmmaBwdWeightShape umma_bwd_weight_shape(int T, int Ci, int Co, eql_dtype_t dtyp
     const int64_t chunks = N > 0 ? (N + kChunkTok - 1) / kChunkTok : 1;
     int64_t want = num_sms / tiles;
     if (want < 1) want = 1;
+    // FP32 plans: the tensor core adds into its FP32 accumulator with truncation, so the error of a partial sum grows
+    // linearly with the number of accumulation steps (measured: ~2.7e-7 of the largest |dw| per 16-token chunk,
+    // independent of the layer shape).  Short token ranges per accumulator keep it well inside the 1e-5 bar; the
+    // partial sums are then added with round-to-nearest by the finalize kernel.
+    if (dtype == EQL_FP32 && want * kMaxChunksPerSplitFp32 < chunks) {
+        const int64_t need = (chunks + kMaxChunksPerSplitFp32 - 1) / kMaxChunksPerSplitFp32;
+        const int64_t waves = (need * tiles + num_sms - 1) / num_sms;          // whole waves of CTAs
+        want = waves * num_sms / tiles;
+        if (want < need) want = need;
+    }
     if (want > chunks) want = chunks;
     s.chunks_per_split = (chunks + want - 1) / want;
     s.splits = (int)((chunks + s.chunks_per_split - 1) / s.chunks_per_split);
