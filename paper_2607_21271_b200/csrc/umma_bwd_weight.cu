@@ -486,7 +486,7 @@ bool umma_bwd_weight_supported(int T, eql_dtype_t dtype) {
     return T == 4 || T == 8;            // FP32 (3xTF32): larger T leaves too few channels per tile
 }
 
-constexpr int64_t kMaxChunksPerSplitFp32 = 12;
+constexpr int64_t kMaxChunksPerSplitFp32 = 12, kMaxChunksPerSplitFp16 = 2048;
 
 UmmaBwdWeightShape umma_bwd_weight_shape(int T, int Ci, int Co, eql_dtype_t dtype, int64_t N, int num_sms) {
     UmmaBwdWeightShape s{};
@@ -516,8 +516,10 @@ UmmaBwdWeightShape umma_bwd_weight_shape(int T, int Ci, int Co, eql_dtype_t dtyp
     // linearly with the number of accumulation steps (measured: ~2.7e-7 of the largest |dw| per 16-token chunk,
     // independent of the layer shape).  Short token ranges per accumulator keep it well inside the 1e-5 bar; the
     // partial sums are then added with round-to-nearest by the finalize kernel.
-    if (dtype == EQL_FP32 && want * kMaxChunksPerSplitFp32 < chunks) {
-        const int64_t need = (chunks + kMaxChunksPerSplitFp32 - 1) / kMaxChunksPerSplitFp32;
+    // (FP16 plans: the same effect against the 3e-3 bar only matters beyond ~10^4 chunks per accumulator.)
+    const int64_t cap = dtype == EQL_FP32 ? kMaxChunksPerSplitFp32 : kMaxChunksPerSplitFp16;
+    if (want * cap < chunks) {
+        const int64_t need = (chunks + cap - 1) / cap;
         const int64_t waves = (need * tiles + num_sms - 1) / num_sms;          // whole waves of CTAs
         want = waves * num_sms / tiles;
         if (want < need) want = need;
