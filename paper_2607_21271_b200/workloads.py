@@ -58,6 +58,18 @@ CONFIGS = {
 # The configuration the headline metric is quoted on.
 HEADLINE = "vit_b_fc1_fp16"
 
+# The shapes of the paper's operator-level benchmark (Tables 1 and 2): batch 32 x 1024 tokens, the p4 group (T = 4),
+# c channels per group element on both sides (total width C = D = 4c), bias, forward and full backward.  The wide
+# ones are the compute-bound end of the path.  Too large for a full oracle pass: tests compare sampled outputs.
+OPERATOR_SHAPES = {
+    **{f"op_c{c}_fp16": Workload(f"op_c{c}_fp16", "fp16", 4, c, c, 32 * 1024, "normal", _FB, 5)
+       for c in (16, 64, 256, 512, 1024, 2048)},
+    **{f"op_c{c}_fp32": Workload(f"op_c{c}_fp32", "fp32", 4, c, c, 32 * 1024, "normal", _FB, 5)
+       for c in (16, 64, 256)},
+}
+
+ALL_WORKLOADS = {**CONFIGS, **OPERATOR_SHAPES}
+
 
 def generate(wl: Workload) -> dict:
     """Draw x, w, bias, dy for a workload, in this fixed order, from PCG64(seed).

@@ -10,7 +10,7 @@ import torch
 
 import paper_2607_21271_b200 as eq
 from oracle import eqlinear_oracle as orc
-from paper_2607_21271_b200.workloads import CONFIGS, Workload, generate
+from paper_2607_21271_b200.workloads import CONFIGS, OPERATOR_SHAPES, Workload, generate, sample_rows
 from tests.harness import TOL, GpuLayer, check_workload, rel_max_err
 
 pytestmark = pytest.mark.gpu
@@ -74,6 +74,38 @@ def test_fp32_long_reductions_stay_inside_the_bar(T, Ci, Co, N):
     wl = Workload("fp32long", "fp32", T, Ci, Co, N, "none", ("fwd", "bwd_data", "bwd_weight"), 31)
     for k, v in check_workload(wl).items():
         assert v <= 0.6 * TOL["fp32"], f"T={T} Ci={Ci} Co={Co} N={N}: {k} error {v:.3e}"
+
+
+# ------------------------------------------------------------------ the paper's operator-benchmark shapes (Tables 1-2)
+@pytest.mark.parametrize("name", ["op_c64_fp16", "op_c256_fp16", "op_c1024_fp16", "op_c64_fp32", "op_c256_fp32"])
+def test_operator_benchmark_shapes_on_sampled_outputs(name):
+    """32 x 1024 tokens, T = 4, c channels per group element on both sides: the GPU runs the full size; the oracle
+    computes a sample of it one piece at a time - sampled token rows x sampled output channels of y (the dense weight
+    of those channels only), sampled rows x sampled input channels of dx, and dw for sampled channel pairs over ALL
+    tokens (dw[o, i, :] depends only on channel i of x and channel o of dy)."""
+    wl = OPERATOR_SHAPES[name]
+    d = generate(wl)
+    T, c, N = wl.T, wl.Ci, wl.N
+    rows = sample_rows(N, 96, seed=1)
+    g = np.random.Generator(np.random.PCG64(77))
+    ch = np.unique(np.concatenate([[0, c - 1], g.choice(c, size=min(c, 10) - 2, replace=False)]))
+    cols = (ch[:, None] * T + np.arange(T)[None, :]).reshape(-1)
+    layer = GpuLayer(T, c, c, wl.dtype, d["w"], d["bias"])
+    try:
+        y = layer.fwd(d["x"])
+        dx = layer.bwd_data(d["dy"])
+        dw, db = layer.bwd_weight(d["x"], d["dy"])
+        assert layer.raw_status() == 0
+    finally:
+        layer.close()
+    tol = TOL[wl.dtype]
+    ry = orc.fwd(d["x"][rows], d["w"][ch], d["bias"][ch])                    # [rows, sampled output channels x T]
+    assert rel_max_err(y[rows][:, cols], ry) <= tol
+    rdx = orc.bwd_data(d["dy"][rows], d["w"][:, ch])                         # [rows, sampled input channels x T]
+    assert rel_max_err(dx[rows][:, cols], rdx) <= tol
+    rdw, rdb = orc.bwd_weight(d["x"][:, cols], d["dy"][:, cols], T)          # [sampled o, sampled i, T], all tokens
+    assert rel_max_err(dw[np.ix_(ch, ch)], rdw) <= tol
+    assert rel_max_err(db[ch], rdb) <= tol
 
 
 # ------------------------------------------------------------------ the two tensor-core kernels of fwd / bwd_data
