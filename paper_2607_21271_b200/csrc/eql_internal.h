@@ -62,14 +62,24 @@ struct UmmaLinearShape {
     int nK;             // chunks of the reduction dimension (16 channels for half, 8 for float)
     int rowsB;          // (2T-2)*CoT rows of the weight image per (tile, chunk)
     size_t image_bytes;
+    // A shape may describe one SEGMENT of a layer's reduction: input channels [cin0, cin0 + Cin) of CinTotal.
+    int cin0, CinTotal;
 };
 bool umma_linear_supported(int T, eql_dtype_t dtype);
 UmmaLinearShape umma_linear_shape(int T, int Cin, int Cout, eql_dtype_t dtype);
+// FP32 plans reduce at most kFp32SegmentChannels channels in one TMEM accumulator (the tensor core adds with
+// truncation, so the error is linear in the accumulation depth); longer reductions run as several launches whose
+// results are added in global memory with round-to-nearest (TMA reduce-add).  Returns the number of segments and
+// their length (a multiple of 16); segment k covers channels [k * len, min(Cin, (k + 1) * len)).
+constexpr int kFp32SegmentChannels = 256;
+int umma_reduction_segments(int Cin, eql_dtype_t dtype, int* seg_len);
+UmmaLinearShape umma_linear_segment(int T, int Cin, int Cout, eql_dtype_t dtype, int k, int seg_len);
+size_t umma_linear_image_bytes(int T, int Cin, int Cout, eql_dtype_t dtype);       // all segments
 // planes[T][Cin][Cout] (float) -> operand image for umma_linear_kernel.
 cudaError_t launch_build_umma_image(const UmmaLinearShape& s, const float* planes, void* image, cudaStream_t stream);
 // out[N, Cout*T] = IDFT( DFT(in[N, Cin*T]) (x) image ) + bias, fp16 I/O, tcgen05 MMA with FP32 accumulation in TMEM.
 cudaError_t launch_umma_linear(const UmmaLinearShape& s, const void* in, void* out, int64_t N, const void* image,
-                               const float* bias_f32, int* status, int num_sms, cudaStream_t stream);
+                               const float* bias_f32, int* status, int num_sms, cudaStream_t stream, bool accumulate = false);
 
 // ---- tcgen05 kernel with resident transformed activations (FP16, T = 4 or 8), umma_linear_res.cu -----
 struct UmmaResShape {

@@ -18,8 +18,8 @@ WorkspaceLayout workspace_layout(int T, int Ci, int Co, eql_dtype_t dtype) {
     l.umma_fwd = off;    l.umma_fwd_bytes = 0;
     l.umma_bwd = off;    l.umma_bwd_bytes = 0;
     if (umma_linear_supported(T, dtype)) {
-        l.umma_fwd_bytes = umma_linear_shape(T, Ci, Co, dtype).image_bytes;
-        l.umma_bwd_bytes = umma_linear_shape(T, Co, Ci, dtype).image_bytes;
+        l.umma_fwd_bytes = umma_linear_image_bytes(T, Ci, Co, dtype);
+        l.umma_bwd_bytes = umma_linear_image_bytes(T, Co, Ci, dtype);
         if (umma_res_supported(T, dtype)) {          // one region serves whichever tensor-core kernel the plan selects
             const size_t rf = umma_res_shape(T, Ci, Co).image_bytes, rb = umma_res_shape(T, Co, Ci).image_bytes;
             if (rf > l.umma_fwd_bytes) l.umma_fwd_bytes = rf;
@@ -62,12 +62,25 @@ eql_status_t build_weights(eqlinear_plan_t p, const void* w, const void* bias, c
                                         (float*)(p->ws + p->lay.planes_fwd), (float*)(p->ws + p->lay.planes_bwd),
                                         (float*)(p->ws + p->lay.bias), s);
     if (e != cudaSuccess) return EQL_ERR_CUDA;
+    // streaming kernel: one operand image per segment of the reduction (one segment except for wide FP32 layers)
+    auto build_segments = [&](int Cin, int Cout, size_t planes_off, size_t image_off) -> cudaError_t {
+        int len = 0;
+        const int nseg = umma_reduction_segments(Cin, p->dtype, &len);
+        size_t off = 0;
+        for (int k = 0; k < nseg; ++k) {
+            const UmmaLinearShape sh = umma_linear_segment(p->T, Cin, Cout, p->dtype, k, len);
+            cudaError_t err = launch_build_umma_image(sh, (const float*)(p->ws + planes_off), p->ws + image_off + off, s);
+            if (err != cudaSuccess) return err;
+            off += sh.image_bytes;
+        }
+        return cudaSuccess;
+    };
     if (p->fwd_kernel == 1) {
-        e = launch_build_umma_image(p->umma_fwd, (const float*)(p->ws + p->lay.planes_fwd), p->ws + p->lay.umma_fwd, s);
+        e = build_segments(p->Ci, p->Co, p->lay.planes_fwd, p->lay.umma_fwd);
         if (e != cudaSuccess) return EQL_ERR_CUDA;
     }
     if (p->bwd_data_kernel == 1) {
-        e = launch_build_umma_image(p->umma_bwd, (const float*)(p->ws + p->lay.planes_bwd), p->ws + p->lay.umma_bwd, s);
+        e = build_segments(p->Co, p->Ci, p->lay.planes_bwd, p->lay.umma_bwd);
         if (e != cudaSuccess) return EQL_ERR_CUDA;
     }
     if (p->fwd_kernel == 2) {
@@ -79,6 +92,23 @@ eql_status_t build_weights(eqlinear_plan_t p, const void* w, const void* bias, c
         if (e != cudaSuccess) return EQL_ERR_CUDA;
     }
     return EQL_OK;
+}
+
+// Streaming tensor-core kernel over every segment of the reduction: the first launch writes out = bias + its share,
+// the others add theirs (one launch in all except for FP32 layers with more than 256 reduced channels).
+cudaError_t run_streaming(eqlinear_plan_t p, int Cin, int Cout, const void* in, void* out, int64_t N, size_t image_off,
+                          const float* bias, cudaStream_t s) {
+    int len = 0;
+    const int nseg = umma_reduction_segments(Cin, p->dtype, &len);
+    size_t off = 0;
+    for (int k = 0; k < nseg; ++k) {
+        const UmmaLinearShape sh = umma_linear_segment(p->T, Cin, Cout, p->dtype, k, len);
+        cudaError_t e = launch_umma_linear(sh, in, out, N, p->ws + image_off + off, k == 0 ? bias : nullptr,
+                                           (int*)(p->ws + p->lay.status), p->num_sms, s, k > 0);
+        if (e != cudaSuccess) return e;
+        off += sh.image_bytes;
+    }
+    return cudaSuccess;
 }
 
 void destroy_pipe(HostPipe* hp) {
@@ -231,11 +261,10 @@ eql_status_t eqlinear_plan(eqlinear_plan_t* plan, int T, int C_in, int C_out, eq
     if (cudaDeviceGetAttribute(&p->num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) { delete p; return EQL_ERR_CUDA; }
     if (umma_linear_supported(T, dtype) && !(flags & EQL_FLAG_FORCE_SIMT)) {
         // 3xTF32 accumulates 1.4e-8 ... 1.6e-8 of relative error per reduced channel (measured: the tensor core adds
-        // into its FP32 accumulator with truncation); beyond 256 channels (4e-6) the margin to the FP32 bar of 1e-5
-        // gets thin and the FFMA kernel is used instead.
-        const int max_red = dtype == EQL_FP32 ? 256 : (1 << 30);
-        p->fwd_kernel = C_in <= max_red ? 1 : 0;
-        p->bwd_data_kernel = C_out <= max_red ? 1 : 0;
+        // into its FP32 accumulator with truncation); FP32 plans therefore reduce at most 256 channels (4e-6) per
+        // accumulator and run longer reductions as segments that are added in global memory (run_streaming below).
+        p->fwd_kernel = 1;
+        p->bwd_data_kernel = 1;
         p->umma_fwd = umma_linear_shape(T, C_in, C_out, dtype);
         p->umma_bwd = umma_linear_shape(T, C_out, C_in, dtype);
         if (umma_bwd_weight_supported(T, dtype)) p->bwd_weight_kernel = 1;
@@ -313,8 +342,7 @@ eql_status_t eqlinear_fwd(eqlinear_plan_t plan, const void* x, void* y, int64_t 
         return e == cudaSuccess ? EQL_OK : EQL_ERR_CUDA;
     }
     if (plan->fwd_kernel == 1) {
-        cudaError_t e = launch_umma_linear(plan->umma_fwd, x, y, N, plan->ws + plan->lay.umma_fwd, bias,
-                                           (int*)(plan->ws + plan->lay.status), plan->num_sms, (cudaStream_t)stream);
+        cudaError_t e = run_streaming(plan, plan->Ci, plan->Co, x, y, N, plan->lay.umma_fwd, bias, (cudaStream_t)stream);
         return e == cudaSuccess ? EQL_OK : EQL_ERR_CUDA;
     }
     cudaError_t e = launch_direct_linear(plan->T, plan->dtype, x, y, N, plan->Ci, plan->Co,
@@ -335,8 +363,7 @@ eql_status_t eqlinear_bwd_data(eqlinear_plan_t plan, const void* dy, void* dx, i
         return e == cudaSuccess ? EQL_OK : EQL_ERR_CUDA;
     }
     if (plan->bwd_data_kernel == 1) {
-        cudaError_t e = launch_umma_linear(plan->umma_bwd, dy, dx, N, plan->ws + plan->lay.umma_bwd, nullptr,
-                                           (int*)(plan->ws + plan->lay.status), plan->num_sms, (cudaStream_t)stream);
+        cudaError_t e = run_streaming(plan, plan->Co, plan->Ci, dy, dx, N, plan->lay.umma_bwd, nullptr, (cudaStream_t)stream);
         return e == cudaSuccess ? EQL_OK : EQL_ERR_CUDA;
     }
     cudaError_t e = launch_direct_linear(plan->T, plan->dtype, dy, dx, N, plan->Co, plan->Ci,

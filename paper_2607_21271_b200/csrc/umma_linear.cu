@@ -67,6 +67,7 @@ struct UmmaParams {
     int CoT, nTiles, nK, rowsB;
     int b_slot_bytes;            // bytes of one B ring slot (rowsB*32, twice that for FP32, rounded up to 128)
     int64_t num_units;
+    int accumulate;              // out += result (TMA reduce-add) instead of out = result: later segments of a reduction
 };
 
 // Optional timeline instrumentation (compiled only with -DEQL_TRACE): CTA 0 records clock64() stamps.
@@ -98,7 +99,7 @@ struct SmemBarriers {
 //   [rowsB - CoT, rowsB)             plane T-1 (k = T/2)
 template <int T, typename IO>
 __global__ void build_image_kernel(const float* __restrict__ planes, int Cin, int Cout, int CoT, int nTiles, int nK,
-                                   int rowsB, IO* __restrict__ image) {
+                                   int rowsB, IO* __restrict__ image, int cin0, int CinTotal) {
     constexpr int E = sizeof(IO), KCH = kRowBytes / E, EPC = 16 / E, NSPLIT = E == 4 ? 2 : 1;
     const int64_t per_blob = (int64_t)NSPLIT * rowsB * KCH;
     const int64_t total = (int64_t)nTiles * nK * per_blob;
@@ -129,7 +130,7 @@ __global__ void build_image_kernel(const float* __restrict__ planes, int Cin, in
         }
         const int cin = kc * KCH + kk, cout = tile * CoT + local;
         float v = 0.f;
-        if (cin < Cin && cout < Cout) v = sign * planes[((size_t)plane * Cin + cin) * Cout + cout];
+        if (cin < Cin && cout < Cout) v = sign * planes[((size_t)plane * CinTotal + cin0 + cin) * Cout + cout];
         if constexpr (E == 2) {
             image[idx] = __float2half_rn(v);
         } else {
@@ -496,7 +497,8 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
                 ptx::fence_proxy_async_smem();
                 __syncwarp();
                 if (lane == 0 && co0 < prm.Cout) {
-                    ptx::tma_store_2d(&tmap_out, co0 * T, (int)((u / nTiles) * kTileM) + quad * 32, staging);
+                    if (prm.accumulate) ptx::tma_reduce_add_2d(&tmap_out, co0 * T, (int)((u / nTiles) * kTileM) + quad * 32, staging);
+                    else ptx::tma_store_2d(&tmap_out, co0 * T, (int)((u / nTiles) * kTileM) + quad * 32, staging);
                     ptx::bulk_commit_group();
                 }
             }
@@ -611,7 +613,31 @@ UmmaLinearShape umma_linear_shape(int T, int Cin, int Cout, eql_dtype_t dtype) {
     s.nK = (Cin + kch - 1) / kch;
     s.rowsB = (2 * T - 2) * s.CoT;
     s.image_bytes = align_up((size_t)s.nTiles * s.nK * s.rowsB * kRowBytes * (s.elem_bytes == 4 ? 2 : 1), kWsAlign);
+    s.cin0 = 0; s.CinTotal = Cin;
     return s;
+}
+
+int umma_reduction_segments(int Cin, eql_dtype_t dtype, int* seg_len) {
+    if (dtype != EQL_FP32 || Cin <= kFp32SegmentChannels) { *seg_len = Cin; return 1; }
+    const int want = (Cin + kFp32SegmentChannels - 1) / kFp32SegmentChannels;
+    const int len = ((Cin + want - 1) / want + 15) / 16 * 16;
+    *seg_len = len;
+    return (Cin + len - 1) / len;
+}
+
+UmmaLinearShape umma_linear_segment(int T, int Cin, int Cout, eql_dtype_t dtype, int k, int seg_len) {
+    const int c0 = k * seg_len;
+    UmmaLinearShape s = umma_linear_shape(T, Cin - c0 < seg_len ? Cin - c0 : seg_len, Cout, dtype);
+    s.cin0 = c0; s.CinTotal = Cin;
+    return s;
+}
+
+size_t umma_linear_image_bytes(int T, int Cin, int Cout, eql_dtype_t dtype) {
+    int len = 0;
+    const int n = umma_reduction_segments(Cin, dtype, &len);
+    size_t total = 0;
+    for (int k = 0; k < n; ++k) total += umma_linear_segment(T, Cin, Cout, dtype, k, len).image_bytes;
+    return total;
 }
 
 cudaError_t launch_build_umma_image(const UmmaLinearShape& s, const float* planes, void* image, cudaStream_t stream) {
@@ -621,13 +647,14 @@ cudaError_t launch_build_umma_image(const UmmaLinearShape& s, const float* plane
         const int64_t total = (int64_t)(s.image_bytes / sizeof(IO));
         const int blocks = (int)((total + 255) / 256 < 4096 ? (total + 255) / 256 : 4096);
         build_image_kernel<TT, IO><<<blocks, 256, 0, stream>>>(planes, s.Cin, s.Cout, s.CoT, s.nTiles, s.nK, s.rowsB,
-                                                                (IO*)image);
+                                                                (IO*)image, s.cin0, s.CinTotal);
         return cudaGetLastError();
     });
 }
 
 cudaError_t launch_umma_linear(const UmmaLinearShape& s, const void* in, void* out, int64_t N, const void* image,
-                               const float* bias_f32, int* status, int num_sms, cudaStream_t stream) {
+                               const float* bias_f32, int* status, int num_sms, cudaStream_t stream, bool accumulate) {
+    if (accumulate && s.elem_bytes != 4) return cudaErrorInvalidValue;       // the reduce-add path exists for float outputs
     EncodeTiledFn enc = encode_tiled_fn();
     if (enc == nullptr) return cudaErrorNotSupported;
     const CUtensorMapDataType dt = s.elem_bytes == 4 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16;
@@ -635,10 +662,12 @@ cudaError_t launch_umma_linear(const UmmaLinearShape& s, const void* in, void* o
     CUtensorMap tmap, tmap_out;
     const cuuint32_t estr[2] = {1, 1};
     {
+        // a segment of the reduction sees only its own columns of the rows (the rest reads as zero fill)
         const cuuint64_t gdim[2] = {(cuuint64_t)s.Cin * s.T, (cuuint64_t)N};
-        const cuuint64_t gstr[1] = {(cuuint64_t)s.Cin * s.T * s.elem_bytes};
+        const cuuint64_t gstr[1] = {(cuuint64_t)s.CinTotal * s.T * s.elem_bytes};
         const cuuint32_t box[2] = {epr, (cuuint32_t)kTileM};
-        if (enc(&tmap, dt, 2, const_cast<void*>(in), gdim, gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+        const char* in_seg = (const char*)in + (size_t)s.cin0 * s.T * s.elem_bytes;
+        if (enc(&tmap, dt, 2, const_cast<char*>(in_seg), gdim, gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                 CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return cudaErrorInvalidValue;
     }
@@ -656,6 +685,7 @@ cudaError_t launch_umma_linear(const UmmaLinearShape& s, const void* in, void* o
     prm.CoT = s.CoT; prm.nTiles = s.nTiles; prm.nK = s.nK; prm.rowsB = s.rowsB;
     prm.b_slot_bytes = (int)align_up((size_t)s.rowsB * kRowBytes * (s.elem_bytes == 4 ? 2 : 1), 128);
     prm.num_units = ((N + kTileM - 1) / kTileM) * s.nTiles;
+    prm.accumulate = accumulate ? 1 : 0;
     const int grid = (int)(prm.num_units < num_sms ? prm.num_units : num_sms);
 
     return dispatch_umma(s.T, s.elem_bytes, [&](auto tc, auto io) {

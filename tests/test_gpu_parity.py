@@ -65,12 +65,14 @@ def test_shapes(dtype, T, Ci, Co):
         assert v <= TOL[dtype], f"T={T} Ci={Ci} Co={Co} {dtype}: {k} error {v:.3e}"
 
 
-@pytest.mark.parametrize("T,Ci,Co,N", [(8, 162, 254, 9473), (8, 297, 219, 4099), (4, 300, 280, 6000), (8, 380, 40, 2049)])
+@pytest.mark.parametrize("T,Ci,Co,N", [(8, 162, 254, 9473), (8, 297, 219, 4099), (4, 300, 280, 6000), (8, 380, 40, 2049),
+                                         (4, 512, 520, 1500), (4, 1040, 72, 700)])
 def test_fp32_long_reductions_stay_inside_the_bar(T, Ci, Co, N):
     """FP32 plans on the tensor cores: the accumulator adds with truncation, so the error grows with the number of
     accumulation steps.  Layers with many channel tiles leave few CTAs per tile, i.e. long token ranges per
-    accumulator (weight gradient), and wide layers have long channel reductions (forward, data gradient); both must
-    stay inside the FP32 bar (these shapes measured 1.8e-5 ... 3.8e-5 on dw before the token range was bounded)."""
+    accumulator (weight gradient), and wide layers have long channel reductions (forward, data gradient: run as
+    segments of at most 256 channels whose results are added in global memory); both must stay inside the FP32 bar
+    (these shapes measured 1.8e-5 ... 3.8e-5 on dw before the token range was bounded)."""
     wl = Workload("fp32long", "fp32", T, Ci, Co, N, "none", ("fwd", "bwd_data", "bwd_weight"), 31)
     for k, v in check_workload(wl).items():
         assert v <= 0.6 * TOL["fp32"], f"T={T} Ci={Ci} Co={Co} N={N}: {k} error {v:.3e}"
