@@ -309,7 +309,7 @@ direct_bwd_weight_kernel(const IO* __restrict__ x, const IO* __restrict__ dy, in
 template <int T>
 __global__ void __launch_bounds__(32 * T)
 bwd_weight_finalize_kernel(const float* __restrict__ part, const float* __restrict__ db_part, int splits, int Ci,
-                           int Co, bool correlation, float* __restrict__ dw, float* __restrict__ db) {
+                           int Co, bool correlation, float* __restrict__ dw, float* __restrict__ db, bool accumulate) {
     __shared__ float planes[T][33];
     const int pair = threadIdx.x & 31, p = threadIdx.x >> 5;
     const int idx = blockIdx.x * 32 + pair;
@@ -320,7 +320,7 @@ bwd_weight_finalize_kernel(const float* __restrict__ part, const float* __restri
         if (o < Co && db != nullptr) {
             float s = 0.f;
             for (int sp = 0; sp < splits; ++sp) s += db_part[(size_t)sp * Co + o];
-            db[o] = s;
+            db[o] = accumulate ? db[o] + s : s;                  // later token blocks add to the earlier ones
         }
     }
     float acc = 0.f;
@@ -352,7 +352,7 @@ bwd_weight_finalize_kernel(const float* __restrict__ part, const float* __restri
         for (int q = 0; q < T; ++q) v[q] = planes[q][pair];
         rdft_inverse<T>(v);
 #pragma unroll
-        for (int r = 0; r < T; ++r) dw[(size_t)idx * T + r] = v[r];
+        for (int r = 0; r < T; ++r) dw[(size_t)idx * T + r] = accumulate ? dw[(size_t)idx * T + r] + v[r] : v[r];
     }
 }
 
@@ -435,13 +435,13 @@ BwdWeightSplit direct_bwd_weight_split(int T, int Ci, int Co, int64_t N) {
 }
 
 cudaError_t launch_bwd_weight_finalize(int T, bool correlation, const float* scratch, int splits, int Ci, int Co,
-                                       float* dw, float* db, cudaStream_t stream) {
+                                       float* dw, float* db, cudaStream_t stream, bool accumulate) {
     const float* part = scratch;
     const float* db_part = scratch + (size_t)splits * T * Co * Ci;
     return dispatch_T(T, [&](auto tc) {
         constexpr int TT = decltype(tc)::value;
         bwd_weight_finalize_kernel<TT><<<finalize_blocks(TT, Ci, Co), 32 * TT, 0, stream>>>(part, db_part, splits, Ci, Co,
-                                                                                             correlation, dw, db);
+                                                                                             correlation, dw, db, accumulate);
         return cudaGetLastError();
     });
 }
@@ -465,7 +465,7 @@ cudaError_t launch_direct_bwd_weight(int T, eql_dtype_t dtype, bool correlation,
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return e;
         bwd_weight_finalize_kernel<TT><<<finalize_blocks(TT, Ci, Co), 32 * TT, 0, stream>>>(
-            part, db_part, split.splits, Ci, Co, correlation, dw, db);
+            part, db_part, split.splits, Ci, Co, correlation, dw, db, false);
         return cudaGetLastError();
     });
 }

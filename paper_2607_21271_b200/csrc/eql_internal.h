@@ -114,6 +114,10 @@ struct UmmaBwdWeightShape {
     size_t scratch_bytes;       // splits * (T*Co*Ci + Co) floats
     int64_t total_chunks;       // 16-token chunks in all
     size_t stash_bytes;         // FP16: saved spectrum of x as operand image, nCiTiles * total_chunks * T*CiT*32 bytes (else 0)
+    // FP32: tokens one launch covers (a multiple of 16, or N itself).  The fields above then describe a launch over
+    // min(N, block_tokens) tokens; the caller runs the blocks one after the other and the finalize kernel adds each
+    // block's result to dw / db.
+    int64_t block_tokens;
 };
 bool umma_bwd_weight_supported(int T, eql_dtype_t dtype);
 UmmaBwdWeightShape umma_bwd_weight_shape(int T, int Ci, int Co, eql_dtype_t dtype, int64_t N, int num_sms);
@@ -127,7 +131,7 @@ cudaError_t launch_umma_bwd_weight_saved(const UmmaBwdWeightShape& s, const void
                                          float* scratch, int* status, cudaStream_t stream);
 // Phase 2 (direct_kernels.cu): fixed-order sum over splits, 1/T, inverse DFT -> dw, db.
 cudaError_t launch_bwd_weight_finalize(int T, bool correlation, const float* scratch, int splits, int Ci, int Co,
-                                       float* dw, float* db, cudaStream_t stream);
+                                       float* dw, float* db, cudaStream_t stream, bool accumulate = false);
 
 }  // namespace eql
 

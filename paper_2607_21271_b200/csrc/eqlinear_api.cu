@@ -401,11 +401,24 @@ eql_status_t eqlinear_bwd_weight(eqlinear_plan_t plan, const void* x, const void
     if (plan->bwd_weight_kernel == 1) {
         UmmaBwdWeightShape bs = umma_bwd_weight_shape(plan->T, plan->Ci, plan->Co, plan->dtype, N, plan->num_sms);
         if (scratch_bytes < bs.scratch_bytes) return EQL_ERR_WORKSPACE;
-        cudaError_t e = launch_umma_bwd_weight(bs, x, dy, N, (float*)scratch, (int*)(plan->ws + plan->lay.status), s);
-        if (e != cudaSuccess) return EQL_ERR_CUDA;
-        e = launch_bwd_weight_finalize(plan->T, (plan->flags & EQL_FLAG_CORRELATION) != 0, (const float*)scratch, bs.splits,
-                                       plan->Ci, plan->Co, (float*)dw, (float*)db, s);
-        return e == cudaSuccess ? EQL_OK : EQL_ERR_CUDA;
+        // One launch, except for FP32 plans with long token ranges per accumulator: those run in blocks of tokens,
+        // one after the other through the same scratch, and the finalize kernel adds each block's result to dw / db.
+        const size_t xrow = (size_t)plan->Ci * plan->T * elem_size(plan->dtype);
+        const size_t yrow = (size_t)plan->Co * plan->T * elem_size(plan->dtype);
+        const int64_t block = bs.block_tokens;
+        for (int64_t n0 = 0; n0 < N; n0 += block) {
+            const int64_t nb = N - n0 < block ? N - n0 : block;
+            if (nb != block || n0 > 0)
+                bs = umma_bwd_weight_shape(plan->T, plan->Ci, plan->Co, plan->dtype, nb, plan->num_sms);
+            if (scratch_bytes < bs.scratch_bytes) return EQL_ERR_WORKSPACE;
+            cudaError_t e = launch_umma_bwd_weight(bs, (const char*)x + n0 * xrow, (const char*)dy + n0 * yrow, nb,
+                                                   (float*)scratch, (int*)(plan->ws + plan->lay.status), s);
+            if (e != cudaSuccess) return EQL_ERR_CUDA;
+            e = launch_bwd_weight_finalize(plan->T, (plan->flags & EQL_FLAG_CORRELATION) != 0, (const float*)scratch,
+                                           bs.splits, plan->Ci, plan->Co, (float*)dw, (float*)db, s, n0 > 0);
+            if (e != cudaSuccess) return EQL_ERR_CUDA;
+        }
+        return EQL_OK;
     }
     BwdWeightSplit split = direct_bwd_weight_split(plan->T, plan->Ci, plan->Co, N);
     if (scratch_bytes < split.scratch_bytes) return EQL_ERR_WORKSPACE;

@@ -487,6 +487,7 @@ bool umma_bwd_weight_supported(int T, eql_dtype_t dtype) {
 }
 
 constexpr int64_t kMaxChunksPerSplitFp32 = 12, kMaxChunksPerSplitFp16 = 2048;
+constexpr size_t kBlockScratchBudget = 30u << 20;          // FP32 token blocks: partial sums of one launch (below the 32 MiB built-in scratch)
 
 UmmaBwdWeightShape umma_bwd_weight_shape(int T, int Ci, int Co, eql_dtype_t dtype, int64_t N, int num_sms) {
     UmmaBwdWeightShape s{};
@@ -512,21 +513,45 @@ UmmaBwdWeightShape umma_bwd_weight_shape(int T, int Ci, int Co, eql_dtype_t dtyp
     const int64_t chunks = N > 0 ? (N + kChunkTok - 1) / kChunkTok : 1;
     int64_t want = num_sms / tiles;
     if (want < 1) want = 1;
-    // FP32 plans: the tensor core adds into its FP32 accumulator with truncation, so the error of a partial sum grows
-    // linearly with the number of accumulation steps (measured: ~2.7e-7 of the largest |dw| per 16-token chunk,
-    // independent of the layer shape).  Short token ranges per accumulator keep it well inside the 1e-5 bar; the
-    // partial sums are then added with round-to-nearest by the finalize kernel.
-    // (FP16 plans: the same effect against the 3e-3 bar only matters beyond ~10^4 chunks per accumulator.)
+    s.block_tokens = N > 0 ? N : 1;
+    // The tensor core adds into its FP32 accumulator with truncation, so the error of a partial sum grows linearly
+    // with the number of accumulation steps (measured: ~2.7e-7 of the largest |dw| per 16-token chunk, independent
+    // of the layer shape).  A CTA therefore accumulates a bounded token range; the partial sums are added with
+    // round-to-nearest by the finalize kernel.
     const int64_t cap = dtype == EQL_FP32 ? kMaxChunksPerSplitFp32 : kMaxChunksPerSplitFp16;
+    int64_t launch_chunks = chunks;                              // chunks covered by one launch
     if (want * cap < chunks) {
-        const int64_t need = (chunks + cap - 1) / cap;
-        const int64_t waves = (need * tiles + num_sms - 1) / num_sms;          // whole waves of CTAs
-        want = waves * num_sms / tiles;
-        if (want < need) want = need;
+        if (dtype == EQL_FP32) {
+            // FP32 (12 chunks per accumulator): a launch of a few whole waves of CTAs covers a block of tokens, and the
+            // blocks run one after the other into the same scratch, which stays within the built-in scratch array
+            const size_t partial = ((size_t)T * Ci * Co + Co) * sizeof(float);
+            int64_t waves = (int64_t)(kBlockScratchBudget / ((size_t)want * partial));
+            if (waves < 1) waves = 1;
+            if (waves > 8) waves = 8;
+            const int64_t max_splits = want * waves;             // the same for every N: no block needs more scratch than the first
+            const int64_t block = max_splits * cap;
+            if (block < chunks) {
+                launch_chunks = block;
+                s.block_tokens = block * kChunkTok;
+                want = max_splits;
+            } else {
+                const int64_t need = (chunks + cap - 1) / cap;
+                const int64_t w = (need * tiles + num_sms - 1) / num_sms;      // whole waves of CTAs
+                want = w * num_sms / tiles;
+                if (want < need) want = need;
+                if (want > max_splits) want = max_splits;
+            }
+        } else {
+            // FP16 (the same effect against the 3e-3 bar only matters beyond ~10^4 chunks per accumulator): more splits
+            const int64_t need = (chunks + cap - 1) / cap;
+            const int64_t w = (need * tiles + num_sms - 1) / num_sms;
+            want = w * num_sms / tiles;
+            if (want < need) want = need;
+        }
     }
-    if (want > chunks) want = chunks;
-    s.chunks_per_split = (chunks + want - 1) / want;
-    s.splits = (int)((chunks + s.chunks_per_split - 1) / s.chunks_per_split);
+    if (want > launch_chunks) want = launch_chunks;
+    s.chunks_per_split = (launch_chunks + want - 1) / want;
+    s.splits = (int)((launch_chunks + s.chunks_per_split - 1) / s.chunks_per_split);
     s.scratch_bytes = align_up((size_t)s.splits * ((size_t)T * Co * Ci + Co) * sizeof(float), kWsAlign);
     s.total_chunks = chunks;
     s.stash_bytes = s.elem_bytes == 2 ? align_up((size_t)s.nCiTiles * chunks * ((size_t)T * s.CiT * 32), kWsAlign) : 0;
