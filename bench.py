@@ -356,23 +356,6 @@ def main():
                                    "tcgen05": bool(kernel_kind[n]),
                                    "traffic": NCU_TRAFFIC_BYTES.get((wl.name, n))} for n in names}}
 
-    # Context for the HBM fraction: the denominator is a copy (half reads, half writes), but on this part a stream of
-    # writes alone is much slower than that (a fill of this workload's output tensor, timed here with the same events),
-    # and the forward pass writes four times what it reads.
-    if rank == 0:
-        yb = sets[0]["y"]
-        for _ in range(3):
-            yb.fill_(0.0)
-        f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        f0.record()
-        for i in range(10):
-            sets[i % n_sets]["y"].fill_(0.0)
-        f1.record()
-        torch.cuda.synchronize(dev)
-        fill_s = f0.elapsed_time(f1) * 1e-3 / 10
-        roofline["write_only_GBps_measured"] = yb.numel() * esz / fill_s / 1e9
-        roofline["fwd_output_fill_us"] = fill_s * 1e6
-
     # end to end through the host-buffer C-ABI call: pinned host buffers, copies inside the timed region
     e2e = None
     if not args.no_e2e:
