@@ -35,10 +35,14 @@
 namespace eql {
 namespace {
 
-constexpr int kThreadsRes = 512;
+
 constexpr int kTmemColsRes = 512;
 constexpr int kResWarpTmaX = 0, kResWarpMma = 1, kResWarpTmaW = 2, kResWarpCompute0 = 4;
-constexpr int kResComputeWarps = 12;
+constexpr int kResComputeWarps = 16;         // at most (barrier array size)
+// Compute warps per kernel: the T = 4 epilogue is short on instruction issue and long on stores, and gains from a
+// fourth warp per TMEM lane quadrant even at 96 registers per thread (Swin layer: 99.7 -> 96.1 us); the T = 8 kernels
+// lose more to the smaller register file than they gain (76 -> 80 us), so they keep three.
+template <int T> struct ResWarps { static constexpr int kCompute = T == 4 ? 16 : 12, kThreads = (4 + kCompute) * 32; };
 constexpr int kItemBytes = 4096;            // raw item: 32 token rows x 128 bytes
 constexpr int kWTileBytes = 4096;           // spectral-weight tile of one plane: [128 channels x 32 B]
 constexpr int kResMaxK = 12;                // resident chunks (barrier array size)
@@ -109,10 +113,12 @@ __global__ void build_image_res_kernel(const float* __restrict__ planes, int Cin
 // instead of three; an MMA costs about the same whatever its width, so this shortens the main loop where the larger
 // x^ buffers fit.
 template <int T, int NTOK, bool PF>
-__global__ void __launch_bounds__(kThreadsRes, 1)
+__global__ void __launch_bounds__(ResWarps<T>::kThreads, 1)
 umma_linear_res_kernel(const __grid_constant__ CUtensorMap tmap_in, const ResParams prm) {
     // NTOK tokens per tile: the accumulator of a unit is T planes x NTOK fp32 TMEM columns.  With T * NTOK = 256 two
     // accumulators alternate, so that the epilogue of a unit overlaps the MMAs of the next one.
+    constexpr int NCW = ResWarps<T>::kCompute;  // compute warps
+    constexpr int kResShares = NCW / 4;         // warps sharing the token column groups of a TMEM lane quadrant
     constexpr int NBUF = 512 / (T * NTOK);
     constexpr int XTILES = PF ? 2 + 3 * (T / 2 - 1) : T;   // plane tiles per chunk
     constexpr int kXChunkBytes = XTILES * NTOK * 32;       // x^ of one 16-channel chunk: tiles of [NTOK tokens x 32 B]
@@ -142,7 +148,7 @@ umma_linear_res_kernel(const __grid_constant__ CUtensorMap tmap_in, const ResPar
         for (int i = 0; i < kResComputeWarps; ++i) { ptx::mbar_init(&bar->full_raw[i], 1); ptx::mbar_init(&bar->empty_raw[i], 1); }
         for (int i = 0; i < kResMaxK; ++i) { ptx::mbar_init(&bar->full_x[i], IPC); ptx::mbar_init(&bar->empty_x[i], 1); }
         for (int i = 0; i < kResMaxWSlots; ++i) { ptx::mbar_init(&bar->full_w[i], 1); ptx::mbar_init(&bar->empty_w[i], 1); }
-        for (int i = 0; i < 2; ++i) { ptx::mbar_init(&bar->full_d[i], 1); ptx::mbar_init(&bar->empty_d[i], kResComputeWarps); }
+        for (int i = 0; i < 2; ++i) { ptx::mbar_init(&bar->full_d[i], 1); ptx::mbar_init(&bar->empty_d[i], NCW); }
         ptx::mbar_init(&bar->mma_done, 1);
         bar->abort_flag = 0;
         ptx::fence_mbar_init();
@@ -421,13 +427,13 @@ umma_linear_res_kernel(const __grid_constant__ CUtensorMap tmap_in, const ResPar
             if (cw == 0 && lane == 0) RES_STAMP(8 * cu + 2);
             ptx::tc_fence_after_sync();
             constexpr int NG = NTOK / 8;                         // groups of 8 tokens
-            for (int g = third; g < NG; g += 3) {
+            for (int g = third; g < NG; g += kResShares) {
                 const int n0 = g * 8;
                 uint32_t in[T][8];
 #pragma unroll
                 for (int p = 0; p < T; ++p) ptx::tmem_ld<8>(acc_base + (uint32_t)(p * NTOK + n0), in[p]);
                 ptx::tmem_ld_wait();
-                if (g + 3 >= NG) {                               // this warp's last read of the accumulator
+                if (g + kResShares >= NG) {                      // this warp's last read of the accumulator
                     ptx::tc_fence_before_sync();
                     __syncwarp();
                     if (lane == 0) ptx::mbar_arrive(&bar->empty_d[buf]);
@@ -596,7 +602,7 @@ cudaError_t launch_umma_linear_res(const UmmaResShape& s, const void* in, void* 
             if (e != cudaSuccess) return e;
             attr_done |= 1ull << (dev & 63);
         }
-        umma_linear_res_kernel<TT, NT, PF><<<grid, kThreadsRes, smem, stream>>>(tmap, prm);
+        umma_linear_res_kernel<TT, NT, PF><<<grid, ResWarps<TT>::kThreads, smem, stream>>>(tmap, prm);
         return cudaGetLastError();
     };
     using I4 = std::integral_constant<int, 4>;
