@@ -155,7 +155,7 @@ def run_reference(args, wl):
 
     d = generate(wl)
     total_budget = 150.0                                   # seconds for warm-up + timed steps
-    per_step = max(0.5, min(15.0, total_budget / max(1, args.steps + args.warmup)))
+    per_step = max(0.1, min(15.0, total_budget / max(1, args.steps + args.warmup)))   # 1000 steps still end in ~3 min
     rows = pick_sample_rows(orc, wl, d, per_step)
     for _ in range(args.warmup):
         oracle_step(orc, wl, d, rows)
