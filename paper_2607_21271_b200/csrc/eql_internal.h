@@ -118,6 +118,8 @@ struct UmmaBwdWeightShape {
     // min(N, block_tokens) tokens; the caller runs the blocks one after the other and the finalize kernel adds each
     // block's result to dw / db.
     int64_t block_tokens;
+    int raw_slots;              // 48 KB raw slots in shared memory (2, or 1 beside a large FP32 stage)
+    int y_slab0;                // first slab of dy inside a raw slot: 16 (fixed layout) or nXs (packed layout)
 };
 bool umma_bwd_weight_supported(int T, eql_dtype_t dtype);
 UmmaBwdWeightShape umma_bwd_weight_shape(int T, int Ci, int Co, eql_dtype_t dtype, int64_t N, int num_sms);

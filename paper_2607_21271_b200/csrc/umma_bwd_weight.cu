@@ -48,6 +48,8 @@ struct BwParams {
     int xhat_bytes, stage_bytes;
     int x_part_bytes, y_part_bytes;   // FP32: bytes of the TF32 "hi" copy of x^ / dy^ inside a stage; the "lo" copy follows it
     int stages;                  // operand stages (2; 1 where the hi/lo copies of FP32 leave no room for two)
+    int raw_slots;               // raw slots of 48 KB (2; 1 where a large FP32 stage leaves room for one only)
+    int y_slab0;                 // first slab of dy inside a raw slot (kMaxXSlabs, or nXs in the packed layout)
     int x3d, y3d;                // tensor maps are 3-D (64 elements, rows, slab index): one load per chunk and tensor
     int part_tma;                // the partial spectra can be written with TMA tensor stores (row pitch a multiple of 16 bytes)
 };
@@ -86,8 +88,8 @@ umma_bwd_weight_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw_base) + 1023) & ~(uintptr_t)1023);
     BwBarriers* bar = reinterpret_cast<BwBarriers*>(smem);
     uint8_t* raw = smem + 1024;                                  // kRawSlots x 48 KB
-    uint8_t* stages = raw + kRawSlots * kRawSlot;                // prm.stages x stage_bytes (+ 8 KB slack after the last)
-    const int NST = prm.stages;
+    uint8_t* stages = raw + prm.raw_slots * kRawSlot;            // prm.stages x stage_bytes (+ 8 KB slack after the last)
+    const int NST = prm.stages, NRAW = prm.raw_slots;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     volatile int* abort_flag = &bar->abort_flag;
@@ -130,8 +132,8 @@ umma_bwd_weight_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
             int64_t c = 0;
             const uint32_t bytes = (uint32_t)(prm.nXs + prm.nYs) * kSlab;
             for (; c < nchunks; ++c) {
-                const int slot = (int)(c % kRawSlots);
-                ok = ptx::mbar_wait(&bar->empty_raw[slot], (uint32_t)((c / kRawSlots) & 1) ^ 1, abort_flag, status, 201);
+                const int slot = NRAW == 2 ? (int)(c & 1) : 0;
+                ok = ptx::mbar_wait(&bar->empty_raw[slot], (uint32_t)((NRAW == 2 ? (c >> 1) : c) & 1) ^ 1, abort_flag, status, 201);
                 if (!ok) break;
                 BW_STAMP(3000 + (int)c);
                 ptx::mbar_arrive_expect_tx(&bar->full_raw[slot], bytes);
@@ -146,17 +148,17 @@ umma_bwd_weight_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
                         ptx::tma_load_2d(dst + s * kSlab, &tmap_x, ci_tile * CiT * T + s * EPR, row, &bar->full_raw[slot]);
                 }
                 if (prm.y3d) {
-                    ptx::tma_load_3d(dst + kMaxXSlabs * kSlab, &tmap_dy, 0, row, co_tile * CoT * T / EPR, &bar->full_raw[slot]);
+                    ptx::tma_load_3d(dst + prm.y_slab0 * kSlab, &tmap_dy, 0, row, co_tile * CoT * T / EPR, &bar->full_raw[slot]);
                 } else {
                     for (int s = 0; s < prm.nYs; ++s)
-                        ptx::tma_load_2d(dst + (kMaxXSlabs + s) * kSlab, &tmap_dy, co_tile * CoT * T + s * EPR, row,
+                        ptx::tma_load_2d(dst + (prm.y_slab0 + s) * kSlab, &tmap_dy, co_tile * CoT * T + s * EPR, row,
                                          &bar->full_raw[slot]);
                 }
             }
             if (!ok) {
-                const int64_t lo = c > kRawSlots ? c - kRawSlots : 0;
+                const int64_t lo = c > NRAW ? c - NRAW : 0;
                 for (int64_t d = lo; d < c; ++d)
-                    ptx::mbar_wait(&bar->full_raw[d % kRawSlots], (uint32_t)((d / kRawSlots) & 1), abort_flag, status, 211, false);
+                    ptx::mbar_wait(&bar->full_raw[NRAW == 2 ? (d & 1) : 0], (uint32_t)((NRAW == 2 ? (d >> 1) : d) & 1), abort_flag, status, 211, false);
             }
         }
     } else if (warp == kWarpMmaBw) {
@@ -214,8 +216,13 @@ umma_bwd_weight_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
         }
     } else if (warp >= kWarpDftX0) {
         // ------------------------------------------------------------ transform warps
-        const bool is_y = warp >= kWarpDftY0;
-        const int wi = is_y ? warp - kWarpDftY0 : warp - kWarpDftX0;
+        // A half warp takes one slab of a chunk.  Fixed layout: warps 4-11 the (up to 16) slabs of x, warps 12-15 the (up
+        // to 8) slabs of dy.  Packed layout (y_slab0 = nXs, an even number): the slabs of dy follow those of x directly, so
+        // a layer with few input channels can give more half warps - and a wider output tile - to dy.
+        const bool packed_slabs = prm.y_slab0 != kMaxXSlabs;
+        const int hw0 = 2 * (warp - kWarpDftX0);                 // first half warp of this warp
+        const bool is_y = packed_slabs ? hw0 >= prm.nXs : warp >= kWarpDftY0;
+        const int wi = packed_slabs ? (is_y ? (hw0 - prm.nXs) >> 1 : hw0 >> 1) : (is_y ? warp - kWarpDftY0 : warp - kWarpDftX0);
         const int half = lane >> 4, row = lane & 15;
         const int slab = 2 * wi + half;
         const bool active = slab < (is_y ? prm.nYs : prm.nXs);
@@ -224,14 +231,14 @@ umma_bwd_weight_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
         for (int i = 0; i < NCH; ++i) dbacc[i] = 0.f;
         bool ok = true;
         for (int64_t c = 0; c < nchunks; ++c) {
-            const int slot = (int)(c % kRawSlots), st = NST == 2 ? (int)(c & 1) : 0;
+            const int slot = NRAW == 2 ? (int)(c & 1) : 0, st = NST == 2 ? (int)(c & 1) : 0;
             const uint32_t sph = (uint32_t)((NST == 2 ? (c >> 1) : c) & 1);
 #ifdef EQL_TRACE
             const bool tr = lane == 0 && (warp == kWarpDftX0 || warp == kWarpDftY0);
             const int tb = (warp == kWarpDftX0 ? 4000 : 5000) + 6 * (int)c;
             if (tr) BW_STAMP(tb);
 #endif
-            ok = ptx::mbar_wait(&bar->full_raw[slot], (uint32_t)((c / kRawSlots) & 1), abort_flag, status, 203);
+            ok = ptx::mbar_wait(&bar->full_raw[slot], (uint32_t)((NRAW == 2 ? (c >> 1) : c) & 1), abort_flag, status, 203);
 #ifdef EQL_TRACE
             if (tr) BW_STAMP(tb + 1);
 #endif
@@ -242,7 +249,7 @@ umma_bwd_weight_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
             if (!ok) break;
             uint32_t wd[32];
             if (active)
-                load_slab_row(raw + slot * kRawSlot + ((is_y ? kMaxXSlabs : 0) + slab) * kSlab + row * 128, row, wd);
+                load_slab_row(raw + slot * kRawSlot + ((is_y ? prm.y_slab0 : 0) + slab) * kSlab + row * 128, row, wd);
             // The rows are in registers: order these generic-proxy reads before the async-proxy (TMA) refill of
             // the slot, then release it so that the refill overlaps the transform.
             ptx::fence_proxy_async_smem();
@@ -453,7 +460,8 @@ bool encode_slabs3d(EncodeTiledFn enc, CUtensorMap* map, const void* base, int64
 
 // Shared memory outside the operand stages: barriers, alignment, two raw slots, and 8 KB of slack after the last stage
 // (the UMMA reads 128 rows of every plane although only CiT are valid).
-constexpr size_t kBwFixedSmem = 1024 + 1024 + (size_t)kRawSlots * kRawSlot + 8192;
+constexpr size_t bw_fixed_smem(int raw_slots) { return 1024 + 1024 + (size_t)raw_slots * kRawSlot + 8192; }
+constexpr size_t kBwFixedSmem = bw_fixed_smem(kRawSlots);
 
 // Bytes per channel of one operand tile of a 16-token chunk: FP16 MN-major 32; FP32 K-major with padded cores 72.
 int bw_chan_bytes(int elem_bytes) { return elem_bytes == 2 ? kChunkTok * 2 : 72; }
@@ -508,6 +516,28 @@ UmmaBwdWeightShape umma_bwd_weight_shape(int T, int Ci, int Co, eql_dtype_t dtyp
     }
     s.nCiTiles = (Ci + s.CiT - 1) / s.CiT;
     s.nXs = (s.CiT * T + epr - 1) / epr;
+    s.raw_slots = kRawSlots;
+    s.y_slab0 = kMaxXSlabs;
+    // FP32 layers with few input channels: the half warps that x leaves idle can transform dy (packed slab layout), which
+    // allows a wider output-channel tile - fewer tiles means fewer CTAs repeating the transform of x and half as many
+    // chunks per CTA at the same MMA count per chunk.  The larger stage may leave room for one raw slot only.
+    if (dtype == EQL_FP32 && s.nXs % 2 == 0 && s.nXs < kMaxXSlabs + kMaxYSlabs) {
+        int max_cot2 = (kMaxXSlabs + kMaxYSlabs - s.nXs) * epr / T;
+        if (max_cot2 > kTmemColsBw / T) max_cot2 = kTmemColsBw / T;
+        max_cot2 = max_cot2 / 16 * 16;
+        if (max_cot2 >= 16) {
+            const int cot2 = balanced_tile(Co, max_cot2, 16);
+            const int n2 = (Co + cot2 - 1) / cot2;
+            if (cot2 <= max_cot2 && n2 < s.nCoTiles) {
+                for (int rs = kRawSlots; rs >= 1; --rs) {
+                    if (bw_fixed_smem(rs) + bw_stage_bytes(T, s.CiT, cot2, s.elem_bytes) <= 227 * 1024) {
+                        s.CoT = cot2; s.nCoTiles = n2; s.raw_slots = rs; s.y_slab0 = s.nXs;
+                        break;
+                    }
+                }
+            }
+        }
+    }
     s.nYs = (s.CoT * T + epr - 1) / epr;
     const int64_t tiles = (int64_t)s.nCiTiles * s.nCoTiles;
     const int64_t chunks = N > 0 ? (N + kChunkTok - 1) / kChunkTok : 1;
@@ -595,8 +625,9 @@ cudaError_t launch_umma_bwd_weight(const UmmaBwdWeightShape& s, const void* x, c
     prm.y_part_bytes = ytiles * s.CoT * chan_bytes;              // one copy of the dy^ tiles
     prm.xhat_bytes = nsplit * prm.x_part_bytes;
     prm.stage_bytes = (int)bw_stage_bytes(s.T, s.CiT, s.CoT, E);
-    prm.stages = kBwFixedSmem + 2 * (size_t)prm.stage_bytes <= 227 * 1024 ? 2 : 1;
-    const size_t smem = kBwFixedSmem + (size_t)prm.stages * prm.stage_bytes;
+    prm.raw_slots = s.raw_slots; prm.y_slab0 = s.y_slab0;
+    prm.stages = bw_fixed_smem(s.raw_slots) + 2 * (size_t)prm.stage_bytes <= 227 * 1024 ? 2 : 1;
+    const size_t smem = bw_fixed_smem(s.raw_slots) + (size_t)prm.stages * prm.stage_bytes;
     if (smem > 227 * 1024) return cudaErrorInvalidConfiguration;
     const int grid = s.splits * s.nCiTiles * s.nCoTiles;
 
