@@ -1,5 +1,5 @@
 // Thin inline-PTX wrappers for sm_100a: mbarrier, TMA (cp.async.bulk / cp.async.bulk.tensor),
-// tcgen05 (TMEM allocation, MMA, commit, load) and proxy fences.  No multicast forms are used anywhere.
+// tcgen05 (TMEM allocation, MMA, commit, load) and proxy fences.  Every copy targets this CTA's own shared memory only.
 #pragma once
 
 #include <cuda.h>
@@ -86,14 +86,14 @@ __device__ __forceinline__ void tc_fence_after_sync() {
 }
 
 // ---------------------------------------------------------------- TMA
-// 2-D tiled load global -> shared (no multicast); completion counted in bytes on `bar`.
+// 2-D tiled load global -> this CTA's shared memory; completion counted in bytes on `bar`.
 __device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* map, int c0, int c1, uint64_t* bar) {
     asm volatile(
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
         ::"r"(smem_u32(smem_dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(smem_u32(bar))
         : "memory");
 }
-// 3-D tiled load global -> shared (no multicast).
+// 3-D tiled load global -> this CTA's shared memory.
 __device__ __forceinline__ void tma_load_3d(void* smem_dst, const CUtensorMap* map, int c0, int c1, int c2, uint64_t* bar) {
     asm volatile(
         "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
