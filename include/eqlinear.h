@@ -128,6 +128,15 @@ eql_status_t eqlinear_plan_info(eqlinear_plan_t plan, eql_info_t* info);
  * EQL_ERR_DEVICE_TIMEOUT if a bounded wait inside one of the plan's kernels gave up. */
 eql_status_t eqlinear_plan_device_status(eqlinear_plan_t plan, void* stream);
 
+/* Sets the plan's device status word back to "ok" (asynchronous on `stream`), e.g. after a reported time-out. */
+eql_status_t eqlinear_plan_clear_device_status(eqlinear_plan_t plan, void* stream);
+
+/* Self-test of that error path: launches (asynchronously on `stream`) a one-warp kernel whose single bounded wait -
+ * the helper every tensor-core kernel of the library waits with - is never satisfied.  The kernel ends by itself
+ * after its poll budget (tens of milliseconds), nothing faults, and eqlinear_plan_device_status then reports
+ * EQL_ERR_DEVICE_TIMEOUT until the status is cleared; the plan stays usable. */
+eql_status_t eqlinear_plan_selftest_expired_wait(eqlinear_plan_t plan, void* stream);
+
 /* Frees the host object only (the workspace is the caller's). NULL is accepted. */
 eql_status_t eqlinear_plan_destroy(eqlinear_plan_t plan);
 

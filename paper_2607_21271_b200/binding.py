@@ -39,6 +39,7 @@ EXPORTED_SYMBOLS = (
     "eqlinear_fwd", "eqlinear_bwd_data", "eqlinear_bwd_weight_scratch_bytes", "eqlinear_bwd_weight",
     "eqlinear_fwd_host", "eqlinear_bwd_data_host", "eqlinear_bwd_weight_host", "eqlinear_step_host", "eqlinear_bwd_weight_static",
     "eqlinear_spectrum_bytes", "eqlinear_fwd_save_spectrum", "eqlinear_bwd_weight_from_spectrum",
+    "eqlinear_plan_clear_device_status", "eqlinear_plan_selftest_expired_wait",
 )
 
 
@@ -84,6 +85,8 @@ def load_library(path: str | None = None) -> ctypes.CDLL:
         "eqlinear_plan_set_weight": [V, V, V, V],
         "eqlinear_plan_info": [V, POINTER(EqlInfo)],
         "eqlinear_plan_device_status": [V, V],
+        "eqlinear_plan_clear_device_status": [V, V],
+        "eqlinear_plan_selftest_expired_wait": [V, V],
         "eqlinear_plan_destroy": [V],
         "eqlinear_fwd": [V, V, V, I64, V],
         "eqlinear_bwd_data": [V, V, V, I64, V],
@@ -161,6 +164,14 @@ def eqlinear_plan_info(plan) -> EqlInfo:
 
 def eqlinear_plan_device_status(plan, stream=0) -> int:
     return load_library().eqlinear_plan_device_status(plan, stream or None)
+
+
+def eqlinear_plan_clear_device_status(plan, stream=0) -> None:
+    _check(load_library().eqlinear_plan_clear_device_status(plan, stream or None), "eqlinear_plan_clear_device_status")
+
+
+def eqlinear_plan_selftest_expired_wait(plan, stream=0) -> None:
+    _check(load_library().eqlinear_plan_selftest_expired_wait(plan, stream or None), "eqlinear_plan_selftest_expired_wait")
 
 
 def eqlinear_plan_destroy(plan) -> None:

@@ -320,6 +320,30 @@ def test_gpu_equivariance_and_adjoint(dtype, T):
         layer.close()
 
 
+# ------------------------------------------------------------------ the error path of the bounded waits
+def test_expired_wait_is_reported_and_the_plan_stays_usable():
+    """Every wait inside the tensor-core kernels is bounded; when one runs out the kernel ends by itself and leaves a code
+    in the plan's status word.  The self-test kernel waits (with the same helper) on a barrier nothing arrives on: the
+    host must read EQL_ERR_DEVICE_TIMEOUT, nothing may fault, and after clearing the status the plan computes as before."""
+    wl = Workload("err", "fp16", 8, 24, 40, 300, "normal", ("fwd",), 27)
+    d = generate(wl)
+    layer = GpuLayer(wl.T, wl.Ci, wl.Co, wl.dtype, d["w"], d["bias"])
+    try:
+        ref = orc.fwd(d["x"], d["w"], d["bias"])
+        assert rel_max_err(layer.fwd(d["x"]), ref) <= TOL["fp16"]
+        assert eq.eqlinear_plan_device_status(layer.plan, layer.stream) == eq.binding.EQL_OK
+        eq.eqlinear_plan_selftest_expired_wait(layer.plan, layer.stream)
+        assert eq.eqlinear_plan_device_status(layer.plan, layer.stream) == eq.binding.EQL_ERR_DEVICE_TIMEOUT
+        assert layer.raw_status() == 901                                             # the code of the wait that gave up
+        torch.cuda.synchronize()                                                     # no sticky CUDA error
+        eq.eqlinear_plan_clear_device_status(layer.plan, layer.stream)
+        assert eq.eqlinear_plan_device_status(layer.plan, layer.stream) == eq.binding.EQL_OK
+        assert rel_max_err(layer.fwd(d["x"]), ref) <= TOL["fp16"]
+        assert eq.eqlinear_plan_device_status(layer.plan, layer.stream) == eq.binding.EQL_OK
+    finally:
+        layer.close()
+
+
 # ------------------------------------------------------------------ host-buffer variants
 @pytest.mark.parametrize("N", [700, 9001])
 def test_host_buffer_variants(N):
