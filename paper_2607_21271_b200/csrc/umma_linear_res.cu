@@ -112,7 +112,7 @@ __global__ void build_image_res_kernel(const float* __restrict__ planes, int Cin
 // complex frequency takes two MMAs of width 2 NTOK ([Re|Im] += Wr [Xr|Xi] and, with A negated, += (-Wi) [Xi|-Xr])
 // instead of three; an MMA costs about the same whatever its width, so this shortens the main loop where the larger
 // x^ buffers fit.
-template <int T, int NTOK, bool PF>
+template <int T, int NTOK, bool PF, bool MERGED>
 __global__ void __launch_bounds__(ResWarps<T>::kThreads, 1)
 umma_linear_res_kernel(const __grid_constant__ CUtensorMap tmap_in, const ResParams prm) {
     // NTOK tokens per tile: the accumulator of a unit is T planes x NTOK fp32 TMEM columns.  With T * NTOK = 256 two
@@ -146,7 +146,7 @@ umma_linear_res_kernel(const __grid_constant__ CUtensorMap tmap_in, const ResPar
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < kResComputeWarps; ++i) { ptx::mbar_init(&bar->full_raw[i], 1); ptx::mbar_init(&bar->empty_raw[i], 1); }
-        for (int i = 0; i < kResMaxK; ++i) { ptx::mbar_init(&bar->full_x[i], IPC); ptx::mbar_init(&bar->empty_x[i], 1); }
+        for (int i = 0; i < kResMaxK; ++i) { ptx::mbar_init(&bar->full_x[i], IPC + (MERGED ? 1 : 0)); ptx::mbar_init(&bar->empty_x[i], 1); }
         for (int i = 0; i < kResMaxWSlots; ++i) { ptx::mbar_init(&bar->full_w[i], 1); ptx::mbar_init(&bar->empty_w[i], 1); }
         for (int i = 0; i < 2; ++i) { ptx::mbar_init(&bar->full_d[i], 1); ptx::mbar_init(&bar->empty_d[i], NCW); }
         ptx::mbar_init(&bar->mma_done, 1);
@@ -171,7 +171,14 @@ umma_linear_res_kernel(const __grid_constant__ CUtensorMap tmap_in, const ResPar
     const int64_t tt0 = u0 / nCT;
     // With a ring of x^ buffers (fewer buffers than chunks) nothing survives a unit: every unit transforms its token
     // tile itself, i.e. is the first and the last of its tile.
-    const bool ring = XR < nK;
+    const bool ring = MERGED || XR < nK;                         // (MERGED implies ring mode: known at compile time there)
+    // Ring mode with equally deep rings: chunk q uses x^ buffer q % 3 and weight slot q % 3, so one "full" barrier
+    // (transform warps + the weight copy) and one "empty" barrier (one commit) per chunk serve both, which halves the
+    // barrier operations of the MMA-issuing thread.
+    // MERGED is a template parameter so that the other modes keep their exact instruction stream.
+    constexpr bool merged = MERGED;                               // host: ring mode with w_slots == x_slots
+    uint64_t* const full_wb = merged ? bar->full_x : bar->full_w;
+    uint64_t* const empty_wb = merged ? bar->empty_x : bar->empty_w;
     auto first_of_tile = [&](int64_t u, int ct) { return ring || u == u0 || ct == 0; };
     auto last_of_tile = [&](int64_t u, int ct) { return ring || u == u1 - 1 || ct == nCT - 1; };
     const int items_per_tile = IPC * nK;
@@ -214,17 +221,17 @@ umma_linear_res_kernel(const __grid_constant__ CUtensorMap tmap_in, const ResPar
             for (int64_t u = u0; u < u1 && ok; ++u, ++ct) {
                 if (ct == nCT) ct = 0;
                 for (int kc = 0; kc < nK; ++kc, ++cw) {
-                    ok = ptx::mbar_wait(&bar->empty_w[slot], eph, abort_flag, status, 302, true, kResSpin);
+                    ok = ptx::mbar_wait(&empty_wb[slot], eph, abort_flag, status, 302, true, kResSpin);
                     if (!ok) break;
-                    ptx::mbar_arrive_expect_tx(&bar->full_w[slot], kWSlot);
+                    ptx::mbar_arrive_expect_tx(&full_wb[slot], kWSlot);
                     ptx::bulk_load_1d(wsm + slot * kWSlot, prm.image + ((size_t)ct * nK + kc) * (size_t)kWSlot, kWSlot,
-                                      &bar->full_w[slot]);
+                                      &full_wb[slot]);
                     if (++slot == w_slots) { slot = 0; eph ^= 1u; }
                 }
             }
             const uint32_t lo = cw > (uint32_t)w_slots ? cw - w_slots : 0;
             for (uint32_t c = lo; c < cw; ++c)
-                ptx::mbar_wait(&bar->full_w[c % w_slots], (c / w_slots) & 1, abort_flag, status, 312, false);
+                ptx::mbar_wait(&full_wb[c % w_slots], (c / w_slots) & 1, abort_flag, status, 312, false);
         }
     } else if (warp == kResWarpMma) {
         // ---------------------------------------------------------------- tensor-core issue (one thread)
@@ -254,7 +261,7 @@ umma_linear_res_kernel(const __grid_constant__ CUtensorMap tmap_in, const ResPar
                 uint32_t xph = ((tc * (uint32_t)nK) / (uint32_t)XR) & 1u;
                 // operands of the unit's first chunk
                 if (first) ok = ptx::mbar_wait(&bar->full_x[xs], xph, abort_flag, status, 304, true, kResSpin);
-                ok = ok && ptx::mbar_wait(&bar->full_w[slot], wph, abort_flag, status, 305, true, kResSpin);
+                if constexpr (!merged) ok = ok && ptx::mbar_wait(&bar->full_w[slot], wph, abort_flag, status, 305, true, kResSpin);
                 if (!ok) break;
                 for (int kc = 0; kc < nK; ++kc) {
                     RES_STAMP(1024 + 4 * (cu * nK + kc));
@@ -288,12 +295,12 @@ umma_linear_res_kernel(const __grid_constant__ CUtensorMap tmap_in, const ResPar
                             // MMAs queued, so that the issue stream has no gap between chunks.
                             RES_STAMP(1024 + 4 * (cu * nK + kc) + 1);
                             if (first) ok = ptx::mbar_wait(&bar->full_x[nxs], nxph, abort_flag, status, 304, true, kResSpin);
-                            ok = ok && ptx::mbar_wait(&bar->full_w[nslot], nwph, abort_flag, status, 305, true, kResSpin);
+                            if constexpr (!merged) ok = ok && ptx::mbar_wait(&bar->full_w[nslot], nwph, abort_flag, status, 305, true, kResSpin);
                             RES_STAMP(1024 + 4 * (cu * nK + kc) + 2);
                         }
                     }
                     mma(dbase + (uint32_t)((T - 1) * NTOK), a0 + (T - 1) * kWTileBytes, b0 + (XTILES - 1) * XT, idesc1, acc);  // k = T/2
-                    ptx::umma_commit(&bar->empty_w[slot]);
+                    if constexpr (!merged) ptx::umma_commit(&bar->empty_w[slot]);
                     if (last) ptx::umma_commit(&bar->empty_x[xs]);  // the x^ buffer may be overwritten once these MMAs retire
                     RES_STAMP(1024 + 4 * (cu * nK + kc) + 3);
                     slot = nslot; wph = nwph;
@@ -545,7 +552,10 @@ UmmaResShape umma_res_shape(int T, int Cin, int Cout) {
         s.paired = true;
         s.w_slots = 3;
     }
-    if (s.fits && s.w_slots == 3 && res_smem_bytes(T, s.nTok, s.paired, s.x_slots, 4, s.n_tw) <= kResSmemLimit) s.w_slots = 4;
+    // (not in ring mode: equal ring depths let one barrier pair serve the weight slot and the x^ buffer of a chunk)
+    if (s.fits && s.w_slots == 3 && s.x_slots == s.nK &&
+        res_smem_bytes(T, s.nTok, s.paired, s.x_slots, 4, s.n_tw) <= kResSmemLimit)
+        s.w_slots = 4;
     return s;
 }
 
@@ -590,27 +600,33 @@ cudaError_t launch_umma_linear_res(const UmmaResShape& s, const void* in, void* 
     const int grid = (int)(prm.num_units < num_sms ? prm.num_units : num_sms);
     const size_t smem = res_smem_bytes(s.T, s.nTok, s.paired, s.x_slots, s.w_slots, s.n_tw);
 
-    auto go = [&](auto tc, auto nt, auto pf) -> cudaError_t {
+    auto go = [&](auto tc, auto nt, auto pf, auto mg) -> cudaError_t {
         constexpr int TT = decltype(tc)::value, NT = decltype(nt)::value;
-        constexpr bool PF = decltype(pf)::value;
+        constexpr bool PF = decltype(pf)::value, MG = decltype(mg)::value;
         static unsigned long long attr_done = 0;
         int dev = 0;
         cudaGetDevice(&dev);
         if (!((attr_done >> (dev & 63)) & 1ull)) {
-            cudaError_t e = cudaFuncSetAttribute(umma_linear_res_kernel<TT, NT, PF>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+            cudaError_t e = cudaFuncSetAttribute(umma_linear_res_kernel<TT, NT, PF, MG>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                  (int)kResSmemLimit);
             if (e != cudaSuccess) return e;
             attr_done |= 1ull << (dev & 63);
         }
-        umma_linear_res_kernel<TT, NT, PF><<<grid, ResWarps<TT>::kThreads, smem, stream>>>(tmap, prm);
+        umma_linear_res_kernel<TT, NT, PF, MG><<<grid, ResWarps<TT>::kThreads, smem, stream>>>(tmap, prm);
         return cudaGetLastError();
     };
     using I4 = std::integral_constant<int, 4>;
     using I8 = std::integral_constant<int, 8>;
     using I64 = std::integral_constant<int, 64>;
     using I128 = std::integral_constant<int, 128>;
-    if (s.T == 4 && s.nTok == 128) return s.paired ? go(I4{}, I128{}, std::true_type{}) : go(I4{}, I128{}, std::false_type{});
-    if (s.T == 8 && s.nTok == 64) return s.paired ? go(I8{}, I64{}, std::true_type{}) : go(I8{}, I64{}, std::false_type{});
+    const bool merged = s.x_slots < s.nK && s.w_slots == s.x_slots;      // ring mode, equally deep rings: one barrier pair per chunk
+    auto pick = [&](auto tc, auto nt) -> cudaError_t {
+        if (merged)
+            return s.paired ? go(tc, nt, std::true_type{}, std::true_type{}) : go(tc, nt, std::false_type{}, std::true_type{});
+        return s.paired ? go(tc, nt, std::true_type{}, std::false_type{}) : go(tc, nt, std::false_type{}, std::false_type{});
+    };
+    if (s.T == 4 && s.nTok == 128) return pick(I4{}, I128{});
+    if (s.T == 8 && s.nTok == 64) return pick(I8{}, I64{});
     return cudaErrorInvalidValue;
 }
 
