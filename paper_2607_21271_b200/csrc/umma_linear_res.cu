@@ -134,7 +134,9 @@ umma_linear_res_kernel(const __grid_constant__ CUtensorMap tmap_in, const ResPar
 
     extern __shared__ uint8_t smem_raw_base[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw_base) + 1023) & ~(uintptr_t)1023);
-    const int nK = prm.nK, nCT = prm.nCT, n_tw = prm.n_tw, w_slots = prm.w_slots, XR = prm.x_slots;
+    // ring mode: three x^ buffers, three weight slots, twelve transform warps, one channel tile (compile-time there)
+    const int nK = prm.nK, nCT = MERGED ? 1 : prm.nCT, n_tw = MERGED ? 12 : prm.n_tw, w_slots = MERGED ? 3 : prm.w_slots,
+              XR = MERGED ? 3 : prm.x_slots;
     uint8_t* raw = smem;                                         // n_tw items
     uint8_t* xhat = raw + n_tw * kItemBytes;                     // XR chunk buffers
     uint8_t* wsm = xhat + XR * kXChunkBytes;                     // w_slots slots
@@ -171,7 +173,7 @@ umma_linear_res_kernel(const __grid_constant__ CUtensorMap tmap_in, const ResPar
     const int64_t tt0 = u0 / nCT;
     // With a ring of x^ buffers (fewer buffers than chunks) nothing survives a unit: every unit transforms its token
     // tile itself, i.e. is the first and the last of its tile.
-    const bool ring = MERGED || XR < nK;                         // (MERGED implies ring mode: known at compile time there)
+    constexpr bool ring = MERGED;                                // the host runs ring mode with equally deep rings only
     // Ring mode with equally deep rings: chunk q uses x^ buffer q % 3 and weight slot q % 3, so one "full" barrier
     // (transform warps + the weight copy) and one "empty" barrier (one commit) per chunk serve both, which halves the
     // barrier operations of the MMA-issuing thread.
@@ -619,7 +621,9 @@ cudaError_t launch_umma_linear_res(const UmmaResShape& s, const void* in, void* 
     using I8 = std::integral_constant<int, 8>;
     using I64 = std::integral_constant<int, 64>;
     using I128 = std::integral_constant<int, 128>;
-    const bool merged = s.x_slots < s.nK && s.w_slots == s.x_slots;      // ring mode, equally deep rings: one barrier pair per chunk
+    const bool merged = s.x_slots < s.nK;                                // ring mode: one barrier pair per chunk
+    // the ring-mode variant has these folded in at compile time
+    if (merged && !(s.x_slots == 3 && s.w_slots == 3 && s.n_tw == 12 && s.nCT == 1)) return cudaErrorInvalidConfiguration;
     auto pick = [&](auto tc, auto nt) -> cudaError_t {
         if (merged)
             return s.paired ? go(tc, nt, std::true_type{}, std::true_type{}) : go(tc, nt, std::false_type{}, std::true_type{});
