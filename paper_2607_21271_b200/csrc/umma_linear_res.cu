@@ -259,8 +259,9 @@ umma_linear_res_kernel(const __grid_constant__ CUtensorMap tmap_in, const ResPar
                 RES_STAMP(512 + 2 * cu + 1);
                 if (!ok) break;
                 // x^ buffer and phase of the tile's chunk 0: chunk kc of the CTA's tc-th tile has running number tc*nK + kc
-                int xs = (int)((tc * (uint32_t)nK) % (uint32_t)XR);
-                uint32_t xph = ((tc * (uint32_t)nK) / (uint32_t)XR) & 1u;
+                // (resident mode has XR == nK: buffer = chunk index, phase = tile parity, no division)
+                int xs = ring ? (int)((tc * (uint32_t)nK) % (uint32_t)XR) : 0;
+                uint32_t xph = ring ? ((tc * (uint32_t)nK) / (uint32_t)XR) & 1u : tc & 1u;
                 // operands of the unit's first chunk
                 if (first) ok = ptx::mbar_wait(&bar->full_x[xs], xph, abort_flag, status, 304, true, kResSpin);
                 if constexpr (!merged) ok = ok && ptx::mbar_wait(&bar->full_w[slot], wph, abort_flag, status, 305, true, kResSpin);
@@ -370,8 +371,8 @@ umma_linear_res_kernel(const __grid_constant__ CUtensorMap tmap_in, const ResPar
                 }
                 // buffer of this chunk (running number qn); the MMAs that read the buffer's previous contents must have retired
                 const uint32_t qn = tc * (uint32_t)nK + (uint32_t)kc;
-                const int xsl = (int)(qn % (uint32_t)XR);
-                const uint32_t use = qn / (uint32_t)XR;
+                const int xsl = ring ? (int)(qn % (uint32_t)XR) : kc;
+                const uint32_t use = ring ? qn / (uint32_t)XR : tc;
                 if (use > 0) {
                     ok = ptx::mbar_wait(&bar->empty_x[xsl], (use - 1) & 1, abort_flag, status, 307, true, 16);
                     if (!ok) break;
