@@ -109,7 +109,10 @@ __global__ void xhat_image_kernel(const __half* __restrict__ x, int64_t N, int C
     for (int p = 0; p < T; ++p) store_plane_run<NCH>(dst + (size_t)p * CiT * 32, packed[p], 256);
 }
 
-template <int T>
+// MERGED (x^ ring as deep as the dy^ stages, i.e. three): chunk c uses stage c % 3 and ring slot c % 3, so one "full"
+// barrier (the group's transform warps + the x^ copy) and one "empty" barrier (one commit) per chunk serve both, and
+// the MMA-issuing thread - which paces this kernel - handles half as many barrier operations.
+template <int T, bool MERGED>
 __global__ void __launch_bounds__(kThreadsBw, 1)
 umma_bwd_weight_saved_kernel(const __grid_constant__ CUtensorMap tmap_dy, const __grid_constant__ CUtensorMap tmap_part,
                              const BwParams prm) {
@@ -129,7 +132,7 @@ umma_bwd_weight_saved_kernel(const __grid_constant__ CUtensorMap tmap_dy, const 
         for (int i = 0; i < kGroups; ++i) {
             ptx::mbar_init(&bar->full_raw[i], 1);
             ptx::mbar_init(&bar->empty_raw[i], kWarpsPerGroup);
-            ptx::mbar_init(&bar->full_ab[i], kWarpsPerGroup);            // the group's warps have stored dy^
+            ptx::mbar_init(&bar->full_ab[i], kWarpsPerGroup + (MERGED ? 1 : 0));   // the group's warps have stored dy^ (+ the x^ copy)
             ptx::mbar_init(&bar->empty_ab[i], 1);
         }
         for (int i = 0; i < kMaxXSlots; ++i) { ptx::mbar_init(&bar->full_x[i], 1); ptx::mbar_init(&bar->empty_x[i], 1); }
@@ -194,22 +197,24 @@ umma_bwd_weight_saved_kernel(const __grid_constant__ CUtensorMap tmap_dy, const 
             // ---- x^ blob of every chunk -> ring slot (freed when the MMAs that read it have retired)
             bool ok = true;
             int64_t nx = 0;
-            const int XS = prm.x_slots;
+            const int XS = MERGED ? kGroups : prm.x_slots;
+            uint64_t* const full_xb = MERGED ? bar->full_ab : bar->full_x;
+            uint64_t* const empty_xb = MERGED ? bar->empty_ab : bar->empty_x;
             const uint8_t* xsrc = prm.ximage + ((size_t)ci_tile * prm.total_chunks + chunk0) * (size_t)prm.xhat_bytes;
             int slot = 0;
             uint32_t eph = 1;
             for (int64_t c = 0; c < nchunks; ++c, ++nx) {
                 if (c > 0 && ++slot == XS) { slot = 0; eph ^= 1u; }
-                ok = ptx::mbar_wait(&bar->empty_x[slot], eph, abort_flag, status, 206);
+                ok = ptx::mbar_wait(&empty_xb[slot], eph, abort_flag, status, 206);
                 if (!ok) break;
                 BW_STAMP(2000 + (int)c);
-                ptx::mbar_arrive_expect_tx(&bar->full_x[slot], (uint32_t)prm.xhat_bytes);
+                ptx::mbar_arrive_expect_tx(&full_xb[slot], (uint32_t)prm.xhat_bytes);
                 ptx::bulk_load_1d(xring + slot * prm.xhat_bytes, xsrc + (size_t)c * prm.xhat_bytes, (uint32_t)prm.xhat_bytes,
-                                  &bar->full_x[slot]);
+                                  &full_xb[slot]);
             }
             if (!ok)
                 for (int64_t d = nx > XS ? nx - XS : 0; d < nx; ++d)
-                    ptx::mbar_wait(&bar->full_x[d % XS], (uint32_t)((d / XS) & 1), abort_flag, status, 212, false);
+                    ptx::mbar_wait(&full_xb[d % XS], (uint32_t)((d / XS) & 1), abort_flag, status, 212, false);
         }
     } else if (warp == kWarpMmaBw) {
         if (lane == 0) {
@@ -217,12 +222,12 @@ umma_bwd_weight_saved_kernel(const __grid_constant__ CUtensorMap tmap_dy, const 
             const uint32_t idesc_real = ptx::umma_idesc_f16_f32_mn_major(128, CoT);
             const uint32_t idesc_cplx = ptx::umma_idesc_f16_f32_mn_major(128, 2 * CoT);
             const uint32_t a_plane = (uint32_t)CiT * 32u, b_tile = (uint32_t)CoT * 32u;
-            const int XS = prm.x_slots;
+            const int XS = MERGED ? kGroups : prm.x_slots;
             int st = 0, xs = 0;                                  // dy^ stage and x^ ring slot of the current chunk
             uint32_t sph = 0, xph = 0;                           // their phase parities
             if (nchunks > 0)
                 ok = ptx::mbar_wait(&bar->full_ab[0], 0, abort_flag, status, 202) &&
-                     ptx::mbar_wait(&bar->full_x[0], 0, abort_flag, status, 207);
+                     (MERGED || ptx::mbar_wait(&bar->full_x[0], 0, abort_flag, status, 207));
             for (int64_t c = 0; c < nchunks && ok; ++c) {
                 BW_STAMP(1000 + 4 * (int)c);
                 ptx::tc_fence_after_sync();
@@ -233,29 +238,30 @@ umma_bwd_weight_saved_kernel(const __grid_constant__ CUtensorMap tmap_dy, const 
                 uint32_t nsph = sph, nxph = xph;
                 if (nst == kGroups) { nst = 0; nsph ^= 1u; }
                 if (nxs == XS) { nxs = 0; nxph ^= 1u; }
-                // MN-major no-swizzle: lbo = stride between 8-token groups (128 B), sbo = stride between 8-channel groups (256 B)
-                ptx::umma_f16(tmem_base, ptx::umma_smem_desc(a0, 128, 256), ptx::umma_smem_desc(b0, 128, 256), idesc_real, acc);
+                // MN-major no-swizzle: lbo = stride between 8-token groups (128 B), sbo = stride between 8-channel groups (256 B);
+                // the descriptors of the chunk's first tiles are built once and advanced by (byte offset >> 4)
+                const uint64_t ad = ptx::umma_smem_desc(a0, 128, 256), bd = ptx::umma_smem_desc(b0, 128, 256);
+                const uint64_t ap = a_plane >> 4, bt1 = b_tile >> 4;
+                ptx::umma_f16(tmem_base, ad, bd, idesc_real, acc);
 #pragma unroll
                 for (int f = 1; f < T / 2; ++f) {
                     const uint32_t d = tmem_base + (uint32_t)((2 * f - 1) * CoT);
-                    const uint32_t bt = b0 + (uint32_t)(1 + 3 * (f - 1)) * b_tile;          // tiles Gr | Gi | -Gr
-                    ptx::umma_f16(d, ptx::umma_smem_desc(a0 + (2 * f - 1) * a_plane, 128, 256),
-                                  ptx::umma_smem_desc(bt, 128, 256), idesc_cplx, acc);       // Xr^T [Gr | Gi]
-                    ptx::umma_f16(d, ptx::umma_smem_desc(a0 + (2 * f) * a_plane, 128, 256),
-                                  ptx::umma_smem_desc(bt + b_tile, 128, 256), idesc_cplx, 1u);  // Xi^T [Gi | -Gr]
+                    const uint64_t bt = bd + (uint64_t)(1 + 3 * (f - 1)) * bt1;             // tiles Gr | Gi | -Gr
+                    ptx::umma_f16(d, ad + (2 * f - 1) * ap, bt, idesc_cplx, acc);            // Xr^T [Gr | Gi]
+                    ptx::umma_f16(d, ad + (2 * f) * ap, bt + bt1, idesc_cplx, 1u);           // Xi^T [Gi | -Gr]
                     if (f == 1 && c + 1 < nchunks) {
                         // The next chunk's operands are checked here, while the tensor pipe still has this chunk's
                         // MMAs queued, so that the issue stream has no gap between chunks.
                         BW_STAMP(1000 + 4 * (int)c + 1);
                         ok = ptx::mbar_wait(&bar->full_ab[nst], nsph, abort_flag, status, 202) &&
-                             ptx::mbar_wait(&bar->full_x[nxs], nxph, abort_flag, status, 207);
+                             (MERGED || ptx::mbar_wait(&bar->full_x[nxs], nxph, abort_flag, status, 207));
                         BW_STAMP(1000 + 4 * (int)c + 2);
                     }
                 }
-                ptx::umma_f16(tmem_base + (uint32_t)((T - 1) * CoT), ptx::umma_smem_desc(a0 + (T - 1) * a_plane, 128, 256),
-                              ptx::umma_smem_desc(b0 + (uint32_t)(1 + 3 * (T / 2 - 1)) * b_tile, 128, 256), idesc_real, acc);
+                ptx::umma_f16(tmem_base + (uint32_t)((T - 1) * CoT), ad + (T - 1) * ap,
+                              bd + (uint64_t)(1 + 3 * (T / 2 - 1)) * bt1, idesc_real, acc);
                 ptx::umma_commit(&bar->empty_ab[st]);
-                ptx::umma_commit(&bar->empty_x[xs]);
+                if constexpr (!MERGED) ptx::umma_commit(&bar->empty_x[xs]);
                 BW_STAMP(1000 + 4 * (int)c + 3);
                 st = nst; xs = nxs; sph = nsph; xph = nxph;
             }
@@ -515,25 +521,28 @@ cudaError_t launch_umma_bwd_weight_saved(const UmmaBwdWeightShape& s, const void
     const int ytiles = 2 + 3 * (s.T / 2 - 1);
     prm.stage_bytes = (int)align_up((size_t)ytiles * s.CoT * 32, 1024);
     const size_t fixed = 1024 + 2048 + (size_t)kGroups * kRawSlot + (size_t)kGroups * prm.stage_bytes + 4096;
-    prm.x_slots = kMaxXSlots;
+    prm.x_slots = kGroups;                                           // three slots: the merged-barrier variant
     while (prm.x_slots > 2 && fixed + (size_t)prm.x_slots * prm.xhat_bytes > 227 * 1024) --prm.x_slots;
     const size_t smem = fixed + (size_t)prm.x_slots * prm.xhat_bytes;
     if (smem > 227 * 1024) return cudaErrorInvalidConfiguration;
     const int grid = s.splits * s.nCiTiles * s.nCoTiles;
 
-    auto go = [&](auto tc) -> cudaError_t {
+    const bool merged = prm.x_slots == kGroups;
+    auto go2 = [&](auto tc, auto mg) -> cudaError_t {
         constexpr int TT = decltype(tc)::value;
+        constexpr bool MG = decltype(mg)::value;
         static unsigned long long attr_done = 0;
         int dev = 0;
         cudaGetDevice(&dev);
         if (!((attr_done >> (dev & 63)) & 1ull)) {
-            cudaError_t e = cudaFuncSetAttribute(umma_bwd_weight_saved_kernel<TT>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+            cudaError_t e = cudaFuncSetAttribute(umma_bwd_weight_saved_kernel<TT, MG>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
             if (e != cudaSuccess) return e;
             attr_done |= 1ull << (dev & 63);
         }
-        umma_bwd_weight_saved_kernel<TT><<<grid, kThreadsBw, smem, stream>>>(my, mp, prm);
+        umma_bwd_weight_saved_kernel<TT, MG><<<grid, kThreadsBw, smem, stream>>>(my, mp, prm);
         return cudaGetLastError();
     };
+    auto go = [&](auto tc) -> cudaError_t { return merged ? go2(tc, std::true_type{}) : go2(tc, std::false_type{}); };
     switch (s.T) {
         case 4: return go(std::integral_constant<int, 4>{});
         case 8: return go(std::integral_constant<int, 8>{});
