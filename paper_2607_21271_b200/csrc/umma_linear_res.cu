@@ -244,9 +244,12 @@ umma_linear_res_kernel(const __grid_constant__ CUtensorMap tmap_in, const ResPar
             bool ok = true;
             const uint32_t idesc1 = ptx::umma_idesc_f16_f32(128, NTOK);          // one plane of tokens
             const uint32_t idesc2 = ptx::umma_idesc_f16_f32(128, 2 * NTOK);      // [Re | Im] planes of a complex frequency
-            auto mma = [](uint32_t d, uint32_t a_addr, uint32_t b_addr, uint32_t idesc, uint32_t accumulate) {
-                ptx::umma_f16(d, ptx::umma_smem_desc_k_sw32(a_addr), ptx::umma_smem_desc_k_sw32(b_addr), idesc, accumulate);
+            // shared-memory descriptors are built once per chunk and advanced by (byte offset >> 4) in their address field
+            // (the tiles stay inside the 256 KB window, so no carry leaves it)
+            auto mma = [](uint32_t d, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+                ptx::umma_f16(d, a_desc, b_desc, idesc, accumulate);
             };
+            constexpr uint64_t kWTileD = kWTileBytes >> 4, kXTileD = XT >> 4;
             int ct = ct0;
             for (int64_t u = u0; u < u1 && ok; ++u, ++cu, ++ct) {
                 if (ct == nCT) ct = 0;
@@ -269,8 +272,8 @@ umma_linear_res_kernel(const __grid_constant__ CUtensorMap tmap_in, const ResPar
                 for (int kc = 0; kc < nK; ++kc) {
                     RES_STAMP(1024 + 4 * (cu * nK + kc));
                     ptx::tc_fence_after_sync();
-                    const uint32_t a0 = ptx::smem_u32(wsm + slot * kWSlot);      // weight tiles, plane p at p * 4 KB
-                    const uint32_t b0 = ptx::smem_u32(xhat + xs * kXChunkBytes); // x^ tiles, plane p at p * XT
+                    const uint64_t a0 = ptx::umma_smem_desc_k_sw32(ptx::smem_u32(wsm + slot * kWSlot));      // weight tiles, plane p at p * 4 KB
+                    const uint64_t b0 = ptx::umma_smem_desc_k_sw32(ptx::smem_u32(xhat + xs * kXChunkBytes)); // x^ tiles, plane p at p * XT
                     const uint32_t acc = kc > 0 ? 1u : 0u;
                     int nslot = slot + 1;
                     uint32_t nwph = wph;
@@ -282,13 +285,13 @@ umma_linear_res_kernel(const __grid_constant__ CUtensorMap tmap_in, const ResPar
 #pragma unroll
                     for (int f = 1; f < T / 2; ++f) {
                         const uint32_t dre = dbase + (uint32_t)((2 * f - 1) * NTOK), dim = dre + NTOK;
-                        const uint32_t wr = a0 + (2 * f - 1) * kWTileBytes, wi = wr + kWTileBytes;
+                        const uint64_t wr = a0 + (2 * f - 1) * kWTileD, wi = wr + kWTileD;
                         if constexpr (PF) {
-                            const uint32_t xr = b0 + (1 + 3 * (f - 1)) * XT, xi = xr + XT;            // tiles Re | Im | -Re
+                            const uint64_t xr = b0 + (1 + 3 * (f - 1)) * kXTileD, xi = xr + kXTileD;  // tiles Re | Im | -Re
                             mma(dre, wr, xr, idesc2, acc);                                                // [Re|Im] += Wr [Xr|Xi]
                             mma(dre, wi, xi, idesc2 | kIdescNegateA, 1u);                                 // [Re|Im] -= Wi [Xi|-Xr]
                         } else {
-                            const uint32_t xr = b0 + (2 * f - 1) * XT, xi = xr + XT;
+                            const uint64_t xr = b0 + (2 * f - 1) * kXTileD, xi = xr + kXTileD;
                             mma(dre, wr, xr, idesc2, acc);                                                // [Re|Im] += Wr [Xr|Xi]
                             mma(dre, wi, xi, idesc1 | kIdescNegateA, 1u);                                 //  Re     -= Wi Xi
                             mma(dim, wi, xr, idesc1, 1u);                                                 //  Im     += Wi Xr
@@ -302,7 +305,7 @@ umma_linear_res_kernel(const __grid_constant__ CUtensorMap tmap_in, const ResPar
                             RES_STAMP(1024 + 4 * (cu * nK + kc) + 2);
                         }
                     }
-                    mma(dbase + (uint32_t)((T - 1) * NTOK), a0 + (T - 1) * kWTileBytes, b0 + (XTILES - 1) * XT, idesc1, acc);  // k = T/2
+                    mma(dbase + (uint32_t)((T - 1) * NTOK), a0 + (T - 1) * kWTileD, b0 + (XTILES - 1) * kXTileD, idesc1, acc);  // k = T/2
                     if constexpr (!merged) ptx::umma_commit(&bar->empty_w[slot]);
                     if (last) ptx::umma_commit(&bar->empty_x[xs]);  // the x^ buffer may be overwritten once these MMAs retire
                     RES_STAMP(1024 + 4 * (cu * nK + kc) + 3);
