@@ -36,9 +36,9 @@ FALLBACK_BF16_TFLOPS = 1590.0
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per launch from the committed ncu capture
 # profiles/umma_kernels_fp16_vit_b_fc1.md (None = not captured for that workload / kernel).
 NCU_TRAFFIC_BYTES = {
-    ("vit_b_fc1_fp16", "fwd"): 48.5e6 + 144.0e6,          # includes the 38.7 MB spectrum of x saved for the weight gradient
-    ("vit_b_fc1_fp16", "bwd_data"): 156.1e6 + 16.5e6,
-    ("vit_b_fc1_fp16", "bwd_weight"): 193.7e6 + 3.6e6,
+    ("vit_b_fc1_fp16", "fwd"): 48.6e6 + 145.4e6,          # includes the 38.7 MB spectrum of x saved for the weight gradient
+    ("vit_b_fc1_fp16", "bwd_data"): 156.1e6 + 17.3e6,
+    ("vit_b_fc1_fp16", "bwd_weight"): 193.7e6 + 3.7e6,
 }
 
 
