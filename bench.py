@@ -249,8 +249,7 @@ def main():
             s["dy"] = dy0 if i == 0 else dy0.clone()
             s["dx"] = torch.empty(wl.N, wl.Din, dtype=td, device=dev)
         sets.append(s)
-    dw = torch.empty(wl.Co, wl.Ci, wl.T, dtype=torch.float32, device=dev)
-    db = torch.empty(wl.Co, dtype=torch.float32, device=dev)
+    grads, dw, db = parallel.grad_buffers(wl.Co, wl.Ci, wl.T, dev)      # one buffer: one all-reduce at N > 1
     sb = eq.eqlinear_bwd_weight_scratch_bytes(plan, wl.N) if has_bwd else 0
     scratch = torch.empty(max(sb, 256), dtype=torch.uint8, device=dev)
     # Training with a saved spectrum: the forward kernel that transforms x once per token tile also writes x^ for
@@ -285,7 +284,7 @@ def main():
             if events is not None:
                 events[3].record()
             if world > 1:
-                parallel.allreduce_weight_grads(dw, db)
+                parallel.allreduce_weight_grads(dw, db, flat=grads)
 
     def barrier():
         if world > 1:

@@ -45,6 +45,27 @@ def _worker(rank, world, port, out_dir):
     dist.destroy_process_group()
 
 
+def _flat_worker(rank, world, port, out_dir):
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    flat, dw, db = parallel.grad_buffers(5, 6, 4, "cpu")
+    assert dw.shape == (5, 6, 4) and db.shape == (5,) and db.data_ptr() % 16 == 0 and dw.data_ptr() == flat.data_ptr()
+    dw.fill_(rank + 1.0); db.fill_(10.0 * (rank + 1))
+    parallel.allreduce_weight_grads(dw, db, flat=flat)            # one collective for both
+    np.savez(os.path.join(out_dir, f"flat{rank}.npz"), dw=dw.numpy(), db=db.numpy())
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_flat_gradient_buffer_is_reduced_in_one_call(tmp_path):
+    world, port = 2, 31500 + os.getpid() % 2000
+    mp.spawn(_flat_worker, args=(world, port, str(tmp_path)), nprocs=world, join=True)
+    for r in range(world):
+        p = np.load(tmp_path / f"flat{r}.npz")
+        assert np.all(p["dw"] == 3.0) and np.all(p["db"] == 30.0)
+
+
 def test_two_ranks_reproduce_the_single_process_result(tmp_path):
     world, port = 2, 29500 + os.getpid() % 2000
     mp.spawn(_worker, args=(world, port, str(tmp_path)), nprocs=world, join=True)
