@@ -216,7 +216,9 @@ def main():
         raise RuntimeError("bench.py needs a CUDA device: the library has no CPU fallback")
     dev = torch.device(f"cuda:{local_rank}")
     torch.cuda.set_device(dev)
-    if world > 1:
+    # EQL_BENCH_FORCE_DIST: run the N > 1 form of the step in a one-rank group (to exercise it on one GPU)
+    use_dist = world > 1 or bool(os.environ.get("EQL_BENCH_FORCE_DIST"))
+    if use_dist:
         dist.init_process_group("nccl", device_id=dev)
     n_gpus = world
 
@@ -264,6 +266,12 @@ def main():
         for s in sets:
             s["spec"] = torch.empty(spec_bytes, dtype=torch.uint8, device=dev)
 
+    # N > 1: the weight gradient goes first, and its all-reduce is issued from a side stream that waits only for it, so
+    # that the exchange overlaps the data gradient of the same step (the step still ends with the summed dw / db:
+    # the compute stream waits for the collective before the step is over).
+    comm_stream = torch.cuda.Stream(device=dev) if use_dist else None
+    dw_ready = torch.cuda.Event() if use_dist else None
+
     def step(s, events=None):
         if events is not None:
             events[0].record()
@@ -274,17 +282,33 @@ def main():
         if events is not None:
             events[1].record()
         if has_bwd:
-            eq.eqlinear_bwd_data(plan, s["dy"], s["dx"], wl.N, stream)
-            if events is not None:
-                events[2].record()
-            if use_saved:
-                eq.eqlinear_bwd_weight_from_spectrum(plan, s["spec"], spec_bytes, s["dy"], dw, db, wl.N, scratch, sb, stream)
+            def weight_grad():
+                if use_saved:
+                    eq.eqlinear_bwd_weight_from_spectrum(plan, s["spec"], spec_bytes, s["dy"], dw, db, wl.N, scratch, sb, stream)
+                else:
+                    eq.eqlinear_bwd_weight(plan, s["x"], s["dy"], dw, db, wl.N, scratch, sb, stream)
+
+            work = None
+            if use_dist:
+                weight_grad()
+                dw_ready.record()
+                with torch.cuda.stream(comm_stream):
+                    comm_stream.wait_event(dw_ready)
+                    work = parallel.allreduce_weight_grads(dw, db, flat=grads, async_op=True)
+                if events is not None:
+                    events[2].record()
+                eq.eqlinear_bwd_data(plan, s["dy"], s["dx"], wl.N, stream)
+                if events is not None:
+                    events[3].record()
+                if work is not None:
+                    work.wait()                                # the compute stream waits for the collective
             else:
-                eq.eqlinear_bwd_weight(plan, s["x"], s["dy"], dw, db, wl.N, scratch, sb, stream)
-            if events is not None:
-                events[3].record()
-            if world > 1:
-                parallel.allreduce_weight_grads(dw, db, flat=grads)
+                eq.eqlinear_bwd_data(plan, s["dy"], s["dx"], wl.N, stream)
+                if events is not None:
+                    events[2].record()
+                weight_grad()
+                if events is not None:
+                    events[3].record()
 
     def barrier():
         if world > 1:
@@ -324,7 +348,7 @@ def main():
     value = wl.N * n_gpus / (ms_per_step * 1e-3)
 
     # per-kernel times (mean over the timed steps), from the events recorded inside the timed region
-    names = ["fwd", "bwd_data", "bwd_weight"] if has_bwd else ["fwd"]
+    names = (["fwd", "bwd_weight", "bwd_data"] if use_dist else ["fwd", "bwd_data", "bwd_weight"]) if has_bwd else ["fwd"]
     kern_ms = {name: statistics.mean(ev[i][k].elapsed_time(ev[i][k + 1]) for i in range(args.steps))
                for k, name in enumerate(names)}
     alg_bytes = {"fwd": wl.N * info.bytes_per_token_fwd, "bwd_data": wl.N * info.bytes_per_token_bwd_data,
@@ -419,7 +443,7 @@ def main():
                 "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
                 "roofline": roofline, "cpu_baseline": cpu_baseline}
         print(json.dumps(line))
-    if world > 1:
+    if use_dist:
         dist.destroy_process_group()
 
 

@@ -29,16 +29,22 @@ def grad_buffers(Co: int, Ci: int, T: int, device):
     return flat, flat[:n].view(Co, Ci, T), flat[n + pad:n + pad + Co]
 
 
-def allreduce_weight_grads(dw, db=None, group=None, flat=None) -> None:
+def allreduce_weight_grads(dw, db=None, group=None, flat=None, async_op=False):
     """Sum dw (and db) over the ranks of `group`, in place.  No-op without an initialised process group.
-    With `flat` (the buffer of grad_buffers that dw and db are views of) one all-reduce covers both."""
+    With `flat` (the buffer of grad_buffers that dw and db are views of) one all-reduce covers both; with
+    `async_op` (flat form only) the collective's work handle is returned instead of being waited for."""
     import torch.distributed as dist
 
-    if not dist.is_available() or not dist.is_initialized() or dist.get_world_size(group) == 1:
-        return
+    if not dist.is_available() or not dist.is_initialized():
+        return None
     if flat is not None:
-        dist.all_reduce(flat, op=dist.ReduceOp.SUM, group=group)
-        return
+        if dist.get_world_size(group) == 1 and not async_op:
+            return None
+        return dist.all_reduce(flat, op=dist.ReduceOp.SUM, group=group, async_op=async_op) if async_op else \
+            dist.all_reduce(flat, op=dist.ReduceOp.SUM, group=group)
+    if dist.get_world_size(group) == 1:
+        return None
     dist.all_reduce(dw, op=dist.ReduceOp.SUM, group=group)
     if db is not None:
         dist.all_reduce(db, op=dist.ReduceOp.SUM, group=group)
+    return None
