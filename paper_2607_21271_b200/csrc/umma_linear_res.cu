@@ -14,11 +14,15 @@
 //   TMA (1-D bulk)              spectral-weight image of (channel tile, 16-channel chunk) -> weight ring
 //   1 thread                    tcgen05.mma kind::f16; complex frequency (Eq. 5) as
 //                                   [Re|Im] += Wr [Xr|Xi],   Re += (-Wi) Xi (A negated by the instruction),   Im += Wi Xr
-//   12 warps                    tcgen05.ld, bias on plane k = 0, inverse DFT (Eq. 7), fp16 rounding; a thread owns one
+//   12 warps (16 for T = 4)     tcgen05.ld, bias on plane k = 0, inverse DFT (Eq. 7), fp16 rounding; a thread owns one
 //                               output channel, so a warp writes 32 channels x T elements of a token as one contiguous run
 //
 // The transform of the next token tile runs while the MMAs of the current tile's last channel tile are in flight
 // (each x^ chunk is rewritten as soon as the MMAs that read it have retired).
+//
+// Two compile-time variants.  Resident mode: all chunks of a token tile stay in shared memory (several channel tiles).
+// Ring mode (one channel tile, any C_in): three x^ chunk buffers and three weight slots used as rings with ONE
+// full/empty barrier pair per chunk for both; this is the variant the data gradient of a wide-output layer runs.
 //
 // Every wait on an mbarrier is bounded: on a time-out the CTA raises an abort flag, records a status code for the
 // host, drains its outstanding copies and MMAs, frees its TMEM and returns.
