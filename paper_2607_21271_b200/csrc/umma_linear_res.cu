@@ -457,21 +457,28 @@ umma_linear_res_kernel(const __grid_constant__ CUtensorMap tmap_in, const ResPar
                 }
                 uint8_t* dst = out_o + (size_t)(row0 + n0) * pitch;
                 const int rows_left = (int)(prm.N - (row0 + n0) < 8 ? prm.N - (row0 + n0) : 8);   // may be <= 0
+                // whole groups of a valid channel (everything but the batch's last tile and the channels past C_out) take
+                // a copy of the loop without per-token predicates
+                auto emit = [&](auto whole_tag) {
+                    constexpr bool kWhole = decltype(whole_tag)::value;
 #pragma unroll
-                for (int j = 0; j < 8; ++j, dst += pitch) {
-                    float v[T];
+                    for (int j = 0; j < 8; ++j, dst += pitch) {
+                        float v[T];
 #pragma unroll
-                    for (int p = 0; p < T; ++p) v[p] = __uint_as_float(in[p][j]);
-                    v[0] += bias_v;
-                    rdft_inverse<T>(v);
-                    if (o_ok && j < rows_left) {
-                        if constexpr (T == 8)
-                            *reinterpret_cast<uint4*>(dst) = make_uint4(pack_h2(v[0], v[1]), pack_h2(v[2], v[3]),
-                                                                        pack_h2(v[4], v[5]), pack_h2(v[6], v[7]));
-                        else
-                            *reinterpret_cast<uint2*>(dst) = make_uint2(pack_h2(v[0], v[1]), pack_h2(v[2], v[3]));
+                        for (int p = 0; p < T; ++p) v[p] = __uint_as_float(in[p][j]);
+                        v[0] += bias_v;
+                        rdft_inverse<T>(v);
+                        if (kWhole || (o_ok && j < rows_left)) {
+                            if constexpr (T == 8)
+                                *reinterpret_cast<uint4*>(dst) = make_uint4(pack_h2(v[0], v[1]), pack_h2(v[2], v[3]),
+                                                                            pack_h2(v[4], v[5]), pack_h2(v[6], v[7]));
+                            else
+                                *reinterpret_cast<uint2*>(dst) = make_uint2(pack_h2(v[0], v[1]), pack_h2(v[2], v[3]));
+                        }
                     }
-                }
+                };
+                if (o_ok && rows_left >= 8) emit(std::true_type{});
+                else emit(std::false_type{});
             }
             if (cw == 0 && lane == 0) RES_STAMP(8 * cu + 4);
         }
