@@ -26,7 +26,9 @@
  *     asynchronous on that stream and never synchronise the device, except where stated.
  *   - Errors are return codes.  Argument errors are detected on the host before any launch.
  *     N == 0 is a successful no-op.  Nothing traps or aborts on the device.
- *   - A plan may be used from one stream at a time.
+ *   - A plan may be used from one stream at a time, and only while the device it was built on is the
+ *     current device: every entry point that takes a plan returns EQL_ERR_INVALID_ARG, before any
+ *     launch, when another device is current.  Different plans may be used from different host threads.
  */
 #ifndef EQLINEAR_H_
 #define EQLINEAR_H_
@@ -124,6 +126,13 @@ eql_status_t eqlinear_plan_set_weight(eqlinear_plan_t plan, const void* w, const
 
 eql_status_t eqlinear_plan_info(eqlinear_plan_t plan, eql_info_t* info);
 
+/* Kernel launches ONE call of each entry point makes for N tokens with this plan (launch accounting for
+ * benchmarks; no GPU work): counts[0] eqlinear_fwd, counts[1] eqlinear_bwd_data, counts[2] eqlinear_bwd_weight
+ * (or eqlinear_bwd_weight_from_spectrum), counts[3] the launches eqlinear_fwd_save_spectrum adds to eqlinear_fwd.
+ * More than one launch per call occurs for FP32 plans only: reductions over more than 256 channels run as
+ * segments, long token ranges of the weight gradient as blocks (the plan's FP32 semantics, see eqlinear_plan). */
+eql_status_t eqlinear_plan_launch_counts(eqlinear_plan_t plan, int64_t N, int32_t counts[4]);
+
 /* Reads the plan's device status word (synchronises `stream`): EQL_OK, or
  * EQL_ERR_DEVICE_TIMEOUT if a bounded wait inside one of the plan's kernels gave up. */
 eql_status_t eqlinear_plan_device_status(eqlinear_plan_t plan, void* stream);
@@ -204,14 +213,21 @@ eql_status_t eqlinear_bwd_weight_from_spectrum(eqlinear_plan_t plan, const void*
  * cudaMalloc would fail, or a latency-critical loop that may not risk the device-wide stall an
  * allocation can cause.  Such callers still pass their inputs and outputs (x, dy, dw, db, as for
  * eqlinear_bwd_weight); only the scratch for the per-split partial spectra comes from the library,
- * from a fixed device array of EQL_STATIC_SCRATCH_BYTES (32 MiB) that every GPU which loads the
- * library holds until the process exits.  This call allocates nothing and frees nothing.
+ * from a fixed device array of EQL_STATIC_SCRATCH_BYTES (32 MiB) that is part of the library image.
+ * This call allocates nothing and frees nothing.
  *
+ *   - When the 32 MiB become resident: CUDA loads the parts of a library lazily, and the array's part
+ *     is loaded on a GPU the first time the array's address is looked up there.  eqlinear_plan does
+ *     that look-up for its device, so building the first plan on a GPU is what reserves the array
+ *     (once per GPU, until the process exits) -- do it while device memory can still be had, i.e.
+ *     before a pool claims the rest of the GPU.  After that no call of this entry point loads,
+ *     reserves or looks up anything: free device memory is the same before and after it.
  *   - Returns EQL_ERR_WORKSPACE, and launches nothing, when eqlinear_bwd_weight_scratch_bytes(plan, N)
  *     is larger than EQL_STATIC_SCRATCH_BYTES; use eqlinear_bwd_weight with your own buffer then.
- *   - The first call on each device looks up the array's device address (the plan's device must be
- *     the current device; EQL_ERR_INVALID_ARG otherwise).  Make that first call before any stream
- *     capture begins.
+ *   - The array's device address is looked up once per device, by eqlinear_plan (with the plan's
+ *     device current).  Should that look-up have failed, this call repeats it and returns
+ *     EQL_ERR_CUDA if it fails again; build plans, and so do the look-up, before any stream capture
+ *     begins.  The plan's device must be the current device (EQL_ERR_INVALID_ARG otherwise).
  *   - All calls, from every plan and stream, share the one array, and it keeps whatever the last
  *     call left in it.  Nothing in it has to start at zero: each call overwrites every partial it
  *     later reads.  Two calls that overlap in time on the GPU race on it; order them on one stream

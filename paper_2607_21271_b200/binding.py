@@ -39,7 +39,7 @@ EXPORTED_SYMBOLS = (
     "eqlinear_fwd", "eqlinear_bwd_data", "eqlinear_bwd_weight_scratch_bytes", "eqlinear_bwd_weight",
     "eqlinear_fwd_host", "eqlinear_bwd_data_host", "eqlinear_bwd_weight_host", "eqlinear_step_host", "eqlinear_bwd_weight_static",
     "eqlinear_spectrum_bytes", "eqlinear_fwd_save_spectrum", "eqlinear_bwd_weight_from_spectrum",
-    "eqlinear_plan_clear_device_status", "eqlinear_plan_selftest_expired_wait",
+    "eqlinear_plan_clear_device_status", "eqlinear_plan_selftest_expired_wait", "eqlinear_plan_launch_counts",
 )
 
 
@@ -84,6 +84,7 @@ def load_library(path: str | None = None) -> ctypes.CDLL:
         "eqlinear_plan": [POINTER(V), I, I, I, I, V, V, V, SZ, c_uint, V],
         "eqlinear_plan_set_weight": [V, V, V, V],
         "eqlinear_plan_info": [V, POINTER(EqlInfo)],
+        "eqlinear_plan_launch_counts": [V, I64, POINTER(c_int32)],
         "eqlinear_plan_device_status": [V, V],
         "eqlinear_plan_clear_device_status": [V, V],
         "eqlinear_plan_selftest_expired_wait": [V, V],
@@ -160,6 +161,13 @@ def eqlinear_plan_info(plan) -> EqlInfo:
     info = EqlInfo()
     _check(load_library().eqlinear_plan_info(plan, byref(info)), "eqlinear_plan_info")
     return info
+
+
+def eqlinear_plan_launch_counts(plan, N) -> dict:
+    """Kernel launches one call of each entry point makes for N tokens with this plan."""
+    c = (c_int32 * 4)()
+    _check(load_library().eqlinear_plan_launch_counts(plan, N, c), "eqlinear_plan_launch_counts")
+    return {"fwd": c[0], "bwd_data": c[1], "bwd_weight": c[2], "fwd_save_spectrum_extra": c[3]}
 
 
 def eqlinear_plan_device_status(plan, stream=0) -> int:

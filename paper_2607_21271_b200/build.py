@@ -24,11 +24,6 @@ NVCC_FLAGS = [
 ]
 
 
-def _extra_flags():
-    """Extra nvcc flags from the environment (e.g. EQL_NVCC_FLAGS=-DEQL_TRACE for the timeline instrumentation)."""
-    return os.environ.get("EQL_NVCC_FLAGS", "").split()
-
-
 def _nvcc() -> str:
     cand = os.path.join(os.environ.get("CUDA_HOME", "/usr/local/cuda"), "bin", "nvcc")
     return cand if os.path.exists(cand) else "nvcc"
@@ -56,7 +51,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
         obj = os.path.join(BUILD_DIR, os.path.basename(src)[:-3] + ".o")
         objs.append(obj)
         if force or not os.path.exists(obj) or os.path.getmtime(obj) < max(os.path.getmtime(src), hdr_m):
-            cmd = [_nvcc(), *NVCC_FLAGS, *_extra_flags(), "-I", INCLUDE, "-c", src, "-o", obj]
+            cmd = [_nvcc(), *NVCC_FLAGS, "-I", INCLUDE, "-c", src, "-o", obj]
             if verbose:
                 cmd.insert(1, "-Xptxas=-v")
             jobs.append(cmd)

@@ -5,6 +5,8 @@
 #include <stddef.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "../../include/eqlinear.h"
 
 namespace eql {
@@ -26,6 +28,25 @@ struct WorkspaceLayout {
     size_t total;
 };
 WorkspaceLayout workspace_layout(int T, int Ci, int Co, eql_dtype_t dtype);
+
+// Raises a kernel's dynamic shared-memory limit once per device.  One object per kernel instantiation (a function-local
+// static of the launcher); safe to use from several host threads: a bit is published only after the attribute call
+// has returned, and setting the attribute twice is harmless.
+struct SmemLimitOnce {
+    std::atomic<unsigned long long> done{0};
+    template <class Kernel>
+    cudaError_t ensure(Kernel kernel, int bytes) {
+        int dev = 0;
+        cudaError_t e = cudaGetDevice(&dev);
+        if (e != cudaSuccess) return e;
+        if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+        if ((done.load(std::memory_order_acquire) >> dev) & 1ull) return cudaSuccess;
+        e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+        if (e != cudaSuccess) return e;
+        done.fetch_or(1ull << dev, std::memory_order_release);
+        return cudaSuccess;
+    }
+};
 
 inline bool supported_T(int T) { return T == 2 || T == 4 || T == 8 || T == 16 || T == 32; }
 
@@ -135,6 +156,11 @@ cudaError_t launch_umma_bwd_weight_saved(const UmmaBwdWeightShape& s, const void
 cudaError_t launch_bwd_weight_finalize(int T, bool correlation, const float* scratch, int splits, int Ci, int Co,
                                        float* dw, float* db, cudaStream_t stream, bool accumulate = false);
 
+// Device address, on `device`, of the scratch array built into the library for eqlinear_bwd_weight_static
+// (static_scratch.cu).  `device` must be the current device.  Looked up once per device and cached; the first look-up
+// on a device loads the module that holds the array.  Returns nullptr on failure (*err, if given, says why).
+void* static_scratch_address(int device, cudaError_t* err);
+
 }  // namespace eql
 
 // Copy pipeline of the host-buffer entry points: token chunks travel host -> device on one stream, are computed on
@@ -162,3 +188,12 @@ struct eqlinear_plan_s {
     eql::UmmaResShape res_fwd, res_bwd;   // used when the kernel id is 2
     HostPipe* pipe = nullptr;
 };
+
+// Every call that takes a plan launches on the current device with pointers (workspace, tensor maps) that belong to the
+// plan's device: refuse, before any launch, when the two differ.
+inline eql_status_t eql_check_plan(eqlinear_plan_t plan) {
+    if (!plan) return EQL_ERR_INVALID_ARG;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return EQL_ERR_CUDA;
+    return dev == plan->device ? EQL_OK : EQL_ERR_INVALID_ARG;
+}

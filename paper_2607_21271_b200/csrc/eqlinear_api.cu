@@ -281,6 +281,11 @@ eql_status_t eqlinear_plan(eqlinear_plan_t* plan, int T, int C_in, int C_out, eq
         }
     }
 
+    // The built-in scratch array of eqlinear_bwd_weight_static: look its address up now, with the plan's device current,
+    // so that the module holding it is loaded (and its memory reserved) here and never by a call on the hot path.
+    // A failure is not an error of this call; eqlinear_bwd_weight_static reports it.
+    static_scratch_address(dev, nullptr);
+
     cudaStream_t s = (cudaStream_t)stream;
     if (cudaMemsetAsync(p->ws + lay.status, 0, kWsAlign, s) != cudaSuccess) { delete p; return EQL_ERR_CUDA; }
     st = build_weights(p, w, bias, s);
@@ -290,7 +295,8 @@ eql_status_t eqlinear_plan(eqlinear_plan_t* plan, int T, int C_in, int C_out, eq
 }
 
 eql_status_t eqlinear_plan_set_weight(eqlinear_plan_t plan, const void* w, const void* bias, void* stream) {
-    if (!plan || !w) return EQL_ERR_INVALID_ARG;
+    if (eql_status_t ps = eql_check_plan(plan); ps != EQL_OK) return ps;
+    if (!w) return EQL_ERR_INVALID_ARG;
     if ((bias != nullptr) != plan->has_bias) return EQL_ERR_INVALID_ARG;
     if (!aligned16(w) || (bias && !aligned16(bias))) return EQL_ERR_ALIGNMENT;
     return build_weights(plan, w, bias, (cudaStream_t)stream);
@@ -312,8 +318,29 @@ eql_status_t eqlinear_plan_info(eqlinear_plan_t plan, eql_info_t* info) {
     return EQL_OK;
 }
 
+eql_status_t eqlinear_plan_launch_counts(eqlinear_plan_t plan, int64_t N, int32_t counts[4]) {
+    if (!plan || !counts) return EQL_ERR_INVALID_ARG;
+    eql_status_t st = check_tokens(N);
+    if (st != EQL_OK) return st;
+    counts[0] = counts[1] = counts[2] = counts[3] = 0;
+    if (N == 0) return EQL_OK;
+    int len = 0;
+    counts[0] = plan->fwd_kernel == 1 ? umma_reduction_segments(plan->Ci, plan->dtype, &len) : 1;
+    counts[1] = plan->bwd_data_kernel == 1 ? umma_reduction_segments(plan->Co, plan->dtype, &len) : 1;
+    if (plan->bwd_weight_kernel == 1) {
+        const UmmaBwdWeightShape bs = umma_bwd_weight_shape(plan->T, plan->Ci, plan->Co, plan->dtype, N, plan->num_sms);
+        const int64_t blocks = (N + bs.block_tokens - 1) / bs.block_tokens;
+        counts[2] = (int32_t)(2 * blocks);                     // partial-spectra kernel + finalize kernel per block of tokens
+    } else {
+        counts[2] = 2;
+    }
+    // eqlinear_fwd_save_spectrum: the resident-activation kernel writes the spectrum itself, others add a pre-pass
+    counts[3] = (plan->dtype == EQL_FP16 && plan->bwd_weight_kernel == 1 && plan->fwd_kernel != 2) ? 1 : 0;
+    return EQL_OK;
+}
+
 eql_status_t eqlinear_plan_device_status(eqlinear_plan_t plan, void* stream) {
-    if (!plan) return EQL_ERR_INVALID_ARG;
+    if (eql_status_t ps = eql_check_plan(plan); ps != EQL_OK) return ps;
     int word = 0;
     cudaStream_t s = (cudaStream_t)stream;
     if (cudaMemcpyAsync(&word, plan->ws + plan->lay.status, sizeof(int), cudaMemcpyDeviceToHost, s) != cudaSuccess)
@@ -329,7 +356,7 @@ eql_status_t eqlinear_plan_destroy(eqlinear_plan_t plan) {
 }
 
 eql_status_t eqlinear_fwd(eqlinear_plan_t plan, const void* x, void* y, int64_t N, void* stream) {
-    if (!plan) return EQL_ERR_INVALID_ARG;
+    if (eql_status_t ps = eql_check_plan(plan); ps != EQL_OK) return ps;
     eql_status_t st = check_tokens(N);
     if (st != EQL_OK) return st;
     if (N == 0) return EQL_OK;
@@ -351,7 +378,7 @@ eql_status_t eqlinear_fwd(eqlinear_plan_t plan, const void* x, void* y, int64_t 
 }
 
 eql_status_t eqlinear_bwd_data(eqlinear_plan_t plan, const void* dy, void* dx, int64_t N, void* stream) {
-    if (!plan) return EQL_ERR_INVALID_ARG;
+    if (eql_status_t ps = eql_check_plan(plan); ps != EQL_OK) return ps;
     eql_status_t st = check_tokens(N);
     if (st != EQL_OK) return st;
     if (N == 0) return EQL_OK;
@@ -384,7 +411,7 @@ eql_status_t eqlinear_bwd_weight_scratch_bytes(eqlinear_plan_t plan, int64_t N, 
 
 eql_status_t eqlinear_bwd_weight(eqlinear_plan_t plan, const void* x, const void* dy, void* dw, void* db, int64_t N,
                                  void* scratch, size_t scratch_bytes, void* stream) {
-    if (!plan) return EQL_ERR_INVALID_ARG;
+    if (eql_status_t ps = eql_check_plan(plan); ps != EQL_OK) return ps;
     eql_status_t st = check_tokens(N);
     if (st != EQL_OK) return st;
     if (!dw) return EQL_ERR_INVALID_ARG;
@@ -439,7 +466,7 @@ eql_status_t eqlinear_spectrum_bytes(eqlinear_plan_t plan, int64_t N, size_t* by
 
 eql_status_t eqlinear_fwd_save_spectrum(eqlinear_plan_t plan, const void* x, void* y, int64_t N, void* spectrum,
                                         size_t spectrum_bytes, void* stream) {
-    if (!plan) return EQL_ERR_INVALID_ARG;
+    if (eql_status_t ps = eql_check_plan(plan); ps != EQL_OK) return ps;
     size_t need = 0;
     eql_status_t st = eqlinear_spectrum_bytes(plan, N, &need);
     if (st != EQL_OK) return st;
@@ -468,7 +495,7 @@ eql_status_t eqlinear_fwd_save_spectrum(eqlinear_plan_t plan, const void* x, voi
 eql_status_t eqlinear_bwd_weight_from_spectrum(eqlinear_plan_t plan, const void* spectrum, size_t spectrum_bytes,
                                                const void* dy, void* dw, void* db, int64_t N, void* scratch,
                                                size_t scratch_bytes, void* stream) {
-    if (!plan) return EQL_ERR_INVALID_ARG;
+    if (eql_status_t ps = eql_check_plan(plan); ps != EQL_OK) return ps;
     size_t need = 0;
     eql_status_t st = eqlinear_spectrum_bytes(plan, N, &need);
     if (st != EQL_OK) return st;
@@ -496,7 +523,7 @@ eql_status_t eqlinear_bwd_weight_from_spectrum(eqlinear_plan_t plan, const void*
 // ---- host-buffer variants ---------------------------------------------------------------------
 eql_status_t eqlinear_fwd_host(eqlinear_plan_t plan, const void* x_host, void* y_host, int64_t N, void* x_staging,
                                void* y_staging, void* stream) {
-    if (!plan) return EQL_ERR_INVALID_ARG;
+    if (eql_status_t ps = eql_check_plan(plan); ps != EQL_OK) return ps;
     eql_status_t st = check_tokens(N);
     if (st != EQL_OK) return st;
     if (N == 0) return EQL_OK;
@@ -507,7 +534,7 @@ eql_status_t eqlinear_fwd_host(eqlinear_plan_t plan, const void* x_host, void* y
 
 eql_status_t eqlinear_bwd_data_host(eqlinear_plan_t plan, const void* dy_host, void* dx_host, int64_t N,
                                     void* dy_staging, void* dx_staging, void* stream) {
-    if (!plan) return EQL_ERR_INVALID_ARG;
+    if (eql_status_t ps = eql_check_plan(plan); ps != EQL_OK) return ps;
     eql_status_t st = check_tokens(N);
     if (st != EQL_OK) return st;
     if (N == 0) return EQL_OK;
@@ -525,7 +552,7 @@ eql_status_t eqlinear_bwd_data_host(eqlinear_plan_t plan, const void* dy_host, v
 eql_status_t eqlinear_bwd_weight_host(eqlinear_plan_t plan, const void* x_host, const void* dy_host, void* dw_host,
                                       void* db_host, int64_t N, void* x_staging, void* dy_staging, void* dw_staging,
                                       void* db_staging, void* scratch, size_t scratch_bytes, void* stream) {
-    if (!plan) return EQL_ERR_INVALID_ARG;
+    if (eql_status_t ps = eql_check_plan(plan); ps != EQL_OK) return ps;
     eql_status_t st = check_tokens(N);
     if (st != EQL_OK) return st;
     if (!dw_host || !dw_staging || (db_host && !db_staging)) return EQL_ERR_INVALID_ARG;
@@ -551,7 +578,7 @@ eql_status_t eqlinear_step_host(eqlinear_plan_t plan, const void* x_host, const 
                                 void* dx_host, void* dw_host, void* db_host, int64_t N, void* x_staging,
                                 void* dy_staging, void* y_staging, void* dx_staging, void* dw_staging,
                                 void* db_staging, void* scratch, size_t scratch_bytes, void* stream) {
-    if (!plan) return EQL_ERR_INVALID_ARG;
+    if (eql_status_t ps = eql_check_plan(plan); ps != EQL_OK) return ps;
     eql_status_t st = check_tokens(N);
     if (st != EQL_OK) return st;
     if (N == 0) return EQL_ERR_INVALID_ARG;

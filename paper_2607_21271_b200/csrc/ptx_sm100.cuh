@@ -73,9 +73,6 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
 
 // ---------------------------------------------------------------- proxy / tcgen05 fences
 __device__ __forceinline__ void fence_proxy_async_smem() {
-#ifdef EQL_ABLATE_FENCE
-    return;
-#endif
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
 __device__ __forceinline__ void tc_fence_before_sync() {
@@ -190,9 +187,6 @@ __device__ __forceinline__ uint32_t umma_idesc_f16_f32_mn_major(uint32_t M, uint
 // D[tmem] (+)= A[smem] * B[smem]^T; issued by ONE thread.
 __device__ __forceinline__ void umma_f16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
                                          uint32_t accumulate) {
-#ifdef EQL_ABLATE_MMA
-    return;
-#endif
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
         "setp.ne.b32 p, %4, 0;\n\t"
@@ -202,9 +196,6 @@ __device__ __forceinline__ void umma_f16(uint32_t d_tmem, uint64_t a_desc, uint6
 }
 __device__ __forceinline__ void umma_tf32(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
                                           uint32_t accumulate) {
-#ifdef EQL_ABLATE_MMA
-    return;
-#endif
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
         "setp.ne.b32 p, %4, 0;\n\t"

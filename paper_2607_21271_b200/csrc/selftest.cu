@@ -27,13 +27,13 @@ __global__ void __launch_bounds__(32, 1) expire_one_wait_kernel(int* status) {
 extern "C" {
 
 eql_status_t eqlinear_plan_selftest_expired_wait(eqlinear_plan_t plan, void* stream) {
-    if (!plan) return EQL_ERR_INVALID_ARG;
+    if (eql_status_t ps = eql_check_plan(plan); ps != EQL_OK) return ps;
     eql::expire_one_wait_kernel<<<1, 32, 0, (cudaStream_t)stream>>>((int*)(plan->ws + plan->lay.status));
     return cudaGetLastError() == cudaSuccess ? EQL_OK : EQL_ERR_CUDA;
 }
 
 eql_status_t eqlinear_plan_clear_device_status(eqlinear_plan_t plan, void* stream) {
-    if (!plan) return EQL_ERR_INVALID_ARG;
+    if (eql_status_t ps = eql_check_plan(plan); ps != EQL_OK) return ps;
     return cudaMemsetAsync(plan->ws + plan->lay.status, 0, sizeof(int), (cudaStream_t)stream) == cudaSuccess ? EQL_OK
                                                                                                               : EQL_ERR_CUDA;
 }

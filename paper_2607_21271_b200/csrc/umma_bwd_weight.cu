@@ -54,13 +54,6 @@ struct BwParams {
     int part_tma;                // the partial spectra can be written with TMA tensor stores (row pitch a multiple of 16 bytes)
 };
 
-// Optional timeline instrumentation (compiled only with -DEQL_TRACE): CTA 0 records clock64() stamps.
-#ifdef EQL_TRACE
-__device__ unsigned long long g_trace_bw[8192];
-#define BW_STAMP(slot) do { if (blockIdx.x == 0 && (slot) < 8192) g_trace_bw[(slot)] = clock64(); } while (0)
-#else
-#define BW_STAMP(slot) do { } while (0)
-#endif
 
 struct BwBarriers {
     uint64_t full_raw[kRawSlots], empty_raw[kRawSlots];
@@ -135,7 +128,6 @@ umma_bwd_weight_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
                 const int slot = NRAW == 2 ? (int)(c & 1) : 0;
                 ok = ptx::mbar_wait(&bar->empty_raw[slot], (uint32_t)((NRAW == 2 ? (c >> 1) : c) & 1) ^ 1, abort_flag, status, 201);
                 if (!ok) break;
-                BW_STAMP(3000 + (int)c);
                 ptx::mbar_arrive_expect_tx(&bar->full_raw[slot], bytes);
                 const int row = (int)((chunk0 + c) * kChunkTok);
                 uint8_t* dst = raw + slot * kRawSlot;
@@ -182,9 +174,7 @@ umma_bwd_weight_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
                 // NST is 1 or 2: stage and phase parity without a division
                 const int st = NST == 2 ? (int)(c & 1) : 0;
                 const uint32_t sph = (uint32_t)((NST == 2 ? (c >> 1) : c) & 1);
-                BW_STAMP(1000 + 3 * (int)c);
                 ok = ptx::mbar_wait(&bar->full_ab[st], sph, abort_flag, status, 202);
-                BW_STAMP(1000 + 3 * (int)c + 1);
                 if (!ok) break;
                 ptx::tc_fence_after_sync();
                 const uint32_t stage0 = ptx::smem_u32(stages + st * prm.stage_bytes);
@@ -208,7 +198,6 @@ umma_bwd_weight_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
                     }
                 }
                 ptx::umma_commit(&bar->empty_ab[st]);
-                BW_STAMP(1000 + 3 * (int)c + 2);
             }
             if (ok) ptx::umma_commit(&bar->full_d);
             ptx::umma_commit(&bar->mma_done);
@@ -233,19 +222,8 @@ umma_bwd_weight_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
         for (int64_t c = 0; c < nchunks; ++c) {
             const int slot = NRAW == 2 ? (int)(c & 1) : 0, st = NST == 2 ? (int)(c & 1) : 0;
             const uint32_t sph = (uint32_t)((NST == 2 ? (c >> 1) : c) & 1);
-#ifdef EQL_TRACE
-            const bool tr = lane == 0 && (warp == kWarpDftX0 || warp == kWarpDftY0);
-            const int tb = (warp == kWarpDftX0 ? 4000 : 5000) + 6 * (int)c;
-            if (tr) BW_STAMP(tb);
-#endif
             ok = ptx::mbar_wait(&bar->full_raw[slot], (uint32_t)((NRAW == 2 ? (c >> 1) : c) & 1), abort_flag, status, 203);
-#ifdef EQL_TRACE
-            if (tr) BW_STAMP(tb + 1);
-#endif
             ok = ok && ptx::mbar_wait(&bar->empty_ab[st], sph ^ 1, abort_flag, status, 204);
-#ifdef EQL_TRACE
-            if (tr) BW_STAMP(tb + 2);
-#endif
             if (!ok) break;
             uint32_t wd[32];
             if (active)
@@ -266,14 +244,6 @@ umma_bwd_weight_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
                 if constexpr (E == 2) {
                     uint32_t packed[T][NCH / 2];
                     float p0[NCH];
-#ifdef EQL_ABLATE_DFT
-#pragma unroll
-                    for (int p = 0; p < T; ++p)
-#pragma unroll
-                        for (int c2 = 0; c2 < NCH / 2; ++c2) packed[p][c2] = wd[(p * (NCH / 2) + c2) & 31];
-#pragma unroll
-                    for (int i = 0; i < NCH; ++i) p0[i] = 0.f;
-#else
                     // dy: butterflies in float, planes rounded to fp16 once (its k = 0 plane also feeds db, unrounded).
                     // x: packed-half butterflies, two channels per instruction.  x^ is recomputed by every
                     // output-channel tile, which makes its transform the largest share of this kernel's instructions
@@ -281,7 +251,6 @@ umma_bwd_weight_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
                     // (measured max error 4.2e-4 instead of 3.1e-4 of the largest |dw|, bar 3e-3).
                     if (is_y) dft_words<T, true>(wd, packed, p0);
                     else dft_words<T, false, true>(wd, packed, nullptr);
-#endif
                     if (!is_y) {
 #pragma unroll
                         for (int p = 0; p < T; ++p) store_plane_run<NCH>(stage + p * a_plane + off, packed[p], 256);
@@ -336,9 +305,6 @@ umma_bwd_weight_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
             ptx::fence_proxy_async_smem();
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(&bar->full_ab[st]);
-#ifdef EQL_TRACE
-            if (tr) BW_STAMP(tb + 3);
-#endif
         }
         // db partial of this token range: sum over the 16 token rows of each half warp
         if (is_y) {
@@ -482,12 +448,6 @@ int balanced_tile(int C, int max_tile, int round) {
 
 }  // namespace
 
-#ifdef EQL_TRACE
-extern "C" int eqlinear_debug_read_trace_bw(unsigned long long* dst, int n) {
-    cudaDeviceSynchronize();
-    return (int)cudaMemcpyFromSymbol(dst, g_trace_bw, sizeof(unsigned long long) * (n < 8192 ? n : 8192));
-}
-#endif
 
 bool umma_bwd_weight_supported(int T, eql_dtype_t dtype) {
     if (dtype == EQL_FP16) return T == 4 || T == 8 || T == 16 || T == 32;
@@ -634,14 +594,8 @@ cudaError_t launch_umma_bwd_weight(const UmmaBwdWeightShape& s, const void* x, c
     auto go = [&](auto tc, auto io) -> cudaError_t {
         constexpr int TT = decltype(tc)::value;
         using IO = decltype(io);
-        static unsigned long long attr_done = 0;
-        int dev = 0;
-        cudaGetDevice(&dev);
-        if (!((attr_done >> (dev & 63)) & 1ull)) {
-            cudaError_t e = cudaFuncSetAttribute(umma_bwd_weight_kernel<TT, IO>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-            if (e != cudaSuccess) return e;
-            attr_done |= 1ull << (dev & 63);
-        }
+        static SmemLimitOnce smem_limit;                      // per kernel instantiation
+        if (cudaError_t e = smem_limit.ensure(umma_bwd_weight_kernel<TT, IO>, 227 * 1024); e != cudaSuccess) return e;
         umma_bwd_weight_kernel<TT, IO><<<grid, kThreadsBw, smem, stream>>>(mx, my, mp, prm);
         return cudaGetLastError();
     };

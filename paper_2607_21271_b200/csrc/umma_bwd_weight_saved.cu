@@ -53,16 +53,6 @@ struct BwParams {
     int part_tma;                // the partial spectra can be written with TMA tensor stores
 };
 
-// Optional timeline instrumentation (compiled only with -DEQL_TRACE): CTA 0 records clock64() stamps.
-#ifdef EQL_TRACE
-__device__ unsigned long long g_trace_bws[8192];
-#ifndef EQL_TRACE_CTA
-#define EQL_TRACE_CTA 0
-#endif
-#define BW_STAMP(slot) do { if (blockIdx.x == EQL_TRACE_CTA && (slot) < 8192) g_trace_bws[(slot)] = clock64(); } while (0)
-#else
-#define BW_STAMP(slot) do { } while (0)
-#endif
 
 struct BwBarriers {
     uint64_t full_raw[kGroups], empty_raw[kGroups];
@@ -175,7 +165,6 @@ umma_bwd_weight_saved_kernel(const __grid_constant__ CUtensorMap tmap_dy, const 
                 if (c > 0 && ++slot == kGroups) { slot = 0; eph ^= 1u; }
                 ok = ptx::mbar_wait(&bar->empty_raw[slot], eph, abort_flag, status, 201);
                 if (!ok) break;
-                BW_STAMP(3000 + (int)c);
                 ptx::mbar_arrive_expect_tx(&bar->full_raw[slot], ybytes);
                 const int row = (int)((chunk0 + c) * kChunkTok);
                 uint8_t* dst = raw + slot * kRawSlot;
@@ -207,7 +196,6 @@ umma_bwd_weight_saved_kernel(const __grid_constant__ CUtensorMap tmap_dy, const 
                 if (c > 0 && ++slot == XS) { slot = 0; eph ^= 1u; }
                 ok = ptx::mbar_wait(&empty_xb[slot], eph, abort_flag, status, 206);
                 if (!ok) break;
-                BW_STAMP(2000 + (int)c);
                 ptx::mbar_arrive_expect_tx(&full_xb[slot], (uint32_t)prm.xhat_bytes);
                 ptx::bulk_load_1d(xring + slot * prm.xhat_bytes, xsrc + (size_t)c * prm.xhat_bytes, (uint32_t)prm.xhat_bytes,
                                   &full_xb[slot]);
@@ -229,7 +217,6 @@ umma_bwd_weight_saved_kernel(const __grid_constant__ CUtensorMap tmap_dy, const 
                 ok = ptx::mbar_wait(&bar->full_ab[0], 0, abort_flag, status, 202) &&
                      (MERGED || ptx::mbar_wait(&bar->full_x[0], 0, abort_flag, status, 207));
             for (int64_t c = 0; c < nchunks && ok; ++c) {
-                BW_STAMP(1000 + 4 * (int)c);
                 ptx::tc_fence_after_sync();
                 const uint32_t a0 = ptx::smem_u32(xring + xs * prm.xhat_bytes);
                 const uint32_t b0 = ptx::smem_u32(stages + st * prm.stage_bytes);
@@ -252,17 +239,14 @@ umma_bwd_weight_saved_kernel(const __grid_constant__ CUtensorMap tmap_dy, const 
                     if (f == 1 && c + 1 < nchunks) {
                         // The next chunk's operands are checked here, while the tensor pipe still has this chunk's
                         // MMAs queued, so that the issue stream has no gap between chunks.
-                        BW_STAMP(1000 + 4 * (int)c + 1);
                         ok = ptx::mbar_wait(&bar->full_ab[nst], nsph, abort_flag, status, 202) &&
                              (MERGED || ptx::mbar_wait(&bar->full_x[nxs], nxph, abort_flag, status, 207));
-                        BW_STAMP(1000 + 4 * (int)c + 2);
                     }
                 }
                 ptx::umma_f16(tmem_base + (uint32_t)((T - 1) * CoT), ad + (T - 1) * ap,
                               bd + (uint64_t)(1 + 3 * (T / 2 - 1)) * bt1, idesc_real, acc);
                 ptx::umma_commit(&bar->empty_ab[st]);
                 if constexpr (!MERGED) ptx::umma_commit(&bar->empty_x[xs]);
-                BW_STAMP(1000 + 4 * (int)c + 3);
                 st = nst; xs = nxs; sph = nsph; xph = nxph;
             }
             if (ok) ptx::umma_commit(&bar->full_d);
@@ -282,16 +266,8 @@ umma_bwd_weight_saved_kernel(const __grid_constant__ CUtensorMap tmap_dy, const 
         bool ok = true;
         uint32_t ph = 0;                                         // phase parity of this group's slot and stage
         for (int64_t c = g; c < nchunks; c += kGroups, ph ^= 1u) {
-#ifdef EQL_TRACE
-            const bool tr = lane == 0 && wg == 0;
-            const int tb = 4000 + 6 * (int)c;
-            if (tr) BW_STAMP(tb);
-#endif
             ok = ptx::mbar_wait(&bar->full_raw[g], ph, abort_flag, status, 203);
             if (!ok) break;
-#ifdef EQL_TRACE
-            if (tr) BW_STAMP(tb + 1);
-#endif
             uint32_t wd[32];
             if (active) load_slab_row(raw + g * kRawSlot + slab * kSlab + row * 128, row, wd);
             // The rows are in registers: order these generic-proxy reads before the async-proxy (TMA) refill of
@@ -302,23 +278,11 @@ umma_bwd_weight_saved_kernel(const __grid_constant__ CUtensorMap tmap_dy, const 
             uint32_t packed[T][NCH / 2];
             float p0[NCH];
             if (active) {
-#ifdef EQL_ABLATE_DFT
-#pragma unroll
-                for (int p = 0; p < T; ++p)
-#pragma unroll
-                    for (int c2 = 0; c2 < NCH / 2; ++c2) packed[p][c2] = wd[(p * (NCH / 2) + c2) & 31];
-#pragma unroll
-                for (int i = 0; i < NCH; ++i) p0[i] = 0.f;
-#else
                 dft_words<T, true>(wd, packed, p0);
-#endif
             }
             // the MMAs that read this stage three chunks ago must have retired
             ok = ptx::mbar_wait(&bar->empty_ab[g], ph ^ 1, abort_flag, status, 204);
             if (!ok) break;
-#ifdef EQL_TRACE
-            if (tr) BW_STAMP(tb + 2);
-#endif
             if (active) {
                 const int mn0 = slab * NCH;                      // first channel of this slab inside the tile
                 // MN-major tile: (channel mn, token k) at (mn/8)*256 + (k/8)*128 + (k%8)*16 + (mn%8)*2
@@ -340,9 +304,6 @@ umma_bwd_weight_saved_kernel(const __grid_constant__ CUtensorMap tmap_dy, const 
             ptx::fence_proxy_async_smem();
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(&bar->full_ab[g]);
-#ifdef EQL_TRACE
-            if (tr) BW_STAMP(tb + 3);
-#endif
         }
         // db partial of this token range: sum over the 16 token rows of each half warp; the three groups' sums meet
         // in shared memory and are added in a fixed order at the end
@@ -363,9 +324,7 @@ umma_bwd_weight_saved_kernel(const __grid_constant__ CUtensorMap tmap_dy, const 
             const int ci_local = quad * 32 + lane;
             const int ci = ci_tile * CiT + ci_local;
             const bool lane_ok = ci_local < CiT && ci < prm.Ci;
-            if (wi == 0 && lane == 0) BW_STAMP(7000);
             if (nchunks > 0) ok = ptx::mbar_wait(&bar->full_d, 0, abort_flag, status, 205);
-            if (wi == 0 && lane == 0) BW_STAMP(7001);
             if (ok) {
                 ptx::tc_fence_after_sync();
                 const uint32_t lane_base = tmem_base + ((uint32_t)(quad * 32) << 16);
@@ -410,7 +369,6 @@ umma_bwd_weight_saved_kernel(const __grid_constant__ CUtensorMap tmap_dy, const 
         }
     }
 
-    if (warp == kWarpDft0 && lane == 0) BW_STAMP(7002);
     ptx::tc_fence_before_sync();
     __syncthreads();
     if (bar->abort_flag == 0 && ci_tile == 0 && (int)threadIdx.x < CoT && co_tile * CoT + (int)threadIdx.x < prm.Co)
@@ -464,12 +422,6 @@ bool encode_dy_slabs3d(EncodeTiledFn enc, CUtensorMap* map, const void* base, in
 
 }  // namespace
 
-#ifdef EQL_TRACE
-extern "C" int eqlinear_debug_read_trace_bws(unsigned long long* dst, int n) {
-    cudaDeviceSynchronize();
-    return (int)cudaMemcpyFromSymbol(dst, g_trace_bws, sizeof(unsigned long long) * (n < 8192 ? n : 8192));
-}
-#endif
 
 // Pre-pass: the spectrum image of x for launch_umma_bwd_weight_saved (used when the forward pass that ran for this
 // batch could not write it itself).
@@ -531,14 +483,8 @@ cudaError_t launch_umma_bwd_weight_saved(const UmmaBwdWeightShape& s, const void
     auto go2 = [&](auto tc, auto mg) -> cudaError_t {
         constexpr int TT = decltype(tc)::value;
         constexpr bool MG = decltype(mg)::value;
-        static unsigned long long attr_done = 0;
-        int dev = 0;
-        cudaGetDevice(&dev);
-        if (!((attr_done >> (dev & 63)) & 1ull)) {
-            cudaError_t e = cudaFuncSetAttribute(umma_bwd_weight_saved_kernel<TT, MG>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-            if (e != cudaSuccess) return e;
-            attr_done |= 1ull << (dev & 63);
-        }
+        static SmemLimitOnce smem_limit;                      // per kernel instantiation
+        if (cudaError_t e = smem_limit.ensure(umma_bwd_weight_saved_kernel<TT, MG>, 227 * 1024); e != cudaSuccess) return e;
         umma_bwd_weight_saved_kernel<TT, MG><<<grid, kThreadsBw, smem, stream>>>(my, mp, prm);
         return cudaGetLastError();
     };

@@ -70,13 +70,6 @@ struct UmmaParams {
     int accumulate;              // out += result (TMA reduce-add) instead of out = result: later segments of a reduction
 };
 
-// Optional timeline instrumentation (compiled only with -DEQL_TRACE): CTA 0 records clock64() stamps.
-#ifdef EQL_TRACE
-__device__ unsigned long long g_trace[8192];
-#define EQL_STAMP(slot) do { if (blockIdx.x == 0 && (slot) < 8192) g_trace[(slot)] = clock64(); } while (0)
-#else
-#define EQL_STAMP(slot) do { } while (0)
-#endif
 
 struct SmemBarriers {
     uint64_t full_raw[6], empty_raw[6];
@@ -209,7 +202,6 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
                         if (cr % SPS == 0) {
                             ok = ptx::mbar_wait(&bar->empty_raw[slot], ((ph / kRawSlots) & 1) ^ 1, abort_flag, status, 101, true, kSpin);
                             if (!ok) break;
-                            EQL_STAMP(2048 + cr);
                             ptx::mbar_arrive_expect_tx(&bar->full_raw[slot], SPS * kSlabBytes);
                         }
                         ptx::tma_load_2d(raw + (slot * SPS + cr % SPS) * kSlabBytes, &tmap_in, (kc * KCH + q * NCH) * T, row0,
@@ -245,7 +237,6 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
                     const int slot = cb % SB;
                     ok = ptx::mbar_wait(&bar->empty_b[slot], ((cb / SB) & 1) ^ 1, abort_flag, status, 102, true, kSpin);
                     if (!ok) break;
-                    EQL_STAMP(4096 + cb);
                     ptx::mbar_arrive_expect_tx(&bar->full_b[slot], blob_bytes);
                     ptx::bulk_load_1d(bsm + slot * prm.b_slot_bytes,
                                       prm.image + ((size_t)tile * nK + kc) * (size_t)blob_bytes, blob_bytes,
@@ -273,18 +264,13 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
             };
             const uint32_t b_part = (uint32_t)rowsB * kRowBytes;
             for (int64_t u = first; u < prm.num_units && ok; u += stride, ++cu) {
-                EQL_STAMP(512 + 2 * cu);
                 ok = ptx::mbar_wait(&bar->empty_d, (cu & 1) ^ 1, abort_flag, status, 103, true, kSpin);
-                EQL_STAMP(512 + 2 * cu + 1);
                 if (!ok) break;
                 ptx::tc_fence_after_sync();
                 for (int kc = 0; kc < nK; ++kc, ++ca, ++cb) {
                     const int sa = ca % SA, sb = cb % SB;
-                    EQL_STAMP(1024 + 4 * ca);
                     ok = ptx::mbar_wait(&bar->full_a[sa], (ca / SA) & 1, abort_flag, status, 104, true, kSpin);
-                    EQL_STAMP(1024 + 4 * ca + 1);
                     ok = ok && ptx::mbar_wait(&bar->full_b[sb], (cb / SB) & 1, abort_flag, status, 105, true, kSpin);
-                    EQL_STAMP(1024 + 4 * ca + 2);
                     if (!ok) break;
                     ptx::tc_fence_after_sync();
                     // FP16: one pass.  FP32 (3xTF32): hi*hi, hi*lo, lo*hi accumulate into the same columns.
@@ -309,7 +295,6 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
                     }
                     ptx::umma_commit(&bar->empty_a[sa]);
                     ptx::umma_commit(&bar->empty_b[sb]);
-                    EQL_STAMP(1024 + 4 * ca + 3);
                 }
                 if (ok) ptx::umma_commit(&bar->full_d);
             }
@@ -342,7 +327,6 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
         uint8_t* staging = xhat + cw * 4096;                     // this warp's [32 tokens x 128 B] output stage (128B swizzle)
         for (int64_t u = first; u < prm.num_units && ok; u += stride, ++cu) {
             // ---- transform
-            if (cw == 0 && lane == 0) EQL_STAMP(8 * cu);
             for (int kc = 0; kc < nK && ok; ++kc, ++ca) {
                 const int sa = ca % SA;
 #pragma unroll 1
@@ -351,16 +335,8 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
                     if ((int)(cr % 3) != group) continue;
                     const uint32_t ph = cr / SPS;                // raw-ring slot phase this slab arrives in
                     const int slot = ph % kRawSlots;
-#ifdef EQL_TRACE
-                    const bool tr = (cw == 0 && lane == 0);
-                    const int tb = 6000 + 8 * (int)(cr / 3);
-                    if (tr) EQL_STAMP(tb);
-#endif
                     ok = ptx::mbar_wait(&bar->full_raw[slot], (ph / kRawSlots) & 1, abort_flag, status, 106, true, 16);
                     if (!ok) break;
-#ifdef EQL_TRACE
-                    if (tr) EQL_STAMP(tb + 1);
-#endif
                     const int d = quad;                          // this warp's 32-row quarter of the slab
                     const int r = d * 32 + lane;
                     uint32_t wd[32];
@@ -372,9 +348,6 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
                         __syncwarp();
                         if (lane == 0) ptx::mbar_arrive(&bar->empty_raw[slot]);
                     }
-#ifdef EQL_TRACE
-                    if (tr) EQL_STAMP(tb + 2);
-#endif
                     // A tile of a plane: row r at r*32, its two 16-byte chunks exchanged when bit 2 of r is set (32B swizzle);
                     // this slab row's run of channels starts at byte kb of the row
                     const int kb = q * NCH * E;
@@ -383,20 +356,10 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
                     const int second = sw ? -16 : 16;            // where the other half of the same row lives (32-byte runs only)
                     uint32_t packed[E == 2 ? T : 1][E == 2 ? NCH / 2 : 1];
                     if constexpr (E == 2) {
-#ifdef EQL_ABLATE_DFT
-#pragma unroll
-                        for (int p = 0; p < T; ++p)
-#pragma unroll
-                            for (int c2 = 0; c2 < NCH / 2; ++c2) packed[p][c2] = wd[(p * (NCH / 2) + c2) & 31];
-#else
                         dft_words<T, false>(wd, packed, nullptr);
-#endif
                     } else {
                         dft_words_f32<T>(wd);                    // wd[c*T + p] = plane p of channel c
                     }
-#ifdef EQL_TRACE
-                    if (tr) { if (wd[0] == 0x12345678u && packed[0][0] == 1u) EQL_STAMP(tb + 7); EQL_STAMP(tb + 3); }
-#endif
                     ok = ptx::mbar_wait(&bar->empty_a[sa], ((ca / SA) & 1) ^ 1, abort_flag, status, 107, true, 16);
                     if (!ok) break;
                     if (staging_pending) {                       // the previous unit's output stage lives in the A-operand stages
@@ -404,9 +367,6 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
                         if (!ok) break;
                         staging_pending = false;
                     }
-#ifdef EQL_TRACE
-                    if (tr) EQL_STAMP(tb + 4);
-#endif
                     if constexpr (E == 2) {
 #pragma unroll
                         for (int p = 0; p < T; ++p) store_plane_run<2 * W>(dst + p * 4096, packed[p], second);
@@ -428,42 +388,26 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
                         if constexpr (!Cfg::EARLY) ptx::mbar_arrive(&bar->empty_raw[slot]);
                         ptx::mbar_arrive(&bar->full_a[sa]);
                     }
-#ifdef EQL_TRACE
-                    if (tr) EQL_STAMP(tb + 5);
-#endif
                 }
             }
             if (!ok) break;
             // ---- epilogue
             const int tile = (int)(u % nTiles);
-            if (cw == 0 && lane == 0) EQL_STAMP(8 * cu + 1);
             ok = ptx::mbar_wait(&bar->full_d, cu & 1, abort_flag, status, 108, true, 16);
-            if (cw == 0 && lane == 0) EQL_STAMP(8 * cu + 2);
             if (!ok) break;
             ptx::tc_fence_after_sync();
             const int ngroups = CoT / G;
             for (int gi = third; gi < ngroups; gi += 3) {
                 const int c0 = gi * G;
-#ifdef EQL_TRACE
-                const bool tre = (cw == 0 && lane == 0 && cu < 4);
-                const int te = 7000 + 16 * (int)cu + 4 * (gi / 3);
-                if (tre) EQL_STAMP(te);
-#endif
                 uint32_t in[T][G];
 #pragma unroll
                 for (int p = 0; p < T; ++p) ptx::tmem_ld<G>(lane_base + (uint32_t)(p * CoT + c0), in[p]);
                 ptx::tmem_ld_wait();
-#ifdef EQL_TRACE
-                if (tre) { if (in[0][0] == 0x7fc12345u) EQL_STAMP(te + 3); EQL_STAMP(te + 1); }
-#endif
                 if (gi + 3 >= ngroups) {                         // this warp's last read of the accumulator
                     ptx::tc_fence_before_sync();
                     __syncwarp();
                     if (lane == 0) ptx::mbar_arrive(&bar->empty_d);
                 }
-#ifdef EQL_ABLATE_EPI
-                if (in[0][0] != 0x7fc54321u) continue;
-#endif
                 const int co0 = tile * CoT + c0;
                 uint32_t o[32];                                  // G channels x T elements = 128 bytes
 #pragma unroll
@@ -471,10 +415,8 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
                     float v[T];
 #pragma unroll
                     for (int p = 0; p < T; ++p) v[p] = __uint_as_float(in[p][g]);
-#ifndef EQL_ABLATE_EPIMATH
                     if (prm.bias != nullptr && co0 + g < prm.Cout) v[0] += __ldg(prm.bias + co0 + g);
                     rdft_inverse<T>(v);
-#endif
                     if constexpr (E == 2) {
 #pragma unroll
                         for (int t = 0; t < T; t += 2) o[(g * T + t) / 2] = pack_h2(v[t], v[t + 1]);
@@ -483,9 +425,6 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
                         for (int t = 0; t < T; ++t) o[g * T + t] = __float_as_uint(v[t]);
                     }
                 }
-#ifdef EQL_TRACE
-                if (tre) { if (o[0] == 0x7fc12345u) EQL_STAMP(te + 3); EQL_STAMP(te + 2); }
-#endif
                 // stage the warp's 32 rows of 128 bytes (chunk j of row l at j ^ (l & 7): the tensor map's 128B swizzle) and
                 // hand them to one asynchronous TMA store; rows >= N and channels >= Cout are clipped by the hardware
                 if (lane == 0) ptx::bulk_wait_group_read0();     // previous group's stage has been read
@@ -509,15 +448,11 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
                 ptx::mbar_arrive(&bar->staging_free);
             }
             staging_pending = true;
-#ifdef EQL_TRACE
-            if (cw == 0 && lane == 0 && cu < 4) EQL_STAMP(7000 + 16 * (int)cu + 15);
-#endif
             if (third >= ngroups) {                              // fewer column groups than shares: nothing to read
                 ptx::tc_fence_before_sync();
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(&bar->empty_d);
             }
-            if (cw == 0 && lane == 0) EQL_STAMP(8 * cu + 3);
         }
     }
 
@@ -585,16 +520,6 @@ int umma_max_cot(int T, int elem_bytes) {
 
 }  // namespace
 
-#ifdef EQL_TRACE
-extern "C" int eqlinear_debug_read_trace(unsigned long long* dst, int n) {
-    cudaDeviceSynchronize();
-    return (int)cudaMemcpyFromSymbol(dst, g_trace, sizeof(unsigned long long) * (n < 8192 ? n : 8192));
-}
-extern "C" int eqlinear_debug_clear_trace() {
-    static unsigned long long zeros[8192];
-    return (int)cudaMemcpyToSymbol(g_trace, zeros, sizeof(zeros));
-}
-#endif
 
 bool umma_linear_supported(int T, eql_dtype_t dtype) {
     if (dtype == EQL_FP16) return T == 4 || T == 8 || T == 16 || T == 32;
@@ -692,15 +617,8 @@ cudaError_t launch_umma_linear(const UmmaLinearShape& s, const void* in, void* o
         constexpr int TT = decltype(tc)::value;
         using IO = decltype(io);
         const size_t smem = umma_smem_bytes<TT, sizeof(IO)>(prm.b_slot_bytes);
-        static unsigned long long attr_done = 0;              // one bit per device (per instantiation)
-        int dev = 0;
-        cudaGetDevice(&dev);
-        if (!((attr_done >> (dev & 63)) & 1ull)) {
-            cudaError_t e = cudaFuncSetAttribute(umma_linear_kernel<TT, IO>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                 227 * 1024);
-            if (e != cudaSuccess) return e;
-            attr_done |= 1ull << (dev & 63);
-        }
+        static SmemLimitOnce smem_limit;                      // per kernel instantiation
+        if (cudaError_t e = smem_limit.ensure(umma_linear_kernel<TT, IO>, 227 * 1024); e != cudaSuccess) return e;
         if (smem > 227 * 1024) return cudaErrorInvalidConfiguration;
         umma_linear_kernel<TT, IO><<<grid, kThreadsUmma, smem, stream>>>(tmap, tmap_out, prm);
         return cudaGetLastError();

@@ -72,13 +72,6 @@ struct ResParams {
     int64_t st_chunks;           // 16-token chunks in all
 };
 
-// Optional timeline instrumentation (compiled only with -DEQL_TRACE): CTA 0 records clock64() stamps.
-#ifdef EQL_TRACE
-__device__ unsigned long long g_trace_res[8192];
-#define RES_STAMP(slot) do { if (blockIdx.x == 0 && (slot) < 8192) g_trace_res[(slot)] = clock64(); } while (0)
-#else
-#define RES_STAMP(slot) do { } while (0)
-#endif
 
 struct ResBarriers {
     uint64_t full_raw[kResComputeWarps], empty_raw[kResComputeWarps];
@@ -259,11 +252,9 @@ umma_linear_res_kernel(const __grid_constant__ CUtensorMap tmap_in, const ResPar
                 if (ct == nCT) ct = 0;
                 const bool first = first_of_tile(u, ct), last = last_of_tile(u, ct);
                 if (first && u != u0) ++tc;
-                RES_STAMP(512 + 2 * cu);
                 const uint32_t buf = cu % NBUF;
                 const uint32_t dbase = tmem_base + buf * (uint32_t)(T * NTOK);
                 ok = ptx::mbar_wait(&bar->empty_d[buf], ((cu / NBUF) & 1) ^ 1, abort_flag, status, 303, true, kResSpin);
-                RES_STAMP(512 + 2 * cu + 1);
                 if (!ok) break;
                 // x^ buffer and phase of the tile's chunk 0: chunk kc of the CTA's tc-th tile has running number tc*nK + kc
                 // (resident mode has XR == nK: buffer = chunk index, phase = tile parity, no division)
@@ -274,7 +265,6 @@ umma_linear_res_kernel(const __grid_constant__ CUtensorMap tmap_in, const ResPar
                 if constexpr (!merged) ok = ok && ptx::mbar_wait(&bar->full_w[slot], wph, abort_flag, status, 305, true, kResSpin);
                 if (!ok) break;
                 for (int kc = 0; kc < nK; ++kc) {
-                    RES_STAMP(1024 + 4 * (cu * nK + kc));
                     ptx::tc_fence_after_sync();
                     const uint64_t a0 = ptx::umma_smem_desc_k_sw32(ptx::smem_u32(wsm + slot * kWSlot));      // weight tiles, plane p at p * 4 KB
                     const uint64_t b0 = ptx::umma_smem_desc_k_sw32(ptx::smem_u32(xhat + xs * kXChunkBytes)); // x^ tiles, plane p at p * XT
@@ -303,16 +293,13 @@ umma_linear_res_kernel(const __grid_constant__ CUtensorMap tmap_in, const ResPar
                         if (f == 1 && kc + 1 < nK) {
                             // The next chunk's operands are checked here, while the tensor pipe still has this chunk's
                             // MMAs queued, so that the issue stream has no gap between chunks.
-                            RES_STAMP(1024 + 4 * (cu * nK + kc) + 1);
                             if (first) ok = ptx::mbar_wait(&bar->full_x[nxs], nxph, abort_flag, status, 304, true, kResSpin);
                             if constexpr (!merged) ok = ok && ptx::mbar_wait(&bar->full_w[nslot], nwph, abort_flag, status, 305, true, kResSpin);
-                            RES_STAMP(1024 + 4 * (cu * nK + kc) + 2);
                         }
                     }
                     mma(dbase + (uint32_t)((T - 1) * NTOK), a0 + (T - 1) * kWTileD, b0 + (XTILES - 1) * kXTileD, idesc1, acc);  // k = T/2
                     if constexpr (!merged) ptx::umma_commit(&bar->empty_w[slot]);
                     if (last) ptx::umma_commit(&bar->empty_x[xs]);  // the x^ buffer may be overwritten once these MMAs retire
-                    RES_STAMP(1024 + 4 * (cu * nK + kc) + 3);
                     slot = nslot; wph = nwph;
                     xs = nxs; xph = nxph;
                     if (!ok) break;
@@ -417,7 +404,6 @@ umma_linear_res_kernel(const __grid_constant__ CUtensorMap tmap_in, const ResPar
         int64_t tt = tt0;
         for (int64_t u = u0; u < u1 && ok; ++u, ++cu, ++ct) {
             if (ct == nCT) { ct = 0; ++tt; }
-            if (cw == 0 && lane == 0) RES_STAMP(8 * cu);
             // ring of x^ buffers (one channel tile): the rest of this tile's chunks, consumed by its MMAs as they arrive
             if (first_of_tile(u, ct)) {
                 transform_tile(tc, pre, nK, tt * NTOK);
@@ -429,7 +415,6 @@ umma_linear_res_kernel(const __grid_constant__ CUtensorMap tmap_in, const ResPar
                 transform_tile(tc, 0, pre, (tt + 1) * NTOK);
                 if (!ok) break;
             }
-            if (cw == 0 && lane == 0) RES_STAMP(8 * cu + 1);
             // ---- epilogue of unit u: thread = output channel, columns = (plane, token)
             const int64_t row0 = tt * NTOK;
             const int o = ct * 128 + quad * 32 + lane;
@@ -441,7 +426,6 @@ umma_linear_res_kernel(const __grid_constant__ CUtensorMap tmap_in, const ResPar
             const uint32_t acc_base = lane_base + buf * (uint32_t)(T * NTOK);
             ok = ptx::mbar_wait(&bar->full_d[buf], (cu / NBUF) & 1, abort_flag, status, 308, true, 16);
             if (!ok) break;
-            if (cw == 0 && lane == 0) RES_STAMP(8 * cu + 2);
             ptx::tc_fence_after_sync();
             constexpr int NG = NTOK / 8;                         // groups of 8 tokens
             for (int g = third; g < NG; g += kResShares) {
@@ -480,7 +464,6 @@ umma_linear_res_kernel(const __grid_constant__ CUtensorMap tmap_in, const ResPar
                 if (o_ok && rows_left >= 8) emit(std::true_type{});
                 else emit(std::false_type{});
             }
-            if (cw == 0 && lane == 0) RES_STAMP(8 * cu + 4);
         }
     }
 
@@ -521,16 +504,6 @@ size_t res_smem_bytes(int T, int nTok, bool paired, int x_slots, int w_slots, in
 
 }  // namespace
 
-#ifdef EQL_TRACE
-extern "C" int eqlinear_debug_read_trace_res(unsigned long long* dst, int n) {
-    cudaDeviceSynchronize();
-    return (int)cudaMemcpyFromSymbol(dst, g_trace_res, sizeof(unsigned long long) * (n < 8192 ? n : 8192));
-}
-extern "C" int eqlinear_debug_clear_trace_res() {
-    static unsigned long long zeros[8192];
-    return (int)cudaMemcpyToSymbol(g_trace_res, zeros, sizeof(zeros));
-}
-#endif
 
 bool umma_res_supported(int T, eql_dtype_t dtype) { return dtype == EQL_FP16 && (T == 4 || T == 8); }
 
@@ -620,15 +593,8 @@ cudaError_t launch_umma_linear_res(const UmmaResShape& s, const void* in, void* 
     auto go = [&](auto tc, auto nt, auto pf, auto mg) -> cudaError_t {
         constexpr int TT = decltype(tc)::value, NT = decltype(nt)::value;
         constexpr bool PF = decltype(pf)::value, MG = decltype(mg)::value;
-        static unsigned long long attr_done = 0;
-        int dev = 0;
-        cudaGetDevice(&dev);
-        if (!((attr_done >> (dev & 63)) & 1ull)) {
-            cudaError_t e = cudaFuncSetAttribute(umma_linear_res_kernel<TT, NT, PF, MG>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                 (int)kResSmemLimit);
-            if (e != cudaSuccess) return e;
-            attr_done |= 1ull << (dev & 63);
-        }
+        static SmemLimitOnce smem_limit;                      // per kernel instantiation
+        if (cudaError_t e = smem_limit.ensure(umma_linear_res_kernel<TT, NT, PF, MG>, (int)kResSmemLimit); e != cudaSuccess) return e;
         umma_linear_res_kernel<TT, NT, PF, MG><<<grid, ResWarps<TT>::kThreads, smem, stream>>>(tmap, prm);
         return cudaGetLastError();
     };

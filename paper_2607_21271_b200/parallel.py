@@ -48,3 +48,48 @@ def allreduce_weight_grads(dw, db=None, group=None, flat=None, async_op=False):
     if db is not None:
         dist.all_reduce(db, op=dist.ReduceOp.SUM, group=group)
     return None
+
+
+def dp_training_step(fwd, weight_grad, data_grad, flat, group=None, side_stream=None, mark=None):
+    """One data-parallel training step of the layer, in the order that hides its one exchange step.
+
+    forward -> weight gradient -> START the all-reduce of the flat dw|db buffer -> data gradient -> wait for the
+    collective.  The weight gradient goes first because it is the only result other ranks need; its sum over ranks then
+    travels while the data gradient (which needs no exchange) is computed, and the step ends only once the summed
+    gradients are in place.  `fwd`, `weight_grad` and `data_grad` are callables that enqueue (GPU) or run (CPU) the
+    three passes.  On CUDA, pass `side_stream`: the collective is issued there behind an event recorded after the
+    weight gradient, so that it overlaps the data-gradient kernel, and the current stream waits for it at the end.
+    `mark(i)`, if given, is called at the phase boundaries (0: start, 1: after fwd, 2: after the weight gradient and the
+    start of the exchange, 3: after the data gradient) so that a caller can record timing events.
+    Returns the list of phase names in the order they ran."""
+    import torch
+
+    order = []
+    if mark:
+        mark(0)
+    fwd()
+    order.append("fwd")
+    if mark:
+        mark(1)
+    weight_grad()
+    order.append("bwd_weight")
+    work = None
+    if side_stream is not None:
+        ready = torch.cuda.Event()
+        ready.record()
+        with torch.cuda.stream(side_stream):
+            side_stream.wait_event(ready)
+            work = allreduce_weight_grads(None, None, group=group, flat=flat, async_op=True)
+    else:
+        work = allreduce_weight_grads(None, None, group=group, flat=flat, async_op=True)
+    order.append("allreduce_start")
+    if mark:
+        mark(2)
+    data_grad()
+    order.append("bwd_data")
+    if mark:
+        mark(3)
+    if work is not None:
+        work.wait()                     # CUDA: the current stream waits for the collective; CPU: blocks until it is done
+    order.append("allreduce_done")
+    return order

@@ -65,7 +65,7 @@ OPERATOR_SHAPES = {
     **{f"op_c{c}_fp16": Workload(f"op_c{c}_fp16", "fp16", 4, c, c, 32 * 1024, "normal", _FB, 5)
        for c in (16, 64, 256, 512, 1024, 2048)},
     **{f"op_c{c}_fp32": Workload(f"op_c{c}_fp32", "fp32", 4, c, c, 32 * 1024, "normal", _FB, 5)
-       for c in (16, 64, 256)},
+       for c in (16, 64, 256, 512, 1024, 2048)},
 }
 
 ALL_WORKLOADS = {**CONFIGS, **OPERATOR_SHAPES}

@@ -79,7 +79,8 @@ def test_fp32_long_reductions_stay_inside_the_bar(T, Ci, Co, N):
 
 
 # ------------------------------------------------------------------ the paper's operator-benchmark shapes (Tables 1-2)
-@pytest.mark.parametrize("name", ["op_c64_fp16", "op_c256_fp16", "op_c1024_fp16", "op_c64_fp32", "op_c256_fp32"])
+@pytest.mark.parametrize("name", ["op_c16_fp16", "op_c64_fp16", "op_c256_fp16", "op_c512_fp16", "op_c1024_fp16", "op_c2048_fp16",
+                                  "op_c16_fp32", "op_c64_fp32", "op_c256_fp32", "op_c512_fp32"])
 def test_operator_benchmark_shapes_on_sampled_outputs(name):
     """32 x 1024 tokens, T = 4, c channels per group element on both sides: the GPU runs the full size; the oracle
     computes a sample of it one piece at a time - sampled token rows x sampled output channels of y (the dense weight
@@ -169,6 +170,41 @@ def test_saved_spectrum_path_matches_oracle(T, Ci, Co, N):
         assert rel_max_err(outs[0][0], rdw) <= TOL["fp16"]
         assert rel_max_err(outs[0][1], rdb) <= TOL["fp16"]
         assert np.array_equal(outs[0][0], outs[1][0]) and np.array_equal(outs[0][1], outs[1][1])
+    finally:
+        layer.close()
+
+
+def test_benchmarked_step_sequence_at_full_size():
+    """The call sequence bench.py times on the headline workload, at its full size (N = 25 216): eqlinear_fwd_save_spectrum,
+    eqlinear_bwd_data, eqlinear_bwd_weight_from_spectrum, every output against the oracle."""
+    wl = CONFIGS["vit_b_fc1_fp16"]
+    d = generate(wl)
+    T, Ci, Co, N = wl.T, wl.Ci, wl.Co, wl.N
+    layer = GpuLayer(T, Ci, Co, "fp16", d["w"], d["bias"])
+    try:
+        info = eq.eqlinear_plan_info(layer.plan)
+        assert (info.fwd_kernel, info.bwd_data_kernel, info.bwd_weight_kernel) == (2, 2, 1)
+        x, dy = torch.from_numpy(d["x"]).cuda(), torch.from_numpy(d["dy"]).cuda()
+        sb = eq.eqlinear_spectrum_bytes(layer.plan, N)
+        spec = torch.full((sb + 64,), 0x7F, dtype=torch.uint8, device="cuda")
+        y = torch.empty(N, Co * T, dtype=torch.float16, device="cuda")
+        dx = torch.empty(N, Ci * T, dtype=torch.float16, device="cuda")
+        dw = torch.full((Co, Ci, T), float("nan"), dtype=torch.float32, device="cuda")
+        db = torch.full((Co,), float("nan"), dtype=torch.float32, device="cuda")
+        scb = eq.eqlinear_bwd_weight_scratch_bytes(layer.plan, N)
+        sc = torch.empty(scb, dtype=torch.uint8, device="cuda")
+        eq.eqlinear_fwd_save_spectrum(layer.plan, x, y, N, spec, sb, layer.stream)
+        eq.eqlinear_bwd_data(layer.plan, dy, dx, N, layer.stream)
+        eq.eqlinear_bwd_weight_from_spectrum(layer.plan, spec, sb, dy, dw, db, N, sc, scb, layer.stream)
+        assert layer.raw_status() == 0
+        assert bool((spec[sb:] == 0x7F).all().item())
+        rdw, rdb = orc.bwd_weight(d["x"], d["dy"], T)
+        errs = {"y": rel_max_err(y.cpu().numpy(), orc.fwd(d["x"], d["w"], d["bias"])),
+                "dx": rel_max_err(dx.cpu().numpy(), orc.bwd_data(d["dy"], d["w"])),
+                "dw": rel_max_err(dw.cpu().numpy(), rdw), "db": rel_max_err(db.cpu().numpy(), rdb)}
+        print({k: f"{v:.2e}" for k, v in errs.items()})
+        for k, v in errs.items():
+            assert v <= TOL["fp16"], f"{k} error {v:.3e}"
     finally:
         layer.close()
 
@@ -287,6 +323,35 @@ def test_runtime_argument_errors():
         assert (info.T, info.C_in, info.C_out) == (4, 8, 8)
         assert info.macs_per_token == 6 * 8 * 8 and info.dense_macs_per_token == 32 * 32
         assert info.bytes_per_token_fwd == (8 + 8) * 4 * 4
+    finally:
+        layer.close()
+
+
+def test_plan_is_refused_on_another_device():
+    """A plan's workspace and tensor maps belong to the GPU it was built on: with another device current every entry
+    point that takes the plan must return EQL_ERR_INVALID_ARG before launching anything (needs two GPUs)."""
+    if torch.cuda.device_count() < 2:
+        pytest.skip("needs a second GPU to make another device current")
+    wl = Workload("dev", "fp16", 8, 24, 40, 64, "normal", ("fwd",), 28)
+    d = generate(wl)
+    layer = GpuLayer(wl.T, wl.Ci, wl.Co, wl.dtype, d["w"], d["bias"])
+    lib, B = eq.load_library(), eq.binding
+    try:
+        x = torch.zeros(64, wl.Din, dtype=torch.float16, device="cuda:0")
+        y = torch.full((64, wl.Dout), -5.0, dtype=torch.float16, device="cuda:0")
+        dw = torch.zeros(wl.Co * wl.Ci * wl.T, dtype=torch.float32, device="cuda:0")
+        sc = torch.zeros(1 << 20, dtype=torch.uint8, device="cuda:0")
+        p = layer.plan
+        with torch.cuda.device(1):
+            assert lib.eqlinear_fwd(p, x.data_ptr(), y.data_ptr(), 64, None) == B.EQL_ERR_INVALID_ARG
+            assert lib.eqlinear_bwd_data(p, y.data_ptr(), x.data_ptr(), 64, None) == B.EQL_ERR_INVALID_ARG
+            assert lib.eqlinear_bwd_weight(p, x.data_ptr(), y.data_ptr(), dw.data_ptr(), None, 64, sc.data_ptr(), 1 << 20,
+                                           None) == B.EQL_ERR_INVALID_ARG
+            assert lib.eqlinear_bwd_weight_static(p, x.data_ptr(), y.data_ptr(), dw.data_ptr(), None, 64, None) == B.EQL_ERR_INVALID_ARG
+            assert lib.eqlinear_plan_set_weight(p, layer.w.data_ptr(), layer.bias.data_ptr(), None) == B.EQL_ERR_INVALID_ARG
+            assert lib.eqlinear_plan_device_status(p, None) == B.EQL_ERR_INVALID_ARG
+        torch.cuda.synchronize()
+        assert bool((y == -5.0).all().item())                                          # nothing ran
     finally:
         layer.close()
 

@@ -58,6 +58,54 @@ def _flat_worker(rank, world, port, out_dir):
     dist.destroy_process_group()
 
 
+def _step_worker(rank, world, port, out_dir):
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    wl = Workload("dp", "fp32", 4, 6, 5, 203, "normal", ("fwd", "bwd_data", "bwd_weight"), 31)
+    d = generate(wl)
+    b, e = parallel.shard_tokens(wl.N, rank, world)
+    flat, dw, db = parallel.grad_buffers(wl.Co, wl.Ci, wl.T, "cpu")
+    out, seen = {}, []
+
+    def fwd():
+        out["y"] = orc.fwd(d["x"][b:e], d["w"], d["bias"])
+
+    def weight_grad():
+        g, s = orc.bwd_weight(d["x"][b:e], d["dy"][b:e], wl.T)
+        dw.copy_(torch.from_numpy(g)); db.copy_(torch.from_numpy(s))
+        out["local_dw"] = g.copy()
+
+    def data_grad():
+        out["dx"] = orc.bwd_data(d["dy"][b:e], d["w"])
+
+    order = parallel.dp_training_step(fwd, weight_grad, data_grad, flat, mark=seen.append)
+    np.savez(os.path.join(out_dir, f"step{rank}.npz"), y=out["y"], dx=out["dx"], dw=dw.numpy(), db=db.numpy(),
+             local_dw=out["local_dw"], order=np.array(order), marks=np.array(seen))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_dp_step_orders_the_exchange_before_the_data_gradient(tmp_path):
+    """The N > 1 step of bench.py: weight gradient first, the all-reduce started before the data gradient and joined
+    before the step returns; every rank ends with the gradients summed over all tokens."""
+    world, port = 2, 33500 + os.getpid() % 2000
+    mp.spawn(_step_worker, args=(world, port, str(tmp_path)), nprocs=world, join=True)
+    wl = Workload("dp", "fp32", 4, 6, 5, 203, "normal", ("fwd", "bwd_data", "bwd_weight"), 31)
+    d = generate(wl)
+    ref_dw, ref_db = orc.bwd_weight(d["x"], d["dy"], wl.T)
+    parts = [np.load(tmp_path / f"step{r}.npz") for r in range(world)]
+    for p in parts:
+        assert list(p["order"]) == ["fwd", "bwd_weight", "allreduce_start", "bwd_data", "allreduce_done"]
+        assert list(p["marks"]) == [0, 1, 2, 3]
+        # (the exchange buffer is float32, as the library's dw / db are)
+        assert np.allclose(p["dw"], ref_dw, rtol=0, atol=1e-5 * np.abs(ref_dw).max())
+        assert np.allclose(p["db"], ref_db, rtol=0, atol=1e-5 * np.abs(ref_db).max())
+        assert not np.allclose(p["local_dw"], ref_dw, rtol=0, atol=1e-2 * np.abs(ref_dw).max())      # the sum really needed the other rank
+    assert np.allclose(np.concatenate([p["y"] for p in parts]), orc.fwd(d["x"], d["w"], d["bias"]), rtol=0, atol=1e-12)
+    assert np.allclose(np.concatenate([p["dx"] for p in parts]), orc.bwd_data(d["dy"], d["w"]), rtol=0, atol=1e-12)
+
+
 def test_flat_gradient_buffer_is_reduced_in_one_call(tmp_path):
     world, port = 2, 31500 + os.getpid() % 2000
     mp.spawn(_flat_worker, args=(world, port, str(tmp_path)), nprocs=world, join=True)
