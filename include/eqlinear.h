@@ -66,14 +66,18 @@ enum {
     /* Among the tensor-core kernels, always take the streaming one (activations transformed per
      * output-channel tile) even where the kernel that keeps the transformed activations of a token
      * tile resident in shared memory applies.  For comparisons and tests. */
-    EQL_FLAG_FORCE_STREAMING = 4u
+    EQL_FLAG_FORCE_STREAMING = 4u,
+    /* Never take the CTA-pair form of the streaming kernel (two SMs sharing each spectral-weight tile through
+     * tcgen05 cta_group::2), which plans of wide FP16 layers select.  For comparisons and tests. */
+    EQL_FLAG_NO_CTA_PAIR = 8u
 };
 
 typedef struct {
     int32_t T, C_in, C_out, dtype;
     uint32_t flags;
     int32_t fwd_kernel;           /* 0 = CUDA-core FFMA kernel, 1 = tcgen05 streaming kernel,
-                                     2 = tcgen05 kernel with resident transformed activations */
+                                     2 = tcgen05 kernel with resident transformed activations,
+                                     3 = tcgen05 streaming kernel run by CTA pairs (cta_group::2) */
     int32_t bwd_data_kernel;
     int32_t bwd_weight_kernel;
     int64_t macs_per_token;       /* Step-2 multiply-accumulates of Algorithm 1 per token, exact count */

@@ -85,8 +85,12 @@ struct UmmaLinearShape {
     size_t image_bytes;
     // A shape may describe one SEGMENT of a layer's reduction: input channels [cin0, cin0 + Cin) of CinTotal.
     int cin0, CinTotal;
+    // CTA-pair form (tcgen05 cta_group::2): two CTAs on two SMs share every weight tile, half each; the operand image is
+    // laid out for it, so a shape is either one or the other.
+    bool pair;
 };
 bool umma_linear_supported(int T, eql_dtype_t dtype);
+bool umma_linear_pair_supported(int T, eql_dtype_t dtype);
 UmmaLinearShape umma_linear_shape(int T, int Cin, int Cout, eql_dtype_t dtype);
 // FP32 plans reduce at most kFp32SegmentChannels channels in one TMEM accumulator (the tensor core adds with
 // truncation, so the error is linear in the accumulation depth); longer reductions run as several launches whose

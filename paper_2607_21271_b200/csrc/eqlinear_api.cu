@@ -39,6 +39,9 @@ namespace {
 using namespace eql;
 
 inline size_t elem_size(eql_dtype_t d) { return d == EQL_FP32 ? 4 : 2; }
+
+// Where the CTA-pair form of the streaming kernel is taken (reduced channels Cin, produced channels Cout).
+inline bool pair_pays(int Cin, int Cout) { (void)Cin; (void)Cout; return true; }
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 eql_status_t check_shape(int T, int Ci, int Co, int dtype) {
@@ -63,24 +66,25 @@ eql_status_t build_weights(eqlinear_plan_t p, const void* w, const void* bias, c
                                         (float*)(p->ws + p->lay.bias), s);
     if (e != cudaSuccess) return EQL_ERR_CUDA;
     // streaming kernel: one operand image per segment of the reduction (one segment except for wide FP32 layers)
-    auto build_segments = [&](int Cin, int Cout, size_t planes_off, size_t image_off) -> cudaError_t {
+    auto build_segments = [&](int Cin, int Cout, size_t planes_off, size_t image_off, bool pair) -> cudaError_t {
         int len = 0;
         const int nseg = umma_reduction_segments(Cin, p->dtype, &len);
         size_t off = 0;
         for (int k = 0; k < nseg; ++k) {
-            const UmmaLinearShape sh = umma_linear_segment(p->T, Cin, Cout, p->dtype, k, len);
+            UmmaLinearShape sh = umma_linear_segment(p->T, Cin, Cout, p->dtype, k, len);
+            sh.pair = pair;
             cudaError_t err = launch_build_umma_image(sh, (const float*)(p->ws + planes_off), p->ws + image_off + off, s);
             if (err != cudaSuccess) return err;
             off += sh.image_bytes;
         }
         return cudaSuccess;
     };
-    if (p->fwd_kernel == 1) {
-        e = build_segments(p->Ci, p->Co, p->lay.planes_fwd, p->lay.umma_fwd);
+    if (p->fwd_kernel == 1 || p->fwd_kernel == 3) {
+        e = build_segments(p->Ci, p->Co, p->lay.planes_fwd, p->lay.umma_fwd, p->fwd_kernel == 3);
         if (e != cudaSuccess) return EQL_ERR_CUDA;
     }
-    if (p->bwd_data_kernel == 1) {
-        e = build_segments(p->Co, p->Ci, p->lay.planes_bwd, p->lay.umma_bwd);
+    if (p->bwd_data_kernel == 1 || p->bwd_data_kernel == 3) {
+        e = build_segments(p->Co, p->Ci, p->lay.planes_bwd, p->lay.umma_bwd, p->bwd_data_kernel == 3);
         if (e != cudaSuccess) return EQL_ERR_CUDA;
     }
     if (p->fwd_kernel == 2) {
@@ -97,12 +101,13 @@ eql_status_t build_weights(eqlinear_plan_t p, const void* w, const void* bias, c
 // Streaming tensor-core kernel over every segment of the reduction: the first launch writes out = bias + its share,
 // the others add theirs (one launch in all except for FP32 layers with more than 256 reduced channels).
 cudaError_t run_streaming(eqlinear_plan_t p, int Cin, int Cout, const void* in, void* out, int64_t N, size_t image_off,
-                          const float* bias, cudaStream_t s) {
+                          const float* bias, cudaStream_t s, bool pair) {
     int len = 0;
     const int nseg = umma_reduction_segments(Cin, p->dtype, &len);
     size_t off = 0;
     for (int k = 0; k < nseg; ++k) {
-        const UmmaLinearShape sh = umma_linear_segment(p->T, Cin, Cout, p->dtype, k, len);
+        UmmaLinearShape sh = umma_linear_segment(p->T, Cin, Cout, p->dtype, k, len);
+        sh.pair = pair;
         cudaError_t e = launch_umma_linear(sh, in, out, N, p->ws + image_off + off, k == 0 ? bias : nullptr,
                                            (int*)(p->ws + p->lay.status), p->num_sms, s, k > 0);
         if (e != cudaSuccess) return e;
@@ -240,7 +245,8 @@ eql_status_t eqlinear_plan(eqlinear_plan_t* plan, int T, int C_in, int C_out, eq
     eql_status_t st = check_shape(T, C_in, C_out, dtype);
     if (st != EQL_OK) return st;
     if (!w || !workspace) return EQL_ERR_INVALID_ARG;
-    if (flags & ~(unsigned)(EQL_FLAG_CORRELATION | EQL_FLAG_FORCE_SIMT | EQL_FLAG_FORCE_STREAMING)) return EQL_ERR_INVALID_ARG;
+    if (flags & ~(unsigned)(EQL_FLAG_CORRELATION | EQL_FLAG_FORCE_SIMT | EQL_FLAG_FORCE_STREAMING | EQL_FLAG_NO_CTA_PAIR))
+        return EQL_ERR_INVALID_ARG;
     if (!aligned16(w) || (bias && !aligned16(bias))) return EQL_ERR_ALIGNMENT;
     if (reinterpret_cast<uintptr_t>(workspace) % kWsAlign != 0) return EQL_ERR_ALIGNMENT;
     WorkspaceLayout lay = workspace_layout(T, C_in, C_out, dtype);
@@ -278,6 +284,11 @@ eql_status_t eqlinear_plan(eqlinear_plan_t* plan, int T, int C_in, int C_out, eq
             p->res_bwd = umma_res_shape(T, C_out, C_in);
             if (prefer(p->res_fwd)) p->fwd_kernel = 2;
             if (prefer(p->res_bwd)) p->bwd_data_kernel = 2;
+        }
+        // Wide layers on the streaming kernel: its CTA-pair form, in which two SMs share every weight tile.
+        if (umma_linear_pair_supported(T, dtype) && !(flags & EQL_FLAG_NO_CTA_PAIR)) {
+            if (p->fwd_kernel == 1 && pair_pays(C_in, C_out)) p->fwd_kernel = 3;
+            if (p->bwd_data_kernel == 1 && pair_pays(C_out, C_in)) p->bwd_data_kernel = 3;
         }
     }
 
@@ -325,8 +336,8 @@ eql_status_t eqlinear_plan_launch_counts(eqlinear_plan_t plan, int64_t N, int32_
     counts[0] = counts[1] = counts[2] = counts[3] = 0;
     if (N == 0) return EQL_OK;
     int len = 0;
-    counts[0] = plan->fwd_kernel == 1 ? umma_reduction_segments(plan->Ci, plan->dtype, &len) : 1;
-    counts[1] = plan->bwd_data_kernel == 1 ? umma_reduction_segments(plan->Co, plan->dtype, &len) : 1;
+    counts[0] = (plan->fwd_kernel == 1 || plan->fwd_kernel == 3) ? umma_reduction_segments(plan->Ci, plan->dtype, &len) : 1;
+    counts[1] = (plan->bwd_data_kernel == 1 || plan->bwd_data_kernel == 3) ? umma_reduction_segments(plan->Co, plan->dtype, &len) : 1;
     if (plan->bwd_weight_kernel == 1) {
         const UmmaBwdWeightShape bs = umma_bwd_weight_shape(plan->T, plan->Ci, plan->Co, plan->dtype, N, plan->num_sms);
         const int64_t blocks = (N + bs.block_tokens - 1) / bs.block_tokens;
@@ -368,8 +379,9 @@ eql_status_t eqlinear_fwd(eqlinear_plan_t plan, const void* x, void* y, int64_t 
                                                (int*)(plan->ws + plan->lay.status), plan->num_sms, (cudaStream_t)stream);
         return e == cudaSuccess ? EQL_OK : EQL_ERR_CUDA;
     }
-    if (plan->fwd_kernel == 1) {
-        cudaError_t e = run_streaming(plan, plan->Ci, plan->Co, x, y, N, plan->lay.umma_fwd, bias, (cudaStream_t)stream);
+    if (plan->fwd_kernel == 1 || plan->fwd_kernel == 3) {
+        cudaError_t e = run_streaming(plan, plan->Ci, plan->Co, x, y, N, plan->lay.umma_fwd, bias, (cudaStream_t)stream,
+                                      plan->fwd_kernel == 3);
         return e == cudaSuccess ? EQL_OK : EQL_ERR_CUDA;
     }
     cudaError_t e = launch_direct_linear(plan->T, plan->dtype, x, y, N, plan->Ci, plan->Co,
@@ -389,8 +401,9 @@ eql_status_t eqlinear_bwd_data(eqlinear_plan_t plan, const void* dy, void* dx, i
                                                (int*)(plan->ws + plan->lay.status), plan->num_sms, (cudaStream_t)stream);
         return e == cudaSuccess ? EQL_OK : EQL_ERR_CUDA;
     }
-    if (plan->bwd_data_kernel == 1) {
-        cudaError_t e = run_streaming(plan, plan->Co, plan->Ci, dy, dx, N, plan->lay.umma_bwd, nullptr, (cudaStream_t)stream);
+    if (plan->bwd_data_kernel == 1 || plan->bwd_data_kernel == 3) {
+        cudaError_t e = run_streaming(plan, plan->Co, plan->Ci, dy, dx, N, plan->lay.umma_bwd, nullptr, (cudaStream_t)stream,
+                                      plan->bwd_data_kernel == 3);
         return e == cudaSuccess ? EQL_OK : EQL_ERR_CUDA;
     }
     cudaError_t e = launch_direct_linear(plan->T, plan->dtype, dy, dx, N, plan->Co, plan->Ci,

@@ -14,6 +14,13 @@
 // Frequency-domain data never leaves the SM (registers, shared memory, TMEM).  The data gradient is the
 // same kernel run on dy with the conjugate-transposed weight image and no bias.
 //
+// CG = 2 ("CTA pair"): the same kernel as a cluster of two CTAs on two SMs that work on two neighbouring token tiles
+// and the same output-channel tile in lockstep.  One tcgen05.mma.cta_group::2 (M = 256) issued by the pair's leader
+// covers both token tiles; its B operand -- the spectral weight tile -- is split in halves between the two CTAs, so
+// each SM loads, holds and feeds to the tensor core only half of every weight tile.  On wide layers, whose main loop
+// is bound by shared-memory and L2 -> SM traffic, that is where the time goes.  Each CTA issues its own loads into its
+// own shared memory; only mbarrier arrivals cross the pair.
+//
 // Every wait on an mbarrier is bounded: on a time-out the CTA raises an abort flag, records a status
 // code for the host, drains its outstanding copies and MMAs, frees its TMEM and returns.
 #include <cuda_fp16.h>
@@ -39,7 +46,7 @@ constexpr int kTmemCols = 512;
 constexpr int kWarpTmaX = 0, kWarpMma = 1, kWarpTmaB = 2, kWarpCompute0 = 4;
 constexpr int kNumComputeWarps = 12;
 
-template <int T, int E> struct UmmaCfg;          // E = bytes per element of the I/O tensors (2: half, 4: float)
+template <int T, int E, int CG = 1> struct UmmaCfg;   // E = bytes per element of the I/O tensors (2: half, 4: float); CG: CTAs per MMA
 // Ring depths.  The raw ring has 3 slots of SPS slabs (16 KB each) that complete on one barrier; with 3 slots every
 // slot is always served by the same warp groups (slab number mod 3 selects the group).  SA transformed-operand
 // stages (T*4 KB each, twice that for the hi/lo halves of FP32), SB weight-image slots.  Measured on the EQ-ViT-B
@@ -48,12 +55,19 @@ template <int T, int E> struct UmmaCfg;          // E = bytes per element of the
 // EARLY: release a raw slot as soon as its rows are in registers (one more fence + arrive per item) instead of after
 // the transformed rows have been stored; used where the raw ring cannot be deep.
 // MAXCOT: output channels per tile (T*CoT fp32 TMEM columns <= 512, and the weight-image slot must fit).
-template <> struct UmmaCfg<4, 2>  { static constexpr int SPS = 2, SA = 4, SB = 2, MAXCOT = 128; static constexpr bool EARLY = false; };
-template <> struct UmmaCfg<8, 2>  { static constexpr int SPS = 2, SA = 2, SB = 2, MAXCOT = 64;  static constexpr bool EARLY = false; };
-template <> struct UmmaCfg<16, 2> { static constexpr int SPS = 1, SA = 2, SB = 1, MAXCOT = 32;  static constexpr bool EARLY = true; };
-template <> struct UmmaCfg<32, 2> { static constexpr int SPS = 1, SA = 1, SB = 1, MAXCOT = 16;  static constexpr bool EARLY = true; };
-template <> struct UmmaCfg<4, 4>  { static constexpr int SPS = 1, SA = 3, SB = 1, MAXCOT = 128; static constexpr bool EARLY = true; };
-template <> struct UmmaCfg<8, 4>  { static constexpr int SPS = 1, SA = 2, SB = 1, MAXCOT = 48;  static constexpr bool EARLY = true; };
+// MERGED (needs SA == SB): chunk q uses operand stage q % SA AND weight slot q % SA, and one "full" barrier (transform
+// warps + the weight copy's bytes) and one "empty" barrier (one commit) per chunk serve both.  The single thread that
+// issues the MMAs then executes one wait and one commit per chunk instead of two each; each costs it ~200 cycles while
+// the tensor core is streaming operands, and on wide layers that thread paces the kernel.
+template <> struct UmmaCfg<4, 2, 1>  { static constexpr int SPS = 2, SA = 3, SB = 3, MAXCOT = 128; static constexpr bool EARLY = false, MERGED = true; };
+template <> struct UmmaCfg<8, 2, 1>  { static constexpr int SPS = 2, SA = 2, SB = 2, MAXCOT = 64;  static constexpr bool EARLY = false, MERGED = true; };
+template <> struct UmmaCfg<16, 2, 1> { static constexpr int SPS = 1, SA = 2, SB = 1, MAXCOT = 32;  static constexpr bool EARLY = true, MERGED = false; };
+template <> struct UmmaCfg<32, 2, 1> { static constexpr int SPS = 1, SA = 1, SB = 1, MAXCOT = 16;  static constexpr bool EARLY = true, MERGED = false; };
+template <> struct UmmaCfg<4, 4, 1>  { static constexpr int SPS = 1, SA = 3, SB = 1, MAXCOT = 128; static constexpr bool EARLY = true, MERGED = false; };
+template <> struct UmmaCfg<8, 4, 1>  { static constexpr int SPS = 1, SA = 2, SB = 1, MAXCOT = 48;  static constexpr bool EARLY = true, MERGED = false; };
+// CTA pairs: a CTA holds half of every weight tile, which leaves room for deeper rings.
+template <> struct UmmaCfg<4, 2, 2>  { static constexpr int SPS = 2, SA = 4, SB = 4, MAXCOT = 128; static constexpr bool EARLY = false, MERGED = true; };
+template <> struct UmmaCfg<8, 2, 2>  { static constexpr int SPS = 2, SA = 2, SB = 2, MAXCOT = 64;  static constexpr bool EARLY = false, MERGED = true; };
 constexpr int kRawSlots = 3;
 constexpr uint32_t kSpin = 256;               // test_wait polls before a single-thread role falls back to try_wait
 
@@ -90,9 +104,15 @@ struct SmemBarriers {
 //   [0, CoT)                         plane 0 (k = 0)
 //   per complex frequency f (4*CoT): Wr | Wi   (multiplied by Re x^)   then   -Wi | Wr   (by Im x^)
 //   [rowsB - CoT, rowsB)             plane T-1 (k = T/2)
+//
+// CTA-pair layout (pair != 0): every B tile (the rows one MMA reads) is split in halves, the first half of its rows
+// for the leader CTA and the second for its peer, and a blob holds first everything the leader loads, then everything
+// the peer loads: [half][hi | lo part][rowsB / 2 rows].  The halves of a real plane are its first and second CoT / 2
+// output channels; the halves of a complex frequency's tiles [Wr | Wi] and [-Wi | Wr] are the rows that produce Re y^
+// (leader) and Im y^ (peer).
 template <int T, typename IO>
 __global__ void build_image_kernel(const float* __restrict__ planes, int Cin, int Cout, int CoT, int nTiles, int nK,
-                                   int rowsB, IO* __restrict__ image, int cin0, int CinTotal) {
+                                   int rowsB, IO* __restrict__ image, int cin0, int CinTotal, int pair) {
     constexpr int E = sizeof(IO), KCH = kRowBytes / E, EPC = 16 / E, NSPLIT = E == 4 ? 2 : 1;
     const int64_t per_blob = (int64_t)NSPLIT * rowsB * KCH;
     const int64_t total = (int64_t)nTiles * nK * per_blob;
@@ -101,26 +121,47 @@ __global__ void build_image_kernel(const float* __restrict__ planes, int Cin, in
         const int within_all = (int)(idx % per_blob);
         const int64_t blob = idx / per_blob;
         const int kc = (int)(blob % nK), tile = (int)(blob / nK);
-        const int part = within_all / (rowsB * KCH), within = within_all % (rowsB * KCH);
-        // destination element `within` of the blob: row n, 16-byte chunk c, element e of the chunk; the chunk holds
-        // k-half (c ^ bit 2 of n) (32-byte swizzle)
+        int part, within, plane, local;
+        float sign = 1.f;
+        if (pair) {
+            const int rowsH = rowsB / 2, H = CoT / 2;
+            const int half = within_all / (NSPLIT * rowsH * KCH), rem = within_all % (NSPLIT * rowsH * KCH);
+            part = rem / (rowsH * KCH);
+            within = rem % (rowsH * KCH);
+            const int n = within / KCH;                              // row inside this CTA's half of the blob
+            if (n < H) {
+                plane = 0; local = half * H + n;
+            } else if (n >= rowsH - H) {
+                plane = T - 1; local = half * H + n - (rowsH - H);
+            } else {
+                const int m = n - H, f = m / (2 * CoT) + 1, second = (m / CoT) & 1;   // second: the tile multiplied by Im x^
+                local = m % CoT;
+                if (!second) plane = half == 0 ? 2 * f - 1 : 2 * f;                  // Wr -> Re y^ | Wi -> Im y^
+                else if (half == 0) { plane = 2 * f; sign = -1.f; }                 // -Wi -> Re y^
+                else plane = 2 * f - 1;                                             // Wr -> Im y^
+            }
+        } else {
+            part = within_all / (rowsB * KCH);
+            within = within_all % (rowsB * KCH);
+            const int n = within / KCH;
+            if (n < CoT) {
+                plane = 0; local = n;
+            } else if (n >= rowsB - CoT) {
+                plane = T - 1; local = n - (rowsB - CoT);
+            } else {
+                const int m = n - CoT, f = m / (4 * CoT) + 1, quarter = (m / CoT) & 3;
+                local = m % CoT;
+                if (quarter == 0) plane = 2 * f - 1;                     // Wr  -> Re y^
+                else if (quarter == 1) plane = 2 * f;                    // Wi  -> Im y^
+                else if (quarter == 2) { plane = 2 * f; sign = -1.f; }   // -Wi -> Re y^
+                else plane = 2 * f - 1;                                  // Wr  -> Im y^
+            }
+        }
+        // destination element `within` of the (half-)blob: row n, 16-byte chunk c, element e of the chunk; the chunk
+        // holds k-half (c ^ bit 2 of n) (32-byte swizzle)
         const int n = within / KCH;
         const int c = (within % KCH) / EPC;
         const int kk = (c ^ ((n >> 2) & 1)) * EPC + within % EPC;
-        int plane, local;
-        float sign = 1.f;
-        if (n < CoT) {
-            plane = 0; local = n;
-        } else if (n >= rowsB - CoT) {
-            plane = T - 1; local = n - (rowsB - CoT);
-        } else {
-            const int m = n - CoT, f = m / (4 * CoT) + 1, quarter = (m / CoT) & 3;
-            local = m % CoT;
-            if (quarter == 0) plane = 2 * f - 1;                     // Wr  -> Re y^
-            else if (quarter == 1) plane = 2 * f;                    // Wi  -> Im y^
-            else if (quarter == 2) { plane = 2 * f; sign = -1.f; }   // -Wi -> Re y^
-            else plane = 2 * f - 1;                                  // Wr  -> Im y^
-        }
         const int cin = kc * KCH + kk, cout = tile * CoT + local;
         float v = 0.f;
         if (cin < Cin && cout < Cout) v = sign * planes[((size_t)plane * CinTotal + cin0 + cin) * Cout + cout];
@@ -135,13 +176,16 @@ __global__ void build_image_kernel(const float* __restrict__ planes, int Cin, in
 }
 
 // ------------------------------------------------------------------------------------------------
-template <int T, typename IO>
+template <int T, typename IO, int CG>
 __global__ void __launch_bounds__(kThreadsUmma, 1)
 umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_constant__ CUtensorMap tmap_out,
                    const UmmaParams prm) {
     constexpr int E = sizeof(IO);               // 2: half I/O, kind::f16;  4: float I/O, kind::tf32 with the 3xTF32 split
-    using Cfg = UmmaCfg<T, E>;
+    using Cfg = UmmaCfg<T, E, CG>;
     constexpr int SPS = Cfg::SPS, SA = Cfg::SA, SB = Cfg::SB;
+    constexpr bool PAIR = CG == 2, MERGED = Cfg::MERGED;
+    static_assert(!MERGED || SA == SB, "one barrier pair per chunk needs equally deep rings");
+    static_assert(!PAIR || MERGED, "the CTA-pair form is written for the merged rings");
     constexpr int SR = kRawSlots * SPS;         // slabs in the raw ring
     constexpr int EPR = 128 / E;                // elements per raw slab row (128 B)
     constexpr int NCH = EPR / T;                // channels per raw slab row
@@ -163,12 +207,17 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
     volatile int* abort_flag = &bar->abort_flag;
     int* status = prm.status;
 
+    // A unit is (token tile, channel tile); a pair takes two neighbouring token tiles per unit, one per CTA.
+    const uint32_t rank = PAIR ? ptx::cluster_ctarank() : 0u;
     if (threadIdx.x == 0) {
         for (int i = 0; i < kRawSlots; ++i) { ptx::mbar_init(&bar->full_raw[i], 1); ptx::mbar_init(&bar->empty_raw[i], 4 * SPS); }
-        for (int i = 0; i < SA; ++i) { ptx::mbar_init(&bar->full_a[i], 4 * SPK); ptx::mbar_init(&bar->empty_a[i], 1); }
+        // "full" of a stage: the transform warps; merged rings: + the weight copy (its producer's arrive.expect_tx);
+        // pair, leader: + the peer CTA's word that its own stage is full
+        const uint32_t full_count = 4 * SPK + (MERGED ? 1 : 0) + ((PAIR && rank == 0) ? 1 : 0);
+        for (int i = 0; i < SA; ++i) { ptx::mbar_init(&bar->full_a[i], full_count); ptx::mbar_init(&bar->empty_a[i], 1); }
         for (int i = 0; i < SB; ++i) { ptx::mbar_init(&bar->full_b[i], 1); ptx::mbar_init(&bar->empty_b[i], 1); }
         ptx::mbar_init(&bar->full_d, 1);
-        ptx::mbar_init(&bar->empty_d, kNumComputeWarps);
+        ptx::mbar_init(&bar->empty_d, kNumComputeWarps * CG);    // pair: the leader's barrier takes both CTAs' warps
         ptx::mbar_init(&bar->mma_done, 1);
         ptx::mbar_init(&bar->staging_free, kNumComputeWarps);
         bar->abort_flag = 0;
@@ -177,16 +226,25 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
         ptx::prefetch_tensormap(&tmap_out);
     }
     if (warp == kWarpMma) {
-        ptx::tmem_alloc(&bar->tmem_base, kTmemCols);
-        ptx::tmem_relinquish();
+        if constexpr (PAIR) { ptx::tmem_alloc_pair(&bar->tmem_base, kTmemCols); ptx::tmem_relinquish_pair(); }
+        else { ptx::tmem_alloc(&bar->tmem_base, kTmemCols); ptx::tmem_relinquish(); }
     }
     ptx::tc_fence_before_sync();
     __syncthreads();
+    if constexpr (PAIR) {                       // the peer's barriers must be initialised before anything arrives on them
+        ptx::cluster_arrive();
+        ptx::cluster_wait();
+    }
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = bar->tmem_base;
 
     const int nK = prm.nK, nTiles = prm.nTiles, CoT = prm.CoT, rowsB = prm.rowsB;
-    const int64_t first = blockIdx.x, stride = gridDim.x;
+    const int64_t first = blockIdx.x / CG, stride = gridDim.x / CG;
+    auto unit_row0 = [&](int64_t u) { return (int)(((u / nTiles) * CG + rank) * kTileM); };
+    const int rowsH = rowsB / CG;                                // weight-image rows this CTA holds per (tile, chunk)
+    // barriers of the weight ring: its own, or (merged rings) those of the operand stages
+    uint64_t* const full_wb = MERGED ? bar->full_a : bar->full_b;
+    uint64_t* const empty_wb = MERGED ? bar->empty_a : bar->empty_b;
 
     if (warp == kWarpTmaX) {
         // ---------------------------------------------------------------- raw activation rows via TMA
@@ -194,7 +252,7 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
             uint32_t cr = 0;                                     // running slab counter; slot phase = cr / SPS
             bool ok = true;
             for (int64_t u = first; u < prm.num_units && ok; u += stride) {
-                const int row0 = (int)(u / nTiles) * kTileM;
+                const int row0 = unit_row0(u);
                 for (int kc = 0; kc < nK && ok; ++kc) {
                     for (int q = 0; q < SPK; ++q, ++cr) {
                         const uint32_t ph = cr / SPS;            // slot phase counter
@@ -230,47 +288,71 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
         if (lane == 0) {
             uint32_t cb = 0;
             bool ok = true;
-            const uint32_t blob_bytes = (uint32_t)rowsB * kRowBytes * NSPLIT;
+            const uint32_t blob_bytes = (uint32_t)rowsH * kRowBytes * NSPLIT;       // pair: this CTA's half of the blob
             for (int64_t u = first; u < prm.num_units && ok; u += stride) {
                 const int tile = (int)(u % nTiles);
                 for (int kc = 0; kc < nK; ++kc, ++cb) {
                     const int slot = cb % SB;
-                    ok = ptx::mbar_wait(&bar->empty_b[slot], ((cb / SB) & 1) ^ 1, abort_flag, status, 102, true, kSpin);
+                    ok = ptx::mbar_wait(&empty_wb[slot], ((cb / SB) & 1) ^ 1, abort_flag, status, 102, true, kSpin);
                     if (!ok) break;
-                    ptx::mbar_arrive_expect_tx(&bar->full_b[slot], blob_bytes);
+                    ptx::mbar_arrive_expect_tx(&full_wb[slot], blob_bytes);
                     ptx::bulk_load_1d(bsm + slot * prm.b_slot_bytes,
-                                      prm.image + ((size_t)tile * nK + kc) * (size_t)blob_bytes, blob_bytes,
-                                      &bar->full_b[slot]);
+                                      prm.image + (((size_t)tile * nK + kc) * CG + rank) * (size_t)blob_bytes, blob_bytes,
+                                      &full_wb[slot]);
                 }
             }
             if (!ok) {
+                // giving up: the copies still in flight must land before this CTA's shared memory goes away (with merged
+                // rings the phase also needs the transform warps, which may have given up too: the wait is bounded)
                 const uint32_t lo = cb > (uint32_t)SB ? cb - SB : 0;
                 for (uint32_t c = lo; c < cb; ++c)
-                    ptx::mbar_wait(&bar->full_b[c % SB], (c / SB) & 1, abort_flag, status, 112, false);
+                    ptx::mbar_wait(&full_wb[c % SB], (c / SB) & 1, abort_flag, status, 112, false);
             }
         }
     } else if (warp == kWarpMma) {
         // ---------------------------------------------------------------- tensor-core issue (one thread)
-        if (lane == 0) {
+        if (lane == 0 && rank == 0) {
             uint32_t ca = 0, cb = 0, cu = 0;
             bool ok = true;
-            const uint32_t idesc_real = E == 2 ? ptx::umma_idesc_f16_f32(kTileM, CoT) : ptx::umma_idesc_tf32_f32(kTileM, CoT);
-            const uint32_t idesc_cplx = E == 2 ? ptx::umma_idesc_f16_f32(kTileM, 2 * CoT) : ptx::umma_idesc_tf32_f32(kTileM, 2 * CoT);
+            constexpr int M = kTileM * CG;
+            const uint32_t idesc_real = E == 2 ? ptx::umma_idesc_f16_f32(M, CoT) : ptx::umma_idesc_tf32_f32(M, CoT);
+            const uint32_t idesc_cplx = E == 2 ? ptx::umma_idesc_f16_f32(M, 2 * CoT) : ptx::umma_idesc_tf32_f32(M, 2 * CoT);
             auto mma = [](uint32_t d, uint32_t a_addr, uint32_t b_addr, uint32_t idesc, uint32_t accumulate) {
-                if constexpr (E == 2)
-                    ptx::umma_f16(d, ptx::umma_smem_desc_k_sw32(a_addr), ptx::umma_smem_desc_k_sw32(b_addr), idesc, accumulate);
-                else
-                    ptx::umma_tf32(d, ptx::umma_smem_desc_k_sw32(a_addr), ptx::umma_smem_desc_k_sw32(b_addr), idesc, accumulate);
+                const uint64_t ad = ptx::umma_smem_desc_k_sw32(a_addr), bd = ptx::umma_smem_desc_k_sw32(b_addr);
+                if constexpr (E == 2) {
+                    if constexpr (PAIR) ptx::umma_f16_pair(d, ad, bd, idesc, accumulate);
+                    else ptx::umma_f16(d, ad, bd, idesc, accumulate);
+                } else {
+                    if constexpr (PAIR) ptx::umma_tf32_pair(d, ad, bd, idesc, accumulate);
+                    else ptx::umma_tf32(d, ad, bd, idesc, accumulate);
+                }
             };
-            const uint32_t b_part = (uint32_t)rowsB * kRowBytes;
+            // a barrier of this CTA and, in a pair, the barrier at the same place in the peer CTA
+            auto commit_both = [&](uint64_t* b) {
+                if constexpr (PAIR) {
+                    ptx::umma_commit_pair(b);
+                    ptx::umma_commit_pair_addr(ptx::map_to_cta(ptx::smem_u32(b), 1u));
+                } else {
+                    ptx::umma_commit(b);
+                }
+            };
+            // Rows of this CTA's weight slot (pair: half tiles).  Real plane: CoT / CG rows; a complex frequency: two
+            // tiles of 2 CoT / CG rows each.
+            const uint32_t b_part = (uint32_t)rowsH * kRowBytes;
+            const uint32_t rows_real = (uint32_t)(CoT / CG), rows_cplx = (uint32_t)(2 * CoT / CG);
             for (int64_t u = first; u < prm.num_units && ok; u += stride, ++cu) {
-                ok = ptx::mbar_wait(&bar->empty_d, (cu & 1) ^ 1, abort_flag, status, 103, true, kSpin);
+                if constexpr (PAIR) ok = ptx::mbar_wait_cluster(&bar->empty_d, (cu & 1) ^ 1, abort_flag, status, 103);
+                else ok = ptx::mbar_wait(&bar->empty_d, (cu & 1) ^ 1, abort_flag, status, 103, true, kSpin);
                 if (!ok) break;
                 ptx::tc_fence_after_sync();
                 for (int kc = 0; kc < nK; ++kc, ++ca, ++cb) {
                     const int sa = ca % SA, sb = cb % SB;
-                    ok = ptx::mbar_wait(&bar->full_a[sa], (ca / SA) & 1, abort_flag, status, 104, true, kSpin);
-                    ok = ok && ptx::mbar_wait(&bar->full_b[sb], (cb / SB) & 1, abort_flag, status, 105, true, kSpin);
+                    if constexpr (PAIR) {
+                        ok = ptx::mbar_wait_cluster(&bar->full_a[sa], (ca / SA) & 1, abort_flag, status, 104, true, kSpin);
+                    } else {
+                        ok = ptx::mbar_wait(&bar->full_a[sa], (ca / SA) & 1, abort_flag, status, 104, true, kSpin);
+                        if constexpr (!MERGED) ok = ok && ptx::mbar_wait(&bar->full_b[sb], (cb / SB) & 1, abort_flag, status, 105, true, kSpin);
+                    }
                     if (!ok) break;
                     ptx::tc_fence_after_sync();
                     // FP16: one pass.  FP32 (3xTF32): hi*hi, hi*lo, lo*hi accumulate into the same columns.
@@ -285,22 +367,37 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
 #pragma unroll
                         for (int f = 1; f < T / 2; ++f) {
                             const uint32_t d = tmem_base + (uint32_t)((2 * f - 1) * CoT);
-                            const uint32_t rb = (uint32_t)(CoT + (f - 1) * 4 * CoT);
+                            const uint32_t rb = rows_real + (uint32_t)(f - 1) * 2 * rows_cplx;
                             mma(d, a0 + (2 * f - 1) * 4096, b0 + rb * kRowBytes, idesc_cplx, acc);
-                            mma(d, a0 + (2 * f) * 4096, b0 + (rb + 2 * CoT) * kRowBytes, idesc_cplx, 1u);
+                            mma(d, a0 + (2 * f) * 4096, b0 + (rb + rows_cplx) * kRowBytes, idesc_cplx, 1u);
                         }
                         // k = T/2
                         mma(tmem_base + (uint32_t)((T - 1) * CoT), a0 + (T - 1) * 4096,
-                            b0 + (uint32_t)(rowsB - CoT) * kRowBytes, idesc_real, acc);
+                            b0 + ((uint32_t)rowsH - rows_real) * kRowBytes, idesc_real, acc);
                     }
-                    ptx::umma_commit(&bar->empty_a[sa]);
-                    ptx::umma_commit(&bar->empty_b[sb]);
+                    commit_both(&bar->empty_a[sa]);
+                    if constexpr (!MERGED) commit_both(&bar->empty_b[sb]);
                 }
-                if (ok) ptx::umma_commit(&bar->full_d);
+                if (ok) commit_both(&bar->full_d);
             }
             // all MMAs issued by this thread must have retired before shared memory and TMEM go away
-            ptx::umma_commit(&bar->mma_done);
+            if constexpr (PAIR) ptx::umma_commit_pair(&bar->mma_done);
+            else ptx::umma_commit(&bar->mma_done);
             ptx::mbar_wait(&bar->mma_done, 0, abort_flag, status, 113, false);
+        } else if (PAIR && lane == 0) {
+            // The peer CTA of a pair issues no MMA.  This thread tells the leader when this CTA's stage of a chunk
+            // (transformed rows and weight half) is full, by arriving on the leader's barrier of the same stage; the
+            // leader's commits release the stage in both CTAs.
+            uint32_t ca = 0;
+            bool ok = true;
+            const uint32_t leader_full0 = ptx::map_to_cta(ptx::smem_u32(&bar->full_a[0]), 0u);
+            for (int64_t u = first; u < prm.num_units && ok; u += stride) {
+                for (int kc = 0; kc < nK; ++kc, ++ca) {
+                    ok = ptx::mbar_wait(&bar->full_a[ca % SA], (ca / SA) & 1, abort_flag, status, 116, true, kSpin);
+                    if (!ok) break;
+                    ptx::mbar_arrive_remote(leader_full0 + (ca % SA) * 8u);
+                }
+            }
         }
     } else if (warp >= kWarpCompute0) {
         // ---------------------------------------------------------------- compute warps: transform, then epilogue
@@ -323,6 +420,12 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
         const uint32_t lane_base = tmem_base + ((uint32_t)(quad * 32) << 16);
         uint32_t ca = 0, cu = 0;
         bool ok = true;
+        // the accumulator of this CTA has been read: tell the MMA-issuing thread (in a pair, the leader CTA's)
+        const uint32_t empty_d_leader = PAIR ? ptx::map_to_cta(ptx::smem_u32(&bar->empty_d), 0u) : 0u;
+        auto release_d = [&]() {
+            if (PAIR && rank != 0) ptx::mbar_arrive_remote(empty_d_leader);
+            else ptx::mbar_arrive(&bar->empty_d);
+        };
         bool staging_pending = false;                            // previous unit's TMA stores may still be reading the stage
         uint8_t* staging = xhat + cw * 4096;                     // this warp's [32 tokens x 128 B] output stage (128B swizzle)
         for (int64_t u = first; u < prm.num_units && ok; u += stride, ++cu) {
@@ -406,7 +509,7 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
                 if (gi + 3 >= ngroups) {                         // this warp's last read of the accumulator
                     ptx::tc_fence_before_sync();
                     __syncwarp();
-                    if (lane == 0) ptx::mbar_arrive(&bar->empty_d);
+                    if (lane == 0) release_d();
                 }
                 const int co0 = tile * CoT + c0;
                 uint32_t o[32];                                  // G channels x T elements = 128 bytes
@@ -436,8 +539,8 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
                 ptx::fence_proxy_async_smem();
                 __syncwarp();
                 if (lane == 0 && co0 < prm.Cout) {
-                    if (prm.accumulate) ptx::tma_reduce_add_2d(&tmap_out, co0 * T, (int)((u / nTiles) * kTileM) + quad * 32, staging);
-                    else ptx::tma_store_2d(&tmap_out, co0 * T, (int)((u / nTiles) * kTileM) + quad * 32, staging);
+                    if (prm.accumulate) ptx::tma_reduce_add_2d(&tmap_out, co0 * T, unit_row0(u) + quad * 32, staging);
+                    else ptx::tma_store_2d(&tmap_out, co0 * T, unit_row0(u) + quad * 32, staging);
                     ptx::bulk_commit_group();
                 }
             }
@@ -451,7 +554,7 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
             if (third >= ngroups) {                              // fewer column groups than shares: nothing to read
                 ptx::tc_fence_before_sync();
                 __syncwarp();
-                if (lane == 0) ptx::mbar_arrive(&bar->empty_d);
+                if (lane == 0) release_d();
             }
         }
     }
@@ -459,9 +562,14 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
     // ---------------------------------------------------------------- teardown (reached by every thread)
     ptx::tc_fence_before_sync();
     __syncthreads();
+    if constexpr (PAIR) {                       // neither CTA may leave while the other can still signal it or read its memory
+        ptx::cluster_arrive();
+        ptx::cluster_wait();
+    }
     if (warp == kWarpMma) {
         ptx::tc_fence_after_sync();
-        ptx::tmem_dealloc(tmem_base, kTmemCols);
+        if constexpr (PAIR) ptx::tmem_dealloc_pair(tmem_base, kTmemCols);
+        else ptx::tmem_dealloc(tmem_base, kTmemCols);
     }
 }
 
@@ -483,9 +591,9 @@ EncodeTiledFn encode_tiled_fn() {
     return fn;
 }
 
-template <int T, int E>
+template <int T, int E, int CG>
 size_t umma_smem_bytes(int b_slot_bytes) {
-    using Cfg = UmmaCfg<T, E>;
+    using Cfg = UmmaCfg<T, E, CG>;
     return 1024 + (size_t)kRawSlots * Cfg::SPS * kSlabBytes + (size_t)Cfg::SA * T * 4096 * (E == 4 ? 2 : 1) +
            (size_t)Cfg::SB * b_slot_bytes + sizeof(SmemBarriers) + 64;
 }
@@ -512,7 +620,7 @@ cudaError_t dispatch_umma(int T, int elem_bytes, F&& f) {
 int umma_max_cot(int T, int elem_bytes) {
     int m = 0;
     dispatch_umma(T, elem_bytes, [&](auto tc, auto io) {
-        m = UmmaCfg<decltype(tc)::value, sizeof(decltype(io))>::MAXCOT;
+        m = UmmaCfg<decltype(tc)::value, sizeof(decltype(io)), 1>::MAXCOT;
         return cudaSuccess;
     });
     return m;
@@ -572,7 +680,7 @@ cudaError_t launch_build_umma_image(const UmmaLinearShape& s, const float* plane
         const int64_t total = (int64_t)(s.image_bytes / sizeof(IO));
         const int blocks = (int)((total + 255) / 256 < 4096 ? (total + 255) / 256 : 4096);
         build_image_kernel<TT, IO><<<blocks, 256, 0, stream>>>(planes, s.Cin, s.Cout, s.CoT, s.nTiles, s.nK, s.rowsB,
-                                                                (IO*)image, s.cin0, s.CinTotal);
+                                                                (IO*)image, s.cin0, s.CinTotal, s.pair ? 1 : 0);
         return cudaGetLastError();
     });
 }
@@ -608,21 +716,56 @@ cudaError_t launch_umma_linear(const UmmaLinearShape& s, const void* in, void* o
     prm.out = out; prm.image = (const uint8_t*)image; prm.bias = bias_f32; prm.status = status;
     prm.N = N; prm.Cin = s.Cin; prm.Cout = s.Cout;
     prm.CoT = s.CoT; prm.nTiles = s.nTiles; prm.nK = s.nK; prm.rowsB = s.rowsB;
-    prm.b_slot_bytes = (int)align_up((size_t)s.rowsB * kRowBytes * (s.elem_bytes == 4 ? 2 : 1), 128);
-    prm.num_units = ((N + kTileM - 1) / kTileM) * s.nTiles;
+    const int cg = s.pair ? 2 : 1;
+    prm.b_slot_bytes = (int)align_up((size_t)(s.rowsB / cg) * kRowBytes * (s.elem_bytes == 4 ? 2 : 1), 256);
+    const int64_t token_tiles = (N + kTileM - 1) / kTileM;
+    prm.num_units = ((token_tiles + cg - 1) / cg) * s.nTiles;    // a pair takes two token tiles per unit
     prm.accumulate = accumulate ? 1 : 0;
-    const int grid = (int)(prm.num_units < num_sms ? prm.num_units : num_sms);
 
     return dispatch_umma(s.T, s.elem_bytes, [&](auto tc, auto io) {
         constexpr int TT = decltype(tc)::value;
         using IO = decltype(io);
-        const size_t smem = umma_smem_bytes<TT, sizeof(IO)>(prm.b_slot_bytes);
-        static SmemLimitOnce smem_limit;                      // per kernel instantiation
-        if (cudaError_t e = smem_limit.ensure(umma_linear_kernel<TT, IO>, 227 * 1024); e != cudaSuccess) return e;
-        if (smem > 227 * 1024) return cudaErrorInvalidConfiguration;
-        umma_linear_kernel<TT, IO><<<grid, kThreadsUmma, smem, stream>>>(tmap, tmap_out, prm);
-        return cudaGetLastError();
+        if (s.pair) {
+            if constexpr (sizeof(IO) == 2 && (TT == 4 || TT == 8)) {
+                const size_t smem = umma_smem_bytes<TT, 2, 2>(prm.b_slot_bytes);
+                if (smem > 227 * 1024) return cudaErrorInvalidConfiguration;
+                static SmemLimitOnce smem_limit;
+                auto kernel = umma_linear_kernel<TT, IO, 2>;
+                if (cudaError_t e = smem_limit.ensure(kernel, 227 * 1024); e != cudaSuccess) return e;
+                cudaLaunchConfig_t cfg{};
+                cudaLaunchAttribute attr[1];
+                attr[0].id = cudaLaunchAttributeClusterDimension;
+                attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+                cfg.blockDim = dim3(kThreadsUmma); cfg.dynamicSmemBytes = smem; cfg.stream = stream;
+                cfg.attrs = attr; cfg.numAttrs = 1;
+                // persistent: as many pairs as can be resident at once (pairs need two SMs of one GPC), at most one per unit
+                static std::atomic<int> max_pairs{0};
+                int pairs = max_pairs.load(std::memory_order_relaxed);
+                if (pairs == 0) {
+                    cfg.gridDim = dim3(2 * (num_sms / 2));
+                    if (cudaError_t e = cudaOccupancyMaxActiveClusters(&pairs, kernel, &cfg); e != cudaSuccess) return e;
+                    if (pairs <= 0) return cudaErrorInvalidConfiguration;
+                    if (pairs > num_sms / 2) pairs = num_sms / 2;
+                    max_pairs.store(pairs, std::memory_order_relaxed);
+                }
+                if (prm.num_units < pairs) pairs = (int)prm.num_units;
+                cfg.gridDim = dim3(2 * pairs);
+                return cudaLaunchKernelEx(&cfg, kernel, tmap, tmap_out, prm);
+            } else {
+                return cudaErrorInvalidConfiguration;
+            }
+        } else {
+            const int grid = (int)(prm.num_units < num_sms ? prm.num_units : num_sms);
+            const size_t smem = umma_smem_bytes<TT, sizeof(IO), 1>(prm.b_slot_bytes);
+            static SmemLimitOnce smem_limit;                      // per kernel instantiation
+            if (cudaError_t e = smem_limit.ensure(umma_linear_kernel<TT, IO, 1>, 227 * 1024); e != cudaSuccess) return e;
+            if (smem > 227 * 1024) return cudaErrorInvalidConfiguration;
+            umma_linear_kernel<TT, IO, 1><<<grid, kThreadsUmma, smem, stream>>>(tmap, tmap_out, prm);
+            return cudaGetLastError();
+        }
     });
 }
+
+bool umma_linear_pair_supported(int T, eql_dtype_t dtype) { return dtype == EQL_FP16 && (T == 4 || T == 8); }
 
 }  // namespace eql
