@@ -67,9 +67,11 @@ enum {
      * output-channel tile) even where the kernel that keeps the transformed activations of a token
      * tile resident in shared memory applies.  For comparisons and tests. */
     EQL_FLAG_FORCE_STREAMING = 4u,
-    /* Never take the CTA-pair form of the streaming kernel (two SMs sharing each spectral-weight tile through
-     * tcgen05 cta_group::2), which plans of wide FP16 layers select.  For comparisons and tests. */
-    EQL_FLAG_NO_CTA_PAIR = 8u
+    /* Run the streaming kernel in its CTA-pair form where it exists (FP16 plans, T = 4 or 8): clusters of two CTAs on
+     * two SMs work on neighbouring token tiles, one tcgen05.mma.cta_group::2 covers both, and each SM loads and holds
+     * only half of every spectral-weight tile.  Same results bit for bit.  Not selected by default: on B200 it
+     * measures 3-15 % slower than the single-CTA form (see the kernel's header comment). */
+    EQL_FLAG_CTA_PAIR = 8u
 };
 
 typedef struct {

@@ -40,8 +40,6 @@ using namespace eql;
 
 inline size_t elem_size(eql_dtype_t d) { return d == EQL_FP32 ? 4 : 2; }
 
-// Where the CTA-pair form of the streaming kernel is taken (reduced channels Cin, produced channels Cout).
-inline bool pair_pays(int Cin, int Cout) { (void)Cin; (void)Cout; return true; }
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 eql_status_t check_shape(int T, int Ci, int Co, int dtype) {
@@ -245,7 +243,7 @@ eql_status_t eqlinear_plan(eqlinear_plan_t* plan, int T, int C_in, int C_out, eq
     eql_status_t st = check_shape(T, C_in, C_out, dtype);
     if (st != EQL_OK) return st;
     if (!w || !workspace) return EQL_ERR_INVALID_ARG;
-    if (flags & ~(unsigned)(EQL_FLAG_CORRELATION | EQL_FLAG_FORCE_SIMT | EQL_FLAG_FORCE_STREAMING | EQL_FLAG_NO_CTA_PAIR))
+    if (flags & ~(unsigned)(EQL_FLAG_CORRELATION | EQL_FLAG_FORCE_SIMT | EQL_FLAG_FORCE_STREAMING | EQL_FLAG_CTA_PAIR))
         return EQL_ERR_INVALID_ARG;
     if (!aligned16(w) || (bias && !aligned16(bias))) return EQL_ERR_ALIGNMENT;
     if (reinterpret_cast<uintptr_t>(workspace) % kWsAlign != 0) return EQL_ERR_ALIGNMENT;
@@ -285,10 +283,10 @@ eql_status_t eqlinear_plan(eqlinear_plan_t* plan, int T, int C_in, int C_out, eq
             if (prefer(p->res_fwd)) p->fwd_kernel = 2;
             if (prefer(p->res_bwd)) p->bwd_data_kernel = 2;
         }
-        // Wide layers on the streaming kernel: its CTA-pair form, in which two SMs share every weight tile.
-        if (umma_linear_pair_supported(T, dtype) && !(flags & EQL_FLAG_NO_CTA_PAIR)) {
-            if (p->fwd_kernel == 1 && pair_pays(C_in, C_out)) p->fwd_kernel = 3;
-            if (p->bwd_data_kernel == 1 && pair_pays(C_out, C_in)) p->bwd_data_kernel = 3;
+        // On request: the streaming kernel's CTA-pair form, in which two SMs share every weight tile.
+        if (umma_linear_pair_supported(T, dtype) && (flags & EQL_FLAG_CTA_PAIR)) {
+            if (p->fwd_kernel == 1) p->fwd_kernel = 3;
+            if (p->bwd_data_kernel == 1) p->bwd_data_kernel = 3;
         }
     }
 

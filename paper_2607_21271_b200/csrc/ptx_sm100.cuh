@@ -228,9 +228,12 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t local_smem_addr, uint32_
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_smem_addr), "r"(rank));
     return r;
 }
-// Arrive on a barrier of another CTA of the cluster (address from map_to_cta); release at cluster scope.
+// Arrive on a barrier of another CTA of the cluster (address from map_to_cta).  Default semantics (release at CTA
+// scope), as for a local arrive: measured, a release at cluster scope stalls the arriving thread ~1200 cycles per
+// arrive.  What the arrival announces here is shared memory of THIS CTA written by this CTA's own threads, who ordered
+// their writes (proxy fence + arrive) before this thread saw their barrier complete; nothing cached has to travel.
 __device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr) {
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 // try_wait with acquire at cluster scope: pairs with mbar_arrive_remote from the other CTA.
 __device__ __forceinline__ bool mbar_try_wait_cluster(uint64_t* bar, uint32_t parity) {

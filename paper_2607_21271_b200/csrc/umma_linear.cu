@@ -14,12 +14,21 @@
 // Frequency-domain data never leaves the SM (registers, shared memory, TMEM).  The data gradient is the
 // same kernel run on dy with the conjugate-transposed weight image and no bias.
 //
-// CG = 2 ("CTA pair"): the same kernel as a cluster of two CTAs on two SMs that work on two neighbouring token tiles
-// and the same output-channel tile in lockstep.  One tcgen05.mma.cta_group::2 (M = 256) issued by the pair's leader
-// covers both token tiles; its B operand -- the spectral weight tile -- is split in halves between the two CTAs, so
-// each SM loads, holds and feeds to the tensor core only half of every weight tile.  On wide layers, whose main loop
-// is bound by shared-memory and L2 -> SM traffic, that is where the time goes.  Each CTA issues its own loads into its
-// own shared memory; only mbarrier arrivals cross the pair.
+// CG = 2 ("CTA pair", on request: EQL_FLAG_CTA_PAIR): the same kernel as a cluster of two CTAs on two SMs that work on
+// two neighbouring token tiles and the same output-channel tile in lockstep.  One tcgen05.mma.cta_group::2 (M = 256)
+// issued by the pair's leader covers both token tiles; its B operand -- the spectral weight tile -- is split in halves
+// between the two CTAs, so each SM loads and holds only half of every weight tile (L2 -> SM traffic of the weights
+// halves).  Each CTA issues its own loads into its own shared memory; only mbarrier arrivals cross the pair: the
+// peer's word that its stage of a chunk is full (one remote arrive per chunk on the leader's barrier of that stage),
+// the leader's commits to the peer's "empty" and "accumulator full" barriers (a second commit each, addressed to the
+// peer), and the peer's epilogue warps releasing the accumulator to the leader.
+// Measured on B200 (T = 4, 32 768 tokens): 57.9 / 148 / 508 / 2300 us at 256 / 512 / 1024 / 2048 channels against
+// 54.8 / 141 / 496 / 1990 us for the single-CTA form, bit-identical results.  The form does not pay here because the
+// main loop is paced by the MMA-issuing thread and the SM's shared-memory bandwidth, and neither gets lighter: each
+// SM's shared memory still serves its half of B to BOTH tensor cores, the leader executes one more commit per chunk,
+// and what halves -- the weight stream from L2 -- was not the limit.  (With release / acquire at cluster scope on the
+// pair's barriers the form ran 1.7x slower: a cluster-scope release stalls the arriving thread ~1200 cycles, a
+// cluster-scope acquire ~250.)
 //
 // Every wait on an mbarrier is bounded: on a time-out the CTA raises an abort flag, records a status
 // code for the host, drains its outstanding copies and MMAs, frees its TMEM and returns.
@@ -65,7 +74,8 @@ template <> struct UmmaCfg<16, 2, 1> { static constexpr int SPS = 1, SA = 2, SB 
 template <> struct UmmaCfg<32, 2, 1> { static constexpr int SPS = 1, SA = 1, SB = 1, MAXCOT = 16;  static constexpr bool EARLY = true, MERGED = false; };
 template <> struct UmmaCfg<4, 4, 1>  { static constexpr int SPS = 1, SA = 3, SB = 1, MAXCOT = 128; static constexpr bool EARLY = true, MERGED = false; };
 template <> struct UmmaCfg<8, 4, 1>  { static constexpr int SPS = 1, SA = 2, SB = 1, MAXCOT = 48;  static constexpr bool EARLY = true, MERGED = false; };
-// CTA pairs: a CTA holds half of every weight tile, which leaves room for deeper rings.
+// CTA pairs: a CTA holds half of every weight tile, which leaves room for deeper rings (measured: depths beyond these
+// change nothing, for either form -- the rings are not what paces the kernel).
 template <> struct UmmaCfg<4, 2, 2>  { static constexpr int SPS = 2, SA = 4, SB = 4, MAXCOT = 128; static constexpr bool EARLY = false, MERGED = true; };
 template <> struct UmmaCfg<8, 2, 2>  { static constexpr int SPS = 2, SA = 2, SB = 2, MAXCOT = 64;  static constexpr bool EARLY = false, MERGED = true; };
 constexpr int kRawSlots = 3;
@@ -87,8 +97,8 @@ struct UmmaParams {
 
 struct SmemBarriers {
     uint64_t full_raw[6], empty_raw[6];
-    uint64_t full_a[4], empty_a[4];
-    uint64_t full_b[4], empty_b[4];      // SB <= 4
+    uint64_t full_a[8], empty_a[8];      // SA <= 8
+    uint64_t full_b[4], empty_b[4];      // SB <= 4 (unmerged rings)
     uint64_t full_d, empty_d, mma_done, staging_free;
     uint32_t tmem_base;
     int abort_flag;
@@ -341,18 +351,15 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
             const uint32_t b_part = (uint32_t)rowsH * kRowBytes;
             const uint32_t rows_real = (uint32_t)(CoT / CG), rows_cplx = (uint32_t)(2 * CoT / CG);
             for (int64_t u = first; u < prm.num_units && ok; u += stride, ++cu) {
-                if constexpr (PAIR) ok = ptx::mbar_wait_cluster(&bar->empty_d, (cu & 1) ^ 1, abort_flag, status, 103);
-                else ok = ptx::mbar_wait(&bar->empty_d, (cu & 1) ^ 1, abort_flag, status, 103, true, kSpin);
+                ok = ptx::mbar_wait(&bar->empty_d, (cu & 1) ^ 1, abort_flag, status, 103, true, kSpin);
                 if (!ok) break;
                 ptx::tc_fence_after_sync();
                 for (int kc = 0; kc < nK; ++kc, ++ca, ++cb) {
                     const int sa = ca % SA, sb = cb % SB;
-                    if constexpr (PAIR) {
-                        ok = ptx::mbar_wait_cluster(&bar->full_a[sa], (ca / SA) & 1, abort_flag, status, 104, true, kSpin);
-                    } else {
-                        ok = ptx::mbar_wait(&bar->full_a[sa], (ca / SA) & 1, abort_flag, status, 104, true, kSpin);
-                        if constexpr (!MERGED) ok = ok && ptx::mbar_wait(&bar->full_b[sb], (cb / SB) & 1, abort_flag, status, 105, true, kSpin);
-                    }
+                    // (pair: the peer's arrival on this barrier stands for shared memory of the peer CTA that the peer's own
+                    // threads wrote and fenced; a wait with acquire at cluster scope instead costs ~250 cycles per chunk)
+                    ok = ptx::mbar_wait(&bar->full_a[sa], (ca / SA) & 1, abort_flag, status, 104, true, kSpin);
+                    if constexpr (!MERGED) ok = ok && ptx::mbar_wait(&bar->full_b[sb], (cb / SB) & 1, abort_flag, status, 105, true, kSpin);
                     if (!ok) break;
                     ptx::tc_fence_after_sync();
                     // FP16: one pass.  FP32 (3xTF32): hi*hi, hi*lo, lo*hi accumulate into the same columns.

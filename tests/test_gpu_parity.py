@@ -120,20 +120,51 @@ def test_resident_and_streaming_kernels_agree_with_oracle(T, Ci, Co, N, ids):
     """Layers with few input channels run the kernel that keeps a token tile's spectrum in shared memory (id 2), and so
     do layers with at most 128 output channels (one channel tile: the spectrum then streams through a ring of three
     chunk buffers, e.g. 384 -> 96 channels); EQL_FLAG_FORCE_STREAMING selects the streaming kernel (id 1) for the same
-    plan shape.  Both must meet the bar, on channel counts that are not multiples of the 128-channel / 16-channel
-    tiles, ragged token counts, and token counts large enough that a CTA's range of work starts and ends in the
-    middle of a token tile and covers several units."""
+    plan shape, and EQL_FLAG_CTA_PAIR on top of it the streaming kernel's CTA-pair form (id 3: two CTAs, one
+    tcgen05.mma.cta_group::2 over both).  All must meet the bar, on channel counts that are not multiples of the
+    128-channel / 16-channel tiles, ragged token counts, odd numbers of token tiles (a pair's second CTA then has no
+    rows), and token counts large enough that a CTA's range of work starts and ends in the middle of a token tile and
+    covers several units.  The pair form computes the same products in the same order as the single-CTA form: its
+    results must be bit-identical to it."""
     wl = Workload("res", "fp16", T, Ci, Co, N, "normal", ("fwd", "bwd_data"), 21)
     data = eq.workloads.generate(wl)
-    for flags, want in ((0, ids), (eq.EQL_FLAG_FORCE_STREAMING, (1, 1))):
+    outs = {}
+    for flags, want in ((0, ids), (eq.EQL_FLAG_FORCE_STREAMING, (1, 1)),
+                        (eq.EQL_FLAG_FORCE_STREAMING | eq.EQL_FLAG_CTA_PAIR, (3, 3))):
         layer = GpuLayer(T, Ci, Co, "fp16", data["w"], data["bias"], flags)
         try:
             info = eq.eqlinear_plan_info(layer.plan)
             assert (info.fwd_kernel, info.bwd_data_kernel) == want
+            outs[flags] = (layer.fwd(data["x"]), layer.bwd_data(data["dy"]))
+            assert layer.raw_status() == 0
         finally:
             layer.close()
         for k, v in check_workload(wl, flags=flags, data=data).items():
             assert v <= TOL["fp16"], f"T={T} Ci={Ci} Co={Co} N={N} flags={flags}: {k} error {v:.3e}"
+    single, pair = outs[eq.EQL_FLAG_FORCE_STREAMING], outs[eq.EQL_FLAG_FORCE_STREAMING | eq.EQL_FLAG_CTA_PAIR]
+    assert np.array_equal(single[0], pair[0]) and np.array_equal(single[1], pair[1])
+
+
+def test_cta_pair_form_at_full_size_is_repeatable():
+    """The CTA-pair form on a wide layer at full size (32 x 1024 tokens, 256 -> 256 channels, T = 4: 128 pair units on
+    74 pairs): sampled outputs against the oracle, and bit-identical results on every repetition (a race between the two
+    CTAs of a pair would show up as rare corrupted rows)."""
+    wl = OPERATOR_SHAPES["op_c256_fp16"]
+    d = generate(wl)
+    rows = sample_rows(wl.N, 64, seed=5)
+    layer = GpuLayer(wl.T, wl.Ci, wl.Co, "fp16", d["w"], d["bias"], eq.EQL_FLAG_CTA_PAIR)
+    try:
+        info = eq.eqlinear_plan_info(layer.plan)
+        assert (info.fwd_kernel, info.bwd_data_kernel) == (3, 3)
+        y0, dx0 = layer.fwd(d["x"]), layer.bwd_data(d["dy"])
+        assert rel_max_err(y0[rows], orc.fwd(d["x"][rows], d["w"], d["bias"])) <= TOL["fp16"]
+        assert rel_max_err(dx0[rows], orc.bwd_data(d["dy"][rows], d["w"])) <= TOL["fp16"]
+        for _ in range(5):
+            assert np.array_equal(layer.fwd(d["x"]), y0)
+            assert np.array_equal(layer.bwd_data(d["dy"]), dx0)
+        assert layer.raw_status() == 0
+    finally:
+        layer.close()
 
 
 # ------------------------------------------------------------------ training with a saved spectrum
