@@ -67,11 +67,13 @@ enum {
      * output-channel tile) even where the kernel that keeps the transformed activations of a token
      * tile resident in shared memory applies.  For comparisons and tests. */
     EQL_FLAG_FORCE_STREAMING = 4u,
-    /* Run the streaming kernel in its CTA-pair form where it exists (FP16 plans, T = 4 or 8): clusters of two CTAs on
-     * two SMs work on neighbouring token tiles, one tcgen05.mma.cta_group::2 covers both, and each SM loads and holds
-     * only half of every spectral-weight tile.  Same results bit for bit.  Not selected by default: on B200 it
-     * measures 3-15 % slower than the single-CTA form (see the kernel's header comment). */
-    EQL_FLAG_CTA_PAIR = 8u
+    /* The streaming kernel has a CTA-pair form (FP16 plans, T = 4 or 8): clusters of two CTAs on two SMs work on
+     * neighbouring token tiles, one tcgen05.mma.cta_group::2 covers both, and each SM loads and holds only half of
+     * every spectral-weight tile.  Same results bit for bit.  Plans take it by themselves for wide layers (512 or
+     * more channels per group element on both sides), where it measures 2-10 % faster; below it measures 2-4 %
+     * slower.  EQL_FLAG_CTA_PAIR takes it wherever it exists, EQL_FLAG_NO_CTA_PAIR never (comparisons, tests). */
+    EQL_FLAG_CTA_PAIR = 8u,
+    EQL_FLAG_NO_CTA_PAIR = 16u
 };
 
 typedef struct {

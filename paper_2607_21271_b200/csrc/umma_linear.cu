@@ -14,21 +14,23 @@
 // Frequency-domain data never leaves the SM (registers, shared memory, TMEM).  The data gradient is the
 // same kernel run on dy with the conjugate-transposed weight image and no bias.
 //
-// CG = 2 ("CTA pair", on request: EQL_FLAG_CTA_PAIR): the same kernel as a cluster of two CTAs on two SMs that work on
-// two neighbouring token tiles and the same output-channel tile in lockstep.  One tcgen05.mma.cta_group::2 (M = 256)
-// issued by the pair's leader covers both token tiles; its B operand -- the spectral weight tile -- is split in halves
-// between the two CTAs, so each SM loads and holds only half of every weight tile (L2 -> SM traffic of the weights
-// halves).  Each CTA issues its own loads into its own shared memory; only mbarrier arrivals cross the pair: the
-// peer's word that its stage of a chunk is full (one remote arrive per chunk on the leader's barrier of that stage),
-// the leader's commits to the peer's "empty" and "accumulator full" barriers (a second commit each, addressed to the
-// peer), and the peer's epilogue warps releasing the accumulator to the leader.
-// Measured on B200 (T = 4, 32 768 tokens): 57.9 / 148 / 508 / 2300 us at 256 / 512 / 1024 / 2048 channels against
-// 54.8 / 141 / 496 / 1990 us for the single-CTA form, bit-identical results.  The form does not pay here because the
-// main loop is paced by the MMA-issuing thread and the SM's shared-memory bandwidth, and neither gets lighter: each
-// SM's shared memory still serves its half of B to BOTH tensor cores, the leader executes one more commit per chunk,
-// and what halves -- the weight stream from L2 -- was not the limit.  (With release / acquire at cluster scope on the
-// pair's barriers the form ran 1.7x slower: a cluster-scope release stalls the arriving thread ~1200 cycles, a
-// cluster-scope acquire ~250.)
+// CG = 2 ("CTA pair"; plans of wide layers, or EQL_FLAG_CTA_PAIR): the same kernel as a cluster of two CTAs on two SMs
+// that work on two neighbouring token tiles and the same output-channel tile in lockstep.  One
+// tcgen05.mma.cta_group::2 (M = 256) issued by the pair's leader covers both token tiles; its B operand -- the
+// spectral weight tile -- is split in halves between the two CTAs, so each SM loads and holds only half of every
+// weight tile (the L2 -> SM traffic of the weights halves).  Each CTA issues its own loads into its own shared memory;
+// only mbarrier arrivals cross the pair: the peer's word that its stage of a chunk is full (one remote arrive per
+// stage on the leader's barrier of that stage), the leader's commits to the peer's "empty" and "accumulator full"
+// barriers (a second commit each, addressed to the peer), and the peer's epilogue warps releasing the accumulator to
+// the leader.
+// Measured on B200 (T = 4, 32 768 tokens, forward): 56.7 / 135 / 476 / 1964 us at 256 / 512 / 1024 / 2048 channels
+// against 54.3 / 138 / 491 / 1937 us for the single-CTA form (data gradient at 2048: 1952 against 2168 us),
+// bit-identical results.  The gain is small because these main loops run at the SM's shared-memory bandwidth
+// (~112 KB cross shared memory per 16-channel chunk: raw rows in and out, x^ in, operand reads, weight refill; at
+// 128 B per cycle that is the measured ~880 cycles per chunk), and of those bytes the pair form removes only half
+// of the weight refill: each SM's shared memory still serves its half of B to BOTH tensor cores.
+// (With release / acquire at cluster scope on the pair's barriers the form ran 1.7x slower: a cluster-scope release
+// stalls the arriving thread ~1200 cycles, a cluster-scope acquire ~250.)
 //
 // Every wait on an mbarrier is bounded: on a time-out the CTA raises an abort flag, records a status
 // code for the host, drains its outstanding copies and MMAs, frees its TMEM and returns.
@@ -68,16 +70,18 @@ template <int T, int E, int CG = 1> struct UmmaCfg;   // E = bytes per element o
 // warps + the weight copy's bytes) and one "empty" barrier (one commit) per chunk serve both.  The single thread that
 // issues the MMAs then executes one wait and one commit per chunk instead of two each; each costs it ~200 cycles while
 // the tensor core is streaming operands, and on wide layers that thread paces the kernel.
-template <> struct UmmaCfg<4, 2, 1>  { static constexpr int SPS = 2, SA = 3, SB = 3, MAXCOT = 128; static constexpr bool EARLY = false, MERGED = true; };
-template <> struct UmmaCfg<8, 2, 1>  { static constexpr int SPS = 2, SA = 2, SB = 2, MAXCOT = 64;  static constexpr bool EARLY = false, MERGED = true; };
-template <> struct UmmaCfg<16, 2, 1> { static constexpr int SPS = 1, SA = 2, SB = 1, MAXCOT = 32;  static constexpr bool EARLY = true, MERGED = false; };
-template <> struct UmmaCfg<32, 2, 1> { static constexpr int SPS = 1, SA = 1, SB = 1, MAXCOT = 16;  static constexpr bool EARLY = true, MERGED = false; };
-template <> struct UmmaCfg<4, 4, 1>  { static constexpr int SPS = 1, SA = 3, SB = 1, MAXCOT = 128; static constexpr bool EARLY = true, MERGED = false; };
-template <> struct UmmaCfg<8, 4, 1>  { static constexpr int SPS = 1, SA = 2, SB = 1, MAXCOT = 48;  static constexpr bool EARLY = true, MERGED = false; };
+// KS: chunks (UMMA K steps) per operand stage and weight slot.  With two, the issuing thread's wait and commit are paid
+// once per 32 reduced channels (the reduction is padded to a multiple of KS chunks with zero channels).
+template <> struct UmmaCfg<4, 2, 1>  { static constexpr int SPS = 1, SA = 2, SB = 2, KS = 2, MAXCOT = 128; static constexpr bool EARLY = true, MERGED = true; };
+template <> struct UmmaCfg<8, 2, 1>  { static constexpr int SPS = 2, SA = 2, SB = 2, KS = 1, MAXCOT = 64;  static constexpr bool EARLY = false, MERGED = true; };
+template <> struct UmmaCfg<16, 2, 1> { static constexpr int SPS = 1, SA = 2, SB = 1, KS = 1, MAXCOT = 32;  static constexpr bool EARLY = true, MERGED = false; };
+template <> struct UmmaCfg<32, 2, 1> { static constexpr int SPS = 1, SA = 1, SB = 1, KS = 1, MAXCOT = 16;  static constexpr bool EARLY = true, MERGED = false; };
+template <> struct UmmaCfg<4, 4, 1>  { static constexpr int SPS = 1, SA = 3, SB = 1, KS = 1, MAXCOT = 128; static constexpr bool EARLY = true, MERGED = false; };
+template <> struct UmmaCfg<8, 4, 1>  { static constexpr int SPS = 1, SA = 2, SB = 1, KS = 1, MAXCOT = 48;  static constexpr bool EARLY = true, MERGED = false; };
 // CTA pairs: a CTA holds half of every weight tile, which leaves room for deeper rings (measured: depths beyond these
 // change nothing, for either form -- the rings are not what paces the kernel).
-template <> struct UmmaCfg<4, 2, 2>  { static constexpr int SPS = 2, SA = 4, SB = 4, MAXCOT = 128; static constexpr bool EARLY = false, MERGED = true; };
-template <> struct UmmaCfg<8, 2, 2>  { static constexpr int SPS = 2, SA = 2, SB = 2, MAXCOT = 64;  static constexpr bool EARLY = false, MERGED = true; };
+template <> struct UmmaCfg<4, 2, 2>  { static constexpr int SPS = 1, SA = 3, SB = 3, KS = 2, MAXCOT = 128; static constexpr bool EARLY = true, MERGED = true; };
+template <> struct UmmaCfg<8, 2, 2>  { static constexpr int SPS = 2, SA = 2, SB = 2, KS = 1, MAXCOT = 64;  static constexpr bool EARLY = false, MERGED = true; };
 constexpr int kRawSlots = 3;
 constexpr uint32_t kSpin = 256;               // test_wait polls before a single-thread role falls back to try_wait
 
@@ -192,7 +196,7 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
                    const UmmaParams prm) {
     constexpr int E = sizeof(IO);               // 2: half I/O, kind::f16;  4: float I/O, kind::tf32 with the 3xTF32 split
     using Cfg = UmmaCfg<T, E, CG>;
-    constexpr int SPS = Cfg::SPS, SA = Cfg::SA, SB = Cfg::SB;
+    constexpr int SPS = Cfg::SPS, SA = Cfg::SA, SB = Cfg::SB, KS = Cfg::KS;
     constexpr bool PAIR = CG == 2, MERGED = Cfg::MERGED;
     static_assert(!MERGED || SA == SB, "one barrier pair per chunk needs equally deep rings");
     static_assert(!PAIR || MERGED, "the CTA-pair form is written for the merged rings");
@@ -203,7 +207,8 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
     constexpr int SPK = KCH / NCH;              // slabs per chunk (= T/4)
     constexpr int NSPLIT = E == 4 ? 2 : 1;      // operand copies: FP32 keeps TF32 hi parts and lo remainders
     constexpr int kAPart = T * 4096;            // T planes x [128 rows x 32 B]
-    constexpr int kAStage = kAPart * NSPLIT;
+    constexpr int kAChunk = kAPart * NSPLIT;    // one chunk's operand tiles
+    constexpr int kAStage = kAChunk * KS;
     constexpr int W = NCH * E / 4;              // 32-bit words one slab row contributes to one plane
 
     extern __shared__ uint8_t smem_raw_base[];
@@ -223,7 +228,7 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
         for (int i = 0; i < kRawSlots; ++i) { ptx::mbar_init(&bar->full_raw[i], 1); ptx::mbar_init(&bar->empty_raw[i], 4 * SPS); }
         // "full" of a stage: the transform warps; merged rings: + the weight copy (its producer's arrive.expect_tx);
         // pair, leader: + the peer CTA's word that its own stage is full
-        const uint32_t full_count = 4 * SPK + (MERGED ? 1 : 0) + ((PAIR && rank == 0) ? 1 : 0);
+        const uint32_t full_count = 4 * SPK * KS + (MERGED ? 1 : 0) + ((PAIR && rank == 0) ? 1 : 0);
         for (int i = 0; i < SA; ++i) { ptx::mbar_init(&bar->full_a[i], full_count); ptx::mbar_init(&bar->empty_a[i], 1); }
         for (int i = 0; i < SB; ++i) { ptx::mbar_init(&bar->full_b[i], 1); ptx::mbar_init(&bar->empty_b[i], 1); }
         ptx::mbar_init(&bar->full_d, 1);
@@ -301,14 +306,16 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
             const uint32_t blob_bytes = (uint32_t)rowsH * kRowBytes * NSPLIT;       // pair: this CTA's half of the blob
             for (int64_t u = first; u < prm.num_units && ok; u += stride) {
                 const int tile = (int)(u % nTiles);
-                for (int kc = 0; kc < nK; ++kc, ++cb) {
+                for (int kc = 0; kc < nK; kc += KS, ++cb) {          // one slot per stage: KS chunks
                     const int slot = cb % SB;
                     ok = ptx::mbar_wait(&empty_wb[slot], ((cb / SB) & 1) ^ 1, abort_flag, status, 102, true, kSpin);
                     if (!ok) break;
-                    ptx::mbar_arrive_expect_tx(&full_wb[slot], blob_bytes);
-                    ptx::bulk_load_1d(bsm + slot * prm.b_slot_bytes,
-                                      prm.image + (((size_t)tile * nK + kc) * CG + rank) * (size_t)blob_bytes, blob_bytes,
-                                      &full_wb[slot]);
+                    ptx::mbar_arrive_expect_tx(&full_wb[slot], KS * blob_bytes);
+#pragma unroll
+                    for (int sub = 0; sub < KS; ++sub)
+                        ptx::bulk_load_1d(bsm + slot * prm.b_slot_bytes + sub * blob_bytes,
+                                          prm.image + (((size_t)tile * nK + kc + sub) * CG + rank) * (size_t)blob_bytes, blob_bytes,
+                                          &full_wb[slot]);
                 }
             }
             if (!ok) {
@@ -354,7 +361,7 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
                 ok = ptx::mbar_wait(&bar->empty_d, (cu & 1) ^ 1, abort_flag, status, 103, true, kSpin);
                 if (!ok) break;
                 ptx::tc_fence_after_sync();
-                for (int kc = 0; kc < nK; ++kc, ++ca, ++cb) {
+                for (int kc = 0; kc < nK; kc += KS, ++ca, ++cb) {    // ca, cb count stages
                     const int sa = ca % SA, sb = cb % SB;
                     // (pair: the peer's arrival on this barrier stands for shared memory of the peer CTA that the peer's own
                     // threads wrote and fenced; a wait with acquire at cluster scope instead costs ~250 cycles per chunk)
@@ -364,10 +371,12 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
                     ptx::tc_fence_after_sync();
                     // FP16: one pass.  FP32 (3xTF32): hi*hi, hi*lo, lo*hi accumulate into the same columns.
 #pragma unroll
+                    for (int sub = 0; sub < KS; ++sub)
+#pragma unroll
                     for (int pass = 0; pass < (E == 4 ? 3 : 1); ++pass) {
-                        const uint32_t a0 = ptx::smem_u32(xhat + sa * kAStage) + (pass == 2 ? kAPart : 0);
-                        const uint32_t b0 = ptx::smem_u32(bsm + sb * prm.b_slot_bytes) + (pass == 1 ? b_part : 0);
-                        const uint32_t acc = (kc > 0 || pass > 0) ? 1u : 0u;
+                        const uint32_t a0 = ptx::smem_u32(xhat + sa * kAStage + sub * kAChunk) + (pass == 2 ? kAPart : 0);
+                        const uint32_t b0 = ptx::smem_u32(bsm + sb * prm.b_slot_bytes) + sub * b_part * NSPLIT + (pass == 1 ? b_part : 0);
+                        const uint32_t acc = (kc > 0 || sub > 0 || pass > 0) ? 1u : 0u;
                         // k = 0
                         mma(tmem_base, a0, b0, idesc_real, acc);
                         // complex frequencies: [Re y^ | Im y^] (+)= Re x^ [Wr|Wi] + Im x^ [-Wi|Wr]
@@ -399,7 +408,7 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
             bool ok = true;
             const uint32_t leader_full0 = ptx::map_to_cta(ptx::smem_u32(&bar->full_a[0]), 0u);
             for (int64_t u = first; u < prm.num_units && ok; u += stride) {
-                for (int kc = 0; kc < nK; ++kc, ++ca) {
+                for (int kc = 0; kc < nK; kc += KS, ++ca) {
                     ok = ptx::mbar_wait(&bar->full_a[ca % SA], (ca / SA) & 1, abort_flag, status, 116, true, kSpin);
                     if (!ok) break;
                     ptx::mbar_arrive_remote(leader_full0 + (ca % SA) * 8u);
@@ -419,7 +428,7 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
         // (a warp that stored into chunk c' has seen the commit of chunk c' - SA, so when it next waits for the
         // commit of chunk c - SA with c - c' <= SA the barrier is at most one phase behind).
         static_assert(kRawSlots == 3 && SPS <= 3, "raw slots must map to fixed warp groups");
-        static_assert((3 + SPK - 1) / SPK <= SA, "empty_a parity wait would be ambiguous");
+        static_assert((3 + SPK * KS - 1) / (SPK * KS) <= SA, "empty_a parity wait would be ambiguous");
         const int cw = warp - kWarpCompute0;
         const int quad = warp & 3;                               // TMEM lane quadrant this warp may read
         const int group = cw >> 2;                               // transform group, and share of the epilogue's column groups
@@ -437,8 +446,9 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
         uint8_t* staging = xhat + cw * 4096;                     // this warp's [32 tokens x 128 B] output stage (128B swizzle)
         for (int64_t u = first; u < prm.num_units && ok; u += stride, ++cu) {
             // ---- transform
-            for (int kc = 0; kc < nK && ok; ++kc, ++ca) {
-                const int sa = ca % SA;
+            for (int kc = 0; kc < nK && ok; ++kc, ++ca) {           // ca counts chunks here; stage = chunk / KS
+                const uint32_t stage = ca / KS;
+                const int sa = stage % SA;
 #pragma unroll 1
                 for (int q = 0; q < SPK; ++q) {
                     const uint32_t cr = ca * SPK + q;            // running slab counter
@@ -462,7 +472,7 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
                     // this slab row's run of channels starts at byte kb of the row
                     const int kb = q * NCH * E;
                     const int sw = (r >> 2) & 1;
-                    uint8_t* dst = xhat + sa * kAStage + r * 32 + (((kb >> 4) ^ sw) << 4) + (kb & 15);
+                    uint8_t* dst = xhat + sa * kAStage + (ca % KS) * kAChunk + r * 32 + (((kb >> 4) ^ sw) << 4) + (kb & 15);
                     const int second = sw ? -16 : 16;            // where the other half of the same row lives (32-byte runs only)
                     uint32_t packed[E == 2 ? T : 1][E == 2 ? NCH / 2 : 1];
                     if constexpr (E == 2) {
@@ -470,7 +480,7 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
                     } else {
                         dft_words_f32<T>(wd);                    // wd[c*T + p] = plane p of channel c
                     }
-                    ok = ptx::mbar_wait(&bar->empty_a[sa], ((ca / SA) & 1) ^ 1, abort_flag, status, 107, true, 16);
+                    ok = ptx::mbar_wait(&bar->empty_a[sa], ((stage / SA) & 1) ^ 1, abort_flag, status, 107, true, 16);
                     if (!ok) break;
                     if (staging_pending) {                       // the previous unit's output stage lives in the A-operand stages
                         ok = ptx::mbar_wait(&bar->staging_free, (cu - 1) & 1, abort_flag, status, 109, true, 16);
@@ -601,7 +611,7 @@ EncodeTiledFn encode_tiled_fn() {
 template <int T, int E, int CG>
 size_t umma_smem_bytes(int b_slot_bytes) {
     using Cfg = UmmaCfg<T, E, CG>;
-    return 1024 + (size_t)kRawSlots * Cfg::SPS * kSlabBytes + (size_t)Cfg::SA * T * 4096 * (E == 4 ? 2 : 1) +
+    return 1024 + (size_t)kRawSlots * Cfg::SPS * kSlabBytes + (size_t)Cfg::SA * Cfg::KS * T * 4096 * (E == 4 ? 2 : 1) +
            (size_t)Cfg::SB * b_slot_bytes + sizeof(SmemBarriers) + 64;
 }
 
@@ -622,6 +632,17 @@ cudaError_t dispatch_umma(int T, int elem_bytes, F&& f) {
         case 8: return f(std::integral_constant<int, 8>{}, float{});
         default: return cudaErrorInvalidValue;
     }
+}
+
+int umma_chunks_per_stage(int T, int elem_bytes, bool pair) {
+    int k = 1;
+    dispatch_umma(T, elem_bytes, [&](auto tc, auto io) {
+        constexpr int TT = decltype(tc)::value, EE = sizeof(decltype(io));
+        k = UmmaCfg<TT, EE, 1>::KS;
+        if constexpr (EE == 2 && (TT == 4 || TT == 8)) { if (pair) k = UmmaCfg<TT, EE, 2>::KS; }
+        return cudaSuccess;
+    });
+    return k;
 }
 
 int umma_max_cot(int T, int elem_bytes) {
@@ -650,7 +671,8 @@ UmmaLinearShape umma_linear_shape(int T, int Cin, int Cout, eql_dtype_t dtype) {
     const int per = (Cout + s.nTiles - 1) / s.nTiles;
     s.CoT = (per + 15) / 16 * 16;
     const int kch = kRowBytes / s.elem_bytes;                    // channels per chunk (one UMMA K step)
-    s.nK = (Cin + kch - 1) / kch;
+    const int ks = umma_chunks_per_stage(T, s.elem_bytes, false);   // (the same for the pair form of every T that has one)
+    s.nK = ((Cin + kch - 1) / kch + ks - 1) / ks * ks;         // whole stages: the padding chunks hold zero channels
     s.rowsB = (2 * T - 2) * s.CoT;
     s.image_bytes = align_up((size_t)s.nTiles * s.nK * s.rowsB * kRowBytes * (s.elem_bytes == 4 ? 2 : 1), kWsAlign);
     s.cin0 = 0; s.CinTotal = Cin;
@@ -724,7 +746,8 @@ cudaError_t launch_umma_linear(const UmmaLinearShape& s, const void* in, void* o
     prm.N = N; prm.Cin = s.Cin; prm.Cout = s.Cout;
     prm.CoT = s.CoT; prm.nTiles = s.nTiles; prm.nK = s.nK; prm.rowsB = s.rowsB;
     const int cg = s.pair ? 2 : 1;
-    prm.b_slot_bytes = (int)align_up((size_t)(s.rowsB / cg) * kRowBytes * (s.elem_bytes == 4 ? 2 : 1), 256);
+    prm.b_slot_bytes = (int)align_up((size_t)(s.rowsB / cg) * kRowBytes * (s.elem_bytes == 4 ? 2 : 1) *
+                                         umma_chunks_per_stage(s.T, s.elem_bytes, s.pair), 256);
     const int64_t token_tiles = (N + kTileM - 1) / kTileM;
     prm.num_units = ((token_tiles + cg - 1) / cg) * s.nTiles;    // a pair takes two token tiles per unit
     prm.accumulate = accumulate ? 1 : 0;

@@ -129,7 +129,7 @@ def test_resident_and_streaming_kernels_agree_with_oracle(T, Ci, Co, N, ids):
     wl = Workload("res", "fp16", T, Ci, Co, N, "normal", ("fwd", "bwd_data"), 21)
     data = eq.workloads.generate(wl)
     outs = {}
-    for flags, want in ((0, ids), (eq.EQL_FLAG_FORCE_STREAMING, (1, 1)),
+    for flags, want in ((0, ids), (eq.EQL_FLAG_FORCE_STREAMING, (1, 1)),   # (narrow layers: no pair form by default)
                         (eq.EQL_FLAG_FORCE_STREAMING | eq.EQL_FLAG_CTA_PAIR, (3, 3))):
         layer = GpuLayer(T, Ci, Co, "fp16", data["w"], data["bias"], flags)
         try:
@@ -146,23 +146,31 @@ def test_resident_and_streaming_kernels_agree_with_oracle(T, Ci, Co, N, ids):
 
 
 def test_cta_pair_form_at_full_size_is_repeatable():
-    """The CTA-pair form on a wide layer at full size (32 x 1024 tokens, 256 -> 256 channels, T = 4: 128 pair units on
-    74 pairs): sampled outputs against the oracle, and bit-identical results on every repetition (a race between the two
-    CTAs of a pair would show up as rare corrupted rows)."""
-    wl = OPERATOR_SHAPES["op_c256_fp16"]
+    """A wide layer at full size (32 x 1024 tokens, 512 -> 512 channels, T = 4): the plan takes the CTA-pair form by
+    itself (id 3).  Sampled outputs against the oracle, bit-identical results on every repetition (a race between the two
+    CTAs of a pair would show up as rare corrupted rows), and bit-identical to the single-CTA form
+    (EQL_FLAG_NO_CTA_PAIR, id 1)."""
+    wl = OPERATOR_SHAPES["op_c512_fp16"]
     d = generate(wl)
     rows = sample_rows(wl.N, 64, seed=5)
-    layer = GpuLayer(wl.T, wl.Ci, wl.Co, "fp16", d["w"], d["bias"], eq.EQL_FLAG_CTA_PAIR)
+    layer = GpuLayer(wl.T, wl.Ci, wl.Co, "fp16", d["w"], d["bias"])
     try:
         info = eq.eqlinear_plan_info(layer.plan)
         assert (info.fwd_kernel, info.bwd_data_kernel) == (3, 3)
         y0, dx0 = layer.fwd(d["x"]), layer.bwd_data(d["dy"])
         assert rel_max_err(y0[rows], orc.fwd(d["x"][rows], d["w"], d["bias"])) <= TOL["fp16"]
         assert rel_max_err(dx0[rows], orc.bwd_data(d["dy"][rows], d["w"])) <= TOL["fp16"]
-        for _ in range(5):
+        for _ in range(4):
             assert np.array_equal(layer.fwd(d["x"]), y0)
             assert np.array_equal(layer.bwd_data(d["dy"]), dx0)
         assert layer.raw_status() == 0
+    finally:
+        layer.close()
+    layer = GpuLayer(wl.T, wl.Ci, wl.Co, "fp16", d["w"], d["bias"], eq.EQL_FLAG_NO_CTA_PAIR)
+    try:
+        info = eq.eqlinear_plan_info(layer.plan)
+        assert (info.fwd_kernel, info.bwd_data_kernel) == (1, 1)
+        assert np.array_equal(layer.fwd(d["x"]), y0) and np.array_equal(layer.bwd_data(d["dy"]), dx0)
     finally:
         layer.close()
 
