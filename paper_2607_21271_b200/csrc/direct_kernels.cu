@@ -18,10 +18,19 @@ template <int BYTES>
 struct VecBytes { using type = uint4; static constexpr int n = BYTES / 16; };
 template <> struct VecBytes<8> { using type = uint2; static constexpr int n = 1; };
 template <> struct VecBytes<4> { using type = uint32_t; static constexpr int n = 1; };
+// group tuples of other sizes (odd or non-power-of-two group orders) are not aligned to a vector: element by element
+constexpr bool vector_tuple(int bytes) { return bytes == 4 || bytes == 8 || (bytes >= 16 && bytes % 16 == 0); }
 
 template <int T, typename IO>
 __device__ __forceinline__ void load_group(const IO* __restrict__ p, float* v) {
-    using V = VecBytes<T * sizeof(IO)>;
+    if constexpr (!vector_tuple(T * sizeof(IO))) {
+#pragma unroll
+        for (int i = 0; i < T; ++i) {
+            if constexpr (sizeof(IO) == 4) v[i] = __ldg(p + i); else v[i] = __half2float(__ldg(p + i));
+        }
+        return;
+    }
+    using V = VecBytes<vector_tuple(T * sizeof(IO)) ? T * sizeof(IO) : 16>;
     union { typename V::type vec[V::n]; IO e[T]; } u;
 #pragma unroll
     for (int i = 0; i < V::n; ++i) u.vec[i] = __ldg(reinterpret_cast<const typename V::type*>(p) + i);
@@ -33,7 +42,14 @@ __device__ __forceinline__ void load_group(const IO* __restrict__ p, float* v) {
 
 template <int T, typename IO>
 __device__ __forceinline__ void store_group(IO* __restrict__ p, const float* v) {
-    using V = VecBytes<T * sizeof(IO)>;
+    if constexpr (!vector_tuple(T * sizeof(IO))) {
+#pragma unroll
+        for (int i = 0; i < T; ++i) {
+            if constexpr (sizeof(IO) == 4) p[i] = v[i]; else p[i] = __float2half_rn(v[i]);
+        }
+        return;
+    }
+    using V = VecBytes<vector_tuple(T * sizeof(IO)) ? T * sizeof(IO) : 16>;
     union { typename V::type vec[V::n]; IO e[T]; } u;
 #pragma unroll
     for (int i = 0; i < T; ++i) {
@@ -44,12 +60,33 @@ __device__ __forceinline__ void store_group(IO* __restrict__ p, const float* v) 
 }
 
 // ---- tile shapes: 256 threads as 16 x 16, each owning TM x TN (row, column) pairs for all T planes
-template <int T> struct DirectCfg;
-template <> struct DirectCfg<2>  { static constexpr int TM = 8, TN = 4, BK = 8; };
-template <> struct DirectCfg<4>  { static constexpr int TM = 8, TN = 4, BK = 8; };
-template <> struct DirectCfg<8>  { static constexpr int TM = 4, TN = 4, BK = 8; };
-template <> struct DirectCfg<16> { static constexpr int TM = 4, TN = 2, BK = 4; };
-template <> struct DirectCfg<32> { static constexpr int TM = 2, TN = 2, BK = 4; };
+template <int T> struct DirectCfg {        // by register budget: T * TM * TN accumulators per thread
+    static constexpr int TM = T <= 4 ? 8 : T <= 8 ? 4 : T <= 16 ? 4 : 2;
+    static constexpr int TN = T <= 8 ? 4 : 2;
+    static constexpr int BK = T <= 8 ? 8 : 4;
+};
+
+// Transforms of one group tuple: butterflies for the power-of-two orders, the twiddle table `tw` (T entries of
+// (cos, sin)(2 pi j / T), filled by fill_twiddles at the start of the kernel) for the others.
+template <int T>
+__device__ __forceinline__ void dft_fwd(float* v, const float2* tw) {
+    if constexpr (rdft_has_butterflies(T)) rdft_forward<T>(v); else rdft_forward_table<T>(v, tw);
+}
+template <int T>
+__device__ __forceinline__ void dft_inv(float* v, const float2* tw) {
+    if constexpr (rdft_has_butterflies(T)) rdft_inverse<T>(v); else rdft_inverse_table<T>(v, tw);
+}
+template <int T>
+__device__ __forceinline__ void fill_twiddles(float2* tw) {
+    if constexpr (!rdft_has_butterflies(T)) {
+        if (threadIdx.x < T) {
+            float s, c;
+            sincospif(2.0f * (float)threadIdx.x / (float)T, &s, &c);
+            tw[threadIdx.x] = make_float2(c, s);
+        }
+        __syncthreads();
+    }
+}
 
 constexpr int kThreads = 256;
 constexpr int kPad = 4;
@@ -64,10 +101,10 @@ __device__ __forceinline__ void plane_mac(float (&acc)[T][TM][TN], const float (
 #pragma unroll
         for (int j = 0; j < TN; ++j) {
             acc[0][i][j] = fmaf(a[0][i], b[0][j], acc[0][i][j]);
-            acc[T - 1][i][j] = fmaf(a[T - 1][i], b[T - 1][j], acc[T - 1][i][j]);
+            if constexpr (T % 2 == 0) acc[T - 1][i][j] = fmaf(a[T - 1][i], b[T - 1][j], acc[T - 1][i][j]);   // k = T/2
         }
 #pragma unroll
-    for (int k = 1; k < T / 2; ++k) {
+    for (int k = 1; k <= (T - 1) / 2; ++k) {
         const int pr = 2 * k - 1, pi = 2 * k;
 #pragma unroll
         for (int i = 0; i < TM; ++i)
@@ -114,6 +151,8 @@ template <int T, typename IO>
 __global__ void plan_weights_kernel(const IO* __restrict__ w, const IO* __restrict__ bias, int Ci, int Co,
                                     bool correlation, float* __restrict__ pf, float* __restrict__ pb,
                                     float* __restrict__ bias_f32) {
+    __shared__ float2 tw[T];
+    fill_twiddles<T>(tw);
     const int idx = blockIdx.x * blockDim.x + threadIdx.x;
     if (idx < Co && bias_f32 != nullptr) {
         if constexpr (sizeof(IO) == 4) bias_f32[idx] = bias[idx]; else bias_f32[idx] = __half2float(bias[idx]);
@@ -125,10 +164,10 @@ __global__ void plan_weights_kernel(const IO* __restrict__ w, const IO* __restri
     for (int r = 0; r < T; ++r) {
         if constexpr (sizeof(IO) == 4) v[r] = w[(size_t)idx * T + r]; else v[r] = __half2float(w[(size_t)idx * T + r]);
     }
-    rdft_forward<T>(v);
+    dft_fwd<T>(v, tw);
 #pragma unroll
     for (int p = 0; p < T; ++p) {
-        const bool imag = (p != 0) && (p != T - 1) && ((p & 1) == 0);
+        const bool imag = plane_is_imag<T>(p);
         float f = v[p] * plane_inverse_scale<T>(p);
         if (imag && correlation) f = -f;
         pf[((size_t)p * Ci + i) * Co + o] = f;
@@ -147,6 +186,8 @@ direct_linear_kernel(const IO* __restrict__ in, IO* __restrict__ out, int64_t N,
     constexpr int TM = C::TM, TN = C::TN, BK = C::BK, BM = 16 * TM, BN = 16 * TN;
     __shared__ __align__(16) float xs[T][BK][BM + kPad];
     __shared__ __align__(16) float ws[T][BK][BN + kPad];
+    __shared__ float2 tw[T];
+    fill_twiddles<T>(tw);
 
     const int tid = threadIdx.x, tm = tid & 15, tn = tid >> 4;
     const int64_t m0 = (int64_t)blockIdx.x * BM;
@@ -168,7 +209,7 @@ direct_linear_kernel(const IO* __restrict__ in, IO* __restrict__ out, int64_t N,
             const int64_t row = m0 + m;
             if (row < N && k0 + kk < Cin) {
                 load_group<T, IO>(in + row * (int64_t)Cin * T + (int64_t)(k0 + kk) * T, v);
-                rdft_forward<T>(v);
+                dft_fwd<T>(v, tw);
             } else {
 #pragma unroll
                 for (int p = 0; p < T; ++p) v[p] = 0.f;
@@ -209,7 +250,7 @@ direct_linear_kernel(const IO* __restrict__ in, IO* __restrict__ out, int64_t N,
 #pragma unroll
             for (int p = 0; p < T; ++p) v[p] = acc[p][i][j];
             if (bias != nullptr) v[0] += __ldg(bias + n);     // a constant over t lives in plane k = 0
-            rdft_inverse<T>(v);
+            dft_inv<T>(v, tw);
             store_group<T, IO>(out + row * (int64_t)Cout * T + (int64_t)n * T, v);
         }
     }
@@ -226,6 +267,8 @@ direct_bwd_weight_kernel(const IO* __restrict__ x, const IO* __restrict__ dy, in
     constexpr int TO = C::TM, TI = C::TN, BK = C::BK, BO = 16 * TO, BI = 16 * TI;
     __shared__ __align__(16) float gs[T][BK][BO + kPad];
     __shared__ __align__(16) float xs[T][BK][BI + kPad];
+    __shared__ float2 tw[T];
+    fill_twiddles<T>(tw);
 
     const int tid = threadIdx.x, to = tid & 15, ti = tid >> 4;
     const int o0 = blockIdx.x * BO, i0 = blockIdx.y * BI, split = blockIdx.z;
@@ -249,7 +292,7 @@ direct_bwd_weight_kernel(const IO* __restrict__ x, const IO* __restrict__ dy, in
             float v[T];
             if (n0 + kk < nend && o0 + o < Co) {
                 load_group<T, IO>(dy + (n0 + kk) * (int64_t)Co * T + (int64_t)(o0 + o) * T, v);
-                rdft_forward<T>(v);
+                dft_fwd<T>(v, tw);
             } else {
 #pragma unroll
                 for (int p = 0; p < T; ++p) v[p] = 0.f;
@@ -262,7 +305,7 @@ direct_bwd_weight_kernel(const IO* __restrict__ x, const IO* __restrict__ dy, in
             float v[T];
             if (n0 + kk < nend && i0 + i < Ci) {
                 load_group<T, IO>(x + (n0 + kk) * (int64_t)Ci * T + (int64_t)(i0 + i) * T, v);
-                rdft_forward<T>(v);
+                dft_fwd<T>(v, tw);
             } else {
 #pragma unroll
                 for (int p = 0; p < T; ++p) v[p] = 0.f;
@@ -311,6 +354,8 @@ __global__ void __launch_bounds__(32 * T)
 bwd_weight_finalize_kernel(const float* __restrict__ part, const float* __restrict__ db_part, int splits, int Ci,
                            int Co, bool correlation, float* __restrict__ dw, float* __restrict__ db, bool accumulate) {
     __shared__ float planes[T][33];
+    __shared__ float2 tw[T];
+    fill_twiddles<T>(tw);
     const int pair = threadIdx.x & 31, p = threadIdx.x >> 5;
     const int idx = blockIdx.x * 32 + pair;
     const size_t plane_stride = (size_t)Co * Ci;
@@ -341,7 +386,7 @@ bwd_weight_finalize_kernel(const float* __restrict__ part, const float* __restri
         for (; sp < splits; ++sp) a0 += __ldg(src + (size_t)sp * step);
         acc = (a0 + a1) + (a2 + a3);
     }
-    const bool imag = (p != 0) && (p != T - 1) && ((p & 1) == 0);
+    const bool imag = plane_is_imag<T>(p);
     acc *= plane_inverse_scale<T>(p);
     if (imag && correlation) acc = -acc;
     planes[p][pair] = acc;
@@ -350,7 +395,7 @@ bwd_weight_finalize_kernel(const float* __restrict__ part, const float* __restri
         float v[T];
 #pragma unroll
         for (int q = 0; q < T; ++q) v[q] = planes[q][pair];
-        rdft_inverse<T>(v);
+        dft_inv<T>(v, tw);
 #pragma unroll
         for (int r = 0; r < T; ++r) dw[(size_t)idx * T + r] = accumulate ? dw[(size_t)idx * T + r] + v[r] : v[r];
     }
@@ -364,10 +409,16 @@ inline int finalize_blocks(int T, int Ci, int Co) {
 
 template <typename F>
 cudaError_t dispatch_T(int T, F&& f) {
-    switch (T) {
+    switch (T) {                                  // the orders supported_T() lists
+        case 1: return f(std::integral_constant<int, 1>{});
         case 2: return f(std::integral_constant<int, 2>{});
+        case 3: return f(std::integral_constant<int, 3>{});
         case 4: return f(std::integral_constant<int, 4>{});
+        case 5: return f(std::integral_constant<int, 5>{});
+        case 6: return f(std::integral_constant<int, 6>{});
+        case 7: return f(std::integral_constant<int, 7>{});
         case 8: return f(std::integral_constant<int, 8>{});
+        case 12: return f(std::integral_constant<int, 12>{});
         case 16: return f(std::integral_constant<int, 16>{});
         case 32: return f(std::integral_constant<int, 32>{});
         default: return cudaErrorInvalidValue;
@@ -413,13 +464,7 @@ cudaError_t launch_direct_linear(int T, eql_dtype_t dtype, const void* in, void*
 }
 
 BwdWeightSplit direct_bwd_weight_split(int T, int Ci, int Co, int64_t N) {
-    int TO = 4, TI = 4, BK = 8;
-    switch (T) {
-        case 2: case 4: TO = 8; TI = 4; BK = 8; break;
-        case 8: TO = 4; TI = 4; BK = 8; break;
-        case 16: TO = 4; TI = 2; BK = 4; break;
-        default: TO = 2; TI = 2; BK = 4; break;
-    }
+    const int TO = T <= 4 ? 8 : T <= 16 ? 4 : 2, TI = T <= 8 ? 4 : 2, BK = T <= 8 ? 8 : 4;       // DirectCfg<T>
     const int64_t tiles = (int64_t)((Co + 16 * TO - 1) / (16 * TO)) * ((Ci + 16 * TI - 1) / (16 * TI));
     int64_t want = (kNumSMs + tiles - 1) / tiles;                // about one block per SM: fewer partial spectra to write and re-read
     const int64_t chunks = (N + BK - 1) / BK;

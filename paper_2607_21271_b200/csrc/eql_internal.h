@@ -48,7 +48,9 @@ struct SmemLimitOnce {
     }
 };
 
-inline bool supported_T(int T) { return T == 2 || T == 4 || T == 8 || T == 16 || T == 32; }
+// Group orders the library is built for: every order up to 8, and 12, 16, 32.  The powers of two use butterflies and (4
+// to 32, 2 not) the tensor-core kernels; the others run the CUDA-core kernels with a table-driven transform.
+inline bool supported_T(int T) { return (T >= 1 && T <= 8) || T == 12 || T == 16 || T == 32; }
 
 // ---- CUDA-core (FFMA) kernels, direct_kernels.cu -------------------------------------------------
 // Spectral weight: w[Co][Ci][T] -> planes_fwd[T][Ci][Co], planes_bwd[T][Co][Ci] (float), bias -> float.

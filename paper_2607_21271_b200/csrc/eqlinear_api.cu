@@ -209,7 +209,7 @@ const char* eqlinear_status_string(eql_status_t status) {
     switch (status) {
         case EQL_OK: return "ok";
         case EQL_ERR_INVALID_ARG: return "invalid argument";
-        case EQL_ERR_UNSUPPORTED: return "unsupported shape (group order must be 2, 4, 8, 16 or 32)";
+        case EQL_ERR_UNSUPPORTED: return "unsupported shape (group order must be 1..8, 12, 16 or 32)";
         case EQL_ERR_ALIGNMENT: return "pointer or row size not 16-byte aligned";
         case EQL_ERR_WORKSPACE: return "workspace, scratch or staging buffer too small";
         case EQL_ERR_ARCH: return "device is not compute capability 10.x (B200)";

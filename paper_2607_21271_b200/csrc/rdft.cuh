@@ -1,10 +1,12 @@
-// Real DFT / inverse real DFT of length T in {1, 2, 4, 8, 16, 32} along the group axis, held entirely
-// in registers (Algorithm 1, steps 1 and 4; Eq. 4 and Eq. 7; the T = 4 case reduces to Eq. 19 and Eq. 21).
+// Real DFT / inverse real DFT of length T along the group axis, held entirely in registers (Algorithm 1, steps 1 and
+// 4; Eq. 4 and Eq. 7; the T = 4 case reduces to Eq. 19 and Eq. 21).  Powers of two up to 32 run radix-2 butterflies;
+// any other length (Algorithm 1 is stated for every cyclic group) is evaluated directly from a twiddle table
+// (rdft_forward_table / rdft_inverse_table below).
 //
 // Real-packed plane order used everywhere in the library (T values in, T values out):
 //   plane 0        : k = 0                    (real)
 //   plane 2k-1, 2k : Re, Im of frequency k    for 0 < k < T/2
-//   plane T-1      : k = T/2                  (real; T >= 2)
+//   plane T-1      : k = T/2                  (real; even T only -- for odd T plane T-1 is Im of k = (T-1)/2)
 //
 // Forward:  X_k = sum_s x_s e^{-2 pi i k s / T}                 (unnormalised, Eq. 4)
 // Inverse:  y_t = P_0 + (-1)^t P_{T-1} + sum_{0<k<T/2} ( P_{2k-1} cos(2 pi k t/T) - P_{2k} sin(2 pi k t/T) )
@@ -181,7 +183,57 @@ EQL_HD void rdft_inverse(float* v) {
 // Scale that turns a true (unnormalised) spectrum plane into the pre-scaled plane rdft_inverse expects.
 template <int T>
 EQL_HD float plane_inverse_scale(int plane) {
-    return (plane == 0 || plane == T - 1) ? (1.0f / T) : (2.0f / T);
+    return (plane == 0 || (T % 2 == 0 && plane == T - 1)) ? (1.0f / T) : (2.0f / T);
+}
+// Plane p holds the imaginary part of a complex frequency (the planes that change sign under conjugation).
+template <int T>
+EQL_HD bool plane_is_imag(int plane) {
+    return plane > 0 && plane % 2 == 0;          // for even T the last plane (k = T/2, real) has an odd index
+}
+
+constexpr bool rdft_has_butterflies(int T) { return T >= 1 && T <= 32 && (T & (T - 1)) == 0; }
+
+// ---- any length: direct evaluation with a table tw[j] = (cos, sin)(2 pi j / T), j = 0..T-1 (shared or global memory).
+// The loops are fully unrolled for a compile-time T, so every table index is a constant.
+template <int T>
+EQL_HD void rdft_forward_table(float* v, const float2* tw) {
+    float out[T];
+    float s0 = 0.f;
+    static_for<T>([&](auto ss) { s0 += v[decltype(ss)::value]; });
+    out[0] = s0;
+    static_for<(T - 1) / 2>([&](auto kk) {
+        constexpr int k = decltype(kk)::value + 1;
+        float re = 0.f, im = 0.f;
+        static_for<T>([&](auto ss) {
+            constexpr int s = decltype(ss)::value, j = (k * s) % T;
+            re += v[s] * tw[j].x;
+            im -= v[s] * tw[j].y;                        // e^{-2 pi i k s / T}
+        });
+        out[2 * k - 1] = re;
+        out[2 * k] = im;
+    });
+    if constexpr (T % 2 == 0) {
+        float a = 0.f;
+        static_for<T>([&](auto ss) { constexpr int s = decltype(ss)::value; a += (s % 2) ? -v[s] : v[s]; });
+        out[T - 1] = a;
+    }
+    static_for<T>([&](auto ss) { v[decltype(ss)::value] = out[decltype(ss)::value]; });
+}
+// Inverse on pre-scaled planes (see the header of this file).
+template <int T>
+EQL_HD void rdft_inverse_table(float* v, const float2* tw) {
+    float out[T];
+    static_for<T>([&](auto tt) {
+        constexpr int t = decltype(tt)::value;
+        float y = v[0];
+        if constexpr (T % 2 == 0) y += (t % 2) ? -v[T - 1] : v[T - 1];
+        static_for<(T - 1) / 2>([&](auto kk) {
+            constexpr int k = decltype(kk)::value + 1, j = (k * t) % T;
+            y += v[2 * k - 1] * tw[j].x - v[2 * k] * tw[j].y;
+        });
+        out[t] = y;
+    });
+    static_for<T>([&](auto tt) { v[decltype(tt)::value] = out[decltype(tt)::value]; });
 }
 
 }  // namespace eql

@@ -58,7 +58,9 @@ def test_ragged_token_counts(dtype, N):
 
 @pytest.mark.parametrize("dtype", ["fp32", "fp16"])
 @pytest.mark.parametrize("T,Ci,Co", [(2, 8, 16), (4, 64, 64), (4, 6, 10), (8, 96, 384), (8, 384, 96),
-                                       (16, 17, 33), (32, 32, 32), (32, 5, 3)])
+                                       (16, 17, 33), (32, 32, 32), (32, 5, 3),
+                                       # Algorithm 1 for other cyclic groups: odd and non-power-of-two orders, and the trivial group
+                                       (1, 16, 8), (3, 8, 16), (5, 8, 24), (6, 12, 20), (7, 8, 8), (12, 10, 6)])
 def test_shapes(dtype, T, Ci, Co):
     wl = Workload("shape", dtype, T, Ci, Co, 333, "normal", ("fwd", "bwd_data", "bwd_weight"), 12)
     for k, v in check_workload(wl).items():
@@ -285,8 +287,9 @@ def test_paper_parity_shape(dtype):
 
 
 @pytest.mark.parametrize("dtype", ["fp32", "fp16"])
-def test_correlation_flag_and_no_bias(dtype):
-    wl = Workload("corr", dtype, 8, 16, 24, 300, "none", ("fwd", "bwd_data", "bwd_weight"), 14)
+@pytest.mark.parametrize("T", [8, 5, 6])
+def test_correlation_flag_and_no_bias(dtype, T):
+    wl = Workload("corr", dtype, T, 16, 24, 300, "none", ("fwd", "bwd_data", "bwd_weight"), 14)
     for k, v in check_workload(wl, flags=eq.EQL_FLAG_CORRELATION).items():
         assert v <= TOL[dtype], f"{k} error {v:.3e}"
 
@@ -396,7 +399,7 @@ def test_plan_is_refused_on_another_device():
 
 
 # ------------------------------------------------------------------ invariants on the GPU output alone
-@pytest.mark.parametrize("dtype,T", [("fp32", 4), ("fp32", 8), ("fp16", 16)])
+@pytest.mark.parametrize("dtype,T", [("fp32", 4), ("fp32", 8), ("fp16", 16), ("fp32", 5), ("fp32", 12)])
 def test_gpu_equivariance_and_adjoint(dtype, T):
     wl = Workload("inv", dtype, T, 16, 24, 512, "normal", ("fwd", "bwd_data", "bwd_weight"), 19)
     d = generate(wl)

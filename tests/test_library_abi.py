@@ -43,7 +43,7 @@ def test_mac_counts_match_the_paper():
     assert spectral * 16 == dense * 6
     assert abs(2 * dense / 1e9 - 0.134) < 1e-3            # Table 1: 0.134 GFLOPs for the dense layer
     # exact count for even T: (2T - 2) N Ci Co; never more than the paper's bound 4NDC/T^2 (T/2+1)
-    for T in (2, 4, 8, 16, 32):
+    for T in (2, 4, 6, 8, 12, 16, 32):
         s, d = eq.eqlinear_count_macs(T, 3, 5, 7)
         assert s == (2 * T - 2) * 7 * 3 * 5
         assert d == 7 * (3 * T) * (5 * T)
@@ -60,10 +60,12 @@ def test_status_strings():
 
 def test_workspace_bytes_validation():
     assert eq.eqlinear_workspace_bytes(8, 96, 384, eq.EQL_FP16) >= 2 * 8 * 96 * 384 * 4
-    for bad_T in (3, 5, 64):
+    for bad_T in (9, 11, 24, 64):
         with pytest.raises(eq.EqlError) as e:
             eq.eqlinear_workspace_bytes(bad_T, 8, 8, eq.EQL_FP32)
         assert e.value.status == binding.EQL_ERR_UNSUPPORTED
+    for T in (1, 3, 5, 6, 7, 12):                          # odd and other non-power-of-two orders are planned for
+        assert eq.eqlinear_workspace_bytes(T, 8, 8, eq.EQL_FP32) >= 2 * T * 64 * 4
     with pytest.raises(eq.EqlError) as e:
         eq.eqlinear_workspace_bytes(4, 0, 8, eq.EQL_FP32)
     assert e.value.status == binding.EQL_ERR_INVALID_ARG
@@ -82,7 +84,7 @@ def test_plan_argument_errors_are_caught_before_any_cuda_call():
     assert lib.eqlinear_plan(ctypes.byref(h), 4, 8, 8, 0, None, None, 256, 1 << 20, 0, None) == binding.EQL_ERR_INVALID_ARG
     assert h.value is None
     # unsupported group order
-    assert lib.eqlinear_plan(ctypes.byref(h), 6, 8, 8, 0, 256, None, 256, 1 << 20, 0, None) == binding.EQL_ERR_UNSUPPORTED
+    assert lib.eqlinear_plan(ctypes.byref(h), 9, 8, 8, 0, 256, None, 256, 1 << 20, 0, None) == binding.EQL_ERR_UNSUPPORTED
     # misaligned weight / workspace
     assert lib.eqlinear_plan(ctypes.byref(h), 4, 8, 8, 0, 260, None, 256, 1 << 20, 0, None) == binding.EQL_ERR_ALIGNMENT
     assert lib.eqlinear_plan(ctypes.byref(h), 4, 8, 8, 0, 256, None, 272, 1 << 20, 0, None) == binding.EQL_ERR_ALIGNMENT
