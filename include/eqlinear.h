@@ -73,7 +73,14 @@ enum {
      * more channels per group element on both sides), where it measures 2-10 % faster; below it measures 2-4 %
      * slower.  EQL_FLAG_CTA_PAIR takes it wherever it exists, EQL_FLAG_NO_CTA_PAIR never (comparisons, tests). */
     EQL_FLAG_CTA_PAIR = 8u,
-    EQL_FLAG_NO_CTA_PAIR = 16u
+    EQL_FLAG_NO_CTA_PAIR = 16u,
+    /* Forward pass only: apply GELU (exact form, x * Phi(x)) to every output element in the epilogue, in FP32, before
+     * the result is rounded and stored -- the fc1 -> GELU pair of a transformer MLP block as one kernel (a pointwise
+     * map applied to each group element alike keeps the layer equivariant).  For inference: eqlinear_bwd_data and
+     * eqlinear_bwd_weight remain the gradients of the LINEAR layer; a caller that trains multiplies dy by GELU'(pre-
+     * activation) itself and therefore needs the unfused forward.  EQL_ERR_UNSUPPORTED for FP32 plans on the tensor
+     * cores with more than 256 input channels (their forward sums segments in global memory). */
+    EQL_FLAG_GELU = 32u
 };
 
 typedef struct {

@@ -31,6 +31,7 @@ EQL_FLAG_FORCE_SIMT = 2
 EQL_FLAG_FORCE_STREAMING = 4
 EQL_FLAG_CTA_PAIR = 8
 EQL_FLAG_NO_CTA_PAIR = 16
+EQL_FLAG_GELU = 32
 
 EQL_STATIC_SCRATCH_BYTES = 32 << 20
 

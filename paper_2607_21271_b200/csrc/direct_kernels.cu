@@ -181,7 +181,7 @@ __global__ void plan_weights_kernel(const IO* __restrict__ w, const IO* __restri
 template <int T, typename IO>
 __global__ void __launch_bounds__(kThreads)
 direct_linear_kernel(const IO* __restrict__ in, IO* __restrict__ out, int64_t N, int Cin, int Cout,
-                     const float* __restrict__ planes, const float* __restrict__ bias) {
+                     const float* __restrict__ planes, const float* __restrict__ bias, int act) {
     using C = DirectCfg<T>;
     constexpr int TM = C::TM, TN = C::TN, BK = C::BK, BM = 16 * TM, BN = 16 * TN;
     __shared__ __align__(16) float xs[T][BK][BM + kPad];
@@ -251,6 +251,10 @@ direct_linear_kernel(const IO* __restrict__ in, IO* __restrict__ out, int64_t N,
             for (int p = 0; p < T; ++p) v[p] = acc[p][i][j];
             if (bias != nullptr) v[0] += __ldg(bias + n);     // a constant over t lives in plane k = 0
             dft_inv<T>(v, tw);
+            if (act) {
+#pragma unroll
+                for (int q = 0; q < T; ++q) v[q] = 0.5f * v[q] * (1.0f + erff(v[q] * 0.70710678118654752440f));   // GELU
+            }
             store_group<T, IO>(out + row * (int64_t)Cout * T + (int64_t)n * T, v);
         }
     }
@@ -447,7 +451,7 @@ cudaError_t launch_plan_weights(int T, eql_dtype_t dtype, bool correlation, cons
 
 cudaError_t launch_direct_linear(int T, eql_dtype_t dtype, const void* in, void* out, int64_t N,
                                  int Cin, int Cout, const float* planes, const float* bias_f32,
-                                 cudaStream_t stream) {
+                                 cudaStream_t stream, int act) {
     return dispatch_T(T, [&](auto tc) {
         constexpr int TT = decltype(tc)::value;
         using C = DirectCfg<TT>;
@@ -455,10 +459,10 @@ cudaError_t launch_direct_linear(int T, eql_dtype_t dtype, const void* in, void*
         dim3 grid((unsigned)((N + BM - 1) / BM), (unsigned)((Cout + BN - 1) / BN));
         if (dtype == EQL_FP32)
             direct_linear_kernel<TT, float><<<grid, kThreads, 0, stream>>>(
-                (const float*)in, (float*)out, N, Cin, Cout, planes, bias_f32);
+                (const float*)in, (float*)out, N, Cin, Cout, planes, bias_f32, act);
         else
             direct_linear_kernel<TT, __half><<<grid, kThreads, 0, stream>>>(
-                (const __half*)in, (__half*)out, N, Cin, Cout, planes, bias_f32);
+                (const __half*)in, (__half*)out, N, Cin, Cout, planes, bias_f32, act);
         return cudaGetLastError();
     });
 }

@@ -61,7 +61,7 @@ cudaError_t launch_plan_weights(int T, eql_dtype_t dtype, bool correlation, cons
 // out[N, Cout*T] = inverse_dft( dft(in[N, Cin*T]) (x) planes[T][Cin][Cout] ) + bias   (bias may be NULL)
 cudaError_t launch_direct_linear(int T, eql_dtype_t dtype, const void* in, void* out, int64_t N,
                                  int Cin, int Cout, const float* planes, const float* bias_f32,
-                                 cudaStream_t stream);
+                                 cudaStream_t stream, int act = 0);
 
 // Split-K layout of the weight-gradient reduction.
 struct BwdWeightSplit {
@@ -90,6 +90,7 @@ struct UmmaLinearShape {
     // CTA-pair form (tcgen05 cta_group::2): two CTAs on two SMs share every weight tile, half each; the operand image is
     // laid out for it, so a shape is either one or the other.
     bool pair;
+    int act;            // 1: GELU on the result before it is stored (forward only)
 };
 bool umma_linear_supported(int T, eql_dtype_t dtype);
 bool umma_linear_pair_supported(int T, eql_dtype_t dtype);
@@ -119,6 +120,7 @@ struct UmmaResShape {
     bool fits;          // the spectrum of one token tile plus the rings fit in shared memory
     bool paired;        // x^ also keeps -Re of the complex frequencies: two MMAs per complex frequency instead of three
     size_t image_bytes;
+    int act;            // 1: GELU on the result before it is stored (forward only)
 };
 bool umma_res_supported(int T, eql_dtype_t dtype);
 UmmaResShape umma_res_shape(int T, int Cin, int Cout);

@@ -99,13 +99,14 @@ eql_status_t build_weights(eqlinear_plan_t p, const void* w, const void* bias, c
 // Streaming tensor-core kernel over every segment of the reduction: the first launch writes out = bias + its share,
 // the others add theirs (one launch in all except for FP32 layers with more than 256 reduced channels).
 cudaError_t run_streaming(eqlinear_plan_t p, int Cin, int Cout, const void* in, void* out, int64_t N, size_t image_off,
-                          const float* bias, cudaStream_t s, bool pair) {
+                          const float* bias, cudaStream_t s, bool pair, int act = 0) {
     int len = 0;
     const int nseg = umma_reduction_segments(Cin, p->dtype, &len);
     size_t off = 0;
     for (int k = 0; k < nseg; ++k) {
         UmmaLinearShape sh = umma_linear_segment(p->T, Cin, Cout, p->dtype, k, len);
         sh.pair = pair;
+        sh.act = act;                                            // (plans with an activation have one segment)
         cudaError_t e = launch_umma_linear(sh, in, out, N, p->ws + image_off + off, k == 0 ? bias : nullptr,
                                            (int*)(p->ws + p->lay.status), p->num_sms, s, k > 0);
         if (e != cudaSuccess) return e;
@@ -244,9 +245,16 @@ eql_status_t eqlinear_plan(eqlinear_plan_t* plan, int T, int C_in, int C_out, eq
     if (st != EQL_OK) return st;
     if (!w || !workspace) return EQL_ERR_INVALID_ARG;
     if (flags & ~(unsigned)(EQL_FLAG_CORRELATION | EQL_FLAG_FORCE_SIMT | EQL_FLAG_FORCE_STREAMING | EQL_FLAG_CTA_PAIR |
-                            EQL_FLAG_NO_CTA_PAIR))
+                            EQL_FLAG_NO_CTA_PAIR | EQL_FLAG_GELU))
         return EQL_ERR_INVALID_ARG;
     if ((flags & EQL_FLAG_CTA_PAIR) && (flags & EQL_FLAG_NO_CTA_PAIR)) return EQL_ERR_INVALID_ARG;
+    {   // The fused activation is applied to the finished sum: FP32 plans whose forward reduction runs as several
+        // segments added in global memory (more than 256 input channels on the tensor cores) cannot take it.
+        int len = 0;
+        if ((flags & EQL_FLAG_GELU) && !(flags & EQL_FLAG_FORCE_SIMT) && umma_linear_supported(T, dtype) &&
+            umma_reduction_segments(C_in, dtype, &len) > 1)
+            return EQL_ERR_UNSUPPORTED;
+    }
     if (!aligned16(w) || (bias && !aligned16(bias))) return EQL_ERR_ALIGNMENT;
     if (reinterpret_cast<uintptr_t>(workspace) % kWsAlign != 0) return EQL_ERR_ALIGNMENT;
     WorkspaceLayout lay = workspace_layout(T, C_in, C_out, dtype);
@@ -376,18 +384,21 @@ eql_status_t eqlinear_fwd(eqlinear_plan_t plan, const void* x, void* y, int64_t 
     if (!x || !y || x == y) return EQL_ERR_INVALID_ARG;
     if (!aligned16(x) || !aligned16(y)) return EQL_ERR_ALIGNMENT;
     const float* bias = plan->has_bias ? (const float*)(plan->ws + plan->lay.bias) : nullptr;
+    const int act = (plan->flags & EQL_FLAG_GELU) ? 1 : 0;
     if (plan->fwd_kernel == 2) {
-        cudaError_t e = launch_umma_linear_res(plan->res_fwd, x, y, N, plan->ws + plan->lay.umma_fwd, bias,
+        UmmaResShape rs = plan->res_fwd;
+        rs.act = act;
+        cudaError_t e = launch_umma_linear_res(rs, x, y, N, plan->ws + plan->lay.umma_fwd, bias,
                                                (int*)(plan->ws + plan->lay.status), plan->num_sms, (cudaStream_t)stream);
         return e == cudaSuccess ? EQL_OK : EQL_ERR_CUDA;
     }
     if (plan->fwd_kernel == 1 || plan->fwd_kernel == 3) {
         cudaError_t e = run_streaming(plan, plan->Ci, plan->Co, x, y, N, plan->lay.umma_fwd, bias, (cudaStream_t)stream,
-                                      plan->fwd_kernel == 3);
+                                      plan->fwd_kernel == 3, act);
         return e == cudaSuccess ? EQL_OK : EQL_ERR_CUDA;
     }
     cudaError_t e = launch_direct_linear(plan->T, plan->dtype, x, y, N, plan->Ci, plan->Co,
-                                         (const float*)(plan->ws + plan->lay.planes_fwd), bias, (cudaStream_t)stream);
+                                         (const float*)(plan->ws + plan->lay.planes_fwd), bias, (cudaStream_t)stream, act);
     return e == cudaSuccess ? EQL_OK : EQL_ERR_CUDA;
 }
 
@@ -495,7 +506,9 @@ eql_status_t eqlinear_fwd_save_spectrum(eqlinear_plan_t plan, const void* x, voi
         if (!x || !y || x == y) return EQL_ERR_INVALID_ARG;
         if (!aligned16(x) || !aligned16(y)) return EQL_ERR_ALIGNMENT;
         const float* bias = plan->has_bias ? (const float*)(plan->ws + plan->lay.bias) : nullptr;
-        cudaError_t e = launch_umma_linear_res(plan->res_fwd, x, y, N, plan->ws + plan->lay.umma_fwd, bias,
+        UmmaResShape rs = plan->res_fwd;
+        rs.act = (plan->flags & EQL_FLAG_GELU) ? 1 : 0;
+        cudaError_t e = launch_umma_linear_res(rs, x, y, N, plan->ws + plan->lay.umma_fwd, bias,
                                                (int*)(plan->ws + plan->lay.status), plan->num_sms, (cudaStream_t)stream,
                                                &bs, spectrum);
         return e == cudaSuccess ? EQL_OK : EQL_ERR_CUDA;

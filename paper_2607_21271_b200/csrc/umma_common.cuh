@@ -23,6 +23,10 @@ __device__ __forceinline__ uint32_t pack_h2(float lo, float hi) {
     return u;
 }
 
+// Exact GELU, x * Phi(x) with the error function (the activation after fc1 in a ViT MLP block), for the forward
+// kernels' optional fused epilogue.
+__device__ __forceinline__ float gelu_erf(float x) { return 0.5f * x * (1.0f + erff(x * 0.70710678118654752440f)); }
+
 // row_base: start of this token's 128-byte row inside a slab written by TMA with 128B swizzle
 // (slab base 1024-byte aligned, rows 128 bytes apart); r: row index inside the slab.
 // wd[0..32) = the row's 64 halves in logical order.

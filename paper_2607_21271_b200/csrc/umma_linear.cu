@@ -96,6 +96,7 @@ struct UmmaParams {
     int b_slot_bytes;            // bytes of one B ring slot (rowsB*32, twice that for FP32, rounded up to 128)
     int64_t num_units;
     int accumulate;              // out += result (TMA reduce-add) instead of out = result: later segments of a reduction
+    int act;                     // 1: GELU on the result (forward of a plan built with EQL_FLAG_GELU)
 };
 
 
@@ -190,7 +191,7 @@ __global__ void build_image_kernel(const float* __restrict__ planes, int Cin, in
 }
 
 // ------------------------------------------------------------------------------------------------
-template <int T, typename IO, int CG>
+template <int T, typename IO, int CG, bool ACT>
 __global__ void __launch_bounds__(kThreadsUmma, 1)
 umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_constant__ CUtensorMap tmap_out,
                    const UmmaParams prm) {
@@ -537,6 +538,10 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
                     for (int p = 0; p < T; ++p) v[p] = __uint_as_float(in[p][g]);
                     if (prm.bias != nullptr && co0 + g < prm.Cout) v[0] += __ldg(prm.bias + co0 + g);
                     rdft_inverse<T>(v);
+                    if constexpr (ACT) {                         // fused GELU: its own instantiation of the kernel
+#pragma unroll
+                        for (int t = 0; t < T; ++t) v[t] = gelu_erf(v[t]);
+                    }
                     if constexpr (E == 2) {
 #pragma unroll
                         for (int t = 0; t < T; t += 2) o[(g * T + t) / 2] = pack_h2(v[t], v[t + 1]);
@@ -751,6 +756,7 @@ cudaError_t launch_umma_linear(const UmmaLinearShape& s, const void* in, void* o
     const int64_t token_tiles = (N + kTileM - 1) / kTileM;
     prm.num_units = ((token_tiles + cg - 1) / cg) * s.nTiles;    // a pair takes two token tiles per unit
     prm.accumulate = accumulate ? 1 : 0;
+    prm.act = s.act;
 
     return dispatch_umma(s.T, s.elem_bytes, [&](auto tc, auto io) {
         constexpr int TT = decltype(tc)::value;
@@ -759,9 +765,9 @@ cudaError_t launch_umma_linear(const UmmaLinearShape& s, const void* in, void* o
             if constexpr (sizeof(IO) == 2 && (TT == 4 || TT == 8)) {
                 const size_t smem = umma_smem_bytes<TT, 2, 2>(prm.b_slot_bytes);
                 if (smem > 227 * 1024) return cudaErrorInvalidConfiguration;
-                static SmemLimitOnce smem_limit;
-                auto kernel = umma_linear_kernel<TT, IO, 2>;
-                if (cudaError_t e = smem_limit.ensure(kernel, 227 * 1024); e != cudaSuccess) return e;
+                static SmemLimitOnce smem_limit[2];
+                auto kernel = prm.act ? umma_linear_kernel<TT, IO, 2, true> : umma_linear_kernel<TT, IO, 2, false>;
+                if (cudaError_t e = smem_limit[prm.act ? 1 : 0].ensure(kernel, 227 * 1024); e != cudaSuccess) return e;
                 cudaLaunchConfig_t cfg{};
                 cudaLaunchAttribute attr[1];
                 attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -787,10 +793,16 @@ cudaError_t launch_umma_linear(const UmmaLinearShape& s, const void* in, void* o
         } else {
             const int grid = (int)(prm.num_units < num_sms ? prm.num_units : num_sms);
             const size_t smem = umma_smem_bytes<TT, sizeof(IO), 1>(prm.b_slot_bytes);
-            static SmemLimitOnce smem_limit;                      // per kernel instantiation
-            if (cudaError_t e = smem_limit.ensure(umma_linear_kernel<TT, IO, 1>, 227 * 1024); e != cudaSuccess) return e;
             if (smem > 227 * 1024) return cudaErrorInvalidConfiguration;
-            umma_linear_kernel<TT, IO, 1><<<grid, kThreadsUmma, smem, stream>>>(tmap, tmap_out, prm);
+            if (prm.act) {
+                static SmemLimitOnce smem_limit_act;              // per kernel instantiation
+                if (cudaError_t e = smem_limit_act.ensure(umma_linear_kernel<TT, IO, 1, true>, 227 * 1024); e != cudaSuccess) return e;
+                umma_linear_kernel<TT, IO, 1, true><<<grid, kThreadsUmma, smem, stream>>>(tmap, tmap_out, prm);
+                return cudaGetLastError();
+            }
+            static SmemLimitOnce smem_limit;                      // per kernel instantiation
+            if (cudaError_t e = smem_limit.ensure(umma_linear_kernel<TT, IO, 1, false>, 227 * 1024); e != cudaSuccess) return e;
+            umma_linear_kernel<TT, IO, 1, false><<<grid, kThreadsUmma, smem, stream>>>(tmap, tmap_out, prm);
             return cudaGetLastError();
         }
     });

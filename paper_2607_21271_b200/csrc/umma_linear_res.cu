@@ -70,6 +70,7 @@ struct ResParams {
     uint8_t* stash;              // nullptr: off
     int st_CiT, st_nCiTiles;     // the weight gradient's input-channel tiling
     int64_t st_chunks;           // 16-token chunks in all
+    int act;                     // 1: GELU on the result (forward of a plan built with EQL_FLAG_GELU)
 };
 
 
@@ -109,7 +110,7 @@ __global__ void build_image_res_kernel(const float* __restrict__ planes, int Cin
 // complex frequency takes two MMAs of width 2 NTOK ([Re|Im] += Wr [Xr|Xi] and, with A negated, += (-Wi) [Xi|-Xr])
 // instead of three; an MMA costs about the same whatever its width, so this shortens the main loop where the larger
 // x^ buffers fit.
-template <int T, int NTOK, bool PF, bool MERGED>
+template <int T, int NTOK, bool PF, bool MERGED, bool ACT>
 __global__ void __launch_bounds__(ResWarps<T>::kThreads, 1)
 umma_linear_res_kernel(const __grid_constant__ CUtensorMap tmap_in, const ResParams prm) {
     // NTOK tokens per tile: the accumulator of a unit is T planes x NTOK fp32 TMEM columns.  With T * NTOK = 256 two
@@ -452,6 +453,10 @@ umma_linear_res_kernel(const __grid_constant__ CUtensorMap tmap_in, const ResPar
                         for (int p = 0; p < T; ++p) v[p] = __uint_as_float(in[p][j]);
                         v[0] += bias_v;
                         rdft_inverse<T>(v);
+                        if constexpr (ACT) {                     // fused GELU: its own instantiation of the kernel
+#pragma unroll
+                            for (int t = 0; t < T; ++t) v[t] = gelu_erf(v[t]);
+                        }
                         if (kWhole || (o_ok && j < rows_left)) {
                             if constexpr (T == 8)
                                 *reinterpret_cast<uint4*>(dst) = make_uint4(pack_h2(v[0], v[1]), pack_h2(v[2], v[3]),
@@ -583,6 +588,7 @@ cudaError_t launch_umma_linear_res(const UmmaResShape& s, const void* in, void* 
     prm.N = N; prm.Cin = s.Cin; prm.Cout = s.Cout; prm.nCT = s.nCT; prm.nK = s.nK;
     prm.w_slots = s.w_slots; prm.n_tw = s.n_tw; prm.x_slots = s.x_slots;
     prm.num_units = ((N + s.nTok - 1) / s.nTok) * s.nCT;
+    prm.act = s.act;
     if (stash != nullptr && stash_shape != nullptr) {
         prm.stash = (uint8_t*)stash;
         prm.st_CiT = stash_shape->CiT; prm.st_nCiTiles = stash_shape->nCiTiles; prm.st_chunks = stash_shape->total_chunks;
@@ -593,9 +599,15 @@ cudaError_t launch_umma_linear_res(const UmmaResShape& s, const void* in, void* 
     auto go = [&](auto tc, auto nt, auto pf, auto mg) -> cudaError_t {
         constexpr int TT = decltype(tc)::value, NT = decltype(nt)::value;
         constexpr bool PF = decltype(pf)::value, MG = decltype(mg)::value;
+        if (prm.act) {
+            static SmemLimitOnce smem_limit_act;              // per kernel instantiation
+            if (cudaError_t e = smem_limit_act.ensure(umma_linear_res_kernel<TT, NT, PF, MG, true>, (int)kResSmemLimit); e != cudaSuccess) return e;
+            umma_linear_res_kernel<TT, NT, PF, MG, true><<<grid, ResWarps<TT>::kThreads, smem, stream>>>(tmap, prm);
+            return cudaGetLastError();
+        }
         static SmemLimitOnce smem_limit;                      // per kernel instantiation
-        if (cudaError_t e = smem_limit.ensure(umma_linear_res_kernel<TT, NT, PF, MG>, (int)kResSmemLimit); e != cudaSuccess) return e;
-        umma_linear_res_kernel<TT, NT, PF, MG><<<grid, ResWarps<TT>::kThreads, smem, stream>>>(tmap, prm);
+        if (cudaError_t e = smem_limit.ensure(umma_linear_res_kernel<TT, NT, PF, MG, false>, (int)kResSmemLimit); e != cudaSuccess) return e;
+        umma_linear_res_kernel<TT, NT, PF, MG, false><<<grid, ResWarps<TT>::kThreads, smem, stream>>>(tmap, prm);
         return cudaGetLastError();
     };
     using I4 = std::integral_constant<int, 4>;

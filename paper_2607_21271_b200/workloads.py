@@ -68,7 +68,15 @@ OPERATOR_SHAPES = {
        for c in (16, 64, 256, 512, 1024, 2048)},
 }
 
-ALL_WORKLOADS = {**CONFIGS, **OPERATOR_SHAPES}
+# The other linear layers of the EQ-ViT-B block the headline layer (fc1) comes from, at the same token count: the fused
+# q/k/v projection is ONE layer with three blocks of output channels (x is read and transformed once for all three),
+# fc2 is the MLP's second layer (384 -> 96 channels per group element).
+BLOCK_SHAPES = {
+    "vit_b_qkv_fp16": Workload("vit_b_qkv_fp16", "fp16", 8, 96, 3 * 96, 128 * 197, "normal", _FB, 6),
+    "vit_b_fc2_fp16": Workload("vit_b_fc2_fp16", "fp16", 8, 384, 96, 128 * 197, "normal", _FB, 7),
+}
+
+ALL_WORKLOADS = {**CONFIGS, **OPERATOR_SHAPES, **BLOCK_SHAPES}
 
 
 def generate(wl: Workload) -> dict:

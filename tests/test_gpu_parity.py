@@ -10,7 +10,7 @@ import torch
 
 import paper_2607_21271_b200 as eq
 from oracle import eqlinear_oracle as orc
-from paper_2607_21271_b200.workloads import CONFIGS, OPERATOR_SHAPES, Workload, generate, sample_rows
+from paper_2607_21271_b200.workloads import BLOCK_SHAPES, CONFIGS, OPERATOR_SHAPES, Workload, generate, sample_rows
 from tests.harness import TOL, GpuLayer, check_workload, rel_max_err
 
 pytestmark = pytest.mark.gpu
@@ -25,6 +25,55 @@ def test_config_matches_oracle(name):
     assert set(errs) >= {"y"}
     for k, v in errs.items():
         assert v <= TOL[wl.dtype], f"{name}: {k} error {v:.3e} above {TOL[wl.dtype]:.0e}"
+
+
+@pytest.mark.parametrize("name", list(BLOCK_SHAPES))
+def test_transformer_block_layers_match_oracle(name):
+    """The fused q/k/v projection (one layer, 96 -> 3 x 96 channels: x is transformed once for the three blocks) and fc2
+    (384 -> 96) of the EQ-ViT-B block, full size, every output against the oracle."""
+    wl = BLOCK_SHAPES[name]
+    for k, v in check_workload(wl).items():
+        assert v <= TOL[wl.dtype], f"{name}: {k} error {v:.3e}"
+
+
+def _gelu(a):
+    from scipy.special import erf
+    return 0.5 * a * (1.0 + erf(a / np.sqrt(2.0)))
+
+
+@pytest.mark.parametrize("dtype,T,Ci,Co,N,flags,kernel", [
+    ("fp16", 8, 96, 384, 1500, 0, 2),                                        # resident-activation kernel (fc1 -> GELU)
+    ("fp16", 8, 96, 384, 1500, eq.EQL_FLAG_FORCE_STREAMING, 1),              # streaming kernel
+    ("fp16", 4, 64, 200, 777, eq.EQL_FLAG_FORCE_STREAMING | eq.EQL_FLAG_CTA_PAIR, 3),   # its CTA-pair form
+    ("fp16", 16, 17, 33, 333, 0, 1),
+    ("fp32", 8, 48, 48, 1000, 0, 1),                                         # 3xTF32
+    ("fp32", 5, 8, 24, 333, 0, 0), ("fp16", 2, 8, 16, 333, 0, 0),            # CUDA-core kernels
+])
+def test_fused_gelu_epilogue(dtype, T, Ci, Co, N, flags, kernel):
+    """EQL_FLAG_GELU: the forward pass returns GELU(layer(x)), applied in FP32 before the one rounding of the output;
+    the gradients of a plan built with the flag remain those of the linear layer."""
+    wl = Workload("gelu", dtype, T, Ci, Co, N, "normal", ("fwd", "bwd_data"), 33)
+    d = generate(wl)
+    layer = GpuLayer(T, Ci, Co, dtype, d["w"], d["bias"], flags | eq.EQL_FLAG_GELU)
+    try:
+        assert eq.eqlinear_plan_info(layer.plan).fwd_kernel == kernel
+        y = layer.fwd(d["x"])
+        dx = layer.bwd_data(d["dy"])
+        assert layer.raw_status() == 0
+    finally:
+        layer.close()
+    assert rel_max_err(y, _gelu(orc.fwd(d["x"], d["w"], d["bias"]))) <= TOL[dtype]
+    assert rel_max_err(dx, orc.bwd_data(d["dy"], d["w"])) <= TOL[dtype]
+
+
+def test_fused_gelu_is_refused_where_the_forward_sum_is_split():
+    """FP32 plans on the tensor cores with more than 256 input channels add segments of the reduction in global memory:
+    no place to apply an activation to the finished sum."""
+    wl = Workload("gelu", "fp32", 4, 300, 16, 64, "normal", ("fwd",), 34)
+    d = generate(wl)
+    with pytest.raises(eq.EqlError) as e:
+        GpuLayer(wl.T, wl.Ci, wl.Co, "fp32", d["w"], d["bias"], eq.EQL_FLAG_GELU)
+    assert e.value.status == eq.binding.EQL_ERR_UNSUPPORTED
 
 
 def test_repeated_full_size_runs_are_identical():

@@ -5,12 +5,13 @@ full-size parity on sampled outputs, and the shapes of the paper's operator-leve
 import numpy as np
 import pytest
 
-from paper_2607_21271_b200.workloads import ALL_WORKLOADS, CONFIGS, HEADLINE, OPERATOR_SHAPES, Workload, generate, sample_rows
+from paper_2607_21271_b200.workloads import (ALL_WORKLOADS, BLOCK_SHAPES, CONFIGS, HEADLINE, OPERATOR_SHAPES, Workload, generate,
+                                              sample_rows)
 
 
 def test_tables_are_consistent():
     assert HEADLINE in CONFIGS
-    assert set(CONFIGS) | set(OPERATOR_SHAPES) == set(ALL_WORKLOADS)
+    assert set(CONFIGS) | set(OPERATOR_SHAPES) | set(BLOCK_SHAPES) == set(ALL_WORKLOADS)
     assert not set(CONFIGS) & set(OPERATOR_SHAPES)
     for name, wl in ALL_WORKLOADS.items():
         assert wl.name == name
