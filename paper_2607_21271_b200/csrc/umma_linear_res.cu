@@ -41,7 +41,7 @@ namespace {
 
 
 constexpr int kTmemColsRes = 512;
-constexpr int kResWarpTmaX = 0, kResWarpMma = 1, kResWarpTmaW = 2, kResWarpCompute0 = 4;
+constexpr int kResWarpTmaX = 0, kResWarpMma = 1, kResWarpTmaW = 2, kResWarpTmaX2 = 3, kResWarpCompute0 = 4;
 constexpr int kResComputeWarps = 16;         // at most (barrier array size)
 // Compute warps per kernel: the T = 4 epilogue is short on instruction issue and long on stores, and gains from a
 // fourth warp per TMEM lane quadrant even at 96 registers per thread (Swin layer: 99.7 -> 96.1 us); the T = 8 kernels
@@ -183,32 +183,44 @@ umma_linear_res_kernel(const __grid_constant__ CUtensorMap tmap_in, const ResPar
     auto last_of_tile = [&](int64_t u, int ct) { return ring || u == u1 - 1 || ct == nCT - 1; };
     const int items_per_tile = IPC * nK;
 
-    if (warp == kResWarpTmaX) {
+    if (warp == kResWarpTmaX || warp == kResWarpTmaX2) {
         // ---------------------------------------------------------------- raw activation rows via TMA
+        // Two producer threads in two warps, one for the even ring slots (= even items) and one for the odd ones: a thread
+        // gets one bulk / tensor copy accepted every ~300 ns whatever its size (measured: L2-resident source, 4 to 64 KB
+        // per copy, any number in flight; the rate scales with the number of issuing warps), and these items are 4 KB.
+        // A layer with many input channels needs one item per ~260 ns and SM at the speed of its MMA loop.
         if (lane == 0) {
-            uint32_t gi = 0;                                     // running item counter; item gi lives in slot gi % n_tw
-            int slot = 0;
+            const int me = warp == kResWarpTmaX ? 0 : 1;         // n_tw is even: slot parity = item parity
+            uint32_t gi = me;                                    // running item counter; item gi lives in slot gi % n_tw
+            int slot = me;
             uint32_t eph = 1;
             bool ok = true;
             int ct = ct0;
             int64_t tt = tt0;
+            uint32_t base = 0;                                   // running number of the tile's first item
             for (int64_t u = u0; u < u1 && ok; ++u, ++ct) {
                 if (ct == nCT) { ct = 0; ++tt; }
                 if (!first_of_tile(u, ct)) continue;
                 const int row0 = (int)tt * NTOK;
-                for (int i = 0; i < items_per_tile; ++i, ++gi) {
+                for (; gi < base + (uint32_t)items_per_tile; gi += 2) {
+                    const int i = (int)(gi - base);
                     ok = ptx::mbar_wait(&bar->empty_raw[slot], eph, abort_flag, status, 301, true, kResSpin);
                     if (!ok) break;
                     ptx::mbar_arrive_expect_tx(&bar->full_raw[slot], kItemBytes);
                     const int s = i / PARTS, h = i % PARTS;      // slab (64 elements of the row), 32-token part
                     ptx::tma_load_2d(raw + slot * kItemBytes, &tmap_in, s * 64, row0 + h * 32, &bar->full_raw[slot]);
-                    if (++slot == n_tw) { slot = 0; eph ^= 1u; }
+                    slot += 2;
+                    if (slot >= n_tw) { slot -= n_tw; eph ^= 1u; }
                 }
+                base += (uint32_t)items_per_tile;
             }
-            // drain: every copy this thread issued must have landed before the CTA may exit
-            const uint32_t lo = gi > (uint32_t)n_tw ? gi - n_tw : 0;
-            for (uint32_t c = lo; c < gi; ++c)
-                ptx::mbar_wait(&bar->full_raw[c % n_tw], (c / n_tw) & 1, abort_flag, status, 311, false);
+            // drain: every copy this thread issued must have landed before the CTA may exit (its items: me, me + 2, ...)
+            if (gi >= 2) {
+                const uint32_t last = gi - 2;                    // last item issued (or the one a failed wait stopped at)
+                const uint32_t lo = last + 2 > (uint32_t)n_tw ? last + 2 - n_tw : me;
+                for (uint32_t c = lo; c <= last; c += 2)
+                    ptx::mbar_wait(&bar->full_raw[c % n_tw], (c / n_tw) & 1, abort_flag, status, 311, false);
+            }
         }
     } else if (warp == kResWarpTmaW) {
         // ---------------------------------------------------------------- spectral-weight tiles via bulk copy
