@@ -10,6 +10,7 @@ if ROOT not in sys.path:
 
 def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (sm_100a); runs the library through its C ABI")
+    config.addinivalue_line("markers", "soak: long opt-in GPU checks (fuzz, > 4 GB tensors, repeated steps); run with -m soak")
 
 
 def _have_gpu() -> bool:
@@ -21,9 +22,15 @@ def _have_gpu() -> bool:
 
 
 def pytest_collection_modifyitems(config, items):
+    # the long checks run only when asked for by name (-m soak), never as part of "-m gpu" or "-m 'not gpu'"
+    if "soak" not in (config.getoption("-m") or ""):
+        skip_soak = pytest.mark.skip(reason="opt-in: run with -m soak")
+        for item in items:
+            if "soak" in item.keywords:
+                item.add_marker(skip_soak)
     if _have_gpu():
         return
     skip = pytest.mark.skip(reason="no CUDA device")
     for item in items:
-        if "gpu" in item.keywords:
+        if "gpu" in item.keywords or "soak" in item.keywords:
             item.add_marker(skip)
