@@ -15,8 +15,8 @@
  *   - Features are dense row-major [N, C*T] with the group index fastest: element (n, c, t) is at
  *     n*C*T + c*T + t.  The weight is [C_out, C_in, T] with the group offset r fastest; the bias
  *     is [C_out].
- *   - x, y, dy, dx, w and bias have the plan's dtype (EQL_FP32: float; EQL_FP16: IEEE half with
- *     float accumulation).  dw and db are always float.
+ *   - x, y, dy, dx, w and bias have the plan's dtype (EQL_FP32: float; EQL_FP16: IEEE half, EQL_BF16: bfloat16,
+ *     both with float accumulation).  dw and db are always float.
  *   - Every tensor pointer is DEVICE memory owned by the caller, 16-byte aligned; outputs must not
  *     alias inputs.  The *_host entry points are the only ones that take host pointers.
  *   - The library allocates no device memory.  The plan keeps its derived weights in a
@@ -53,7 +53,9 @@ typedef enum {
     EQL_ERR_DEVICE_TIMEOUT = 7    /* a bounded wait inside a kernel ran out                    */
 } eql_status_t;
 
-typedef enum { EQL_FP32 = 0, EQL_FP16 = 1 } eql_dtype_t;
+/* EQL_FP16 / EQL_BF16: 16-bit I/O (IEEE half / bfloat16) with float accumulation; the spectra of the activations and of
+ * the weight are rounded to the same 16-bit type once, everything else is float. */
+typedef enum { EQL_FP32 = 0, EQL_FP16 = 1, EQL_BF16 = 2 } eql_dtype_t;
 
 /* Plan flags. */
 enum {

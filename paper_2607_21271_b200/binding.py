@@ -25,6 +25,7 @@ EQL_ERR_DEVICE_TIMEOUT = 7
 
 EQL_FP32 = 0
 EQL_FP16 = 1
+EQL_BF16 = 2
 
 EQL_FLAG_CORRELATION = 1
 EQL_FLAG_FORCE_SIMT = 2

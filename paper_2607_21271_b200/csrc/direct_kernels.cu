@@ -5,6 +5,7 @@
 // group tuple as it is loaded, the per-frequency complex products (Eq. 5) accumulate in registers,
 // and the inverse DFT (Eq. 7) plus bias runs in the epilogue; no frequency-domain tensor touches
 // global memory except the weight-gradient's split partials.
+#include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
 #include "eql_internal.h"
@@ -12,6 +13,15 @@
 
 namespace eql {
 namespace {
+
+// element <-> float for the three I/O types
+__device__ __forceinline__ float to_f32(float v) { return v; }
+__device__ __forceinline__ float to_f32(__half v) { return __half2float(v); }
+__device__ __forceinline__ float to_f32(__nv_bfloat16 v) { return __bfloat162float(v); }
+template <typename IO> __device__ __forceinline__ IO from_f32(float v);
+template <> __device__ __forceinline__ float from_f32<float>(float v) { return v; }
+template <> __device__ __forceinline__ __half from_f32<__half>(float v) { return __float2half_rn(v); }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
 
 // ---- group-tuple loads and stores (T contiguous elements, T*sizeof(IO) in {4, 8, 16, 32, ...} bytes)
 template <int BYTES>
@@ -26,7 +36,7 @@ __device__ __forceinline__ void load_group(const IO* __restrict__ p, float* v) {
     if constexpr (!vector_tuple(T * sizeof(IO))) {
 #pragma unroll
         for (int i = 0; i < T; ++i) {
-            if constexpr (sizeof(IO) == 4) v[i] = __ldg(p + i); else v[i] = __half2float(__ldg(p + i));
+            v[i] = to_f32(__ldg(p + i));
         }
         return;
     }
@@ -35,9 +45,7 @@ __device__ __forceinline__ void load_group(const IO* __restrict__ p, float* v) {
 #pragma unroll
     for (int i = 0; i < V::n; ++i) u.vec[i] = __ldg(reinterpret_cast<const typename V::type*>(p) + i);
 #pragma unroll
-    for (int i = 0; i < T; ++i) {
-        if constexpr (sizeof(IO) == 4) v[i] = u.e[i]; else v[i] = __half2float(u.e[i]);
-    }
+    for (int i = 0; i < T; ++i) v[i] = to_f32(u.e[i]);
 }
 
 template <int T, typename IO>
@@ -45,16 +53,14 @@ __device__ __forceinline__ void store_group(IO* __restrict__ p, const float* v) 
     if constexpr (!vector_tuple(T * sizeof(IO))) {
 #pragma unroll
         for (int i = 0; i < T; ++i) {
-            if constexpr (sizeof(IO) == 4) p[i] = v[i]; else p[i] = __float2half_rn(v[i]);
+            p[i] = from_f32<IO>(v[i]);
         }
         return;
     }
     using V = VecBytes<vector_tuple(T * sizeof(IO)) ? T * sizeof(IO) : 16>;
     union { typename V::type vec[V::n]; IO e[T]; } u;
 #pragma unroll
-    for (int i = 0; i < T; ++i) {
-        if constexpr (sizeof(IO) == 4) u.e[i] = v[i]; else u.e[i] = __float2half_rn(v[i]);
-    }
+    for (int i = 0; i < T; ++i) u.e[i] = from_f32<IO>(v[i]);
 #pragma unroll
     for (int i = 0; i < V::n; ++i) reinterpret_cast<typename V::type*>(p)[i] = u.vec[i];
 }
@@ -155,14 +161,14 @@ __global__ void plan_weights_kernel(const IO* __restrict__ w, const IO* __restri
     fill_twiddles<T>(tw);
     const int idx = blockIdx.x * blockDim.x + threadIdx.x;
     if (idx < Co && bias_f32 != nullptr) {
-        if constexpr (sizeof(IO) == 4) bias_f32[idx] = bias[idx]; else bias_f32[idx] = __half2float(bias[idx]);
+        bias_f32[idx] = to_f32(bias[idx]);
     }
     if (idx >= Ci * Co) return;
     const int o = idx / Ci, i = idx - o * Ci;
     float v[T];
 #pragma unroll
     for (int r = 0; r < T; ++r) {
-        if constexpr (sizeof(IO) == 4) v[r] = w[(size_t)idx * T + r]; else v[r] = __half2float(w[(size_t)idx * T + r]);
+        v[r] = to_f32(w[(size_t)idx * T + r]);
     }
     dft_fwd<T>(v, tw);
 #pragma unroll
@@ -442,6 +448,9 @@ cudaError_t launch_plan_weights(int T, eql_dtype_t dtype, bool correlation, cons
         if (dtype == EQL_FP32)
             plan_weights_kernel<TT, float><<<blocks, threads, 0, stream>>>(
                 (const float*)w, (const float*)bias, Ci, Co, correlation, planes_fwd, planes_bwd, bdst);
+        else if (dtype == EQL_BF16)
+            plan_weights_kernel<TT, __nv_bfloat16><<<blocks, threads, 0, stream>>>(
+                (const __nv_bfloat16*)w, (const __nv_bfloat16*)bias, Ci, Co, correlation, planes_fwd, planes_bwd, bdst);
         else
             plan_weights_kernel<TT, __half><<<blocks, threads, 0, stream>>>(
                 (const __half*)w, (const __half*)bias, Ci, Co, correlation, planes_fwd, planes_bwd, bdst);
@@ -460,6 +469,9 @@ cudaError_t launch_direct_linear(int T, eql_dtype_t dtype, const void* in, void*
         if (dtype == EQL_FP32)
             direct_linear_kernel<TT, float><<<grid, kThreads, 0, stream>>>(
                 (const float*)in, (float*)out, N, Cin, Cout, planes, bias_f32, act);
+        else if (dtype == EQL_BF16)
+            direct_linear_kernel<TT, __nv_bfloat16><<<grid, kThreads, 0, stream>>>(
+                (const __nv_bfloat16*)in, (__nv_bfloat16*)out, N, Cin, Cout, planes, bias_f32, act);
         else
             direct_linear_kernel<TT, __half><<<grid, kThreads, 0, stream>>>(
                 (const __half*)in, (__half*)out, N, Cin, Cout, planes, bias_f32, act);
@@ -508,6 +520,9 @@ cudaError_t launch_direct_bwd_weight(int T, eql_dtype_t dtype, bool correlation,
         if (dtype == EQL_FP32)
             direct_bwd_weight_kernel<TT, float><<<grid, kThreads, 0, stream>>>(
                 (const float*)x, (const float*)dy, N, Ci, Co, split.tokens_per_split, part, db_part);
+        else if (dtype == EQL_BF16)
+            direct_bwd_weight_kernel<TT, __nv_bfloat16><<<grid, kThreads, 0, stream>>>(
+                (const __nv_bfloat16*)x, (const __nv_bfloat16*)dy, N, Ci, Co, split.tokens_per_split, part, db_part);
         else
             direct_bwd_weight_kernel<TT, __half><<<grid, kThreads, 0, stream>>>(
                 (const __half*)x, (const __half*)dy, N, Ci, Co, split.tokens_per_split, part, db_part);

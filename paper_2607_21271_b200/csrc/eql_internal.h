@@ -79,7 +79,8 @@ cudaError_t launch_direct_bwd_weight(int T, eql_dtype_t dtype, bool correlation,
 // ---- tcgen05 tensor-core kernels (FP16 I/O), umma_linear.cu ----------------------------------------
 struct UmmaLinearShape {
     int T, Cin, Cout;
-    int elem_bytes;     // 2: half I/O (kind::f16), 4: float I/O (kind::tf32, 3xTF32 split)
+    int elem_bytes;     // 2: half or bfloat16 I/O (kind::f16), 4: float I/O (kind::tf32, 3xTF32 split)
+    bool bf16;          // elem_bytes == 2: the elements are bfloat16 instead of IEEE half
     int CoT;            // output channels per tile: multiple of 16, T*CoT <= 512 TMEM columns
     int nTiles;         // output-channel tiles
     int nK;             // chunks of the reduction dimension (16 channels for half, 8 for float)
@@ -121,9 +122,10 @@ struct UmmaResShape {
     bool paired;        // x^ also keeps -Re of the complex frequencies: two MMAs per complex frequency instead of three
     size_t image_bytes;
     int act;            // 1: GELU on the result before it is stored (forward only)
+    bool bf16;          // bfloat16 I/O instead of IEEE half
 };
 bool umma_res_supported(int T, eql_dtype_t dtype);
-UmmaResShape umma_res_shape(int T, int Cin, int Cout);
+UmmaResShape umma_res_shape(int T, int Cin, int Cout, eql_dtype_t dtype = EQL_FP16);
 cudaError_t launch_build_umma_res_image(const UmmaResShape& s, const float* planes, void* image, cudaStream_t stream);
 struct UmmaBwdWeightShape;
 // stash (optional): also write the spectrum of `in` as the operand image of the saved-spectrum weight-gradient kernel
@@ -134,7 +136,8 @@ cudaError_t launch_umma_linear_res(const UmmaResShape& s, const void* in, void* 
 // ---- tcgen05 weight-gradient kernel (FP16 inputs; FP32 inputs with the 3xTF32 split), umma_bwd_weight.cu --------------------------------
 struct UmmaBwdWeightShape {
     int T, Ci, Co;
-    int elem_bytes;             // 2: half inputs (kind::f16), 4: float inputs (kind::tf32, 3xTF32 split)
+    int elem_bytes;             // 2: half or bfloat16 inputs (kind::f16), 4: float inputs (kind::tf32, 3xTF32 split)
+    bool bf16;                  // elem_bytes == 2: bfloat16 instead of IEEE half
     int CiT, nCiTiles;          // input-channel tile (UMMA M side, <= 128 lanes, CiT*T <= 1024)
     int CoT, nCoTiles;          // output-channel tile (UMMA N side, T*CoT <= 512 TMEM columns)
     int nXs, nYs;               // 64-element raw slabs of x / dy per 16-token chunk

@@ -21,7 +21,7 @@ WorkspaceLayout workspace_layout(int T, int Ci, int Co, eql_dtype_t dtype) {
         l.umma_fwd_bytes = umma_linear_image_bytes(T, Ci, Co, dtype);
         l.umma_bwd_bytes = umma_linear_image_bytes(T, Co, Ci, dtype);
         if (umma_res_supported(T, dtype)) {          // one region serves whichever tensor-core kernel the plan selects
-            const size_t rf = umma_res_shape(T, Ci, Co).image_bytes, rb = umma_res_shape(T, Co, Ci).image_bytes;
+            const size_t rf = umma_res_shape(T, Ci, Co, dtype).image_bytes, rb = umma_res_shape(T, Co, Ci, dtype).image_bytes;
             if (rf > l.umma_fwd_bytes) l.umma_fwd_bytes = rf;
             if (rb > l.umma_bwd_bytes) l.umma_bwd_bytes = rb;
         }
@@ -43,7 +43,7 @@ inline size_t elem_size(eql_dtype_t d) { return d == EQL_FP32 ? 4 : 2; }
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 eql_status_t check_shape(int T, int Ci, int Co, int dtype) {
-    if (dtype != EQL_FP32 && dtype != EQL_FP16) return EQL_ERR_INVALID_ARG;
+    if (dtype != EQL_FP32 && dtype != EQL_FP16 && dtype != EQL_BF16) return EQL_ERR_INVALID_ARG;
     if (T < 1 || Ci < 1 || Co < 1) return EQL_ERR_INVALID_ARG;
     if (!supported_T(T)) return EQL_ERR_UNSUPPORTED;
     if ((int64_t)Ci * T > (1 << 20) || (int64_t)Co * T > (1 << 20)) return EQL_ERR_UNSUPPORTED;
@@ -288,8 +288,8 @@ eql_status_t eqlinear_plan(eqlinear_plan_t* plan, int T, int C_in, int C_out, eq
             auto prefer = [](const UmmaResShape& r) {
                 return r.fits && r.w_slots >= 3 && 2 * r.Cout >= 128 * r.nCT;
             };
-            p->res_fwd = umma_res_shape(T, C_in, C_out);
-            p->res_bwd = umma_res_shape(T, C_out, C_in);
+            p->res_fwd = umma_res_shape(T, C_in, C_out, dtype);
+            p->res_bwd = umma_res_shape(T, C_out, C_in, dtype);
             if (prefer(p->res_fwd)) p->fwd_kernel = 2;
             if (prefer(p->res_bwd)) p->bwd_data_kernel = 2;
         }

@@ -168,11 +168,12 @@ __device__ __forceinline__ uint64_t umma_smem_desc_k_sw32(uint32_t smem_addr) {
     d |= (uint64_t)6 << 61;                       // SWIZZLE_32B
     return d;
 }
-// Instruction descriptor for kind::f16 with F16 A/B (both K-major), F32 accumulator, M x N tile.
-__device__ __forceinline__ uint32_t umma_idesc_f16_f32(uint32_t M, uint32_t N) {
+// Instruction descriptor for kind::f16 with 16-bit A/B (both K-major), F32 accumulator, M x N tile.
+// fmt: operand format, 0 = F16 (IEEE half), 1 = BF16.
+__device__ __forceinline__ uint32_t umma_idesc_f16_f32(uint32_t M, uint32_t N, uint32_t fmt = 0u) {
     return (1u << 4)                // D format: F32
-           | (0u << 7)              // A format: F16
-           | (0u << 10)             // B format: F16
+           | (fmt << 7)             // A format
+           | (fmt << 10)            // B format
            | ((N >> 3) << 17)       // N / 8
            | ((M >> 4) << 24);      // M / 16
 }
@@ -181,8 +182,8 @@ __device__ __forceinline__ uint32_t umma_idesc_tf32_f32(uint32_t M, uint32_t N) 
     return (1u << 4) | (2u << 7) | (2u << 10) | ((N >> 3) << 17) | ((M >> 4) << 24);
 }
 // Same, with both operands MN-major ("transposed": the M resp. N index is the contiguous one in shared memory).
-__device__ __forceinline__ uint32_t umma_idesc_f16_f32_mn_major(uint32_t M, uint32_t N) {
-    return umma_idesc_f16_f32(M, N) | (1u << 15) | (1u << 16);
+__device__ __forceinline__ uint32_t umma_idesc_f16_f32_mn_major(uint32_t M, uint32_t N, uint32_t fmt = 0u) {
+    return umma_idesc_f16_f32(M, N, fmt) | (1u << 15) | (1u << 16);
 }
 // D[tmem] (+)= A[smem] * B[smem]^T; issued by ONE thread.
 __device__ __forceinline__ void umma_f16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,

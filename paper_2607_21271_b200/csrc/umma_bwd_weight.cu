@@ -157,8 +157,9 @@ umma_bwd_weight_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
         if (lane == 0) {
             bool ok = true;
             constexpr uint32_t kMnMajor = (1u << 15) | (1u << 16);       // both operands MN-major
-            const uint32_t idesc_real = E == 2 ? (ptx::umma_idesc_f16_f32(128, CoT) | kMnMajor) : ptx::umma_idesc_tf32_f32(128, CoT);
-            const uint32_t idesc_cplx = E == 2 ? (ptx::umma_idesc_f16_f32(128, 2 * CoT) | kMnMajor) : ptx::umma_idesc_tf32_f32(128, 2 * CoT);
+            constexpr uint32_t kFmt = H16<IO>::kUmmaFormat;                // half or bfloat16 operands
+            const uint32_t idesc_real = E == 2 ? (ptx::umma_idesc_f16_f32(128, CoT, kFmt) | kMnMajor) : ptx::umma_idesc_tf32_f32(128, CoT);
+            const uint32_t idesc_cplx = E == 2 ? (ptx::umma_idesc_f16_f32(128, 2 * CoT, kFmt) | kMnMajor) : ptx::umma_idesc_tf32_f32(128, 2 * CoT);
             const uint32_t a_plane = (uint32_t)CiT * TOKB, b_tile = (uint32_t)CoT * TOKB;
             // FP16, MN-major no-swizzle tiles: lbo = stride between 8-token groups (128 B), sbo = stride between 8-channel groups
             // (256 B).  FP32, K-major no-swizzle tiles: lbo = stride between 4-token core matrices, sbo = between 8-channel groups.
@@ -249,8 +250,10 @@ umma_bwd_weight_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
                     // output-channel tile, which makes its transform the largest share of this kernel's instructions
                     // (-10 % kernel time); the weight gradient averages the extra rounding over the token sum
                     // (measured max error 4.2e-4 instead of 3.1e-4 of the largest |dw|, bar 3e-3).
-                    if (is_y) dft_words<T, true>(wd, packed, p0);
-                    else dft_words<T, false, true>(wd, packed, nullptr);
+                    // (bfloat16 inputs: float butterflies for both -- a packed bfloat16 butterfly keeps 8 bits per rounding)
+                    if (is_y) dft_words<T, true, false, IO>(wd, packed, p0);
+                    else if constexpr (H16<IO>::kIsHalf) dft_words<T, false, true>(wd, packed, nullptr);
+                    else dft_words<T, false, false, IO>(wd, packed, nullptr);
                     if (!is_y) {
 #pragma unroll
                         for (int p = 0; p < T; ++p) store_plane_run<NCH>(stage + p * a_plane + off, packed[p], 256);
@@ -450,7 +453,7 @@ int balanced_tile(int C, int max_tile, int round) {
 
 
 bool umma_bwd_weight_supported(int T, eql_dtype_t dtype) {
-    if (dtype == EQL_FP16) return T == 4 || T == 8 || T == 16 || T == 32;
+    if (dtype == EQL_FP16 || dtype == EQL_BF16) return T == 4 || T == 8 || T == 16 || T == 32;
     return T == 4 || T == 8;            // FP32 (3xTF32): larger T leaves too few channels per tile
 }
 
@@ -461,6 +464,7 @@ UmmaBwdWeightShape umma_bwd_weight_shape(int T, int Ci, int Co, eql_dtype_t dtyp
     UmmaBwdWeightShape s{};
     s.T = T; s.Ci = Ci; s.Co = Co;
     s.elem_bytes = dtype == EQL_FP32 ? 4 : 2;
+    s.bf16 = dtype == EQL_BF16;
     const int epr = 128 / s.elem_bytes;                          // elements per raw slab row
     int max_cit = kMaxXSlabs * epr / T;                          // at most 16 raw slabs of x per chunk
     if (max_cit > 128) max_cit = 128;                            // UMMA M = 128 TMEM lanes
@@ -603,6 +607,15 @@ cudaError_t launch_umma_bwd_weight(const UmmaBwdWeightShape& s, const void* x, c
         if (s.T == 4) return go(std::integral_constant<int, 4>{}, float{});
         if (s.T == 8) return go(std::integral_constant<int, 8>{}, float{});
         return cudaErrorInvalidValue;
+    }
+    if (s.bf16) {
+        switch (s.T) {
+            case 4: return go(std::integral_constant<int, 4>{}, __nv_bfloat16{});
+            case 8: return go(std::integral_constant<int, 8>{}, __nv_bfloat16{});
+            case 16: return go(std::integral_constant<int, 16>{}, __nv_bfloat16{});
+            case 32: return go(std::integral_constant<int, 32>{}, __nv_bfloat16{});
+            default: return cudaErrorInvalidValue;
+        }
     }
     switch (s.T) {
         case 4: return go(std::integral_constant<int, 4>{}, __half{});

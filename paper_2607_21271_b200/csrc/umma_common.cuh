@@ -3,6 +3,7 @@
 // group DFT of the 64/T channels they hold, planes rounded to fp16 once and packed channel-pairwise).
 #pragma once
 
+#include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
 #include <cstring>
@@ -22,6 +23,38 @@ __device__ __forceinline__ uint32_t pack_h2(float lo, float hi) {
     memcpy(&u, &h, 4);
     return u;
 }
+
+// The 16-bit I/O flavours of the tensor-core kernels: IEEE half and bfloat16 (same byte geometry, different
+// conversions and UMMA operand format code).  The float specialisation only lets shared code compile.
+template <typename IO> struct H16;
+template <> struct H16<__half> {
+    static constexpr uint32_t kUmmaFormat = 0u;
+    static constexpr bool kIsHalf = true;
+    static __device__ __forceinline__ float2 unpack(uint32_t u) { return unpack_h2(u); }
+    static __device__ __forceinline__ uint32_t pack(float lo, float hi) { return pack_h2(lo, hi); }
+    static __device__ __forceinline__ __half narrow(float v) { return __float2half_rn(v); }
+};
+template <> struct H16<__nv_bfloat16> {
+    static constexpr uint32_t kUmmaFormat = 1u;
+    static constexpr bool kIsHalf = false;
+    static __device__ __forceinline__ float2 unpack(uint32_t u) {          // bf16 -> f32 is a 16-bit shift
+        return make_float2(__uint_as_float(u << 16), __uint_as_float(u & 0xFFFF0000u));
+    }
+    static __device__ __forceinline__ uint32_t pack(float lo, float hi) {
+        __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
+        uint32_t u;
+        memcpy(&u, &h, 4);
+        return u;
+    }
+    static __device__ __forceinline__ __nv_bfloat16 narrow(float v) { return __float2bfloat16_rn(v); }
+};
+template <> struct H16<float> {
+    static constexpr uint32_t kUmmaFormat = 0u;
+    static constexpr bool kIsHalf = false;
+    static __device__ __forceinline__ float2 unpack(uint32_t) { return make_float2(0.f, 0.f); }
+    static __device__ __forceinline__ uint32_t pack(float, float) { return 0u; }
+    static __device__ __forceinline__ float narrow(float v) { return v; }
+};
 
 // Exact GELU, x * Phi(x) with the error function (the activation after fc1 in a ViT MLP block), for the forward
 // kernels' optional fused epilogue.
@@ -44,8 +77,9 @@ __device__ __forceinline__ void load_slab_row(const uint8_t* row_base, int r, ui
 // HALF_MATH = false: butterflies in float, each plane rounded to half once.
 // HALF_MATH = true : two channels per instruction in packed half arithmetic (every butterfly output rounded
 //                    to half; about twice as cheap, error stays well inside the FP16 parity bar).
-template <int T, bool WANT_PLANE0, bool HALF_MATH = false>
+template <int T, bool WANT_PLANE0, bool HALF_MATH = false, typename IO = __half>
 __device__ __forceinline__ void dft_words(const uint32_t (&wd)[32], uint32_t (&packed)[T][(64 / T) / 2], float* plane0) {
+    static_assert(!HALF_MATH || H16<IO>::kIsHalf, "packed-half butterflies exist for IEEE half only");
     constexpr int NCH = 64 / T;
 #pragma unroll
     for (int cp = 0; cp < NCH / 2; ++cp) {
@@ -70,8 +104,8 @@ __device__ __forceinline__ void dft_words(const uint32_t (&wd)[32], uint32_t (&p
             float v0[T], v1[T];
 #pragma unroll
             for (int t = 0; t < T; t += 2) {
-                const float2 a = unpack_h2(wd[((2 * cp) * T + t) / 2]);
-                const float2 b = unpack_h2(wd[((2 * cp + 1) * T + t) / 2]);
+                const float2 a = H16<IO>::unpack(wd[((2 * cp) * T + t) / 2]);
+                const float2 b = H16<IO>::unpack(wd[((2 * cp + 1) * T + t) / 2]);
                 v0[t] = a.x; v0[t + 1] = a.y;
                 v1[t] = b.x; v1[t + 1] = b.y;
             }
@@ -79,7 +113,7 @@ __device__ __forceinline__ void dft_words(const uint32_t (&wd)[32], uint32_t (&p
             rdft_forward<T>(v1);
             if constexpr (WANT_PLANE0) { plane0[2 * cp] = v0[0]; plane0[2 * cp + 1] = v1[0]; }
 #pragma unroll
-            for (int p = 0; p < T; ++p) packed[p][cp] = pack_h2(v0[p], v1[p]);
+            for (int p = 0; p < T; ++p) packed[p][cp] = H16<IO>::pack(v0[p], v1[p]);
         }
     }
 }

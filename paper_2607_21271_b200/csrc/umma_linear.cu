@@ -181,7 +181,7 @@ __global__ void build_image_kernel(const float* __restrict__ planes, int Cin, in
         float v = 0.f;
         if (cin < Cin && cout < Cout) v = sign * planes[((size_t)plane * CinTotal + cin0 + cin) * Cout + cout];
         if constexpr (E == 2) {
-            image[idx] = __float2half_rn(v);
+            image[idx] = H16<IO>::narrow(v);
         } else {
             uint32_t hi, lo;
             split_tf32(v, hi, lo);
@@ -333,8 +333,9 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
             uint32_t ca = 0, cb = 0, cu = 0;
             bool ok = true;
             constexpr int M = kTileM * CG;
-            const uint32_t idesc_real = E == 2 ? ptx::umma_idesc_f16_f32(M, CoT) : ptx::umma_idesc_tf32_f32(M, CoT);
-            const uint32_t idesc_cplx = E == 2 ? ptx::umma_idesc_f16_f32(M, 2 * CoT) : ptx::umma_idesc_tf32_f32(M, 2 * CoT);
+            constexpr uint32_t kFmt = H16<IO>::kUmmaFormat;      // half or bfloat16 operands
+            const uint32_t idesc_real = E == 2 ? ptx::umma_idesc_f16_f32(M, CoT, kFmt) : ptx::umma_idesc_tf32_f32(M, CoT);
+            const uint32_t idesc_cplx = E == 2 ? ptx::umma_idesc_f16_f32(M, 2 * CoT, kFmt) : ptx::umma_idesc_tf32_f32(M, 2 * CoT);
             auto mma = [](uint32_t d, uint32_t a_addr, uint32_t b_addr, uint32_t idesc, uint32_t accumulate) {
                 const uint64_t ad = ptx::umma_smem_desc_k_sw32(a_addr), bd = ptx::umma_smem_desc_k_sw32(b_addr);
                 if constexpr (E == 2) {
@@ -477,7 +478,7 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
                     const int second = sw ? -16 : 16;            // where the other half of the same row lives (32-byte runs only)
                     uint32_t packed[E == 2 ? T : 1][E == 2 ? NCH / 2 : 1];
                     if constexpr (E == 2) {
-                        dft_words<T, false>(wd, packed, nullptr);
+                        dft_words<T, false, false, IO>(wd, packed, nullptr);
                     } else {
                         dft_words_f32<T>(wd);                    // wd[c*T + p] = plane p of channel c
                     }
@@ -544,7 +545,7 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
                     }
                     if constexpr (E == 2) {
 #pragma unroll
-                        for (int t = 0; t < T; t += 2) o[(g * T + t) / 2] = pack_h2(v[t], v[t + 1]);
+                        for (int t = 0; t < T; t += 2) o[(g * T + t) / 2] = H16<IO>::pack(v[t], v[t + 1]);
                     } else {
 #pragma unroll
                         for (int t = 0; t < T; ++t) o[g * T + t] = __float_as_uint(v[t]);
@@ -622,7 +623,16 @@ size_t umma_smem_bytes(int b_slot_bytes) {
 
 // Calls f(integral_constant<T>, element type tag) for the supported (T, dtype) pairs.
 template <typename F>
-cudaError_t dispatch_umma(int T, int elem_bytes, F&& f) {
+cudaError_t dispatch_umma(int T, int elem_bytes, F&& f, bool bf16 = false) {
+    if (elem_bytes == 2 && bf16) {
+        switch (T) {
+            case 4: return f(std::integral_constant<int, 4>{}, __nv_bfloat16{});
+            case 8: return f(std::integral_constant<int, 8>{}, __nv_bfloat16{});
+            case 16: return f(std::integral_constant<int, 16>{}, __nv_bfloat16{});
+            case 32: return f(std::integral_constant<int, 32>{}, __nv_bfloat16{});
+            default: return cudaErrorInvalidValue;
+        }
+    }
     if (elem_bytes == 2) {
         switch (T) {
             case 4: return f(std::integral_constant<int, 4>{}, __half{});
@@ -663,7 +673,7 @@ int umma_max_cot(int T, int elem_bytes) {
 
 
 bool umma_linear_supported(int T, eql_dtype_t dtype) {
-    if (dtype == EQL_FP16) return T == 4 || T == 8 || T == 16 || T == 32;
+    if (dtype == EQL_FP16 || dtype == EQL_BF16) return T == 4 || T == 8 || T == 16 || T == 32;
     return T == 4 || T == 8;            // FP32 (3xTF32): the hi/lo operand stages of larger T do not fit in shared memory
 }
 
@@ -671,6 +681,7 @@ UmmaLinearShape umma_linear_shape(int T, int Cin, int Cout, eql_dtype_t dtype) {
     UmmaLinearShape s{};
     s.T = T; s.Cin = Cin; s.Cout = Cout;
     s.elem_bytes = dtype == EQL_FP32 ? 4 : 2;
+    s.bf16 = dtype == EQL_BF16;
     const int max_cot = umma_max_cot(T, s.elem_bytes);           // T planes x CoT fp32 TMEM columns <= 512
     s.nTiles = (Cout + max_cot - 1) / max_cot;
     const int per = (Cout + s.nTiles - 1) / s.nTiles;
@@ -716,7 +727,7 @@ cudaError_t launch_build_umma_image(const UmmaLinearShape& s, const float* plane
         build_image_kernel<TT, IO><<<blocks, 256, 0, stream>>>(planes, s.Cin, s.Cout, s.CoT, s.nTiles, s.nK, s.rowsB,
                                                                 (IO*)image, s.cin0, s.CinTotal, s.pair ? 1 : 0);
         return cudaGetLastError();
-    });
+    }, s.bf16);
 }
 
 cudaError_t launch_umma_linear(const UmmaLinearShape& s, const void* in, void* out, int64_t N, const void* image,
@@ -805,9 +816,9 @@ cudaError_t launch_umma_linear(const UmmaLinearShape& s, const void* in, void* o
             umma_linear_kernel<TT, IO, 1, false><<<grid, kThreadsUmma, smem, stream>>>(tmap, tmap_out, prm);
             return cudaGetLastError();
         }
-    });
+    }, s.bf16);
 }
 
-bool umma_linear_pair_supported(int T, eql_dtype_t dtype) { return dtype == EQL_FP16 && (T == 4 || T == 8); }
+bool umma_linear_pair_supported(int T, eql_dtype_t dtype) { return (dtype == EQL_FP16 || dtype == EQL_BF16) && (T == 4 || T == 8); }
 
 }  // namespace eql

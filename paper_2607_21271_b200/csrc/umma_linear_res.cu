@@ -86,9 +86,9 @@ struct ResBarriers {
 // Spectral-weight operand image: planes[p][cin][cout] (float, scaled, conjugated for the data gradient) ->
 // for every (channel tile ct, chunk kc, plane p) one [128 x 16] half tile in the canonical K-major layout with
 // 32-byte swizzle: byte b of row n lives at n*32 + (((b>>4) ^ ((n>>2)&1))<<4) + (b&15); row n = channel ct*128 + n.
-template <int T>
+template <int T, typename IO>
 __global__ void build_image_res_kernel(const float* __restrict__ planes, int Cin, int Cout, int nCT, int nK,
-                                       __half* __restrict__ image) {
+                                       IO* __restrict__ image) {
     const int64_t total = (int64_t)nCT * nK * T * 128 * 16;
     for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
          idx += (int64_t)gridDim.x * blockDim.x) {
@@ -101,7 +101,7 @@ __global__ void build_image_res_kernel(const float* __restrict__ planes, int Cin
         const int cin = kc * 16 + kk, cout = ct * 128 + n;
         float v = 0.f;
         if (cin < Cin && cout < Cout) v = planes[((size_t)p * Cin + cin) * Cout + cout];
-        image[idx] = __float2half_rn(v);
+        image[idx] = H16<IO>::narrow(v);
     }
 }
 
@@ -110,9 +110,10 @@ __global__ void build_image_res_kernel(const float* __restrict__ planes, int Cin
 // complex frequency takes two MMAs of width 2 NTOK ([Re|Im] += Wr [Xr|Xi] and, with A negated, += (-Wi) [Xi|-Xr])
 // instead of three; an MMA costs about the same whatever its width, so this shortens the main loop where the larger
 // x^ buffers fit.
-template <int T, int NTOK, bool PF, bool MERGED, bool ACT>
+template <int T, int NTOK, bool PF, bool MERGED, bool ACT, typename IO>
 __global__ void __launch_bounds__(ResWarps<T>::kThreads, 1)
 umma_linear_res_kernel(const __grid_constant__ CUtensorMap tmap_in, const ResParams prm) {
+    // IO: IEEE half or bfloat16 (same byte geometry; conversions and the UMMA operand format differ)
     // NTOK tokens per tile: the accumulator of a unit is T planes x NTOK fp32 TMEM columns.  With T * NTOK = 256 two
     // accumulators alternate, so that the epilogue of a unit overlaps the MMAs of the next one.
     constexpr int NCW = ResWarps<T>::kCompute;  // compute warps
@@ -252,8 +253,8 @@ umma_linear_res_kernel(const __grid_constant__ CUtensorMap tmap_in, const ResPar
             int slot = 0;                                        // weight-ring slot of the current chunk
             uint32_t wph = 0;                                    // its phase parity
             bool ok = true;
-            const uint32_t idesc1 = ptx::umma_idesc_f16_f32(128, NTOK);          // one plane of tokens
-            const uint32_t idesc2 = ptx::umma_idesc_f16_f32(128, 2 * NTOK);      // [Re | Im] planes of a complex frequency
+            const uint32_t idesc1 = ptx::umma_idesc_f16_f32(128, NTOK, H16<IO>::kUmmaFormat);      // one plane of tokens
+            const uint32_t idesc2 = ptx::umma_idesc_f16_f32(128, 2 * NTOK, H16<IO>::kUmmaFormat);  // [Re | Im] planes of a complex frequency
             // shared-memory descriptors are built once per chunk and advanced by (byte offset >> 4) in their address field
             // (the tiles stay inside the 256 KB window, so no carry leaves it)
             auto mma = [](uint32_t d, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
@@ -356,9 +357,9 @@ umma_linear_res_kernel(const __grid_constant__ CUtensorMap tmap_in, const ResPar
                 // Ring mode has the transform on the critical path (every chunk is transformed right before its MMAs):
                 // packed-half butterflies there, two channels per instruction (-5 % kernel time, max error 5.5e-4
                 // instead of 4.7e-4 of the largest output, bar 3e-3).  Resident mode: float butterflies, one rounding.
-                if (ring) dft_words<T, false, true>(wd, packed, nullptr);
-                else
-                dft_words<T, false>(wd, packed, nullptr);
+                // (packed-half butterflies exist for IEEE half only: bfloat16 keeps 8 significand bits per rounding)
+                if constexpr (ring && H16<IO>::kIsHalf) dft_words<T, false, true>(wd, packed, nullptr);
+                else dft_words<T, false, false, IO>(wd, packed, nullptr);
                 const int s = i / PARTS, h = i % PARTS;
                 const int kc = s / SPK, q = s % SPK;
                 const int r = h * 32 + lane;                     // token row inside the tile
@@ -471,10 +472,10 @@ umma_linear_res_kernel(const __grid_constant__ CUtensorMap tmap_in, const ResPar
                         }
                         if (kWhole || (o_ok && j < rows_left)) {
                             if constexpr (T == 8)
-                                *reinterpret_cast<uint4*>(dst) = make_uint4(pack_h2(v[0], v[1]), pack_h2(v[2], v[3]),
-                                                                            pack_h2(v[4], v[5]), pack_h2(v[6], v[7]));
+                                *reinterpret_cast<uint4*>(dst) = make_uint4(H16<IO>::pack(v[0], v[1]), H16<IO>::pack(v[2], v[3]),
+                                                                            H16<IO>::pack(v[4], v[5]), H16<IO>::pack(v[6], v[7]));
                             else
-                                *reinterpret_cast<uint2*>(dst) = make_uint2(pack_h2(v[0], v[1]), pack_h2(v[2], v[3]));
+                                *reinterpret_cast<uint2*>(dst) = make_uint2(H16<IO>::pack(v[0], v[1]), H16<IO>::pack(v[2], v[3]));
                         }
                     }
                 };
@@ -522,11 +523,12 @@ size_t res_smem_bytes(int T, int nTok, bool paired, int x_slots, int w_slots, in
 }  // namespace
 
 
-bool umma_res_supported(int T, eql_dtype_t dtype) { return dtype == EQL_FP16 && (T == 4 || T == 8); }
+bool umma_res_supported(int T, eql_dtype_t dtype) { return (dtype == EQL_FP16 || dtype == EQL_BF16) && (T == 4 || T == 8); }
 
-UmmaResShape umma_res_shape(int T, int Cin, int Cout) {
+UmmaResShape umma_res_shape(int T, int Cin, int Cout, eql_dtype_t dtype) {
     UmmaResShape s{};
     s.T = T; s.Cin = Cin; s.Cout = Cout;
+    s.bf16 = dtype == EQL_BF16;
     s.nTok = 512 / T;                                            // one accumulator filling the 512 TMEM columns
     s.nK = (Cin + 15) / 16;
     s.nCT = (Cout + 127) / 128;
@@ -569,10 +571,14 @@ UmmaResShape umma_res_shape(int T, int Cin, int Cout) {
 cudaError_t launch_build_umma_res_image(const UmmaResShape& s, const float* planes, void* image, cudaStream_t stream) {
     const int64_t total = (int64_t)s.nCT * s.nK * s.T * 128 * 16;
     const int blocks = (int)((total + 255) / 256 < 4096 ? (total + 255) / 256 : 4096);
-    if (s.T == 4)
-        build_image_res_kernel<4><<<blocks, 256, 0, stream>>>(planes, s.Cin, s.Cout, s.nCT, s.nK, (__half*)image);
+    if (s.T == 4 && !s.bf16)
+        build_image_res_kernel<4, __half><<<blocks, 256, 0, stream>>>(planes, s.Cin, s.Cout, s.nCT, s.nK, (__half*)image);
+    else if (s.T == 8 && !s.bf16)
+        build_image_res_kernel<8, __half><<<blocks, 256, 0, stream>>>(planes, s.Cin, s.Cout, s.nCT, s.nK, (__half*)image);
+    else if (s.T == 4)
+        build_image_res_kernel<4, __nv_bfloat16><<<blocks, 256, 0, stream>>>(planes, s.Cin, s.Cout, s.nCT, s.nK, (__nv_bfloat16*)image);
     else if (s.T == 8)
-        build_image_res_kernel<8><<<blocks, 256, 0, stream>>>(planes, s.Cin, s.Cout, s.nCT, s.nK, (__half*)image);
+        build_image_res_kernel<8, __nv_bfloat16><<<blocks, 256, 0, stream>>>(planes, s.Cin, s.Cout, s.nCT, s.nK, (__nv_bfloat16*)image);
     else
         return cudaErrorInvalidValue;
     return cudaGetLastError();
@@ -608,19 +614,23 @@ cudaError_t launch_umma_linear_res(const UmmaResShape& s, const void* in, void* 
     const int grid = (int)(prm.num_units < num_sms ? prm.num_units : num_sms);
     const size_t smem = res_smem_bytes(s.T, s.nTok, s.paired, s.x_slots, s.w_slots, s.n_tw);
 
+    auto launch = [&](auto kernel, SmemLimitOnce& once, int threads) -> cudaError_t {
+        if (cudaError_t e = once.ensure(kernel, (int)kResSmemLimit); e != cudaSuccess) return e;
+        kernel<<<grid, threads, smem, stream>>>(tmap, prm);
+        return cudaGetLastError();
+    };
     auto go = [&](auto tc, auto nt, auto pf, auto mg) -> cudaError_t {
         constexpr int TT = decltype(tc)::value, NT = decltype(nt)::value;
         constexpr bool PF = decltype(pf)::value, MG = decltype(mg)::value;
-        if (prm.act) {
-            static SmemLimitOnce smem_limit_act;              // per kernel instantiation
-            if (cudaError_t e = smem_limit_act.ensure(umma_linear_res_kernel<TT, NT, PF, MG, true>, (int)kResSmemLimit); e != cudaSuccess) return e;
-            umma_linear_res_kernel<TT, NT, PF, MG, true><<<grid, ResWarps<TT>::kThreads, smem, stream>>>(tmap, prm);
-            return cudaGetLastError();
+        static SmemLimitOnce once[4];                         // per kernel instantiation: (activation, element type)
+        constexpr int threads = ResWarps<TT>::kThreads;
+        if (s.bf16) {
+            if (stash != nullptr) return cudaErrorInvalidValue;   // the saved-spectrum path is built for IEEE half
+            if (prm.act) return launch(umma_linear_res_kernel<TT, NT, PF, MG, true, __nv_bfloat16>, once[3], threads);
+            return launch(umma_linear_res_kernel<TT, NT, PF, MG, false, __nv_bfloat16>, once[2], threads);
         }
-        static SmemLimitOnce smem_limit;                      // per kernel instantiation
-        if (cudaError_t e = smem_limit.ensure(umma_linear_res_kernel<TT, NT, PF, MG, false>, (int)kResSmemLimit); e != cudaSuccess) return e;
-        umma_linear_res_kernel<TT, NT, PF, MG, false><<<grid, ResWarps<TT>::kThreads, smem, stream>>>(tmap, prm);
-        return cudaGetLastError();
+        if (prm.act) return launch(umma_linear_res_kernel<TT, NT, PF, MG, true, __half>, once[1], threads);
+        return launch(umma_linear_res_kernel<TT, NT, PF, MG, false, __half>, once[0], threads);
     };
     using I4 = std::integral_constant<int, 4>;
     using I8 = std::integral_constant<int, 8>;

@@ -17,7 +17,7 @@ import numpy as np
 @dataclass(frozen=True)
 class Workload:
     name: str
-    dtype: str            # "fp32" | "fp16"  (fp16 = half I/O, float accumulate)
+    dtype: str            # "fp32" | "fp16" | "bf16"  (fp16 / bf16 = 16-bit I/O, float accumulate)
     T: int                # order of the cyclic group
     Ci: int               # input channels per group element
     Co: int               # output channels per group element
@@ -36,7 +36,9 @@ class Workload:
 
     @property
     def np_dtype(self):
-        return np.float32 if self.dtype == "fp32" else np.float16
+        """Host array type of the inputs.  numpy has no bfloat16: bf16 workloads are float32 arrays whose values are
+        exactly representable in bfloat16 (the device copy is an exact narrowing)."""
+        return np.float16 if self.dtype == "fp16" else np.float32
 
     def with_tokens(self, N: int) -> "Workload":
         return replace(self, N=N, name=f"{self.name}@N={N}")
@@ -91,6 +93,11 @@ def generate(wl: Workload) -> dict:
     """
     g = np.random.Generator(np.random.PCG64(wl.seed))
     dt = wl.np_dtype
+    if wl.dtype == "bf16":
+        narrow = round_to_bf16
+    else:
+        def narrow(a):
+            return a.astype(dt)
     x = g.standard_normal((wl.N, wl.Ci * wl.T), dtype=np.float32)
     w = g.standard_normal((wl.Co, wl.Ci, wl.T), dtype=np.float32) / np.float32(np.sqrt(wl.Ci * wl.T))
     b = g.standard_normal(wl.Co, dtype=np.float32) * np.float32(np.sqrt(0.02))
@@ -100,8 +107,15 @@ def generate(wl: Workload) -> dict:
     elif wl.bias == "zero":
         bias = np.zeros(wl.Co, dtype=dt)
     else:
-        bias = b.astype(dt)
-    return {"x": x.astype(dt), "w": w.astype(dt), "bias": bias, "dy": dy.astype(dt)}
+        bias = narrow(b)
+    return {"x": narrow(x), "w": narrow(w), "bias": bias, "dy": narrow(dy)}
+
+
+def round_to_bf16(a: np.ndarray) -> np.ndarray:
+    """float32 values rounded to the nearest bfloat16 (ties to even), returned as float32."""
+    u = np.ascontiguousarray(a, dtype=np.float32).view(np.uint32).astype(np.uint64)
+    u = (u + 0x7FFF + ((u >> 16) & 1)) & 0xFFFF0000
+    return u.astype(np.uint32).view(np.float32).reshape(a.shape)
 
 
 def sample_rows(N: int, count: int, seed: int = 0) -> np.ndarray:

@@ -8,16 +8,30 @@ import torch
 import paper_2607_21271_b200 as eq
 from oracle import eqlinear_oracle as orc
 
-TOL = {"fp32": 1e-5, "fp16": 3e-3}          # max|err| / max|ref|, the stated parity bars
+# max|err| / max|ref|.  FP32 and FP16: the stated parity bars.  BF16 (not among the stated configurations): derived from
+# the arithmetic -- the scheme is the FP16 one (spectra of activations and weight rounded once, float accumulation, one
+# rounding of the output) with unit roundoff u = 2^-9 instead of 2^-11; the FP16 path measures 0.8-1.3 u_half against
+# its bar of 6 u_half, the BF16 bar is the same 6 u = 1.2e-2.
+TOL = {"fp32": 1e-5, "fp16": 3e-3, "bf16": 6 * 2.0 ** -9}
 CANARY = 64                                  # guard elements after every output buffer
 
 
 def torch_dtype(dtype: str):
-    return torch.float32 if dtype == "fp32" else torch.float16
+    return {"fp32": torch.float32, "fp16": torch.float16, "bf16": torch.bfloat16}[dtype]
 
 
 def eql_dtype(dtype: str) -> int:
-    return eq.EQL_FP32 if dtype == "fp32" else eq.EQL_FP16
+    return {"fp32": eq.EQL_FP32, "fp16": eq.EQL_FP16, "bf16": eq.EQL_BF16}[dtype]
+
+
+def to_device(a: np.ndarray, dtype: str, dev):
+    """Host array of a workload -> device tensor of the plan's dtype (bf16 inputs are float32 arrays holding
+    bfloat16-representable values: the narrowing is exact)."""
+    return torch.from_numpy(np.ascontiguousarray(a)).to(dev).to(torch_dtype(dtype))
+
+
+def to_host(t) -> np.ndarray:
+    return (t.float() if t.dtype == torch.bfloat16 else t).cpu().numpy()
 
 
 def rel_max_err(got: np.ndarray, ref: np.ndarray) -> float:
@@ -33,8 +47,8 @@ class GpuLayer:
         self.T, self.Ci, self.Co, self.dtype = T, Ci, Co, dtype
         self.dev = torch.device(device)
         self.td = torch_dtype(dtype)
-        self.w = torch.from_numpy(np.ascontiguousarray(w)).to(self.dev)
-        self.bias = None if bias is None else torch.from_numpy(np.ascontiguousarray(bias)).to(self.dev)
+        self.w = to_device(w, dtype, self.dev)
+        self.bias = None if bias is None else to_device(bias, dtype, self.dev)
         self.ws_bytes = eq.eqlinear_workspace_bytes(T, Ci, Co, eql_dtype(dtype))
         self.ws = torch.empty(self.ws_bytes + 256, dtype=torch.uint8, device=self.dev)
         assert self.ws.data_ptr() % 256 == 0
@@ -66,26 +80,26 @@ class GpuLayer:
 
     def fwd(self, x_np):
         N = x_np.shape[0]
-        x = torch.from_numpy(np.ascontiguousarray(x_np)).to(self.dev)
+        x = to_device(x_np, self.dtype, self.dev)
         buf, y = self._out(N, self.Co * self.T)
         eq.eqlinear_fwd(self.plan, x if N else None, buf if N else None, N, self.stream)
         torch.cuda.synchronize(self.dev)
         assert self._canary_ok(buf, N * self.Co * self.T), "fwd wrote past its output"
-        return y.cpu().numpy()
+        return to_host(y)
 
     def bwd_data(self, dy_np):
         N = dy_np.shape[0]
-        dy = torch.from_numpy(np.ascontiguousarray(dy_np)).to(self.dev)
+        dy = to_device(dy_np, self.dtype, self.dev)
         buf, dx = self._out(N, self.Ci * self.T)
         eq.eqlinear_bwd_data(self.plan, dy if N else None, buf if N else None, N, self.stream)
         torch.cuda.synchronize(self.dev)
         assert self._canary_ok(buf, N * self.Ci * self.T), "bwd_data wrote past its output"
-        return dx.cpu().numpy()
+        return to_host(dx)
 
     def bwd_weight(self, x_np, dy_np, want_db=True):
         N = x_np.shape[0]
-        x = torch.from_numpy(np.ascontiguousarray(x_np)).to(self.dev)
-        dy = torch.from_numpy(np.ascontiguousarray(dy_np)).to(self.dev)
+        x = to_device(x_np, self.dtype, self.dev)
+        dy = to_device(dy_np, self.dtype, self.dev)
         nw = self.Co * self.Ci * self.T
         wbuf, _ = self._out(1, nw, torch.float32)
         bbuf, _ = self._out(1, self.Co, torch.float32)

@@ -66,6 +66,51 @@ def test_fused_gelu_epilogue(dtype, T, Ci, Co, N, flags, kernel):
     assert rel_max_err(dx, orc.bwd_data(d["dy"], d["w"])) <= TOL[dtype]
 
 
+# ------------------------------------------------------------------ bfloat16 I/O
+@pytest.mark.parametrize("T,Ci,Co,N,flags,kernels", [
+    (8, 96, 384, 1500, 0, (2, 2, 1)),                                         # resident activations / ring mode / tcgen05 dW
+    (4, 24, 96, 1111, 0, (2, 1, 1)),
+    (8, 96, 384, 1000, eq.EQL_FLAG_FORCE_STREAMING, (1, 1, 1)),               # streaming kernel
+    (4, 100, 130, 515, eq.EQL_FLAG_FORCE_STREAMING | eq.EQL_FLAG_CTA_PAIR, (3, 3, 1)),   # CTA pairs
+    (16, 17, 33, 333, 0, (1, 1, 1)), (32, 32, 32, 500, 0, (1, 1, 1)),
+    (5, 8, 24, 333, 0, (0, 0, 0)), (2, 8, 16, 333, 0, (0, 0, 0)),             # CUDA-core kernels
+])
+def test_bf16_matches_oracle(T, Ci, Co, N, flags, kernels):
+    """EQL_BF16: bfloat16 inputs and outputs, float accumulation -- every pass of every kernel family against the oracle
+    fed the same bfloat16-representable values.  The bar is derived in tests/harness.py (6 unit roundoffs, as for FP16)."""
+    wl = Workload("bf16", "bf16", T, Ci, Co, N, "normal", ("fwd", "bwd_data", "bwd_weight"), 35)
+    d = generate(wl)
+    layer = GpuLayer(T, Ci, Co, "bf16", d["w"], d["bias"], flags)
+    try:
+        info = eq.eqlinear_plan_info(layer.plan)
+        assert (info.fwd_kernel, info.bwd_data_kernel, info.bwd_weight_kernel) == kernels
+        with pytest.raises(eq.EqlError) as e:                                 # the saved-spectrum path is FP16 only
+            eq.eqlinear_spectrum_bytes(layer.plan, N)
+        assert e.value.status == eq.binding.EQL_ERR_UNSUPPORTED
+    finally:
+        layer.close()
+    errs = check_workload(wl, flags=flags, data=d)
+    print({k: f"{v:.2e}" for k, v in errs.items()})
+    for k, v in errs.items():
+        assert v <= TOL["bf16"], f"T={T} Ci={Ci} Co={Co} N={N} flags={flags}: {k} error {v:.3e}"
+
+
+def test_bf16_full_size_headline_shape_with_gelu():
+    """The headline layer's shape in bfloat16 at full size, forward with the fused GELU, data and weight gradients."""
+    wl = Workload("bf16_fc1", "bf16", 8, 96, 384, 128 * 197, "normal", ("fwd", "bwd_data", "bwd_weight"), 36)
+    d = generate(wl)
+    errs = check_workload(wl, passes=("bwd_data", "bwd_weight"), data=d)
+    layer = GpuLayer(wl.T, wl.Ci, wl.Co, "bf16", d["w"], d["bias"], eq.EQL_FLAG_GELU)
+    try:
+        errs["gelu(y)"] = rel_max_err(layer.fwd(d["x"]), _gelu(orc.fwd(d["x"], d["w"], d["bias"])))
+        assert layer.raw_status() == 0
+    finally:
+        layer.close()
+    print({k: f"{v:.2e}" for k, v in errs.items()})
+    for k, v in errs.items():
+        assert v <= TOL["bf16"], f"{k} error {v:.3e}"
+
+
 def test_fused_gelu_is_refused_where_the_forward_sum_is_split():
     """FP32 plans on the tensor cores with more than 256 input channels add segments of the reduction in global memory:
     no place to apply an activation to the finished sum."""

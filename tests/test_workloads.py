@@ -9,6 +9,23 @@ from paper_2607_21271_b200.workloads import (ALL_WORKLOADS, BLOCK_SHAPES, CONFIG
                                               sample_rows)
 
 
+def test_bf16_rounding_is_round_to_nearest_even():
+    """bf16 workloads are float32 arrays of bfloat16-representable values: the rounding must be the IEEE one (checked
+    against torch's conversion, and on the tie cases by hand)."""
+    import torch
+    from paper_2607_21271_b200.workloads import round_to_bf16
+    g = np.random.Generator(np.random.PCG64(3))
+    a = (g.standard_normal(100000) * np.exp(g.uniform(-20, 20, 100000))).astype(np.float32)
+    ref = torch.from_numpy(a).to(torch.bfloat16).float().numpy()
+    assert np.array_equal(round_to_bf16(a), ref)
+    ties = np.array([1.0 + 2.0 ** -8, 1.0 + 3 * 2.0 ** -8, -(1.0 + 2.0 ** -8)], dtype=np.float32)   # halfway cases
+    assert np.array_equal(round_to_bf16(ties), np.array([1.0, 1.0 + 2.0 ** -6, -1.0], dtype=np.float32))
+    wl = Workload("b", "bf16", 4, 8, 8, 16, "normal", ("fwd",), 1)
+    d = generate(wl)
+    for k in ("x", "w", "bias", "dy"):
+        assert d[k].dtype == np.float32 and np.array_equal(round_to_bf16(d[k]), d[k])
+
+
 def test_tables_are_consistent():
     assert HEADLINE in CONFIGS
     assert set(CONFIGS) | set(OPERATOR_SHAPES) | set(BLOCK_SHAPES) == set(ALL_WORKLOADS)
