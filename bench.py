@@ -53,6 +53,17 @@ FALLBACK_BF16_TFLOPS = 1590.0
 L2_BYTES = 126e6
 
 
+def torch_dtype_of(wl):
+    import torch
+    return {"fp32": torch.float32, "fp16": torch.float16, "bf16": torch.bfloat16}[wl.dtype]
+
+
+def host_np(t):
+    """Device tensor -> numpy (bfloat16 widened to float32 first: numpy has no bfloat16)."""
+    import torch
+    return (t.float() if t.dtype == torch.bfloat16 else t).cpu().numpy()
+
+
 def load_peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
@@ -237,14 +248,14 @@ def check_against_oracle(orc, wl, d, outs):
     res = {"rows": int(len(rows)), "channels": [int(len(ch_i)), int(len(ch_o))]}
     bias = None if d["bias"] is None else d["bias"][ch_o]
     if "y" in outs:
-        res["y"] = rel(outs["y"][rows][:, cols_o].cpu().numpy(), orc.fwd(d["x"][rows], d["w"][ch_o], bias))
+        res["y"] = rel(host_np(outs["y"][rows][:, cols_o]), orc.fwd(d["x"][rows], d["w"][ch_o], bias))
     if "dx" in outs:
-        res["dx"] = rel(outs["dx"][rows][:, cols_i].cpu().numpy(), orc.bwd_data(d["dy"][rows], d["w"][:, ch_i]))
+        res["dx"] = rel(host_np(outs["dx"][rows][:, cols_i]), orc.bwd_data(d["dy"][rows], d["w"][:, ch_i]))
     if "dw" in outs:
         rdw, rdb = orc.bwd_weight(d["x"][:, cols_i], d["dy"][:, cols_o], T)
         res["dw"] = rel(outs["dw"].cpu().numpy()[np.ix_(ch_o, ch_i)], rdw)
         res["db"] = rel(outs["db"].cpu().numpy()[ch_o], rdb)
-    tol = 1e-5 if wl.dtype == "fp32" else 3e-3
+    tol = {"fp32": 1e-5, "fp16": 3e-3, "bf16": 6 * 2.0 ** -9}[wl.dtype]      # bf16: six unit roundoffs, as the FP16 bar
     res["tolerance"] = tol
     res["ok"] = all(res[k] <= tol for k in ("y", "dx", "dw", "db") if k in res)
     return res
@@ -294,18 +305,18 @@ def dense_context(wl, d, dev, iters=8):
     import torch.nn.functional as F
 
     T, Ci, Co = wl.T, wl.Ci, wl.Co
-    td = torch.float32 if wl.dtype == "fp32" else torch.float16
-    w = torch.from_numpy(d["w"]).to(dev)
+    td = torch_dtype_of(wl)
+    w = torch.from_numpy(d["w"]).to(dev).to(td)
     t_idx = torch.arange(T, device=dev)
     r = (t_idx[:, None] - t_idx[None, :]) % T                       # [t, s] -> group offset (t - s) mod T
     W = w[:, :, r].permute(0, 2, 1, 3).reshape(Co * T, Ci * T).contiguous()   # W[(o,t),(i,s)] = w[o,i,(t-s) mod T]
-    b = None if d["bias"] is None else torch.from_numpy(d["bias"]).to(dev).repeat_interleave(T)
-    x = torch.from_numpy(d["x"]).to(dev).requires_grad_(True)
-    dy = torch.from_numpy(d["dy"]).to(dev) if "bwd_weight" in wl.passes else None
+    b = None if d["bias"] is None else torch.from_numpy(d["bias"]).to(dev).to(td).repeat_interleave(T)
+    x = torch.from_numpy(d["x"]).to(dev).to(td).requires_grad_(True)
+    dy = torch.from_numpy(d["dy"]).to(dev).to(td) if "bwd_weight" in wl.passes else None
     W.requires_grad_(True)
     if b is not None:
         b.requires_grad_(True)
-    modes = [("fp16", None)] if td == torch.float16 else [("fp32_tf32_off", False), ("fp32_tf32_on", True)]
+    modes = [(wl.dtype, None)] if td != torch.float32 else [("fp32_tf32_off", False), ("fp32_tf32_on", True)]
     res = {}
     old = torch.backends.cuda.matmul.allow_tf32
     try:
@@ -351,15 +362,15 @@ def run_workload(args, wl, rt):
     dev, world, rank, local_rank, use_dist = rt["dev"], rt["world"], rt["rank"], rt["local_rank"], rt["use_dist"]
     n_gpus = world
     peaks = load_peaks()
-    td = torch.float32 if wl.dtype == "fp32" else torch.float16
-    code = eq.EQL_FP32 if wl.dtype == "fp32" else eq.EQL_FP16
+    td = torch_dtype_of(wl)
+    code = {"fp32": eq.EQL_FP32, "fp16": eq.EQL_FP16, "bf16": eq.EQL_BF16}[wl.dtype]
     esz = 4 if wl.dtype == "fp32" else 2
     has_bwd = "bwd_weight" in wl.passes
     d = generate(wl)
     stream = torch.cuda.current_stream(dev).cuda_stream
 
-    w = torch.from_numpy(d["w"]).to(dev)
-    b = None if d["bias"] is None else torch.from_numpy(d["bias"]).to(dev)
+    w = torch.from_numpy(d["w"]).to(dev).to(td)
+    b = None if d["bias"] is None else torch.from_numpy(d["bias"]).to(dev).to(td)
     ws_bytes = eq.eqlinear_workspace_bytes(wl.T, wl.Ci, wl.Co, code)
     ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
     flags = eq.EQL_FLAG_FORCE_SIMT if args.force_simt else 0
@@ -374,8 +385,8 @@ def run_workload(args, wl, rt):
     # a 256 MB buffer is overwritten, and the step time is the sum of the per-call event times (the flush excluded).
     flush_l2 = n_sets * bytes_per_set < 2.5 * L2_BYTES
     flush_buf = torch.empty(int(2 * L2_BYTES + 4e6), dtype=torch.uint8, device=dev) if flush_l2 else None
-    x0 = torch.from_numpy(d["x"]).to(dev)
-    dy0 = torch.from_numpy(d["dy"]).to(dev) if has_bwd else None
+    x0 = torch.from_numpy(d["x"]).to(dev).to(td)
+    dy0 = torch.from_numpy(d["dy"]).to(dev).to(td) if has_bwd else None
     sets = []
     for i in range(n_sets):
         s = {"x": x0 if i == 0 else x0.clone(), "y": torch.empty(wl.N, wl.Dout, dtype=td, device=dev)}
@@ -512,7 +523,7 @@ def run_workload(args, wl, rt):
     # plans compute in TF32 with the 3xTF32 split (three tensor-core products per spectral product), against the fp32
     # matmul throughput with TF32 allowed measured in this run; their CUDA-core kernels against the FFMA figure.
     fp32_peaks = measure_fp32_peaks(dev) if wl.dtype == "fp32" else None
-    if wl.dtype == "fp16":
+    if wl.dtype in ("fp16", "bf16"):
         tc_peak, tc_flops, tc_note = peaks["bf16_tflops"], flops, f"bf16 dense matmul, of {peaks['source']}"
     elif kernel_kind[dom]:
         tc_peak, tc_flops, tc_note = fp32_peaks["tf32_tflops"], 3 * flops, "fp32 matmul with TF32 allowed, measured in this run; 3xTF32 = 3 products per spectral product"
@@ -521,7 +532,7 @@ def run_workload(args, wl, rt):
     tc_time = tc_flops / (tc_peak * 1e12)
     traffic = load_committed_traffic()
     if tc_time > hbm_time:
-        head = {"bound": "tensor" if (wl.dtype == "fp16" or kernel_kind[dom]) else "alu", "kernel": f"eqlinear_{dom}",
+        head = {"bound": "tensor" if (wl.dtype != "fp32" or kernel_kind[dom]) else "alu", "kernel": f"eqlinear_{dom}",
                 "achieved": tc_flops / dom_s / 1e12, "peak": tc_peak, "unit": "TFLOP/s", "frac": tc_flops / dom_s / 1e12 / tc_peak}
     else:
         head = {"bound": "hbm", "kernel": f"eqlinear_{dom}", "achieved": alg_bytes[dom] / dom_s / 1e9,
@@ -567,11 +578,11 @@ def run_workload(args, wl, rt):
     # end to end through the host-buffer C-ABI call: pinned host buffers, copies inside the timed region
     e2e = None
     if not args.no_e2e:
-        xh = torch.from_numpy(d["x"]).pin_memory()
+        xh = torch.from_numpy(d["x"]).to(td).pin_memory()
         yh = torch.empty(wl.N, wl.Dout, dtype=td).pin_memory()
         s0 = sets[0]
         if has_bwd:
-            dyh = torch.from_numpy(d["dy"]).pin_memory()
+            dyh = torch.from_numpy(d["dy"]).to(td).pin_memory()
             dxh = torch.empty(wl.N, wl.Din, dtype=td).pin_memory()
             dwh = torch.empty(wl.Co, wl.Ci, wl.T, dtype=torch.float32).pin_memory()
             dbh = torch.empty(wl.Co, dtype=torch.float32).pin_memory()
@@ -629,7 +640,7 @@ def run_workload(args, wl, rt):
         return None
     return {"metric": metric_name(wl), "value": value, "unit": "tokens/s", "n_gpus": n_gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "f16" if wl.dtype == "fp16" else "f32",
+            "scaling": "weak", "vs_baseline": None, "dtype": {"fp16": "f16", "bf16": "bf16", "fp32": "f32"}[wl.dtype],
             "data": "synthetic",
             "config": workload_config(wl, n_gpus, {"l2": ("flushed before every step (256 MB overwrite), step time = sum of the calls' event times"
                                                           if flush_l2 else f"rotating {n_sets} buffer sets "

@@ -76,6 +76,8 @@ OPERATOR_SHAPES = {
 BLOCK_SHAPES = {
     "vit_b_qkv_fp16": Workload("vit_b_qkv_fp16", "fp16", 8, 96, 3 * 96, 128 * 197, "normal", _FB, 6),
     "vit_b_fc2_fp16": Workload("vit_b_fc2_fp16", "fp16", 8, 384, 96, 128 * 197, "normal", _FB, 7),
+    # the headline layer with bfloat16 I/O
+    "vit_b_fc1_bf16": Workload("vit_b_fc1_bf16", "bf16", 8, 96, 384, 128 * 197, "zero", _FB, 2),
 }
 
 ALL_WORKLOADS = {**CONFIGS, **OPERATOR_SHAPES, **BLOCK_SHAPES}

@@ -32,7 +32,7 @@ def test_tables_are_consistent():
     assert not set(CONFIGS) & set(OPERATOR_SHAPES)
     for name, wl in ALL_WORKLOADS.items():
         assert wl.name == name
-        assert wl.dtype in ("fp32", "fp16") and wl.bias in ("none", "zero", "normal")
+        assert wl.dtype in ("fp32", "fp16", "bf16") and wl.bias in ("none", "zero", "normal")
         assert wl.Din == wl.Ci * wl.T and wl.Dout == wl.Co * wl.T
         esz = 4 if wl.dtype == "fp32" else 2
         assert (wl.Din * esz) % 16 == 0 and (wl.Dout * esz) % 16 == 0          # rows are whole 16-byte units
