@@ -463,6 +463,40 @@ def test_runtime_argument_errors():
         layer.close()
 
 
+def test_plan_on_a_second_stream():
+    """A plan is not tied to the stream it was built on: built on one stream (the build is ordered before later use by a
+    stream synchronisation here), then used from another non-default stream, with results equal bit for bit to those on
+    the first."""
+    wl = Workload("stream", "fp16", 8, 96, 200, 3000, "normal", ("fwd", "bwd_data", "bwd_weight"), 29)
+    d = generate(wl)
+    layer = GpuLayer(wl.T, wl.Ci, wl.Co, wl.dtype, d["w"], d["bias"])
+    try:
+        y0, dx0 = layer.fwd(d["x"]), layer.bwd_data(d["dy"])
+        dw0, db0 = layer.bwd_weight(d["x"], d["dy"])
+        torch.cuda.synchronize()
+        side = torch.cuda.Stream()
+        x, dy = torch.from_numpy(d["x"]).cuda(), torch.from_numpy(d["dy"]).cuda()
+        y = torch.empty(wl.N, wl.Dout, dtype=torch.float16, device="cuda")
+        dx = torch.empty(wl.N, wl.Din, dtype=torch.float16, device="cuda")
+        dw = torch.empty(wl.Co, wl.Ci, wl.T, dtype=torch.float32, device="cuda")
+        db = torch.empty(wl.Co, dtype=torch.float32, device="cuda")
+        sb = eq.eqlinear_bwd_weight_scratch_bytes(layer.plan, wl.N)
+        sc = torch.empty(sb, dtype=torch.uint8, device="cuda")
+        torch.cuda.synchronize()
+        with torch.cuda.stream(side):
+            s = side.cuda_stream
+            eq.eqlinear_fwd(layer.plan, x, y, wl.N, s)
+            eq.eqlinear_bwd_data(layer.plan, dy, dx, wl.N, s)
+            eq.eqlinear_bwd_weight(layer.plan, x, dy, dw, db, wl.N, sc, sb, s)
+            assert eq.eqlinear_plan_device_status(layer.plan, s) == eq.binding.EQL_OK
+        side.synchronize()
+        assert np.array_equal(y.cpu().numpy(), y0) and np.array_equal(dx.cpu().numpy(), dx0)
+        assert np.array_equal(dw.cpu().numpy(), dw0) and np.array_equal(db.cpu().numpy(), db0)
+        assert rel_max_err(y0, orc.fwd(d["x"], d["w"], d["bias"])) <= TOL["fp16"]
+    finally:
+        layer.close()
+
+
 def test_plan_is_refused_on_another_device():
     """A plan's workspace and tensor maps belong to the GPU it was built on: with another device current every entry
     point that takes the plan must return EQL_ERR_INVALID_ARG before launching anything (needs two GPUs)."""

@@ -41,8 +41,8 @@ def brute_fwd(x, w, b, T, correlation=False):
     return y.reshape(N, Co * T)
 
 
-@pytest.mark.parametrize("T", [1, 2, 3, 4, 5, 8, 16])
-@pytest.mark.parametrize("Ci,Co,N", [(1, 1, 1), (3, 2, 2), (2, 5, 3)])
+@pytest.mark.parametrize("T", [1, 2, 3, 4, 5, 6, 7, 8, 12, 16, 32])
+@pytest.mark.parametrize("Ci,Co,N", [(1, 1, 1), (3, 2, 2), (2, 5, 3), (8, 3, 5)])
 @pytest.mark.parametrize("correlation", [False, True])
 def test_forward_matches_brute_force(T, Ci, Co, N, correlation):
     x, w, b = rnd(1, N, Ci * T), rnd(2, Co, Ci, T), rnd(3, Co)
@@ -53,7 +53,7 @@ def test_forward_matches_brute_force(T, Ci, Co, N, correlation):
     assert np.abs(got_nb - brute_fwd(x, w, None, T, correlation)).max() <= 1e-13 * max(1.0, np.abs(ref).max())
 
 
-@pytest.mark.parametrize("T", [1, 2, 3, 4, 5, 8])
+@pytest.mark.parametrize("T", [1, 2, 3, 4, 5, 6, 7, 8, 12])
 @pytest.mark.parametrize("correlation", [False, True])
 def test_gradients_match_finite_structure(T, correlation):
     """The layer is linear, so its exact gradients are read off scalar by scalar:
