@@ -366,6 +366,7 @@ bwd_weight_finalize_kernel(const float* __restrict__ part, const float* __restri
     __shared__ float planes[T][33];
     __shared__ float2 tw[T];
     fill_twiddles<T>(tw);
+    asm volatile("griddepcontrol.wait;" ::: "memory");         // launched to overlap the tail of the kernel that writes `part`
     const int pair = threadIdx.x & 31, p = threadIdx.x >> 5;
     const int idx = blockIdx.x * 32 + pair;
     const size_t plane_stride = (size_t)Co * Ci;
@@ -501,9 +502,8 @@ cudaError_t launch_bwd_weight_finalize(int T, bool correlation, const float* scr
     const float* db_part = scratch + (size_t)splits * T * Co * Ci;
     return dispatch_T(T, [&](auto tc) {
         constexpr int TT = decltype(tc)::value;
-        bwd_weight_finalize_kernel<TT><<<finalize_blocks(TT, Ci, Co), 32 * TT, 0, stream>>>(part, db_part, splits, Ci, Co,
-                                                                                             correlation, dw, db, accumulate);
-        return cudaGetLastError();
+        return launch_overlapped(bwd_weight_finalize_kernel<TT>, dim3(finalize_blocks(TT, Ci, Co)), dim3(32 * TT), 0, stream,
+                                 part, db_part, splits, Ci, Co, correlation, dw, db, accumulate);
     });
 }
 
@@ -528,9 +528,8 @@ cudaError_t launch_direct_bwd_weight(int T, eql_dtype_t dtype, bool correlation,
                 (const __half*)x, (const __half*)dy, N, Ci, Co, split.tokens_per_split, part, db_part);
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return e;
-        bwd_weight_finalize_kernel<TT><<<finalize_blocks(TT, Ci, Co), 32 * TT, 0, stream>>>(
-            part, db_part, split.splits, Ci, Co, correlation, dw, db, false);
-        return cudaGetLastError();
+        return launch_overlapped(bwd_weight_finalize_kernel<TT>, dim3(finalize_blocks(TT, Ci, Co)), dim3(32 * TT), 0, stream,
+                                 (const float*)part, (const float*)db_part, split.splits, Ci, Co, correlation, dw, db, false);
     });
 }
 

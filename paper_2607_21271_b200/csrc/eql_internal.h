@@ -50,6 +50,20 @@ struct SmemLimitOnce {
 
 // Group orders the library is built for: every order up to 8, and 12, 16, 32.  The powers of two use butterflies and (4
 // to 32, 2 not) the tensor-core kernels; the others run the CUDA-core kernels with a table-driven transform.
+// Launches `kernel` so that it may start while the kernel before it in the stream is finishing (programmatic dependent
+// launch); the kernel must call ptx::grid_dependency_wait() before its first access to global memory.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_overlapped(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                                     Args&&... args) {
+    cudaLaunchConfig_t cfg{};
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = stream;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 inline bool supported_T(int T) { return (T >= 1 && T <= 8) || T == 12 || T == 16 || T == 32; }
 
 // ---- CUDA-core (FFMA) kernels, direct_kernels.cu -------------------------------------------------

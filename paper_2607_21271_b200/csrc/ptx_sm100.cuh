@@ -82,6 +82,15 @@ __device__ __forceinline__ void tc_fence_after_sync() {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 }
 
+// ---------------------------------------------------------------- programmatic dependent launch
+// A kernel launched with the programmatic-stream-serialization attribute may be scheduled while the kernel before it
+// in the stream is still running (as SMs become free); grid_dependency_wait() returns once that kernel has completed
+// and its memory is visible, so everything above it (barrier set-up, TMEM allocation) overlaps the predecessor's tail.
+// Nothing that touches global memory may come before it.  Without the attribute, or behind a kernel that never calls
+// grid_launch_dependents(), both are no-ops / the wait is already satisfied.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ---------------------------------------------------------------- TMA
 // 2-D tiled load global -> this CTA's shared memory; completion counted in bytes on `bar`.
 __device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* map, int c0, int c1, uint64_t* bar) {

@@ -106,6 +106,11 @@ umma_bwd_weight_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
     __syncthreads();
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = bar->tmem_base;
+    // This kernel may have been scheduled while the kernel before it in the stream is still finishing: everything above
+    // (barriers, tensor memory) overlapped that; nothing below may run before its results are visible.  The kernel
+    // behind this one gets the same head start.
+    ptx::grid_dependency_wait();
+    ptx::grid_launch_dependents();
 
     // unit -> (token range, input-channel tile, output-channel tile); output tile fastest so that the
     // CTAs sharing the same x rows run at the same time
@@ -600,8 +605,7 @@ cudaError_t launch_umma_bwd_weight(const UmmaBwdWeightShape& s, const void* x, c
         using IO = decltype(io);
         static SmemLimitOnce smem_limit;                      // per kernel instantiation
         if (cudaError_t e = smem_limit.ensure(umma_bwd_weight_kernel<TT, IO>, 227 * 1024); e != cudaSuccess) return e;
-        umma_bwd_weight_kernel<TT, IO><<<grid, kThreadsBw, smem, stream>>>(mx, my, mp, prm);
-        return cudaGetLastError();
+        return launch_overlapped(umma_bwd_weight_kernel<TT, IO>, dim3(grid), dim3(kThreadsBw), smem, stream, mx, my, mp, prm);
     };
     if (E == 4) {
         if (s.T == 4) return go(std::integral_constant<int, 4>{}, float{});

@@ -141,6 +141,11 @@ umma_bwd_weight_saved_kernel(const __grid_constant__ CUtensorMap tmap_dy, const 
     __syncthreads();
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = bar->tmem_base;
+    // This kernel may have been scheduled while the kernel before it in the stream is still finishing: everything above
+    // (barriers, tensor memory) overlapped that; nothing below may run before its results are visible.  The kernel
+    // behind this one gets the same head start.
+    ptx::grid_dependency_wait();
+    ptx::grid_launch_dependents();
 
     // unit -> (token range, input-channel tile, output-channel tile); output tile fastest so that the
     // CTAs sharing the same x^ blobs run at the same time
@@ -485,8 +490,7 @@ cudaError_t launch_umma_bwd_weight_saved(const UmmaBwdWeightShape& s, const void
         constexpr bool MG = decltype(mg)::value;
         static SmemLimitOnce smem_limit;                      // per kernel instantiation
         if (cudaError_t e = smem_limit.ensure(umma_bwd_weight_saved_kernel<TT, MG>, 227 * 1024); e != cudaSuccess) return e;
-        umma_bwd_weight_saved_kernel<TT, MG><<<grid, kThreadsBw, smem, stream>>>(my, mp, prm);
-        return cudaGetLastError();
+        return launch_overlapped(umma_bwd_weight_saved_kernel<TT, MG>, dim3(grid), dim3(kThreadsBw), smem, stream, my, mp, prm);
     };
     auto go = [&](auto tc) -> cudaError_t { return merged ? go2(tc, std::true_type{}) : go2(tc, std::false_type{}); };
     switch (s.T) {

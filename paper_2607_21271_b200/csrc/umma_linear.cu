@@ -253,6 +253,11 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
     }
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = bar->tmem_base;
+    // This kernel may have been scheduled while the kernel before it in the stream is still finishing: everything above
+    // (barriers, tensor memory) overlapped that; nothing below may run before its results are visible.  The kernel
+    // behind this one gets the same head start.
+    ptx::grid_dependency_wait();
+    ptx::grid_launch_dependents();
 
     const int nK = prm.nK, nTiles = prm.nTiles, CoT = prm.CoT, rowsB = prm.rowsB;
     const int64_t first = blockIdx.x / CG, stride = gridDim.x / CG;
@@ -780,11 +785,13 @@ cudaError_t launch_umma_linear(const UmmaLinearShape& s, const void* in, void* o
                 auto kernel = prm.act ? umma_linear_kernel<TT, IO, 2, true> : umma_linear_kernel<TT, IO, 2, false>;
                 if (cudaError_t e = smem_limit[prm.act ? 1 : 0].ensure(kernel, 227 * 1024); e != cudaSuccess) return e;
                 cudaLaunchConfig_t cfg{};
-                cudaLaunchAttribute attr[1];
+                cudaLaunchAttribute attr[2];
                 attr[0].id = cudaLaunchAttributeClusterDimension;
                 attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+                attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;     // see ptx::grid_dependency_wait
+                attr[1].val.programmaticStreamSerializationAllowed = 1;
                 cfg.blockDim = dim3(kThreadsUmma); cfg.dynamicSmemBytes = smem; cfg.stream = stream;
-                cfg.attrs = attr; cfg.numAttrs = 1;
+                cfg.attrs = attr; cfg.numAttrs = 2;
                 // persistent: as many pairs as can be resident at once (pairs need two SMs of one GPC), at most one per unit
                 static std::atomic<int> max_pairs{0};
                 int pairs = max_pairs.load(std::memory_order_relaxed);
@@ -808,13 +815,11 @@ cudaError_t launch_umma_linear(const UmmaLinearShape& s, const void* in, void* o
             if (prm.act) {
                 static SmemLimitOnce smem_limit_act;              // per kernel instantiation
                 if (cudaError_t e = smem_limit_act.ensure(umma_linear_kernel<TT, IO, 1, true>, 227 * 1024); e != cudaSuccess) return e;
-                umma_linear_kernel<TT, IO, 1, true><<<grid, kThreadsUmma, smem, stream>>>(tmap, tmap_out, prm);
-                return cudaGetLastError();
+                return launch_overlapped(umma_linear_kernel<TT, IO, 1, true>, dim3(grid), dim3(kThreadsUmma), smem, stream, tmap, tmap_out, prm);
             }
             static SmemLimitOnce smem_limit;                      // per kernel instantiation
             if (cudaError_t e = smem_limit.ensure(umma_linear_kernel<TT, IO, 1, false>, 227 * 1024); e != cudaSuccess) return e;
-            umma_linear_kernel<TT, IO, 1, false><<<grid, kThreadsUmma, smem, stream>>>(tmap, tmap_out, prm);
-            return cudaGetLastError();
+            return launch_overlapped(umma_linear_kernel<TT, IO, 1, false>, dim3(grid), dim3(kThreadsUmma), smem, stream, tmap, tmap_out, prm);
         }
     }, s.bf16);
 }

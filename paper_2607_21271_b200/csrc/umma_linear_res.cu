@@ -163,6 +163,11 @@ umma_linear_res_kernel(const __grid_constant__ CUtensorMap tmap_in, const ResPar
     __syncthreads();
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = bar->tmem_base;
+    // This kernel may have been scheduled while the kernel before it in the stream is still finishing: everything above
+    // (barriers, tensor memory) overlapped that; nothing below may run before its results are visible.  The kernel
+    // behind this one gets the same head start.
+    ptx::grid_dependency_wait();
+    ptx::grid_launch_dependents();
 
     // this CTA's contiguous range of units; unit u = token tile (u / nCT), channel tile (u % nCT)
     const int64_t u0 = prm.num_units * (int64_t)blockIdx.x / gridDim.x;
@@ -616,8 +621,7 @@ cudaError_t launch_umma_linear_res(const UmmaResShape& s, const void* in, void* 
 
     auto launch = [&](auto kernel, SmemLimitOnce& once, int threads) -> cudaError_t {
         if (cudaError_t e = once.ensure(kernel, (int)kResSmemLimit); e != cudaSuccess) return e;
-        kernel<<<grid, threads, smem, stream>>>(tmap, prm);
-        return cudaGetLastError();
+        return launch_overlapped(kernel, dim3(grid), dim3(threads), smem, stream, tmap, prm);
     };
     auto go = [&](auto tc, auto nt, auto pf, auto mg) -> cudaError_t {
         constexpr int TT = decltype(tc)::value, NT = decltype(nt)::value;
