@@ -23,14 +23,14 @@ pytestmark = pytest.mark.soak
 def test_random_shapes_match_the_oracle():
     """Every pass of every kernel family on random shapes: both dtypes, every supported group order, ragged token counts,
     all bias kinds, the correlation flag, the streaming / CTA-pair / CUDA-core kernels forced at random, and for FP16 the
-    saved-spectrum path.  Stops at the first device time-out."""
+    saved-spectrum path; bfloat16 plans and the fused GELU epilogue at random.  Stops at the first device time-out."""
     count = int(os.environ.get("EQL_SOAK_SHAPES", "300"))
     rng = random.Random(int(os.environ.get("EQL_SOAK_SEED", "0")))
     bad, kinds = [], {}
     for it in range(count):
-        dtype = rng.choice(["fp16", "fp32"])
+        dtype = rng.choice(["fp16", "fp16", "fp32", "fp32", "bf16"])
         T = rng.choice([4, 4, 8, 8, 8, 8, 16, 16, 32, 32, 2, 3, 5, 6, 7, 12, 1])
-        e = 2 if dtype == "fp16" else 4
+        e = 4 if dtype == "fp32" else 2
         step = next(s for s in range(1, 17) if (s * T * e) % 16 == 0)      # row bytes C*T*e must be a multiple of 16
         cmax = 600 if T <= 8 else 96 if T <= 16 else 48
         if not (T in (4, 8, 16, 32)):
@@ -54,6 +54,9 @@ def test_random_shapes_match_the_oracle():
         elif r < 0.35:
             flags |= eq.EQL_FLAG_FORCE_SIMT
         corr = bool(flags & eq.EQL_FLAG_CORRELATION)
+        gelu = rng.random() < 0.2 and not (dtype == "fp32" and T in (4, 8) and Ci > 256 and not flags & eq.EQL_FLAG_FORCE_SIMT)
+        if gelu:
+            flags |= eq.EQL_FLAG_GELU
         wl = Workload("fz", dtype, T, Ci, Co, N, rng.choice(["normal", "zero", "none"]), ("fwd", "bwd_data", "bwd_weight"), 1000 + it)
         d = generate(wl)
         layer = GpuLayer(T, Ci, Co, dtype, d["w"], d["bias"], flags)
@@ -62,7 +65,11 @@ def test_random_shapes_match_the_oracle():
         kinds[key] = kinds.get(key, 0) + 1
         errs = {}
         try:
-            errs["y"] = rel_max_err(layer.fwd(d["x"]), orc.fwd(d["x"], d["w"], d["bias"], corr))
+            ref_y = orc.fwd(d["x"], d["w"], d["bias"], corr)
+            if gelu:
+                from scipy.special import erf
+                ref_y = 0.5 * ref_y * (1.0 + erf(ref_y / np.sqrt(2.0)))
+            errs["y"] = rel_max_err(layer.fwd(d["x"]), ref_y)
             errs["dx"] = rel_max_err(layer.bwd_data(d["dy"]), orc.bwd_data(d["dy"], d["w"], corr))
             dw, db = layer.bwd_weight(d["x"], d["dy"])
             rdw, rdb = orc.bwd_weight(d["x"], d["dy"], T, corr)
@@ -79,7 +86,7 @@ def test_random_shapes_match_the_oracle():
                 db2 = torch.full((Co,), float("nan"), dtype=torch.float32, device="cuda")
                 eq.eqlinear_bwd_weight_from_spectrum(layer.plan, spec, sb, dy_t, dw2, db2, N, sc, scb, layer.stream)
                 torch.cuda.synchronize()
-                errs["y_s"] = rel_max_err(y2.cpu().numpy(), orc.fwd(d["x"], d["w"], d["bias"], corr))
+                errs["y_s"] = rel_max_err(y2.cpu().numpy(), ref_y)
                 errs["dw_s"], errs["db_s"] = rel_max_err(dw2.cpu().numpy(), rdw), rel_max_err(db2.cpu().numpy(), rdb)
                 if not bool((spec[sb:] == 0x7F).all().item()):
                     errs["spectrum_overrun"] = 1.0
