@@ -402,7 +402,7 @@ def run_workload(args, wl, rt):
     # x is the small tensor of the layer (else writing x^ costs more than repeating the transform).
     # Also on very wide layers, where the weight gradient repeats the transform of x once per output-channel tile
     # (16 times at 2048 channels) and the pre-pass that writes x^ is cheap next to the GEMMs.
-    use_saved = (has_bwd and not args.no_saved_spectrum and wl.dtype == "fp16" and info.bwd_weight_kernel == 1
+    use_saved = (has_bwd and not args.no_saved_spectrum and wl.dtype != "fp32" and info.bwd_weight_kernel == 1
                  and ((info.fwd_kernel == 2 and wl.Co >= 2 * wl.Ci) or wl.Co >= 1024))
     spec_bytes = eq.eqlinear_spectrum_bytes(plan, wl.N) if use_saved else 0
     if use_saved:

@@ -195,11 +195,11 @@ eql_status_t eqlinear_bwd_weight(eqlinear_plan_t plan, const void* x, const void
                                  void* dw, void* db, int64_t N,
                                  void* scratch, size_t scratch_bytes, void* stream);
 
-/* ---- training with a saved spectrum (FP16 plans whose weight gradient runs on the tensor cores) --
+/* ---- training with a saved spectrum (FP16 / BF16 plans whose weight gradient runs on the tensor cores) --
  * Algorithm 1 transforms x once for the forward pass; the weight gradient needs the same spectrum
  * x^ again, and computing it there is the largest share of that kernel's instructions (every
  * output-channel tile repeats it).  These three calls let the forward pass save x^ -- rounded to
- * fp16, in the operand layout of the weight-gradient kernel -- so that the weight gradient reads it
+ * the plan's 16-bit type, in the operand layout of the weight-gradient kernel -- so that the weight gradient reads it
  * back instead of x.  (The paper's kernels keep no frequency-domain tensor in global memory; this
  * is an optional trade of N*C_in*T*2 bytes of device memory and one extra write of that size for a
  * shorter backward pass.)  The buffer's layout is private to the library; it is valid for the plan

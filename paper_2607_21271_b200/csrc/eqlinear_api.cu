@@ -356,7 +356,7 @@ eql_status_t eqlinear_plan_launch_counts(eqlinear_plan_t plan, int64_t N, int32_
         counts[2] = 2;
     }
     // eqlinear_fwd_save_spectrum: the resident-activation kernel writes the spectrum itself, others add a pre-pass
-    counts[3] = (plan->dtype == EQL_FP16 && plan->bwd_weight_kernel == 1 && plan->fwd_kernel != 2) ? 1 : 0;
+    counts[3] = (plan->dtype != EQL_FP32 && plan->bwd_weight_kernel == 1 && plan->fwd_kernel != 2) ? 1 : 0;
     return EQL_OK;
 }
 
@@ -485,7 +485,7 @@ eql_status_t eqlinear_spectrum_bytes(eqlinear_plan_t plan, int64_t N, size_t* by
     if (!plan || !bytes) return EQL_ERR_INVALID_ARG;
     eql_status_t st = check_tokens(N);
     if (st != EQL_OK) return st;
-    if (plan->dtype != EQL_FP16 || plan->bwd_weight_kernel != 1) return EQL_ERR_UNSUPPORTED;
+    if (plan->dtype == EQL_FP32 || plan->bwd_weight_kernel != 1) return EQL_ERR_UNSUPPORTED;
     *bytes = umma_bwd_weight_shape(plan->T, plan->Ci, plan->Co, plan->dtype, N > 0 ? N : 1, plan->num_sms).stash_bytes;
     return EQL_OK;
 }

@@ -70,8 +70,8 @@ struct BwBarriers {
 // [CiT channels x 16 tokens] tile:  (channel mn, token k) at (mn/8)*256 + (k/8)*128 + (k%8)*16 + (mn%8)*2.
 // The six output-channel tiles of the EQ-ViT-B layer then share one transform of x instead of repeating it.
 // One half warp per 64-element slab of a token row, one token per lane; rows >= N and channels >= Ci are zero.
-template <int T>
-__global__ void xhat_image_kernel(const __half* __restrict__ x, int64_t N, int Ci, int CiT, int nXs, int64_t total_chunks,
+template <int T, typename IO>
+__global__ void xhat_image_kernel(const IO* __restrict__ x, int64_t N, int Ci, int CiT, int nXs, int64_t total_chunks,
                                   uint8_t* __restrict__ image) {
     constexpr int NCH = 64 / T;
     const int64_t blob = blockIdx.x;                             // = ci_tile * total_chunks + chunk
@@ -91,7 +91,7 @@ __global__ void xhat_image_kernel(const __half* __restrict__ x, int64_t N, int C
         wd[4 * j] = v.x; wd[4 * j + 1] = v.y; wd[4 * j + 2] = v.z; wd[4 * j + 3] = v.w;
     }
     uint32_t packed[T][NCH / 2];
-    dft_words<T, false>(wd, packed, nullptr);
+    dft_words<T, false, false, IO>(wd, packed, nullptr);
     const int mn0 = hw * NCH;
     const int off = (mn0 >> 3) * 256 + (row >> 3) * 128 + (row & 7) * 16 + (mn0 & 7) * 2;
     uint8_t* dst = image + (size_t)blob * ((size_t)T * CiT * 32) + off;
@@ -102,7 +102,7 @@ __global__ void xhat_image_kernel(const __half* __restrict__ x, int64_t N, int C
 // MERGED (x^ ring as deep as the dy^ stages, i.e. three): chunk c uses stage c % 3 and ring slot c % 3, so one "full"
 // barrier (the group's transform warps + the x^ copy) and one "empty" barrier (one commit) per chunk serve both, and
 // the MMA-issuing thread - which paces this kernel - handles half as many barrier operations.
-template <int T, bool MERGED>
+template <int T, bool MERGED, typename IO>
 __global__ void __launch_bounds__(kThreadsBw, 1)
 umma_bwd_weight_saved_kernel(const __grid_constant__ CUtensorMap tmap_dy, const __grid_constant__ CUtensorMap tmap_part,
                              const BwParams prm) {
@@ -212,8 +212,8 @@ umma_bwd_weight_saved_kernel(const __grid_constant__ CUtensorMap tmap_dy, const 
     } else if (warp == kWarpMmaBw) {
         if (lane == 0) {
             bool ok = true;
-            const uint32_t idesc_real = ptx::umma_idesc_f16_f32_mn_major(128, CoT);
-            const uint32_t idesc_cplx = ptx::umma_idesc_f16_f32_mn_major(128, 2 * CoT);
+            const uint32_t idesc_real = ptx::umma_idesc_f16_f32_mn_major(128, CoT, H16<IO>::kUmmaFormat);
+            const uint32_t idesc_cplx = ptx::umma_idesc_f16_f32_mn_major(128, 2 * CoT, H16<IO>::kUmmaFormat);
             const uint32_t a_plane = (uint32_t)CiT * 32u, b_tile = (uint32_t)CoT * 32u;
             const int XS = MERGED ? kGroups : prm.x_slots;
             int st = 0, xs = 0;                                  // dy^ stage and x^ ring slot of the current chunk
@@ -283,7 +283,7 @@ umma_bwd_weight_saved_kernel(const __grid_constant__ CUtensorMap tmap_dy, const 
             uint32_t packed[T][NCH / 2];
             float p0[NCH];
             if (active) {
-                dft_words<T, true>(wd, packed, p0);
+                dft_words<T, true, false, IO>(wd, packed, p0);
             }
             // the MMAs that read this stage three chunks ago must have retired
             ok = ptx::mbar_wait(&bar->empty_ab[g], ph ^ 1, abort_flag, status, 204);
@@ -436,10 +436,15 @@ cudaError_t launch_xhat_image(const UmmaBwdWeightShape& s, const void* x, int64_
     if (blobs > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
     const int xthreads = (s.nXs * 16 + 31) / 32 * 32;
     switch (s.T) {
-        case 4: xhat_image_kernel<4><<<(unsigned)blobs, xthreads, 0, stream>>>((const __half*)x, N, s.Ci, s.CiT, s.nXs, s.total_chunks, (uint8_t*)stash); break;
-        case 8: xhat_image_kernel<8><<<(unsigned)blobs, xthreads, 0, stream>>>((const __half*)x, N, s.Ci, s.CiT, s.nXs, s.total_chunks, (uint8_t*)stash); break;
-        case 16: xhat_image_kernel<16><<<(unsigned)blobs, xthreads, 0, stream>>>((const __half*)x, N, s.Ci, s.CiT, s.nXs, s.total_chunks, (uint8_t*)stash); break;
-        case 32: xhat_image_kernel<32><<<(unsigned)blobs, xthreads, 0, stream>>>((const __half*)x, N, s.Ci, s.CiT, s.nXs, s.total_chunks, (uint8_t*)stash); break;
+#define EQL_XHAT(TT)                                                                                                        \
+    case TT:                                                                                                               \
+        if (s.bf16) xhat_image_kernel<TT, __nv_bfloat16><<<(unsigned)blobs, xthreads, 0, stream>>>(                        \
+            (const __nv_bfloat16*)x, N, s.Ci, s.CiT, s.nXs, s.total_chunks, (uint8_t*)stash);                              \
+        else xhat_image_kernel<TT, __half><<<(unsigned)blobs, xthreads, 0, stream>>>(                                      \
+            (const __half*)x, N, s.Ci, s.CiT, s.nXs, s.total_chunks, (uint8_t*)stash);                                     \
+        break;
+        EQL_XHAT(4) EQL_XHAT(8) EQL_XHAT(16) EQL_XHAT(32)
+#undef EQL_XHAT
         default: return cudaErrorInvalidValue;
     }
     return cudaGetLastError();
@@ -488,9 +493,13 @@ cudaError_t launch_umma_bwd_weight_saved(const UmmaBwdWeightShape& s, const void
     auto go2 = [&](auto tc, auto mg) -> cudaError_t {
         constexpr int TT = decltype(tc)::value;
         constexpr bool MG = decltype(mg)::value;
-        static SmemLimitOnce smem_limit;                      // per kernel instantiation
-        if (cudaError_t e = smem_limit.ensure(umma_bwd_weight_saved_kernel<TT, MG>, 227 * 1024); e != cudaSuccess) return e;
-        return launch_overlapped(umma_bwd_weight_saved_kernel<TT, MG>, dim3(grid), dim3(kThreadsBw), smem, stream, my, mp, prm);
+        static SmemLimitOnce smem_limit[2];                   // per kernel instantiation
+        if (s.bf16) {
+            if (cudaError_t e = smem_limit[1].ensure(umma_bwd_weight_saved_kernel<TT, MG, __nv_bfloat16>, 227 * 1024); e != cudaSuccess) return e;
+            return launch_overlapped(umma_bwd_weight_saved_kernel<TT, MG, __nv_bfloat16>, dim3(grid), dim3(kThreadsBw), smem, stream, my, mp, prm);
+        }
+        if (cudaError_t e = smem_limit[0].ensure(umma_bwd_weight_saved_kernel<TT, MG, __half>, 227 * 1024); e != cudaSuccess) return e;
+        return launch_overlapped(umma_bwd_weight_saved_kernel<TT, MG, __half>, dim3(grid), dim3(kThreadsBw), smem, stream, my, mp, prm);
     };
     auto go = [&](auto tc) -> cudaError_t { return merged ? go2(tc, std::true_type{}) : go2(tc, std::false_type{}); };
     switch (s.T) {

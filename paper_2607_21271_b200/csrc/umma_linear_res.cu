@@ -629,7 +629,6 @@ cudaError_t launch_umma_linear_res(const UmmaResShape& s, const void* in, void* 
         static SmemLimitOnce once[4];                         // per kernel instantiation: (activation, element type)
         constexpr int threads = ResWarps<TT>::kThreads;
         if (s.bf16) {
-            if (stash != nullptr) return cudaErrorInvalidValue;   // the saved-spectrum path is built for IEEE half
             if (prm.act) return launch(umma_linear_res_kernel<TT, NT, PF, MG, true, __nv_bfloat16>, once[3], threads);
             return launch(umma_linear_res_kernel<TT, NT, PF, MG, false, __nv_bfloat16>, once[2], threads);
         }

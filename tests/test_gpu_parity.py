@@ -84,12 +84,31 @@ def test_bf16_matches_oracle(T, Ci, Co, N, flags, kernels):
     try:
         info = eq.eqlinear_plan_info(layer.plan)
         assert (info.fwd_kernel, info.bwd_data_kernel, info.bwd_weight_kernel) == kernels
-        with pytest.raises(eq.EqlError) as e:                                 # the saved-spectrum path is FP16 only
-            eq.eqlinear_spectrum_bytes(layer.plan, N)
-        assert e.value.status == eq.binding.EQL_ERR_UNSUPPORTED
+        saved = {}
+        if info.bwd_weight_kernel == 1:                                       # training with a saved spectrum, in bfloat16
+            x = torch.from_numpy(d["x"]).cuda().to(torch.bfloat16)
+            dy = torch.from_numpy(d["dy"]).cuda().to(torch.bfloat16)
+            sb = eq.eqlinear_spectrum_bytes(layer.plan, N)
+            spec = torch.full((sb + 64,), 0x7F, dtype=torch.uint8, device="cuda")
+            y = torch.empty(N, Co * T, dtype=torch.bfloat16, device="cuda")
+            eq.eqlinear_fwd_save_spectrum(layer.plan, x, y, N, spec, sb, layer.stream)
+            scb = eq.eqlinear_bwd_weight_scratch_bytes(layer.plan, N)
+            sc = torch.empty(scb, dtype=torch.uint8, device="cuda")
+            dw = torch.full((Co, Ci, T), float("nan"), dtype=torch.float32, device="cuda")
+            db = torch.full((Co,), float("nan"), dtype=torch.float32, device="cuda")
+            eq.eqlinear_bwd_weight_from_spectrum(layer.plan, spec, sb, dy, dw, db, N, sc, scb, layer.stream)
+            assert layer.raw_status() == 0
+            assert bool((spec[sb:] == 0x7F).all().item())
+            rdw, rdb = orc.bwd_weight(d["x"], d["dy"], T)
+            saved = {"y_saved": rel_max_err(y.float().cpu().numpy(), orc.fwd(d["x"], d["w"], d["bias"])),
+                     "dw_saved": rel_max_err(dw.cpu().numpy(), rdw), "db_saved": rel_max_err(db.cpu().numpy(), rdb)}
+        else:
+            with pytest.raises(eq.EqlError) as e:                             # no saved-spectrum path behind CUDA-core kernels
+                eq.eqlinear_spectrum_bytes(layer.plan, N)
+            assert e.value.status == eq.binding.EQL_ERR_UNSUPPORTED
     finally:
         layer.close()
-    errs = check_workload(wl, flags=flags, data=d)
+    errs = {**check_workload(wl, flags=flags, data=d), **saved}
     print({k: f"{v:.2e}" for k, v in errs.items()})
     for k, v in errs.items():
         assert v <= TOL["bf16"], f"T={T} Ci={Ci} Co={Co} N={N} flags={flags}: {k} error {v:.3e}"
