@@ -124,8 +124,8 @@ eql_status_t eqlinear_workspace_bytes(int T, int C_in, int C_out, eql_dtype_t dt
  * conjugate-transposed data-gradient product, with the 1/T of the inverse DFT folded in -- and a
  * copy of the bias in `workspace`.
  *   T            group order: 1 to 8, 12, 16 or 32 (Algorithm 1 holds for every cyclic group; the paper's own kernels
- *                cover T = 4).  Powers of two from 4 run on the tensor cores, the other orders -- odd ones
- *                included -- on CUDA-core kernels with a table-driven real DFT
+ *                cover T = 4).  Powers of two from 4 run on the tensor cores (T = 2: forward and data gradient of
+ *                16-bit plans), the other orders -- odd ones included -- on CUDA-core kernels with a table-driven real DFT
  *   C_in, C_out  channels per group element, >= 1; C_in*T*elem and C_out*T*elem must be
  *                multiples of 16 bytes
  *   w            device, [C_out, C_in, T], plan dtype

@@ -72,6 +72,7 @@ template <int T, int E, int CG = 1> struct UmmaCfg;   // E = bytes per element o
 // the tensor core is streaming operands, and on wide layers that thread paces the kernel.
 // KS: chunks (UMMA K steps) per operand stage and weight slot.  With two, the issuing thread's wait and commit are paid
 // once per 32 reduced channels (the reduction is padded to a multiple of KS chunks with zero channels).
+template <> struct UmmaCfg<2, 2, 1>  { static constexpr int SPS = 1, SA = 3, SB = 3, KS = 2, MAXCOT = 256; static constexpr bool EARLY = true, MERGED = true; };
 template <> struct UmmaCfg<4, 2, 1>  { static constexpr int SPS = 1, SA = 2, SB = 2, KS = 2, MAXCOT = 128; static constexpr bool EARLY = true, MERGED = true; };
 template <> struct UmmaCfg<8, 2, 1>  { static constexpr int SPS = 2, SA = 2, SB = 2, KS = 1, MAXCOT = 64;  static constexpr bool EARLY = false, MERGED = true; };
 template <> struct UmmaCfg<16, 2, 1> { static constexpr int SPS = 1, SA = 2, SB = 1, KS = 1, MAXCOT = 32;  static constexpr bool EARLY = true, MERGED = false; };
@@ -205,7 +206,10 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
     constexpr int EPR = 128 / E;                // elements per raw slab row (128 B)
     constexpr int NCH = EPR / T;                // channels per raw slab row
     constexpr int KCH = kRowBytes / E;          // channels per chunk = one UMMA K step (16 halves / 8 floats)
-    constexpr int SPK = KCH / NCH;              // slabs per chunk (= T/4)
+    constexpr int SPK = KCH >= NCH ? KCH / NCH : 1;   // slabs per chunk (= T/4; one slab holds both chunks of a stage at T = 2)
+    constexpr int CPS = NCH > KCH ? NCH / KCH : 1;    // chunks per slab (2 at T = 2: a 128-byte row is 32 channels)
+    static_assert(CPS == 1 || CPS == KS, "a slab that spans chunks must span exactly one stage");
+    constexpr int SLABS_PER_STAGE = SPK * KS / CPS;
     constexpr int NSPLIT = E == 4 ? 2 : 1;      // operand copies: FP32 keeps TF32 hi parts and lo remainders
     constexpr int kAPart = T * 4096;            // T planes x [128 rows x 32 B]
     constexpr int kAChunk = kAPart * NSPLIT;    // one chunk's operand tiles
@@ -229,7 +233,7 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
         for (int i = 0; i < kRawSlots; ++i) { ptx::mbar_init(&bar->full_raw[i], 1); ptx::mbar_init(&bar->empty_raw[i], 4 * SPS); }
         // "full" of a stage: the transform warps; merged rings: + the weight copy (its producer's arrive.expect_tx);
         // pair, leader: + the peer CTA's word that its own stage is full
-        const uint32_t full_count = 4 * SPK * KS + (MERGED ? 1 : 0) + ((PAIR && rank == 0) ? 1 : 0);
+        const uint32_t full_count = 4 * SLABS_PER_STAGE + (MERGED ? 1 : 0) + ((PAIR && rank == 0) ? 1 : 0);
         for (int i = 0; i < SA; ++i) { ptx::mbar_init(&bar->full_a[i], full_count); ptx::mbar_init(&bar->empty_a[i], 1); }
         for (int i = 0; i < SB; ++i) { ptx::mbar_init(&bar->full_b[i], 1); ptx::mbar_init(&bar->empty_b[i], 1); }
         ptx::mbar_init(&bar->full_d, 1);
@@ -274,7 +278,7 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
             bool ok = true;
             for (int64_t u = first; u < prm.num_units && ok; u += stride) {
                 const int row0 = unit_row0(u);
-                for (int kc = 0; kc < nK && ok; ++kc) {
+                for (int kc = 0; kc < nK && ok; kc += CPS) {
                     for (int q = 0; q < SPK; ++q, ++cr) {
                         const uint32_t ph = cr / SPS;            // slot phase counter
                         const int slot = ph % kRawSlots;
@@ -435,7 +439,7 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
         // (a warp that stored into chunk c' has seen the commit of chunk c' - SA, so when it next waits for the
         // commit of chunk c - SA with c - c' <= SA the barrier is at most one phase behind).
         static_assert(kRawSlots == 3 && SPS <= 3, "raw slots must map to fixed warp groups");
-        static_assert((3 + SPK * KS - 1) / (SPK * KS) <= SA, "empty_a parity wait would be ambiguous");
+        static_assert((3 + SLABS_PER_STAGE - 1) / SLABS_PER_STAGE <= SA, "empty_a parity wait would be ambiguous");
         const int cw = warp - kWarpCompute0;
         const int quad = warp & 3;                               // TMEM lane quadrant this warp may read
         const int group = cw >> 2;                               // transform group, and share of the epilogue's column groups
@@ -453,12 +457,12 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
         uint8_t* staging = xhat + cw * 4096;                     // this warp's [32 tokens x 128 B] output stage (128B swizzle)
         for (int64_t u = first; u < prm.num_units && ok; u += stride, ++cu) {
             // ---- transform
-            for (int kc = 0; kc < nK && ok; ++kc, ++ca) {           // ca counts chunks here; stage = chunk / KS
+            for (int kc = 0; kc < nK && ok; kc += CPS, ca += CPS) {   // ca counts chunks here; stage = chunk / KS
                 const uint32_t stage = ca / KS;
                 const int sa = stage % SA;
 #pragma unroll 1
                 for (int q = 0; q < SPK; ++q) {
-                    const uint32_t cr = ca * SPK + q;            // running slab counter
+                    const uint32_t cr = (ca / CPS) * SPK + q;    // running slab counter
                     if ((int)(cr % 3) != group) continue;
                     const uint32_t ph = cr / SPS;                // raw-ring slot phase this slab arrives in
                     const int slot = ph % kRawSlots;
@@ -494,7 +498,14 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
                         if (!ok) break;
                         staging_pending = false;
                     }
-                    if constexpr (E == 2) {
+                    if constexpr (E == 2 && CPS == 2) {
+                        // the row's 32 channels are the stage's two chunks: 16 channels (one full 32-byte operand row) each
+#pragma unroll
+                        for (int p = 0; p < T; ++p) {
+                            store_plane_run<16>(dst + p * 4096, &packed[p][0], second);
+                            store_plane_run<16>(dst + kAChunk + p * 4096, &packed[p][8], second);
+                        }
+                    } else if constexpr (E == 2) {
 #pragma unroll
                         for (int p = 0; p < T; ++p) store_plane_run<2 * W>(dst + p * 4096, packed[p], second);
                     } else {
@@ -631,6 +642,7 @@ template <typename F>
 cudaError_t dispatch_umma(int T, int elem_bytes, F&& f, bool bf16 = false) {
     if (elem_bytes == 2 && bf16) {
         switch (T) {
+            case 2: return f(std::integral_constant<int, 2>{}, __nv_bfloat16{});
             case 4: return f(std::integral_constant<int, 4>{}, __nv_bfloat16{});
             case 8: return f(std::integral_constant<int, 8>{}, __nv_bfloat16{});
             case 16: return f(std::integral_constant<int, 16>{}, __nv_bfloat16{});
@@ -640,6 +652,7 @@ cudaError_t dispatch_umma(int T, int elem_bytes, F&& f, bool bf16 = false) {
     }
     if (elem_bytes == 2) {
         switch (T) {
+            case 2: return f(std::integral_constant<int, 2>{}, __half{});
             case 4: return f(std::integral_constant<int, 4>{}, __half{});
             case 8: return f(std::integral_constant<int, 8>{}, __half{});
             case 16: return f(std::integral_constant<int, 16>{}, __half{});
@@ -678,7 +691,7 @@ int umma_max_cot(int T, int elem_bytes) {
 
 
 bool umma_linear_supported(int T, eql_dtype_t dtype) {
-    if (dtype == EQL_FP16 || dtype == EQL_BF16) return T == 4 || T == 8 || T == 16 || T == 32;
+    if (dtype == EQL_FP16 || dtype == EQL_BF16) return T == 2 || T == 4 || T == 8 || T == 16 || T == 32;
     return T == 4 || T == 8;            // FP32 (3xTF32): the hi/lo operand stages of larger T do not fit in shared memory
 }
 
@@ -690,7 +703,8 @@ UmmaLinearShape umma_linear_shape(int T, int Cin, int Cout, eql_dtype_t dtype) {
     const int max_cot = umma_max_cot(T, s.elem_bytes);           // T planes x CoT fp32 TMEM columns <= 512
     s.nTiles = (Cout + max_cot - 1) / max_cot;
     const int per = (Cout + s.nTiles - 1) / s.nTiles;
-    s.CoT = (per + 15) / 16 * 16;
+    const int gran = T == 2 ? 32 : 16;                          // the epilogue drains 128 output bytes (64 / T channels) at a time
+    s.CoT = (per + gran - 1) / gran * gran;
     const int kch = kRowBytes / s.elem_bytes;                    // channels per chunk (one UMMA K step)
     const int ks = umma_chunks_per_stage(T, s.elem_bytes, false);   // (the same for the pair form of every T that has one)
     s.nK = ((Cin + kch - 1) / kch + ks - 1) / ks * ks;         // whole stages: the padding chunks hold zero channels

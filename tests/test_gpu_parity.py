@@ -47,7 +47,8 @@ def _gelu(a):
     ("fp16", 4, 64, 200, 777, eq.EQL_FLAG_FORCE_STREAMING | eq.EQL_FLAG_CTA_PAIR, 3),   # its CTA-pair form
     ("fp16", 16, 17, 33, 333, 0, 1),
     ("fp32", 8, 48, 48, 1000, 0, 1),                                         # 3xTF32
-    ("fp32", 5, 8, 24, 333, 0, 0), ("fp16", 2, 8, 16, 333, 0, 0),            # CUDA-core kernels
+    ("fp16", 2, 40, 300, 333, 0, 1),                                        # T = 2 on the streaming kernel
+    ("fp32", 5, 8, 24, 333, 0, 0), ("fp16", 2, 8, 16, 333, eq.EQL_FLAG_FORCE_SIMT, 0),   # CUDA-core kernels
 ])
 def test_fused_gelu_epilogue(dtype, T, Ci, Co, N, flags, kernel):
     """EQL_FLAG_GELU: the forward pass returns GELU(layer(x)), applied in FP32 before the one rounding of the output;
@@ -73,7 +74,8 @@ def test_fused_gelu_epilogue(dtype, T, Ci, Co, N, flags, kernel):
     (8, 96, 384, 1000, eq.EQL_FLAG_FORCE_STREAMING, (1, 1, 1)),               # streaming kernel
     (4, 100, 130, 515, eq.EQL_FLAG_FORCE_STREAMING | eq.EQL_FLAG_CTA_PAIR, (3, 3, 1)),   # CTA pairs
     (16, 17, 33, 333, 0, (1, 1, 1)), (32, 32, 32, 500, 0, (1, 1, 1)),
-    (5, 8, 24, 333, 0, (0, 0, 0)), (2, 8, 16, 333, 0, (0, 0, 0)),             # CUDA-core kernels
+    (2, 8, 16, 333, 0, (1, 1, 0)), (2, 72, 264, 1000, 0, (1, 1, 0)),          # T = 2: streaming kernel, CUDA-core weight gradient
+    (5, 8, 24, 333, 0, (0, 0, 0)),                                            # CUDA-core kernels
 ])
 def test_bf16_matches_oracle(T, Ci, Co, N, flags, kernels):
     """EQL_BF16: bfloat16 inputs and outputs, float accumulation -- every pass of every kernel family against the oracle
@@ -171,7 +173,7 @@ def test_ragged_token_counts(dtype, N):
 
 @pytest.mark.parametrize("dtype", ["fp32", "fp16"])
 @pytest.mark.parametrize("T,Ci,Co", [(2, 8, 16), (4, 64, 64), (4, 6, 10), (8, 96, 384), (8, 384, 96),
-                                       (16, 17, 33), (32, 32, 32), (32, 5, 3),
+                                       (16, 17, 33), (32, 32, 32), (32, 5, 3), (2, 136, 520),
                                        # Algorithm 1 for other cyclic groups: odd and non-power-of-two orders, and the trivial group
                                        (1, 16, 8), (3, 8, 16), (5, 8, 24), (6, 12, 20), (7, 8, 8), (12, 10, 6)])
 def test_shapes(dtype, T, Ci, Co):
