@@ -82,7 +82,17 @@ enum {
      * eqlinear_bwd_weight remain the gradients of the LINEAR layer; a caller that trains multiplies dy by GELU'(pre-
      * activation) itself and therefore needs the unfused forward.  EQL_ERR_UNSUPPORTED for FP32 plans on the tensor
      * cores with more than 256 input channels (their forward sums segments in global memory). */
-    EQL_FLAG_GELU = 32u
+    EQL_FLAG_GELU = 32u,
+    /* The group is the DIHEDRAL group D_T (the T rotations of the cyclic group and their T reflections, order 2T) --
+     * the reflection extension the paper's Conclusion names as future work.  T is the number of rotations (2, 3, 4, 5,
+     * 6 or 8); features are [N, C * 2T] and the weight [C_out, C_in, 2T] with the group index g = f*T + t fastest
+     * (element r^t s^f: rotation t, reflection flag f; s r = r^-1 s), and the layer is the group convolution
+     *     y[n, o, g] = bias[o] + sum_i sum_h w[o, i, h^-1 g] x[n, i, h],
+     * whose restriction to the rotations is the cyclic layer.  Algorithm 1 carries over with the group's irreducible
+     * representations in place of the DFT frequencies (one- and two-dimensional real blocks); the kernels run on the
+     * CUDA cores.  Not combinable with EQL_FLAG_CORRELATION, EQL_FLAG_FORCE_STREAMING or EQL_FLAG_CTA_PAIR.
+     * Size the workspace with eqlinear_workspace_bytes_flags. */
+    EQL_FLAG_DIHEDRAL = 64u
 };
 
 typedef struct {
@@ -116,6 +126,9 @@ eql_status_t eqlinear_count_macs(int T, int C_in, int C_out, int64_t N,
 
 /* Size in bytes of the device workspace a plan of this shape needs. */
 eql_status_t eqlinear_workspace_bytes(int T, int C_in, int C_out, eql_dtype_t dtype, size_t* bytes);
+
+/* The same for a plan built with `flags` (EQL_FLAG_DIHEDRAL changes the tuple length and hence the size). */
+eql_status_t eqlinear_workspace_bytes_flags(int T, int C_in, int C_out, eql_dtype_t dtype, unsigned flags, size_t* bytes);
 
 /* ---- plan (Algorithm 1, step 1 for the weight: the spectral weight, computed once) ---------- */
 

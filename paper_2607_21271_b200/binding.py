@@ -33,6 +33,7 @@ EQL_FLAG_FORCE_STREAMING = 4
 EQL_FLAG_CTA_PAIR = 8
 EQL_FLAG_NO_CTA_PAIR = 16
 EQL_FLAG_GELU = 32
+EQL_FLAG_DIHEDRAL = 64
 
 EQL_STATIC_SCRATCH_BYTES = 32 << 20
 
@@ -44,6 +45,7 @@ EXPORTED_SYMBOLS = (
     "eqlinear_fwd_host", "eqlinear_bwd_data_host", "eqlinear_bwd_weight_host", "eqlinear_step_host", "eqlinear_bwd_weight_static",
     "eqlinear_spectrum_bytes", "eqlinear_fwd_save_spectrum", "eqlinear_bwd_weight_from_spectrum",
     "eqlinear_plan_clear_device_status", "eqlinear_plan_selftest_expired_wait", "eqlinear_plan_launch_counts",
+    "eqlinear_workspace_bytes_flags",
 )
 
 
@@ -85,6 +87,7 @@ def load_library(path: str | None = None) -> ctypes.CDLL:
     sigs = {
         "eqlinear_count_macs": [I, I, I, I64, POINTER(I64), POINTER(I64)],
         "eqlinear_workspace_bytes": [I, I, I, I, POINTER(SZ)],
+        "eqlinear_workspace_bytes_flags": [I, I, I, I, c_uint, POINTER(SZ)],
         "eqlinear_plan": [POINTER(V), I, I, I, I, V, V, V, SZ, c_uint, V],
         "eqlinear_plan_set_weight": [V, V, V, V],
         "eqlinear_plan_info": [V, POINTER(EqlInfo)],
@@ -146,6 +149,12 @@ def eqlinear_count_macs(T: int, C_in: int, C_out: int, N: int) -> tuple[int, int
 def eqlinear_workspace_bytes(T: int, C_in: int, C_out: int, dtype: int) -> int:
     out = c_size_t(0)
     _check(load_library().eqlinear_workspace_bytes(T, C_in, C_out, dtype, byref(out)), "eqlinear_workspace_bytes")
+    return out.value
+
+
+def eqlinear_workspace_bytes_flags(T: int, C_in: int, C_out: int, dtype: int, flags: int) -> int:
+    out = c_size_t(0)
+    _check(load_library().eqlinear_workspace_bytes_flags(T, C_in, C_out, dtype, flags, byref(out)), "eqlinear_workspace_bytes_flags")
     return out.value
 
 

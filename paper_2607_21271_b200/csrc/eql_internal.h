@@ -27,7 +27,8 @@ struct WorkspaceLayout {
     size_t umma_fwd_bytes, umma_bwd_bytes;
     size_t total;
 };
-WorkspaceLayout workspace_layout(int T, int Ci, int Co, eql_dtype_t dtype);
+// T: length of a group tuple (the cyclic order, or 2 x rotations for a dihedral plan, which has no tensor-core images)
+WorkspaceLayout workspace_layout(int T, int Ci, int Co, eql_dtype_t dtype, bool tensor_cores = true);
 
 // Raises a kernel's dynamic shared-memory limit once per device.  One object per kernel instantiation (a function-local
 // static of the launcher); safe to use from several host threads: a bit is published only after the attribute call
@@ -181,6 +182,18 @@ cudaError_t launch_umma_bwd_weight_saved(const UmmaBwdWeightShape& s, const void
 cudaError_t launch_bwd_weight_finalize(int T, bool correlation, const float* scratch, int splits, int Ci, int Co,
                                        float* dw, float* db, cudaStream_t stream, bool accumulate = false);
 
+// ---- dihedral group D_T on the CUDA cores (dihedral_kernels.cu); T = number of rotations, tuples have 2T elements ----
+bool dihedral_supported_T(int T);
+int64_t dihedral_macs_per_pair(int T);
+cudaError_t launch_dihedral_plan_weights(int T, eql_dtype_t dtype, const void* w, const void* bias, int Ci, int Co,
+                                         float* planes_fwd, float* planes_bwd, float* bias_f32, cudaStream_t stream);
+cudaError_t launch_dihedral_linear(int T, eql_dtype_t dtype, const void* in, void* out, int64_t N, int Cin, int Cout,
+                                   const float* planes, const float* bias_f32, cudaStream_t stream, int act);
+BwdWeightSplit dihedral_bwd_weight_split(int T, int Ci, int Co, int64_t N);
+cudaError_t launch_dihedral_bwd_weight(int T, eql_dtype_t dtype, const void* x, const void* dy, float* dw, float* db,
+                                       int64_t N, int Ci, int Co, const BwdWeightSplit& split, float* scratch,
+                                       cudaStream_t stream);
+
 // Device address, on `device`, of the scratch array built into the library for eqlinear_bwd_weight_static
 // (static_scratch.cu).  `device` must be the current device.  Looked up once per device and cached; the first look-up
 // on a device loads the module that holds the array.  Returns nullptr on failure (*err, if given, says why).
@@ -200,7 +213,9 @@ struct HostPipe {
 
 // The host object behind eqlinear_plan_t.
 struct eqlinear_plan_s {
-    int T, Ci, Co;
+    int T, Ci, Co;                  // T: elements per group tuple (cyclic order; 2 x rot for a dihedral plan)
+    bool dihedral = false;          // EQL_FLAG_DIHEDRAL
+    int rot = 0;                    // dihedral plans: number of rotations (the T the caller passed)
     eql_dtype_t dtype;
     unsigned flags;
     bool has_bias;

@@ -8,7 +8,7 @@
 
 namespace eql {
 
-WorkspaceLayout workspace_layout(int T, int Ci, int Co, eql_dtype_t dtype) {
+WorkspaceLayout workspace_layout(int T, int Ci, int Co, eql_dtype_t dtype, bool tensor_cores) {
     WorkspaceLayout l{};
     size_t off = 0;
     l.status = off;      off += kWsAlign;
@@ -17,7 +17,7 @@ WorkspaceLayout workspace_layout(int T, int Ci, int Co, eql_dtype_t dtype) {
     l.planes_bwd = off;  off += align_up((size_t)T * Ci * Co * sizeof(float), kWsAlign);
     l.umma_fwd = off;    l.umma_fwd_bytes = 0;
     l.umma_bwd = off;    l.umma_bwd_bytes = 0;
-    if (umma_linear_supported(T, dtype)) {
+    if (tensor_cores && umma_linear_supported(T, dtype)) {
         l.umma_fwd_bytes = umma_linear_image_bytes(T, Ci, Co, dtype);
         l.umma_bwd_bytes = umma_linear_image_bytes(T, Co, Ci, dtype);
         if (umma_res_supported(T, dtype)) {          // one region serves whichever tensor-core kernel the plan selects
@@ -42,10 +42,17 @@ inline size_t elem_size(eql_dtype_t d) { return d == EQL_FP32 ? 4 : 2; }
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-eql_status_t check_shape(int T, int Ci, int Co, int dtype) {
+// T: the group parameter the caller passed (cyclic order, or rotations of a dihedral plan); *tuple = elements per tuple
+eql_status_t check_shape(int T, int Ci, int Co, int dtype, unsigned flags = 0, int* tuple = nullptr) {
     if (dtype != EQL_FP32 && dtype != EQL_FP16 && dtype != EQL_BF16) return EQL_ERR_INVALID_ARG;
     if (T < 1 || Ci < 1 || Co < 1) return EQL_ERR_INVALID_ARG;
-    if (!supported_T(T)) return EQL_ERR_UNSUPPORTED;
+    if (flags & EQL_FLAG_DIHEDRAL) {
+        if (!dihedral_supported_T(T)) return EQL_ERR_UNSUPPORTED;
+        T = 2 * T;
+    } else if (!supported_T(T)) {
+        return EQL_ERR_UNSUPPORTED;
+    }
+    if (tuple) *tuple = T;
     if ((int64_t)Ci * T > (1 << 20) || (int64_t)Co * T > (1 << 20)) return EQL_ERR_UNSUPPORTED;
     const size_t e = elem_size((eql_dtype_t)dtype);
     if (((size_t)Ci * T * e) % 16 != 0 || ((size_t)Co * T * e) % 16 != 0) return EQL_ERR_ALIGNMENT;
@@ -59,6 +66,12 @@ eql_status_t check_tokens(int64_t N) {
 }
 
 eql_status_t build_weights(eqlinear_plan_t p, const void* w, const void* bias, cudaStream_t s) {
+    if (p->dihedral) {
+        cudaError_t de = launch_dihedral_plan_weights(p->rot, p->dtype, w, bias, p->Ci, p->Co,
+                                                      (float*)(p->ws + p->lay.planes_fwd), (float*)(p->ws + p->lay.planes_bwd),
+                                                      (float*)(p->ws + p->lay.bias), s);
+        return de == cudaSuccess ? EQL_OK : EQL_ERR_CUDA;
+    }
     cudaError_t e = launch_plan_weights(p->T, p->dtype, (p->flags & EQL_FLAG_CORRELATION) != 0, w, bias, p->Ci, p->Co,
                                         (float*)(p->ws + p->lay.planes_fwd), (float*)(p->ws + p->lay.planes_bwd),
                                         (float*)(p->ws + p->lay.bias), s);
@@ -230,10 +243,15 @@ eql_status_t eqlinear_count_macs(int T, int C_in, int C_out, int64_t N, int64_t*
 }
 
 eql_status_t eqlinear_workspace_bytes(int T, int C_in, int C_out, eql_dtype_t dtype, size_t* bytes) {
+    return eqlinear_workspace_bytes_flags(T, C_in, C_out, dtype, 0u, bytes);
+}
+
+eql_status_t eqlinear_workspace_bytes_flags(int T, int C_in, int C_out, eql_dtype_t dtype, unsigned flags, size_t* bytes) {
     if (!bytes) return EQL_ERR_INVALID_ARG;
-    eql_status_t st = check_shape(T, C_in, C_out, dtype);
+    int tuple = 0;
+    eql_status_t st = check_shape(T, C_in, C_out, dtype, flags, &tuple);
     if (st != EQL_OK) return st;
-    *bytes = workspace_layout(T, C_in, C_out, dtype).total;
+    *bytes = workspace_layout(tuple, C_in, C_out, dtype, !(flags & EQL_FLAG_DIHEDRAL)).total;
     return EQL_OK;
 }
 
@@ -241,23 +259,27 @@ eql_status_t eqlinear_plan(eqlinear_plan_t* plan, int T, int C_in, int C_out, eq
                            const void* bias, void* workspace, size_t workspace_bytes, unsigned flags, void* stream) {
     if (!plan) return EQL_ERR_INVALID_ARG;
     *plan = nullptr;
-    eql_status_t st = check_shape(T, C_in, C_out, dtype);
+    int tuple = 0;
+    eql_status_t st = check_shape(T, C_in, C_out, dtype, flags, &tuple);
     if (st != EQL_OK) return st;
     if (!w || !workspace) return EQL_ERR_INVALID_ARG;
+    const bool dihedral = (flags & EQL_FLAG_DIHEDRAL) != 0;
+    // the dihedral group runs on the CUDA-core kernels of its own; flags that pick cyclic kernels or readings do not apply
+    if (dihedral && (flags & (EQL_FLAG_CORRELATION | EQL_FLAG_FORCE_STREAMING | EQL_FLAG_CTA_PAIR))) return EQL_ERR_INVALID_ARG;
     if (flags & ~(unsigned)(EQL_FLAG_CORRELATION | EQL_FLAG_FORCE_SIMT | EQL_FLAG_FORCE_STREAMING | EQL_FLAG_CTA_PAIR |
-                            EQL_FLAG_NO_CTA_PAIR | EQL_FLAG_GELU))
+                            EQL_FLAG_NO_CTA_PAIR | EQL_FLAG_GELU | EQL_FLAG_DIHEDRAL))
         return EQL_ERR_INVALID_ARG;
     if ((flags & EQL_FLAG_CTA_PAIR) && (flags & EQL_FLAG_NO_CTA_PAIR)) return EQL_ERR_INVALID_ARG;
     {   // The fused activation is applied to the finished sum: FP32 plans whose forward reduction runs as several
         // segments added in global memory (more than 256 input channels on the tensor cores) cannot take it.
         int len = 0;
-        if ((flags & EQL_FLAG_GELU) && !(flags & EQL_FLAG_FORCE_SIMT) && umma_linear_supported(T, dtype) &&
+        if ((flags & EQL_FLAG_GELU) && !(flags & (EQL_FLAG_FORCE_SIMT | EQL_FLAG_DIHEDRAL)) && umma_linear_supported(T, dtype) &&
             umma_reduction_segments(C_in, dtype, &len) > 1)
             return EQL_ERR_UNSUPPORTED;
     }
     if (!aligned16(w) || (bias && !aligned16(bias))) return EQL_ERR_ALIGNMENT;
     if (reinterpret_cast<uintptr_t>(workspace) % kWsAlign != 0) return EQL_ERR_ALIGNMENT;
-    WorkspaceLayout lay = workspace_layout(T, C_in, C_out, dtype);
+    WorkspaceLayout lay = workspace_layout(tuple, C_in, C_out, dtype, !dihedral);
     if (workspace_bytes < lay.total) return EQL_ERR_WORKSPACE;
 
     int dev = 0;
@@ -268,12 +290,13 @@ eql_status_t eqlinear_plan(eqlinear_plan_t* plan, int T, int C_in, int C_out, eq
 
     eqlinear_plan_s* p = new (std::nothrow) eqlinear_plan_s();
     if (!p) return EQL_ERR_INVALID_ARG;
-    p->T = T; p->Ci = C_in; p->Co = C_out; p->dtype = dtype; p->flags = flags;
+    p->T = tuple; p->Ci = C_in; p->Co = C_out; p->dtype = dtype; p->flags = flags;
+    p->dihedral = dihedral; p->rot = dihedral ? T : 0;
     p->has_bias = bias != nullptr; p->device = dev; p->ws = (char*)workspace; p->lay = lay;
     p->fwd_kernel = p->bwd_data_kernel = p->bwd_weight_kernel = 0;
     p->num_sms = kNumSMs;
     if (cudaDeviceGetAttribute(&p->num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) { delete p; return EQL_ERR_CUDA; }
-    if (umma_linear_supported(T, dtype) && !(flags & EQL_FLAG_FORCE_SIMT)) {
+    if (!dihedral && umma_linear_supported(T, dtype) && !(flags & EQL_FLAG_FORCE_SIMT)) {
         // 3xTF32 accumulates 1.4e-8 ... 1.6e-8 of relative error per reduced channel (measured: the tensor core adds
         // into its FP32 accumulator with truncation); FP32 plans therefore reduce at most 256 channels (4e-6) per
         // accumulator and run longer reductions as segments that are added in global memory (run_streaming below).
@@ -326,12 +349,14 @@ eql_status_t eqlinear_plan_set_weight(eqlinear_plan_t plan, const void* w, const
 eql_status_t eqlinear_plan_info(eqlinear_plan_t plan, eql_info_t* info) {
     if (!plan || !info) return EQL_ERR_INVALID_ARG;
     const int64_t e = (int64_t)elem_size(plan->dtype);
-    info->T = plan->T; info->C_in = plan->Ci; info->C_out = plan->Co; info->dtype = plan->dtype;
+    info->T = plan->dihedral ? plan->rot : plan->T; info->C_in = plan->Ci; info->C_out = plan->Co; info->dtype = plan->dtype;
     info->flags = plan->flags;
     info->fwd_kernel = plan->fwd_kernel;
     info->bwd_data_kernel = plan->bwd_data_kernel;
     info->bwd_weight_kernel = plan->bwd_weight_kernel;
     eqlinear_count_macs(plan->T, plan->Ci, plan->Co, 1, &info->macs_per_token, &info->dense_macs_per_token);
+    if (plan->dihedral)            // one product per one-dimensional irrep, eight per two-dimensional one
+        info->macs_per_token = dihedral_macs_per_pair(plan->rot) * plan->Ci * plan->Co;
     info->bytes_per_token_fwd = (int64_t)(plan->Ci + plan->Co) * plan->T * e;
     info->bytes_per_token_bwd_data = info->bytes_per_token_fwd;
     info->bytes_per_token_bwd_weight = info->bytes_per_token_fwd;
@@ -397,6 +422,11 @@ eql_status_t eqlinear_fwd(eqlinear_plan_t plan, const void* x, void* y, int64_t 
                                       plan->fwd_kernel == 3, act);
         return e == cudaSuccess ? EQL_OK : EQL_ERR_CUDA;
     }
+    if (plan->dihedral) {
+        cudaError_t de = launch_dihedral_linear(plan->rot, plan->dtype, x, y, N, plan->Ci, plan->Co,
+                                                (const float*)(plan->ws + plan->lay.planes_fwd), bias, (cudaStream_t)stream, act);
+        return de == cudaSuccess ? EQL_OK : EQL_ERR_CUDA;
+    }
     cudaError_t e = launch_direct_linear(plan->T, plan->dtype, x, y, N, plan->Ci, plan->Co,
                                          (const float*)(plan->ws + plan->lay.planes_fwd), bias, (cudaStream_t)stream, act);
     return e == cudaSuccess ? EQL_OK : EQL_ERR_CUDA;
@@ -419,6 +449,11 @@ eql_status_t eqlinear_bwd_data(eqlinear_plan_t plan, const void* dy, void* dx, i
                                       plan->bwd_data_kernel == 3);
         return e == cudaSuccess ? EQL_OK : EQL_ERR_CUDA;
     }
+    if (plan->dihedral) {
+        cudaError_t de = launch_dihedral_linear(plan->rot, plan->dtype, dy, dx, N, plan->Co, plan->Ci,
+                                                (const float*)(plan->ws + plan->lay.planes_bwd), nullptr, (cudaStream_t)stream, 0);
+        return de == cudaSuccess ? EQL_OK : EQL_ERR_CUDA;
+    }
     cudaError_t e = launch_direct_linear(plan->T, plan->dtype, dy, dx, N, plan->Co, plan->Ci,
                                          (const float*)(plan->ws + plan->lay.planes_bwd), nullptr, (cudaStream_t)stream);
     return e == cudaSuccess ? EQL_OK : EQL_ERR_CUDA;
@@ -430,6 +465,8 @@ eql_status_t eqlinear_bwd_weight_scratch_bytes(eqlinear_plan_t plan, int64_t N, 
     if (st != EQL_OK) return st;
     if (plan->bwd_weight_kernel == 1)
         *bytes = umma_bwd_weight_shape(plan->T, plan->Ci, plan->Co, plan->dtype, N > 0 ? N : 1, plan->num_sms).scratch_bytes;
+    else if (plan->dihedral)
+        *bytes = dihedral_bwd_weight_split(plan->rot, plan->Ci, plan->Co, N > 0 ? N : 1).scratch_bytes;
     else
         *bytes = direct_bwd_weight_split(plan->T, plan->Ci, plan->Co, N > 0 ? N : 1).scratch_bytes;
     return EQL_OK;
@@ -472,6 +509,13 @@ eql_status_t eqlinear_bwd_weight(eqlinear_plan_t plan, const void* x, const void
             if (e != cudaSuccess) return EQL_ERR_CUDA;
         }
         return EQL_OK;
+    }
+    if (plan->dihedral) {
+        BwdWeightSplit ds = dihedral_bwd_weight_split(plan->rot, plan->Ci, plan->Co, N);
+        if (scratch_bytes < ds.scratch_bytes) return EQL_ERR_WORKSPACE;
+        cudaError_t de = launch_dihedral_bwd_weight(plan->rot, plan->dtype, x, dy, (float*)dw, (float*)db, N, plan->Ci, plan->Co,
+                                                    ds, (float*)scratch, s);
+        return de == cudaSuccess ? EQL_OK : EQL_ERR_CUDA;
     }
     BwdWeightSplit split = direct_bwd_weight_split(plan->T, plan->Ci, plan->Co, N);
     if (scratch_bytes < split.scratch_bytes) return EQL_ERR_WORKSPACE;

@@ -45,11 +45,12 @@ class GpuLayer:
 
     def __init__(self, T, Ci, Co, dtype, w, bias, flags=0, device="cuda:0"):
         self.T, self.Ci, self.Co, self.dtype = T, Ci, Co, dtype
+        self.L = 2 * T if flags & eq.EQL_FLAG_DIHEDRAL else T        # elements per group tuple
         self.dev = torch.device(device)
         self.td = torch_dtype(dtype)
         self.w = to_device(w, dtype, self.dev)
         self.bias = None if bias is None else to_device(bias, dtype, self.dev)
-        self.ws_bytes = eq.eqlinear_workspace_bytes(T, Ci, Co, eql_dtype(dtype))
+        self.ws_bytes = eq.eqlinear_workspace_bytes_flags(T, Ci, Co, eql_dtype(dtype), flags & eq.EQL_FLAG_DIHEDRAL)
         self.ws = torch.empty(self.ws_bytes + 256, dtype=torch.uint8, device=self.dev)
         assert self.ws.data_ptr() % 256 == 0
         self.stream = torch.cuda.current_stream(self.dev).cuda_stream
@@ -81,26 +82,26 @@ class GpuLayer:
     def fwd(self, x_np):
         N = x_np.shape[0]
         x = to_device(x_np, self.dtype, self.dev)
-        buf, y = self._out(N, self.Co * self.T)
+        buf, y = self._out(N, self.Co * self.L)
         eq.eqlinear_fwd(self.plan, x if N else None, buf if N else None, N, self.stream)
         torch.cuda.synchronize(self.dev)
-        assert self._canary_ok(buf, N * self.Co * self.T), "fwd wrote past its output"
+        assert self._canary_ok(buf, N * self.Co * self.L), "fwd wrote past its output"
         return to_host(y)
 
     def bwd_data(self, dy_np):
         N = dy_np.shape[0]
         dy = to_device(dy_np, self.dtype, self.dev)
-        buf, dx = self._out(N, self.Ci * self.T)
+        buf, dx = self._out(N, self.Ci * self.L)
         eq.eqlinear_bwd_data(self.plan, dy if N else None, buf if N else None, N, self.stream)
         torch.cuda.synchronize(self.dev)
-        assert self._canary_ok(buf, N * self.Ci * self.T), "bwd_data wrote past its output"
+        assert self._canary_ok(buf, N * self.Ci * self.L), "bwd_data wrote past its output"
         return to_host(dx)
 
     def bwd_weight(self, x_np, dy_np, want_db=True):
         N = x_np.shape[0]
         x = to_device(x_np, self.dtype, self.dev)
         dy = to_device(dy_np, self.dtype, self.dev)
-        nw = self.Co * self.Ci * self.T
+        nw = self.Co * self.Ci * self.L
         wbuf, _ = self._out(1, nw, torch.float32)
         bbuf, _ = self._out(1, self.Co, torch.float32)
         sb = eq.eqlinear_bwd_weight_scratch_bytes(self.plan, N)
@@ -110,7 +111,7 @@ class GpuLayer:
         torch.cuda.synchronize(self.dev)
         assert self._canary_ok(wbuf, nw), "bwd_weight wrote past dw"
         assert self._canary_ok(bbuf, self.Co), "bwd_weight wrote past db"
-        dw = wbuf[:nw].view(self.Co, self.Ci, self.T).cpu().numpy()
+        dw = wbuf[:nw].view(self.Co, self.Ci, self.L).cpu().numpy()
         db = bbuf[:self.Co].cpu().numpy() if want_db else None
         return dw, db
 
