@@ -1,13 +1,14 @@
-// Fused EQ-Linear forward / data-gradient on the 5th-generation tensor cores (tcgen05 + TMEM), FP16 I/O,
-// FP32 accumulation.  One persistent CTA per SM; a work unit is (128-token tile, output-channel tile).
+// Fused EQ-Linear forward / data-gradient on the 5th-generation tensor cores (tcgen05 + TMEM): 16-bit I/O (IEEE half or
+// bfloat16, kind::f16) or float I/O (kind::tf32 with the 3xTF32 split), FP32 accumulation.  One persistent CTA per SM;
+// a work unit is (128-token tile, output-channel tile).
 //
 //   TMA (2-D, 128B swizzle)      raw rows of x            -> shared "slabs" [128 rows x 128 B]
-//   12 compute warps, phase 1    group DFT (Eq. 4) in registers, planes rounded to fp16 once
+//   12 compute warps, phase 1    group DFT (Eq. 4) in registers, planes rounded to the operand type once
 //                                -> shared A operands, one [128 x 16] K-major tile per real-packed plane
 //   TMA (1-D bulk)               spectral-weight image of this (tile, 16-channel chunk) -> shared B operands
 //   1 thread                     tcgen05.mma kind::f16: one product per real frequency, and the complex
 //                                product of Eq. 5 as the real 2x2 block [Xr|Xi] x [[Wr,Wi],[-Wi,Wr]] -> TMEM
-//   12 compute warps, phase 2    tcgen05.ld, bias on plane k = 0, inverse DFT (Eq. 7) in registers, fp16 rounding,
+//   12 compute warps, phase 2    tcgen05.ld, bias on plane k = 0, inverse DFT (Eq. 7) in registers, one rounding,
 //                                [32 tokens x 128 B] staged in shared memory (the idle A-operand stages) and written
 //                                with asynchronous, fully coalesced TMA tensor stores
 //

@@ -1,5 +1,5 @@
-// Fused EQ-Linear forward / data-gradient with the transformed activations RESIDENT in shared memory (FP16 I/O,
-// FP32 accumulation in TMEM, T = 4 or 8).  Used where the spectrum of one token tile fits on chip
+// Fused EQ-Linear forward / data-gradient with the transformed activations RESIDENT in shared memory (16-bit I/O: IEEE
+// half or bfloat16; FP32 accumulation in TMEM, T = 4 or 8).  Used where the spectrum of one token tile fits on chip
 // (C_in * T * 2 bytes * 512/T tokens <= ~150 KB), i.e. the layers with few input channels.
 //
 // Compared with the streaming kernel (umma_linear.cu) the roles of the two operands are exchanged: the
