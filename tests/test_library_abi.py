@@ -77,6 +77,23 @@ def test_workspace_bytes_validation():
     assert e.value.status == binding.EQL_ERR_INVALID_ARG
 
 
+def test_workspace_bytes_with_flags():
+    """The dihedral flag doubles the tuple length (2T elements per channel) and has its own list of group orders."""
+    D = binding.EQL_FLAG_DIHEDRAL
+    plain = eq.eqlinear_workspace_bytes_flags(5, 8, 8, eq.EQL_FP32, 0)
+    assert plain == eq.eqlinear_workspace_bytes(5, 8, 8, eq.EQL_FP32)
+    dih = eq.eqlinear_workspace_bytes_flags(5, 8, 8, eq.EQL_FP32, D)
+    assert dih >= 2 * 10 * 64 * 4 and dih > plain
+    for bad_T in (1, 7, 12, 16):
+        with pytest.raises(eq.EqlError) as e:
+            eq.eqlinear_workspace_bytes_flags(bad_T, 8, 8, eq.EQL_FP32, D)
+        assert e.value.status == binding.EQL_ERR_UNSUPPORTED
+    with pytest.raises(eq.EqlError) as e:                  # D_3 in half precision: 3 channels * 6 * 2 bytes = 36-byte rows
+        eq.eqlinear_workspace_bytes_flags(3, 3, 4, eq.EQL_FP16, D)
+    assert e.value.status == binding.EQL_ERR_ALIGNMENT
+    assert eq.eqlinear_workspace_bytes(8, 96, 384, eq.EQL_BF16) == eq.eqlinear_workspace_bytes(8, 96, 384, eq.EQL_FP16)
+
+
 def test_plan_argument_errors_are_caught_before_any_cuda_call():
     lib = eq.load_library()
     h = ctypes.c_void_p(1234)
